@@ -1,0 +1,195 @@
+/*
+ * specbound.h -- C ABI of the B200 (sm_100a) bounded self-speculative decode step.
+ *
+ * The method is SpecBound: a frozen Llama-style decoder drafts tokens from its own shallow
+ * layers and verifies them with its own deep layers, producing exactly the tokens plain greedy
+ * decoding would (paper: abstract; Section 3.3, last paragraph; Section 5).
+ *
+ * Conventions
+ *   - Every function returns SB_OK (0) or a negative sb_status.  Nothing throws, aborts or traps.
+ *     On error no output argument is written and the context is unchanged unless stated.
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are ordinary
+ *     host memory, read or written only during the call.
+ *   - Device memory is BORROWED: the caller allocates and frees weights, workspace and scratch and
+ *     owns the stream.  The library allocates no device memory.  sb_create pins one small host
+ *     mailbox (a few KB) that sb_destroy releases.
+ *   - Matrices are row-major [out_features, in_features] in the config's storage dtype, no biases,
+ *     LM head untied from the embedding.  Layers are numbered 1..n_layers as in the paper.
+ *   - One context = one sequence on one GPU.  A context is not thread-safe.
+ *   - Functions that return host scalars synchronise the context's stream themselves.
+ *   - Device-side waits are bounded; if one expires the call returns SB_ERR_DEVICE_TIMEOUT and the
+ *     CUDA context stays usable.
+ */
+#ifndef SPECBOUND_H
+#define SPECBOUND_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sb_ctx sb_ctx;
+
+typedef enum {
+    SB_OK = 0,
+    SB_ERR_ARG = -1,            /* NULL / out-of-range argument                                   */
+    SB_ERR_STATE = -2,          /* call out of order (no weights, no row in flight, wrong depth)   */
+    SB_ERR_CAPACITY = -3,       /* sequence, workspace or scratch too small                        */
+    SB_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed                               */
+    SB_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired                              */
+    SB_ERR_UNSUPPORTED = -6     /* shape/dtype combination the kernels do not cover                */
+} sb_status;
+
+typedef enum { SB_F32 = 0, SB_BF16 = 1 } sb_dtype;
+
+#define SB_MAX_W 8        /* most rows one pass may carry (w_max <= 8) */
+#define SB_MAX_LAYERS 64
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float rope_base, rms_eps;
+    int32_t dtype;   /* sb_dtype: storage of weights and of the KV cache; arithmetic is fp32 */
+    int32_t max_seq; /* most positions the KV cache holds                                   */
+    int32_t kv_page; /* tokens per KV page (power of two, >= 16)                            */
+} sb_config;
+
+typedef struct { /* device pointers */
+    const void *attn_norm /*[d]*/, *wq /*[H*hd,d]*/, *wk /*[Hkv*hd,d]*/, *wv /*[Hkv*hd,d]*/, *wo /*[d,H*hd]*/,
+        *mlp_norm /*[d]*/, *w_gate /*[F,d]*/, *w_up /*[F,d]*/, *w_down /*[d,F]*/;
+} sb_layer_weights;
+
+typedef struct {
+    const void *embed /*[V,d]*/, *final_norm /*[d]*/, *lm_head /*[V,d]*/; /* device */
+    const sb_layer_weights* layers;                                      /* HOST array [n_layers] */
+} sb_weights;
+
+typedef struct {
+    int64_t rounds, rows, accepted_drafts, emitted, probes, layer_steps, layer_row_steps;
+    int64_t exit_hist[SB_MAX_LAYERS + 1]; /* [l] = rows that exited at layer l; [0] = failed by d_max */
+    int64_t width_hist[SB_MAX_W + 1];     /* [w] = rounds verified with w rows                       */
+    double us_prefill, us_decode;         /* host wall time around the two phases                    */
+    double us_draft, us_verify;           /* device time (CUDA events) of draft phases / unified passes */
+    int64_t verify_layer_steps;           /* layer passes inside us_verify                           */
+    int64_t kernel_launches;              /* kernels launched by the call                            */
+} sb_stats;
+
+typedef struct { /* trace of one speculation round, filled by sb_generate when asked to */
+    int32_t w, D, emitted, accepted_drafts;
+    int32_t exit_layer[SB_MAX_W]; /* 0 = no exit by d_max */
+    int32_t draft[SB_MAX_W];      /* -1 = none            */
+    int32_t g[SB_MAX_W];          /* final greedy token of each row */
+    float conf[SB_MAX_W];         /* confidence at the exit layer (or at d_max) */
+} sb_round;
+
+typedef struct {
+    int32_t n;       /* positions whose KV is complete in every layer                      */
+    int32_t pending; /* last committed token, not yet forwarded (-1 before prefill)         */
+    int32_t rows;    /* rows in flight in the current round                                 */
+    int32_t depth[SB_MAX_W];
+} sb_state;
+
+/* ---- context -------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a context of this shape needs (KV pages + activations + scratch).
+ * Returns 0 if the config is invalid. */
+size_t sb_workspace_bytes(const sb_config* cfg);
+
+/* workspace: device, >= sb_workspace_bytes(cfg), 1024-byte aligned; stays the caller's.
+ * cuda_stream: a cudaStream_t (NULL = default stream) on which all work of the context runs. */
+int sb_create(const sb_config* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream, sb_ctx** out);
+void sb_destroy(sb_ctx* ctx);
+
+/* Records the (device) weight pointers of a frozen base model (paper Section 4.1: the base
+ * parameters are never modified) and prepares the TMA descriptors of every matrix.  The weights
+ * must outlive the context.  Errors: SB_ERR_ARG (NULL / misaligned pointer: 16 bytes needed). */
+int sb_load_weights(sb_ctx* ctx, const sb_weights* w);
+
+/* Forget the sequence: n = 0, no pending token, no rows in flight.  KV pages stay allocated. */
+int sb_reset(sb_ctx* ctx);
+int sb_get_state(sb_ctx* ctx, sb_state* out);
+/* Copy the cached hidden state of in-flight row `row` (fp32 [d_model]) to host memory. */
+int sb_read_hidden(sb_ctx* ctx, int32_t row, float* host_out);
+
+/* ---- the decode step ------------------------------------------------------------------------ */
+
+/* Prefill (Section 4.3: identical to the base model): all n_prompt tokens (host) through all
+ * layers; first_token (host) receives the first generated token, which becomes `pending`. */
+int sb_prefill(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t* first_token);
+
+/* Draft-phase primitives (Section 3.3).  push: a new row at depth 0 whose input token is `token`,
+ * at position n + rows.  advance: run layers for every in-flight row whose depth is below
+ * `to_layer`, lazily filling the KV of earlier rows together with the newer ones (the cache
+ * manager's "Reuse"), until all rows with smaller depth reach `to_layer`. */
+int sb_draft_push(sb_ctx* ctx, int32_t token);
+int sb_draft_advance(sb_ctx* ctx, int32_t to_layer);
+
+/* (a) Exit decision of Section 3.2 (Eq. 1-2) for the newest row, whose depth must equal `layer`:
+ * final RMSNorm -> shared LM head -> logits / tau_l -> conf = max softmax, token = argmax,
+ * exit_flag = (conf >= threshold).  One fused kernel; logits never reach HBM.  Outputs are host. */
+int sb_exit_confidence(sb_ctx* ctx, int32_t layer, float tau_l, float threshold, float* conf, int32_t* token,
+                       int32_t* exit_flag);
+
+/* (b) Unified parallel pass (Section 3.3; appendix "Illustration of Long Shallow Chains") over
+ * the w rows in flight: alignment to the deepest row, layers D+1..L for all rows, final greedy
+ * token of each row, greedy acceptance against drafts[i] (host; -1 = row i has no draft),
+ * KV rollback.  out_tokens (host, [w]) receives the n_out committed tokens.  w must equal the
+ * number of rows in flight. */
+int sb_verify(sb_ctx* ctx, const int32_t* drafts, int32_t w, int32_t* out_tokens, int32_t* n_out);
+
+/* Whole generation: prefill, then rounds of draft + verify until n_gen tokens are out.
+ * tau (host) [d_max]: tau[l-1] = temperature T_l of layer l.  threshold: exit when conf >= it
+ * (<= 0: always exit at layer 1; > 1: never exit).  rounds (host, nullable) [max_rounds] receives
+ * the per-round trace; n_rounds (nullable) their number.  stats nullable.
+ * Errors: SB_ERR_ARG (d_max not in [1, n_layers-1], w_max not in [1, SB_MAX_W], tau <= 0, NaN
+ * threshold, token id outside the vocabulary), SB_ERR_CAPACITY (n_prompt + n_gen + w_max > max_seq). */
+int sb_generate(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t n_gen, int32_t d_max, int32_t w_max,
+                const float* tau, float threshold, int32_t* out_tokens, int32_t* n_out, sb_stats* stats,
+                sb_round* rounds, int32_t max_rounds, int32_t* n_rounds);
+
+/* Plain greedy autoregressive decoding with the same kernels (one row, all layers per token):
+ * the baseline the paper's speed-ups are measured against (Section 3.4). */
+int sb_generate_ar(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t n_gen, int32_t* out_tokens,
+                   int32_t* n_out, sb_stats* stats);
+
+/* ---- stateless kernel entry points (micro-benchmarks, unit parity) ---------------------------- */
+
+/* Scratch bytes the two calls below need for this shape. */
+size_t sb_k_scratch_bytes(const sb_config* cfg);
+
+/* Exit-confidence kernel on m rows of hidden states (Section 3.2, Eq. 2):
+ * h device fp32 [m, d]; final_norm / lm_head device in cfg->dtype; tau_l > 0.
+ * conf device fp32 [m], token device int32 [m]; logits_dbg nullable device fp32 [m, vocab]
+ * (debug dump only).  scratch: device, >= sb_k_scratch_bytes, 1024-byte aligned. */
+int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const void* final_norm, const void* lm_head,
+                         float tau_l, float* conf, int32_t* token, float* logits_dbg, void* scratch,
+                         size_t scratch_bytes, void* cuda_stream);
+
+/* One decoder layer for m rows at positions first_pos .. first_pos+m-1 (the verify pass of one
+ * layer, Section 3.3): h device fp32 [m, d] in/out.  k_cache / v_cache: device, cfg->dtype,
+ * [n_pages, kv_page, n_kv_heads*head_dim]; page_table device int32 [ceil(max_seq / kv_page)]
+ * maps logical page -> physical page.  Appends K,V of the m rows, attends causally over
+ * positions 0 .. own position. */
+int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_t m, void* k_cache, void* v_cache,
+               const int32_t* page_table, int32_t first_pos, void* scratch, size_t scratch_bytes, void* cuda_stream);
+
+/* ---- helpers ---------------------------------------------------------------------------------- */
+
+/* Eq. 1: out[l-1] = 1 + alpha (1 - l/L) for l = 1..L (host). */
+int sb_tau_schedule(float alpha, int32_t L, float* out);
+/* Eq. 5: analytic speed-up for acceptance rate a, draft width w, depth bound d_max. */
+double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
+
+/* Options: SB_OPT_GEMM 0 = CUDA-core streaming kernels, 1 = TMA + tcgen05 kernels (bf16 only). */
+enum { SB_OPT_GEMM = 1 };
+int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);
+/* Process-wide default for contexts and stateless calls created afterwards. */
+int sb_set_default_option(int32_t key, int32_t value);
+
+const char* sb_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECBOUND_H */

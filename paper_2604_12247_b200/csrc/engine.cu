@@ -1,0 +1,685 @@
+// Host side of the SpecBound library: context, workspace layout, the layer step, the round loop
+// of Section 3.3 and the C ABI declared in include/specbound.h.  Every arithmetic step runs in a
+// kernel; the host only sequences launches and reads the few integers that gate the next launch
+// (exit flag after a probe, acceptance count after a round).
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "gemm_tc.cuh"
+#include "sb_internal.cuh"
+
+namespace sb {
+
+static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
+
+struct Dims {
+    int L, d, H, Hkv, hd, F, V, qd, kvd;
+    int page, page_shift, n_pages, max_seq, chunk;
+    float rope_base, eps;
+    bool f32;
+};
+
+static int pick_gemm(bool f32) {
+    if (f32 || !tc_available()) return 0;
+    return g_default_gemm < 0 ? 1 : g_default_gemm;
+}
+
+static bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+static bool make_dims(const sb_config* c, Dims* o) {
+    if (!c) return false;
+    if (c->n_layers < 1 || c->n_layers > SB_MAX_LAYERS || c->d_model < 8 || c->n_heads < 1 || c->n_kv_heads < 1 ||
+        c->d_ffn < 8 || c->vocab < 2 || c->max_seq < 1)
+        return false;
+    if (c->n_heads % c->n_kv_heads) return false;
+    if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->d_model % 8 || c->d_ffn % 8) return false;
+    if (c->dtype != SB_F32 && c->dtype != SB_BF16) return false;
+    if (!is_pow2(c->kv_page) || c->kv_page < 16) return false;
+    if (!(c->rope_base > 0.f) || !(c->rms_eps > 0.f)) return false;
+    o->L = c->n_layers; o->d = c->d_model; o->H = c->n_heads; o->Hkv = c->n_kv_heads; o->hd = c->head_dim;
+    o->F = c->d_ffn; o->V = c->vocab; o->qd = o->H * o->hd; o->kvd = o->Hkv * o->hd;
+    o->page = c->kv_page; o->page_shift = 0;
+    while ((1 << o->page_shift) < o->page) ++o->page_shift;
+    o->max_seq = c->max_seq;
+    o->n_pages = (c->max_seq + o->page - 1) / o->page;
+    // split-KV chunk: fixed per context so that a row's attention never depends on its companions
+    int ch = 32;
+    while (ch < 256 && ch * 64 < c->max_seq) ch <<= 1;
+    o->chunk = ch;
+    o->rope_base = c->rope_base; o->eps = c->rms_eps; o->f32 = c->dtype == SB_F32;
+    return true;
+}
+
+// Scratch shared by the context and the stateless entry points.
+struct Work {
+    int* page_table;
+    float* h;              // [8][d] hidden-state cache: one vector per in-flight row
+    void *act_a, *act_o, *act_f;
+    float *p_qkv, *p_o, *p_gu, *p_down;   // split-K partials [kMaxSplit][8][N]
+    float* q;              // [8][qd]
+    float* attn_part;
+    SoftTriple* head_part;
+    unsigned int* ticket;
+    int* res;              // result block: conf[8] | token[8] | flag[8] | accept[10] (32-bit words)
+    int* toks;             // [max_seq + 8] device token log
+    unsigned int* status;  // device status word of the bounded waits
+    void* k_cache;         // [L][n_pages][page][kvd]
+    void* v_cache;
+};
+
+struct Carver {
+    char* base;
+    size_t off = 0;
+    template <typename P> void take(P*& p, size_t bytes) {
+        off = (off + 1023) & ~size_t(1023);
+        p = reinterpret_cast<P*>(base ? base + off : nullptr);
+        off += bytes;
+    }
+};
+
+static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
+    Carver c{base};
+    Work tmp;
+    Work& W = w ? *w : tmp;
+    size_t es = D.f32 ? 4 : 2, act_rows = D.f32 ? 8 : 16;
+    c.take(W.page_table, sizeof(int) * D.n_pages);
+    c.take(W.h, sizeof(float) * kMaxW * D.d);
+    c.take(W.act_a, es * act_rows * D.d);
+    c.take(W.act_o, es * act_rows * D.qd);
+    c.take(W.act_f, es * act_rows * D.F);
+    size_t ps = sizeof(float) * kMaxSplit * kMaxW;
+    c.take(W.p_qkv, ps * (D.qd + 2 * D.kvd));
+    c.take(W.p_o, ps * D.d);
+    c.take(W.p_gu, ps * 2 * D.F);
+    c.take(W.p_down, ps * D.d);
+    c.take(W.q, sizeof(float) * kMaxW * D.qd);
+    int max_chunks = (D.max_seq + kMaxW + D.chunk - 1) / D.chunk + 1;
+    c.take(W.attn_part, sizeof(float) * (size_t)max_chunks * kMaxW * D.H * (D.hd + 2));
+    c.take(W.head_part, sizeof(SoftTriple) * kHeadMaxCtas * kMaxW);
+    c.take(W.ticket, 64);
+    c.take(W.res, sizeof(int) * 64);
+    c.take(W.status, 64);
+    if (with_state) {
+        c.take(W.toks, sizeof(int) * (D.max_seq + 16));
+        size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
+        c.take(W.k_cache, kv);
+        c.take(W.v_cache, kv);
+    }
+    return (c.off + 1023) & ~size_t(1023);
+}
+
+struct Exec {   // everything a launch sequence needs
+    Dims D;
+    Work W;
+    cudaStream_t st;
+    int gemm;   // 0 simt, 1 tcgen05
+    int64_t launches = 0;
+    // which normalised activation act_a currently holds
+    const void* act_gain = nullptr;
+    int act_r0 = 0, act_m = 0;
+    TcPlanCache* plans = nullptr;
+};
+
+#define SB_T(E, call)                          \
+    do {                                       \
+        if ((E).D.f32) { using T = float; call; } \
+        else { using T = __nv_bfloat16; call; }   \
+    } while (0)
+
+static void ensure_act(Exec& e, const void* gain, int r0, int m) {
+    if (e.act_gain == gain && r0 >= e.act_r0 && r0 + m <= e.act_r0 + e.act_m) return;
+    SB_T(e, launch_resid_norm<T>(e.st, e.W.h, nullptr, 0, e.D.d, (const T*)gain, e.D.eps, e.W.act_a, r0, m));
+    e.launches++;
+    e.act_gain = gain; e.act_r0 = r0; e.act_m = m;
+}
+
+// out = act x W^T for up to three matrices; returns the number of split-K partials written
+static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, const void* act, float* out, int r0, int m) {
+    GemmArgs a{};
+    int tot = 0;
+    for (int j = 0; j < n_mats; ++j) { a.W[j] = W[j]; tot += N[j]; a.n_end[j] = tot; }
+    for (int j = n_mats; j < 3; ++j) { a.W[j] = nullptr; a.n_end[j] = 0x7fffffff; }
+    a.n_mats = n_mats; a.K = K; a.act = act; a.out = out; a.n_total = tot; a.r0 = r0; a.m = m;
+    e.launches++;
+    if (e.gemm == 1 && !e.D.f32) return launch_gemm_tc(e.st, a, e.plans, e.W.status);
+    SB_T(e, launch_gemm_simt<T>(e.st, a));
+    return 1;
+}
+
+// One decoder layer for rows r0 .. r0+m-1 (row i sits at position pos0 + i).  Ends by adding the
+// MLP output to the hidden rows and, if next_gain is given, leaving their RMSNorm in act_a.
+static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int r0, int m, int pos0,
+                       const void* next_gain) {
+    const Dims& D = e.D;
+    Work& W = e.W;
+    ensure_act(e, lw.attn_norm, r0, m);
+    const void* wqkv[3] = {lw.wq, lw.wk, lw.wv};
+    int nqkv[3] = {D.qd, D.kvd, D.kvd};
+    int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.act_a, W.p_qkv, r0, m);
+    RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
+                pos0, r0, m, D.rope_base};
+    SB_T(e, launch_rope_append<T>(e.st, ra));
+    AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, W.act_o, D.H, D.Hkv, D.hd, D.page, D.page_shift,
+                pos0, r0, m, D.chunk};
+    SB_T(e, launch_attention<T>(e.st, aa));
+    e.launches += 3;
+    const void* wo[1] = {lw.wo};
+    int no[1] = {D.d};
+    int s_o = gemm(e, wo, no, 1, D.qd, W.act_o, W.p_o, r0, m);
+    SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_o, s_o, D.d, (const T*)lw.mlp_norm, D.eps, W.act_a, r0, m));
+    const void* wgu[2] = {lw.w_gate, lw.w_up};
+    int ngu[2] = {D.F, D.F};
+    int s_gu = gemm(e, wgu, ngu, 2, D.d, W.act_a, W.p_gu, r0, m);
+    SB_T(e, launch_swiglu<T>(e.st, W.p_gu, s_gu, D.F, W.act_f, r0, m));
+    const void* wd[1] = {lw.w_down};
+    int nd[1] = {D.d};
+    int s_d = gemm(e, wd, nd, 1, D.F, W.act_f, W.p_down, r0, m);
+    SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_down, s_d, D.d, (const T*)next_gain, D.eps, W.act_a, r0, m));
+    e.launches += 3;
+    e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
+}
+
+// exit-confidence / final-head kernel on rows r0 .. r0+m-1; act_a must hold their final RMSNorm
+static void head(Exec& e, const void* lm_head, int r0, int m, float tau, float threshold, float* conf, int* token,
+                 int* flag, float* logits_dbg) {
+    HeadArgs a{lm_head, e.D.V, e.D.d, e.W.act_a, r0, m, 1.f / tau, threshold, conf, token, flag, logits_dbg,
+               e.W.head_part, e.W.ticket};
+    e.launches++;
+    if (e.gemm == 1 && !e.D.f32) { launch_head_tc(e.st, a, e.plans, e.W.status); return; }
+    SB_T(e, launch_head_simt<T>(e.st, a, 148 * 4));
+}
+
+}  // namespace sb
+
+using namespace sb;
+
+struct sb_ctx {
+    sb_config cfg;
+    Exec e;
+    sb_weights w;
+    sb_layer_weights layers[SB_MAX_LAYERS];
+    bool loaded = false;
+    int* mailbox = nullptr;   // pinned host
+    int n = 0, pending = -1, rows = 0;
+    int depth[SB_MAX_W];
+    cudaEvent_t ev[3];
+    TcPlanCache plans;
+
+    void* kc(int layer) const {
+        size_t es = e.D.f32 ? 4 : 2;
+        return (char*)e.W.k_cache + es * (size_t)(layer - 1) * e.D.n_pages * e.D.page * e.D.kvd;
+    }
+    void* vc(int layer) const {
+        size_t es = e.D.f32 ? 4 : 2;
+        return (char*)e.W.v_cache + es * (size_t)(layer - 1) * e.D.n_pages * e.D.page * e.D.kvd;
+    }
+    float* conf_d() const { return reinterpret_cast<float*>(e.W.res); }
+    int* token_d() const { return e.W.res + 8; }
+    int* flag_d() const { return e.W.res + 16; }
+    int* accept_d() const { return e.W.res + 24; }
+};
+
+static int cuda_ok(cudaError_t err) { return err == cudaSuccess ? SB_OK : SB_ERR_CUDA; }
+
+// copy the 40-word result block to the pinned mailbox and wait for it; also surfaces launch errors
+// and expired device waits
+static int fetch_results(sb_ctx* c) {
+    if (cudaMemcpyAsync(c->mailbox, c->e.W.res, sizeof(int) * 40, cudaMemcpyDeviceToHost, c->e.st) != cudaSuccess)
+        return SB_ERR_CUDA;
+    if (cudaMemcpyAsync(c->mailbox + 48, c->e.W.status, sizeof(int), cudaMemcpyDeviceToHost, c->e.st) != cudaSuccess)
+        return SB_ERR_CUDA;
+    if (cudaStreamSynchronize(c->e.st) != cudaSuccess) return SB_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return SB_ERR_CUDA;
+    if (c->mailbox[48] != 0) return SB_ERR_DEVICE_TIMEOUT;
+    return SB_OK;
+}
+
+static void run_layer(sb_ctx* c, int layer, int r0, int m, const void* next_gain) {
+    layer_step(c->e, c->layers[layer - 1], c->kc(layer), c->vc(layer), r0, m, c->n, next_gain);
+    for (int i = r0; i < r0 + m; ++i) c->depth[i] = layer;
+}
+
+// run layer `layer` on the trailing rows whose depth is layer-1; returns rows advanced
+static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats* st) {
+    int r0 = c->rows;
+    while (r0 > 0 && c->depth[r0 - 1] == layer - 1) --r0;
+    int m = c->rows - r0;
+    if (m == 0) return 0;
+    run_layer(c, layer, r0, m, next_gain);
+    if (st) { st->layer_steps++; st->layer_row_steps += m; }
+    return m;
+}
+
+extern "C" {
+
+size_t sb_workspace_bytes(const sb_config* cfg) {
+    Dims D;
+    if (!make_dims(cfg, &D)) return 0;
+    return carve(D, nullptr, true, nullptr);
+}
+
+size_t sb_k_scratch_bytes(const sb_config* cfg) {
+    Dims D;
+    if (!make_dims(cfg, &D)) return 0;
+    return carve(D, nullptr, false, nullptr);
+}
+
+int sb_create(const sb_config* cfg, void* workspace, size_t bytes, void* stream, sb_ctx** out) {
+    Dims D;
+    if (!out || !workspace || !make_dims(cfg, &D)) return SB_ERR_ARG;
+    if ((uintptr_t)workspace & 1023) return SB_ERR_ARG;
+    if (bytes < carve(D, nullptr, true, nullptr)) return SB_ERR_CAPACITY;
+    sb_ctx* c = new (std::nothrow) sb_ctx();
+    if (!c) return SB_ERR_CUDA;
+    c->cfg = *cfg;
+    c->e.D = D;
+    c->e.st = (cudaStream_t)stream;
+    carve(D, (char*)workspace, true, &c->e.W);
+    c->e.gemm = pick_gemm(D.f32);
+    c->e.plans = &c->plans;
+    if (cudaHostAlloc((void**)&c->mailbox, sizeof(int) * 64, cudaHostAllocDefault) != cudaSuccess) {
+        delete c;
+        return SB_ERR_CUDA;
+    }
+    for (auto& ev : c->ev) cudaEventCreate(&ev);
+    launch_init_pages(c->e.st, c->e.W.page_table, D.n_pages);
+    cudaMemsetAsync(c->e.W.ticket, 0, 64, c->e.st);
+    cudaMemsetAsync(c->e.W.status, 0, 64, c->e.st);
+    cudaMemsetAsync(c->e.W.res, 0, sizeof(int) * 64, c->e.st);
+    if (cudaStreamSynchronize(c->e.st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+        sb_destroy(c);
+        return SB_ERR_CUDA;
+    }
+    for (int i = 0; i < SB_MAX_W; ++i) c->depth[i] = 0;
+    *out = c;
+    return SB_OK;
+}
+
+void sb_destroy(sb_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->e.st);
+    for (auto& ev : c->ev) cudaEventDestroy(ev);
+    if (c->mailbox) cudaFreeHost(c->mailbox);
+    delete c;
+}
+
+int sb_load_weights(sb_ctx* c, const sb_weights* w) {
+    if (!c || !w || !w->embed || !w->final_norm || !w->lm_head || !w->layers) return SB_ERR_ARG;
+    auto bad = [](const void* p) { return !p || ((uintptr_t)p & 15); };
+    if (bad(w->embed) || bad(w->final_norm) || bad(w->lm_head)) return SB_ERR_ARG;
+    for (int l = 0; l < c->e.D.L; ++l) {
+        const sb_layer_weights& s = w->layers[l];
+        const void* ps[9] = {s.attn_norm, s.wq, s.wk, s.wv, s.wo, s.mlp_norm, s.w_gate, s.w_up, s.w_down};
+        for (const void* p : ps)
+            if (bad(p)) return SB_ERR_ARG;
+    }
+    c->w = *w;
+    for (int l = 0; l < c->e.D.L; ++l) c->layers[l] = w->layers[l];
+    c->w.layers = c->layers;
+    c->plans.clear();
+    c->loaded = true;
+    return SB_OK;
+}
+
+int sb_reset(sb_ctx* c) {
+    if (!c) return SB_ERR_ARG;
+    c->n = 0; c->pending = -1; c->rows = 0;
+    c->e.act_gain = nullptr;
+    return SB_OK;
+}
+
+int sb_get_state(sb_ctx* c, sb_state* out) {
+    if (!c || !out) return SB_ERR_ARG;
+    out->n = c->n; out->pending = c->pending; out->rows = c->rows;
+    for (int i = 0; i < SB_MAX_W; ++i) out->depth[i] = i < c->rows ? c->depth[i] : 0;
+    return SB_OK;
+}
+
+int sb_read_hidden(sb_ctx* c, int32_t row, float* host_out) {
+    if (!c || !host_out || row < 0 || row >= c->rows) return SB_ERR_ARG;
+    if (cudaMemcpyAsync(host_out, c->e.W.h + (size_t)row * c->e.D.d, sizeof(float) * c->e.D.d, cudaMemcpyDeviceToHost,
+                        c->e.st) != cudaSuccess)
+        return SB_ERR_CUDA;
+    return cuda_ok(cudaStreamSynchronize(c->e.st));
+}
+
+int sb_set_option(sb_ctx* c, int32_t key, int32_t value) {
+    if (!c) return SB_ERR_ARG;
+    if (key == SB_OPT_GEMM) {
+        if (value != 0 && value != 1) return SB_ERR_ARG;
+        if (value == 1 && (c->e.D.f32 || !tc_available())) return SB_ERR_UNSUPPORTED;
+        c->e.gemm = value;
+        return SB_OK;
+    }
+    return SB_ERR_ARG;
+}
+
+int sb_set_default_option(int32_t key, int32_t value) {
+    if (key == SB_OPT_GEMM && (value == 0 || value == 1 || value == -1)) {
+        if (value == 1 && !tc_available()) return SB_ERR_UNSUPPORTED;
+        g_default_gemm = value;
+        return SB_OK;
+    }
+    return SB_ERR_ARG;
+}
+
+static int check_tokens(const sb_ctx* c, const int32_t* t, int n) {
+    for (int i = 0; i < n; ++i)
+        if (t[i] < 0 || t[i] >= c->e.D.V) return SB_ERR_ARG;
+    return SB_OK;
+}
+
+int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* first_token) {
+    if (!c || !prompt || !first_token || n_prompt < 1) return SB_ERR_ARG;
+    if (!c->loaded) return SB_ERR_STATE;
+    if (c->n != 0 || c->rows != 0) return SB_ERR_STATE;
+    if (n_prompt + 1 > c->e.D.max_seq) return SB_ERR_CAPACITY;
+    if (check_tokens(c, prompt, n_prompt)) return SB_ERR_ARG;
+    Exec& e = c->e;
+    if (cudaMemcpyAsync(e.W.toks, prompt, sizeof(int) * n_prompt, cudaMemcpyHostToDevice, e.st) != cudaSuccess)
+        return SB_ERR_CUDA;
+    int m = 0;
+    for (int p0 = 0; p0 < n_prompt; p0 += m) {
+        m = n_prompt - p0 < kMaxW ? n_prompt - p0 : kMaxW;
+        bool last = p0 + m == n_prompt;
+        SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, e.W.toks + p0, 0, 0, m, e.W.h));
+        e.launches++;
+        e.act_gain = nullptr;
+        c->n = p0;
+        for (int l = 1; l <= e.D.L; ++l) {
+            const void* next = l < e.D.L ? c->layers[l].attn_norm : (last ? c->w.final_norm : nullptr);
+            layer_step(e, c->layers[l - 1], c->kc(l), c->vc(l), 0, m, c->n, next);
+        }
+    }
+    c->n = n_prompt;
+    ensure_act(e, c->w.final_norm, m - 1, 1);
+    head(e, c->w.lm_head, m - 1, 1, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
+    int rc = fetch_results(c);
+    if (rc) return rc;
+    c->pending = c->mailbox[8 + (m - 1)];
+    c->rows = 0;
+    *first_token = c->pending;
+    return SB_OK;
+}
+
+int sb_draft_push(sb_ctx* c, int32_t token) {
+    if (!c) return SB_ERR_ARG;
+    if (!c->loaded || c->pending < 0) return SB_ERR_STATE;
+    if (token < 0 || token >= c->e.D.V) return SB_ERR_ARG;
+    if (c->rows >= SB_MAX_W) return SB_ERR_CAPACITY;
+    if (c->n + c->rows + 1 > c->e.D.max_seq) return SB_ERR_CAPACITY;
+    Exec& e = c->e;
+    SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, nullptr, token, c->rows, 1, e.W.h));
+    e.launches++;
+    c->depth[c->rows++] = 0;
+    return SB_OK;
+}
+
+int sb_draft_advance(sb_ctx* c, int32_t to_layer) {
+    if (!c) return SB_ERR_ARG;
+    if (!c->loaded || c->rows < 1) return SB_ERR_STATE;
+    if (to_layer < 1 || to_layer > c->e.D.L) return SB_ERR_ARG;
+    for (int l = 1; l <= to_layer; ++l) advance_suffix(c, l, c->w.final_norm, nullptr);
+    return cuda_ok(cudaGetLastError());
+}
+
+static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf, int32_t* token, int32_t* flag) {
+    int r = c->rows - 1;
+    ensure_act(c->e, c->w.final_norm, r, 1);
+    head(c->e, c->w.lm_head, r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
+    int rc = fetch_results(c);
+    if (rc) return rc;
+    memcpy(conf, &c->mailbox[r], sizeof(float));
+    *token = c->mailbox[8 + r];
+    *flag = c->mailbox[16 + r];
+    (void)layer;
+    return SB_OK;
+}
+
+int sb_exit_confidence(sb_ctx* c, int32_t layer, float tau_l, float threshold, float* conf, int32_t* token,
+                       int32_t* exit_flag) {
+    if (!c || !conf || !token || !exit_flag) return SB_ERR_ARG;
+    if (!c->loaded || c->rows < 1) return SB_ERR_STATE;
+    if (layer < 1 || layer > c->e.D.L || !(tau_l > 0.f) || threshold != threshold) return SB_ERR_ARG;
+    if (c->depth[c->rows - 1] != layer) return SB_ERR_STATE;
+    return probe(c, layer, tau_l, threshold, conf, token, exit_flag);
+}
+
+// alignment + unified pass + final head + acceptance + rollback
+static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, int32_t* out_tokens, int32_t* n_out,
+                       sb_stats* st, sb_round* tr) {
+    Exec& e = c->e;
+    int D = 0;
+    for (int i = 0; i < w; ++i) D = c->depth[i] > D ? c->depth[i] : D;
+    for (int l = 1; l <= D; ++l) advance_suffix(c, l, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm, st);
+    for (int l = D + 1; l <= e.D.L; ++l) {
+        run_layer(c, l, 0, w, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
+        if (st) { st->layer_steps++; st->layer_row_steps += w; st->verify_layer_steps++; }
+    }
+    ensure_act(e, c->w.final_norm, 0, w);
+    head(e, c->w.lm_head, 0, w, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
+    int d8[kMaxW];
+    for (int i = 0; i < kMaxW; ++i) d8[i] = i < w ? drafts[i] : -1;
+    launch_accept(e.st, c->token_d(), d8, w, max_emit, c->accept_d());
+    e.launches++;
+    cudaEventRecord(c->ev[2], e.st);
+    int rc = fetch_results(c);
+    if (rc) return rc;
+    int emit = c->mailbox[24], acc = c->mailbox[25];
+    for (int i = 0; i < emit; ++i) out_tokens[i] = c->mailbox[26 + i];
+    *n_out = emit;
+    if (tr) {
+        tr->w = w; tr->D = D; tr->emitted = emit; tr->accepted_drafts = acc;
+        for (int i = 0; i < kMaxW; ++i) { tr->g[i] = c->mailbox[26 + i]; tr->draft[i] = d8[i]; }
+    }
+    if (st) { st->accepted_drafts += acc; st->emitted += emit; st->rounds++; st->rows += w; st->width_hist[w]++; }
+    c->n += emit;                       // rollback: KV at positions >= n is dead and will be overwritten
+    c->pending = c->mailbox[26 + emit - 1];
+    c->rows = 0;
+    e.act_gain = nullptr;
+    return SB_OK;
+}
+
+int sb_verify(sb_ctx* c, const int32_t* drafts, int32_t w, int32_t* out_tokens, int32_t* n_out) {
+    if (!c || !drafts || !out_tokens || !n_out) return SB_ERR_ARG;
+    if (!c->loaded) return SB_ERR_STATE;
+    if (w < 1 || w > SB_MAX_W) return SB_ERR_ARG;
+    if (w != c->rows) return SB_ERR_STATE;
+    for (int i = 0; i < w; ++i)
+        if (drafts[i] < -1 || drafts[i] >= c->e.D.V) return SB_ERR_ARG;
+    return verify_rows(c, drafts, w, w, out_tokens, n_out, nullptr, nullptr);
+}
+
+static double now_us() {
+    return std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_gen, int32_t d_max, int32_t w_max,
+                const float* tau, float threshold, int32_t* out_tokens, int32_t* n_out, sb_stats* stats,
+                sb_round* rounds, int32_t max_rounds, int32_t* n_rounds) {
+    if (!c || !prompt || !tau || !out_tokens || !n_out || n_prompt < 1 || n_gen < 1) return SB_ERR_ARG;
+    if (!c->loaded) return SB_ERR_STATE;
+    if (d_max < 1 || d_max > c->e.D.L - 1 || w_max < 1 || w_max > SB_MAX_W || threshold != threshold) return SB_ERR_ARG;
+    for (int l = 0; l < d_max; ++l)
+        if (!(tau[l] > 0.f)) return SB_ERR_ARG;
+    if (n_prompt + n_gen + w_max > c->e.D.max_seq) return SB_ERR_CAPACITY;
+    if (check_tokens(c, prompt, n_prompt)) return SB_ERR_ARG;
+    sb_stats local;
+    sb_stats* st = stats ? stats : &local;
+    memset(st, 0, sizeof(*st));
+    Exec& e = c->e;
+    int64_t launches0 = e.launches;
+    sb_reset(c);
+    double t0 = now_us();
+    int first;
+    int rc = sb_prefill(c, prompt, n_prompt, &first);
+    if (rc) return rc;
+    double t1 = now_us();
+    st->us_prefill = t1 - t0;
+    int produced = 0, nr = 0;
+    out_tokens[produced++] = first;
+    st->emitted = 1;
+    while (produced < n_gen) {
+        sb_round R;
+        memset(&R, 0, sizeof(R));
+        int drafts[kMaxW];
+        for (int i = 0; i < kMaxW; ++i) { drafts[i] = -1; R.draft[i] = -1; }
+        int cur = c->pending;
+        cudaEventRecord(c->ev[0], e.st);
+        for (;;) {                              // draft phase (Section 3.3)
+            if ((rc = sb_draft_push(c, cur))) return rc;
+            int r = c->rows - 1;
+            bool exited = false;
+            for (int l = 1; l <= d_max; ++l) {
+                advance_suffix(c, l, c->w.final_norm, st);
+                float conf; int tok, flag;
+                if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag))) return rc;
+                st->probes++;
+                R.conf[r] = conf;
+                if (flag) { drafts[r] = tok; R.exit_layer[r] = l; exited = true; break; }
+            }
+            st->exit_hist[exited ? R.exit_layer[r] : 0]++;
+            if (!exited) break;                 // difficult token: the depth bound ends the round
+            if (c->rows == w_max) break;        // long shallow chain: the width bound ends the round
+            cur = drafts[r];
+        }
+        cudaEventRecord(c->ev[1], e.st);
+        int w = c->rows, emit = 0;
+        if ((rc = verify_rows(c, drafts, w, n_gen - produced, out_tokens + produced, &emit, st, &R))) return rc;
+        produced += emit;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]) == cudaSuccess) st->us_draft += 1e3 * ms;
+        if (cudaEventElapsedTime(&ms, c->ev[1], c->ev[2]) == cudaSuccess) st->us_verify += 1e3 * ms;
+        if (rounds && nr < max_rounds) rounds[nr] = R;
+        ++nr;
+    }
+    st->us_decode = now_us() - t1;
+    st->kernel_launches = e.launches - launches0;
+    *n_out = produced;
+    if (n_rounds) *n_rounds = nr;
+    return SB_OK;
+}
+
+int sb_generate_ar(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_gen, int32_t* out_tokens, int32_t* n_out,
+                   sb_stats* stats) {
+    if (!c || !prompt || !out_tokens || !n_out || n_prompt < 1 || n_gen < 1) return SB_ERR_ARG;
+    if (!c->loaded) return SB_ERR_STATE;
+    if (n_prompt + n_gen > c->e.D.max_seq) return SB_ERR_CAPACITY;
+    if (check_tokens(c, prompt, n_prompt)) return SB_ERR_ARG;
+    sb_stats local;
+    sb_stats* st = stats ? stats : &local;
+    memset(st, 0, sizeof(*st));
+    Exec& e = c->e;
+    int64_t launches0 = e.launches;
+    sb_reset(c);
+    double t0 = now_us();
+    int first;
+    int rc = sb_prefill(c, prompt, n_prompt, &first);
+    if (rc) return rc;
+    double t1 = now_us();
+    st->us_prefill = t1 - t0;
+    // token log on the device: toks[n_prompt + i] = i-th generated token.  Each step embeds the
+    // previous token straight from the log, so the host never has to look at a token in between.
+    int* log = e.W.toks + n_prompt;
+    if (cudaMemcpyAsync(log, &first, sizeof(int), cudaMemcpyHostToDevice, e.st) != cudaSuccess) return SB_ERR_CUDA;
+    for (int i = 1; i < n_gen; ++i) {
+        SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, log + i - 1, 0, 0, 1, e.W.h));
+        e.launches++;
+        e.act_gain = nullptr;
+        for (int l = 1; l <= e.D.L; ++l)
+            layer_step(e, c->layers[l - 1], c->kc(l), c->vc(l), 0, 1, c->n, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
+        head(e, c->w.lm_head, 0, 1, 1.f, 2.f, c->conf_d(), log + i, c->flag_d(), nullptr);
+        c->n += 1;
+        st->layer_steps += e.D.L; st->layer_row_steps += e.D.L; st->rounds++; st->rows++;
+    }
+    if (cudaMemcpyAsync(out_tokens, log, sizeof(int) * n_gen, cudaMemcpyDeviceToHost, e.st) != cudaSuccess)
+        return SB_ERR_CUDA;
+    rc = fetch_results(c);
+    if (rc) return rc;
+    c->pending = out_tokens[n_gen - 1];
+    st->emitted = n_gen;
+    st->us_decode = now_us() - t1;
+    st->kernel_launches = e.launches - launches0;
+    *n_out = n_gen;
+    return SB_OK;
+}
+
+int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const void* final_norm, const void* lm_head,
+                         float tau_l, float* conf, int32_t* token, float* logits_dbg, void* scratch, size_t scratch_bytes,
+                         void* stream) {
+    Dims D;
+    if (!make_dims(cfg, &D) || !h || !final_norm || !lm_head || !conf || !token || !scratch) return SB_ERR_ARG;
+    if (m < 1 || m > SB_MAX_W || !(tau_l > 0.f)) return SB_ERR_ARG;
+    if (((uintptr_t)scratch & 1023) || ((uintptr_t)lm_head & 15)) return SB_ERR_ARG;
+    if (scratch_bytes < carve(D, nullptr, false, nullptr)) return SB_ERR_CAPACITY;
+    Exec e;
+    e.D = D;
+    e.st = (cudaStream_t)stream;
+    carve(D, (char*)scratch, false, &e.W);
+    e.gemm = pick_gemm(D.f32);
+    TcPlanCache plans;
+    e.plans = &plans;
+    cudaMemsetAsync(e.W.ticket, 0, 64, e.st);
+    cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    cudaMemcpyAsync(e.W.h, h, sizeof(float) * m * D.d, cudaMemcpyDeviceToDevice, e.st);
+    ensure_act(e, final_norm, 0, m);
+    head(e, lm_head, 0, m, tau_l, 2.f, reinterpret_cast<float*>(e.W.res), e.W.res + 8, e.W.res + 16, logits_dbg);
+    cudaMemcpyAsync(conf, e.W.res, sizeof(float) * m, cudaMemcpyDeviceToDevice, e.st);
+    cudaMemcpyAsync(token, e.W.res + 8, sizeof(int) * m, cudaMemcpyDeviceToDevice, e.st);
+    return cuda_ok(cudaGetLastError());
+}
+
+int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_t m, void* k_cache, void* v_cache,
+               const int32_t* page_table, int32_t first_pos, void* scratch, size_t scratch_bytes, void* stream) {
+    Dims D;
+    if (!make_dims(cfg, &D) || !lw || !h || !k_cache || !v_cache || !page_table || !scratch) return SB_ERR_ARG;
+    if (m < 1 || m > SB_MAX_W || first_pos < 0) return SB_ERR_ARG;
+    if (first_pos + m > D.max_seq) return SB_ERR_CAPACITY;
+    if ((uintptr_t)scratch & 1023) return SB_ERR_ARG;
+    if (scratch_bytes < carve(D, nullptr, false, nullptr)) return SB_ERR_CAPACITY;
+    const void* ps[9] = {lw->attn_norm, lw->wq, lw->wk, lw->wv, lw->wo, lw->mlp_norm, lw->w_gate, lw->w_up, lw->w_down};
+    for (const void* p : ps)
+        if (!p || ((uintptr_t)p & 15)) return SB_ERR_ARG;
+    Exec e;
+    e.D = D;
+    e.st = (cudaStream_t)stream;
+    carve(D, (char*)scratch, false, &e.W);
+    e.W.page_table = const_cast<int*>(page_table);
+    e.W.h = reinterpret_cast<float*>(h);   // rows 0..m-1 of the caller's buffer are the hidden cache
+    e.gemm = pick_gemm(D.f32);
+    TcPlanCache plans;
+    e.plans = &plans;
+    cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    layer_step(e, *lw, k_cache, v_cache, 0, m, first_pos, nullptr);
+    return cuda_ok(cudaGetLastError());
+}
+
+int sb_tau_schedule(float alpha, int32_t L, float* out) {
+    if (!out || L < 1 || !(alpha >= 0.f)) return SB_ERR_ARG;
+    for (int l = 1; l <= L; ++l) out[l - 1] = 1.f + alpha * (1.f - (float)l / (float)L);
+    return SB_OK;
+}
+
+double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max) {
+    double num = (double)L * a * (1.0 - std::pow(a, (double)w));
+    return num / ((1.0 - a) * ((double)w * d_max + L - d_max));
+}
+
+const char* sb_strerror(int s) {
+    switch (s) {
+        case SB_OK: return "ok";
+        case SB_ERR_ARG: return "bad argument";
+        case SB_ERR_STATE: return "call out of order";
+        case SB_ERR_CAPACITY: return "capacity exceeded";
+        case SB_ERR_CUDA: return "CUDA error";
+        case SB_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case SB_ERR_UNSUPPORTED: return "unsupported configuration";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,26 @@
+// Interface of the TMA + tcgen05 weight-streaming kernels (bf16 models).
+#pragma once
+#include <cuda_runtime.h>
+
+#include <map>
+#include <vector>
+
+#include "sb_internal.cuh"
+
+namespace sb {
+
+constexpr int kMaxSplit = 8;   // most split-K partials a GEMM may leave for its consumer
+
+struct TcPlan;                 // tensor maps + work decomposition of one GEMM call shape
+struct TcPlanCache {
+    std::map<std::vector<uint64_t>, TcPlan*> plans;
+    void clear();
+    ~TcPlanCache() { clear(); }
+};
+
+bool tc_available();
+// returns the number of split-K partials written to a.out
+int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status);
+void launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status);
+
+}  // namespace sb

@@ -1,0 +1,148 @@
+// Internal declarations shared by the translation units of the SpecBound sm_100a library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/specbound.h"
+
+namespace sb {
+
+constexpr int kMaxW = SB_MAX_W;
+constexpr int kHeadMaxCtas = 1024;   // upper bound of CTAs of one exit-confidence launch
+
+// ---------------------------------------------------------------------------------------------
+// Activation operand of the skinny GEMMs.
+//   fp32 models : float [8][K]                      (row i of the round in row i)
+//   bf16 models : bf16  [16][K], row i = high part, row 8+i = low part of the fp32 value
+//                 (x = hi + lo keeps 16 mantissa bits, so the bf16 tensor-core product of a
+//                  weight with an activation is as accurate as an fp32 one)
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct Act;
+template <> struct Act<float> {
+    using type = float;
+    static constexpr int rows = 8;
+    __device__ static void store(float* a, int row, int k, int K, float v) { a[(size_t)row * K + k] = v; }
+    __device__ static float load(const float* a, int row, int k, int K) { return a[(size_t)row * K + k]; }
+};
+template <> struct Act<__nv_bfloat16> {
+    using type = __nv_bfloat16;
+    static constexpr int rows = 16;
+    __device__ static void store(__nv_bfloat16* a, int row, int k, int K, float v) {
+        __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        a[(size_t)row * K + k] = hi;
+        a[(size_t)(row + 8) * K + k] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+    __device__ static float load(const __nv_bfloat16* a, int row, int k, int K) {
+        return __bfloat162float(a[(size_t)row * K + k]) + __bfloat162float(a[(size_t)(row + 8) * K + k]);
+    }
+};
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Partial result of the temperature-scaled softmax of Eq. 2 over a slice of the vocabulary:
+// m = largest raw logit, idx = its (lowest) index, s = sum exp((z - m) / T).
+struct SoftTriple {
+    float m;
+    int idx;
+    float s;
+};
+__device__ __forceinline__ SoftTriple soft_empty() { return SoftTriple{-INFINITY, 0x7fffffff, 0.f}; }
+__device__ __forceinline__ SoftTriple soft_merge(SoftTriple a, SoftTriple b, float inv_t) {
+    // larger logit wins; equal logits: lower index wins
+    bool a_wins = (a.m > b.m) || (a.m == b.m && a.idx < b.idx);
+    SoftTriple hi = a_wins ? a : b, lo = a_wins ? b : a;
+    float s = hi.s;
+    if (lo.s > 0.f) s += lo.s * expf((lo.m - hi.m) * inv_t);
+    return SoftTriple{hi.m, hi.idx, s};
+}
+__device__ __forceinline__ void soft_push(SoftTriple& t, float z, int idx, float inv_t) {
+    if (z > t.m) {   // strictly larger: a later equal logit never replaces an earlier index
+        t.s = t.s * expf((t.m - z) * inv_t) + 1.f;   // exp(-inf) = 0 handles the first element
+        t.m = z;
+        t.idx = idx;
+    } else {
+        t.s += expf((z - t.m) * inv_t);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Launch arguments
+// ---------------------------------------------------------------------------------------------
+struct GemmArgs {          // out[s][row][n] = sum_k act[row][k] * W[n][k]   for rows r0 .. r0+m-1
+    const void* W[3];      // up to three matrices sharing K and the activation operand
+    int n_end[3];          // cumulative row counts: matrix j owns output columns [n_end[j-1], n_end[j])
+    int n_mats;
+    int K;
+    const void* act;       // Act<T> layout
+    float* out;            // [n_split][8][n_total]
+    int n_total;
+    int r0, m;
+};
+
+struct HeadArgs {          // exit-confidence / final-head kernel
+    const void* W;         // lm_head [V, K]
+    int V, K;
+    const void* act;       // Act<T> layout: final-RMSNorm of the hidden rows
+    int r0, m;
+    float inv_tau;
+    float threshold;
+    float* conf;           // [8]   indexed by row
+    int* token;            // [8]
+    int* exit_flag;        // [8]   conf >= threshold
+    float* logits_dbg;     // nullable [m][V] (row r0 first)
+    SoftTriple* part;      // scratch [kHeadMaxCtas][8]
+    unsigned int* ticket;  // scratch counter, zero between launches (the kernel re-zeroes it)
+};
+
+struct AttnArgs {
+    const float* q;        // [8][H*hd]
+    const void* k_cache;   // [n_pages][page][kvd]
+    const void* v_cache;
+    const int* page_table;
+    float* part;           // [n_chunks][8][H][hd+2]
+    void* act_out;         // Act<T> [.][H*hd]
+    int H, Hkv, hd, page, page_shift;
+    int pos0;              // position of row 0
+    int r0, m;
+    int chunk;             // tokens per split (fixed per context)
+};
+
+struct RopeArgs {
+    const float* qkv;      // partials [n_split][8][qd + 2 kvd]
+    int n_split;
+    float* q;              // [8][qd]
+    void* k_cache;
+    void* v_cache;
+    const int* page_table;
+    int H, Hkv, hd, page, page_shift;
+    int pos0, r0, m;
+    float rope_base;
+};
+
+// ---- launchers (kernels_small.cu) ----
+template <typename T> void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, int tok_scalar,
+                                        int row0, int m, float* h);
+template <typename T> void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d,
+                                             const T* gain, float eps, void* act, int r0, int m);
+template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a);
+template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
+template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
+void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result);
+void launch_init_pages(cudaStream_t st, int* page_table, int n_pages);
+
+// ---- launchers (gemm_simt.cu) ----
+template <typename T> void launch_gemm_simt(cudaStream_t st, const GemmArgs& a);
+template <typename T> void launch_head_simt(cudaStream_t st, const HeadArgs& a, int n_ctas);
+
+}  // namespace sb
