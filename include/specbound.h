@@ -70,9 +70,15 @@ typedef struct {
     int64_t exit_hist[SB_MAX_LAYERS + 1]; /* [l] = rows that exited at layer l; [0] = failed by d_max */
     int64_t width_hist[SB_MAX_W + 1];     /* [w] = rounds verified with w rows                       */
     double us_prefill, us_decode;         /* host wall time around the two phases                    */
-    double us_draft, us_verify;           /* device time (CUDA events) of draft phases / unified passes */
-    int64_t verify_layer_steps;           /* layer passes inside us_verify                           */
+    double us_decode_dev;                 /* device time of the decode phase (CUDA events on the stream) */
+    double us_draft, us_verify;           /* device time of draft phases / of verification (alignment,
+                                             unified pass, final head, acceptance)                    */
+    double us_unified;                    /* device time of the unified passes alone (layers D+1..L) */
+    int64_t unified_layer_steps;          /* layer passes inside us_unified                          */
+    int64_t unified_kv_positions;         /* sum over those passes of the KV length they attended over */
+    double us_probe_kernels;              /* device time of the exit-confidence kernels of the draft phase */
     int64_t kernel_launches;              /* kernels launched by the call                            */
+    int64_t h2d_bytes, d2h_bytes;         /* bytes copied host->device / device->host by the call    */
 } sb_stats;
 
 typedef struct { /* trace of one speculation round, filled by sb_generate when asked to */

@@ -206,7 +206,8 @@ struct sb_ctx {
     int* mailbox = nullptr;   // pinned host
     int n = 0, pending = -1, rows = 0;
     int depth[SB_MAX_W];
-    cudaEvent_t ev[3];
+    cudaEvent_t ev[9];   // 0 draft start, 1 verify start, 2 round end, 3/4 unified pass, 5/6 probe kernel, 7/8 decode phase
+    int64_t h2d = 0, d2h = 0;
     TcPlanCache plans;
 
     void* kc(int layer) const {
@@ -234,6 +235,7 @@ static int fetch_results(sb_ctx* c) {
         return SB_ERR_CUDA;
     if (cudaStreamSynchronize(c->e.st) != cudaSuccess) return SB_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return SB_ERR_CUDA;
+    c->d2h += sizeof(int) * 41;
     if (c->mailbox[48] != 0) return SB_ERR_DEVICE_TIMEOUT;
     return SB_OK;
 }
@@ -382,6 +384,7 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
     Exec& e = c->e;
     if (cudaMemcpyAsync(e.W.toks, prompt, sizeof(int) * n_prompt, cudaMemcpyHostToDevice, e.st) != cudaSuccess)
         return SB_ERR_CUDA;
+    c->h2d += sizeof(int) * n_prompt;
     int m = 0;
     for (int p0 = 0; p0 < n_prompt; p0 += m) {
         m = n_prompt - p0 < kMaxW ? n_prompt - p0 : kMaxW;
@@ -427,12 +430,19 @@ int sb_draft_advance(sb_ctx* c, int32_t to_layer) {
     return cuda_ok(cudaGetLastError());
 }
 
-static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf, int32_t* token, int32_t* flag) {
+static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf, int32_t* token, int32_t* flag,
+                 sb_stats* st = nullptr) {
     int r = c->rows - 1;
     ensure_act(c->e, c->w.final_norm, r, 1);
+    cudaEventRecord(c->ev[5], c->e.st);
     head(c->e, c->w.lm_head, r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
+    cudaEventRecord(c->ev[6], c->e.st);
     int rc = fetch_results(c);
     if (rc) return rc;
+    if (st) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev[5], c->ev[6]) == cudaSuccess) st->us_probe_kernels += 1e3 * ms;
+    }
     memcpy(conf, &c->mailbox[r], sizeof(float));
     *token = c->mailbox[8 + r];
     *flag = c->mailbox[16 + r];
@@ -456,10 +466,12 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     int D = 0;
     for (int i = 0; i < w; ++i) D = c->depth[i] > D ? c->depth[i] : D;
     for (int l = 1; l <= D; ++l) advance_suffix(c, l, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm, st);
+    cudaEventRecord(c->ev[3], e.st);
     for (int l = D + 1; l <= e.D.L; ++l) {
         run_layer(c, l, 0, w, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
-        if (st) { st->layer_steps++; st->layer_row_steps += w; st->verify_layer_steps++; }
+        if (st) { st->layer_steps++; st->layer_row_steps += w; st->unified_layer_steps++; st->unified_kv_positions += c->n + w; }
     }
+    cudaEventRecord(c->ev[4], e.st);
     ensure_act(e, c->w.final_norm, 0, w);
     head(e, c->w.lm_head, 0, w, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
     int d8[kMaxW];
@@ -469,6 +481,10 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     cudaEventRecord(c->ev[2], e.st);
     int rc = fetch_results(c);
     if (rc) return rc;
+    if (st) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]) == cudaSuccess) st->us_unified += 1e3 * ms;
+    }
     int emit = c->mailbox[24], acc = c->mailbox[25];
     for (int i = 0; i < emit; ++i) out_tokens[i] = c->mailbox[26 + i];
     *n_out = emit;
@@ -512,7 +528,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
     sb_stats* st = stats ? stats : &local;
     memset(st, 0, sizeof(*st));
     Exec& e = c->e;
-    int64_t launches0 = e.launches;
+    int64_t launches0 = e.launches, h2d0 = c->h2d, d2h0 = c->d2h;
     sb_reset(c);
     double t0 = now_us();
     int first;
@@ -520,6 +536,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
     if (rc) return rc;
     double t1 = now_us();
     st->us_prefill = t1 - t0;
+    cudaEventRecord(c->ev[7], e.st);
     int produced = 0, nr = 0;
     out_tokens[produced++] = first;
     st->emitted = 1;
@@ -537,7 +554,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
             for (int l = 1; l <= d_max; ++l) {
                 advance_suffix(c, l, c->w.final_norm, st);
                 float conf; int tok, flag;
-                if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag))) return rc;
+                if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag, st))) return rc;
                 st->probes++;
                 R.conf[r] = conf;
                 if (flag) { drafts[r] = tok; R.exit_layer[r] = l; exited = true; break; }
@@ -557,8 +574,17 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
         if (rounds && nr < max_rounds) rounds[nr] = R;
         ++nr;
     }
+    cudaEventRecord(c->ev[8], e.st);
+    cudaEventSynchronize(c->ev[8]);
     st->us_decode = now_us() - t1;
+    {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev[7], c->ev[8]) == cudaSuccess) st->us_decode_dev = 1e3 * ms;
+    }
+    c->d2h += sizeof(int) * produced;   // the caller's token buffer is host memory written from the mailbox
     st->kernel_launches = e.launches - launches0;
+    st->h2d_bytes = c->h2d - h2d0;
+    st->d2h_bytes = c->d2h - d2h0;
     *n_out = produced;
     if (n_rounds) *n_rounds = nr;
     return SB_OK;
@@ -574,7 +600,7 @@ int sb_generate_ar(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n
     sb_stats* st = stats ? stats : &local;
     memset(st, 0, sizeof(*st));
     Exec& e = c->e;
-    int64_t launches0 = e.launches;
+    int64_t launches0 = e.launches, h2d0 = c->h2d, d2h0 = c->d2h;
     sb_reset(c);
     double t0 = now_us();
     int first;
@@ -582,6 +608,7 @@ int sb_generate_ar(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n
     if (rc) return rc;
     double t1 = now_us();
     st->us_prefill = t1 - t0;
+    cudaEventRecord(c->ev[7], e.st);
     // token log on the device: toks[n_prompt + i] = i-th generated token.  Each step embeds the
     // previous token straight from the log, so the host never has to look at a token in between.
     int* log = e.W.toks + n_prompt;
@@ -596,13 +623,22 @@ int sb_generate_ar(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n
         c->n += 1;
         st->layer_steps += e.D.L; st->layer_row_steps += e.D.L; st->rounds++; st->rows++;
     }
+    cudaEventRecord(c->ev[8], e.st);
     if (cudaMemcpyAsync(out_tokens, log, sizeof(int) * n_gen, cudaMemcpyDeviceToHost, e.st) != cudaSuccess)
         return SB_ERR_CUDA;
+    c->d2h += sizeof(int) * n_gen;
+    c->h2d += sizeof(int);
     rc = fetch_results(c);
     if (rc) return rc;
     c->pending = out_tokens[n_gen - 1];
     st->emitted = n_gen;
     st->us_decode = now_us() - t1;
+    {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev[7], c->ev[8]) == cudaSuccess) st->us_decode_dev = 1e3 * ms;
+    }
+    st->h2d_bytes = c->h2d - h2d0;
+    st->d2h_bytes = c->d2h - d2h0;
     st->kernel_launches = e.launches - launches0;
     *n_out = n_gen;
     return SB_OK;
