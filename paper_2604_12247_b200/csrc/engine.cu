@@ -122,6 +122,7 @@ struct Exec {   // everything a launch sequence needs
     const void* act_gain = nullptr;
     int act_r0 = 0, act_m = 0;
     TcPlanCache* plans = nullptr;
+    int err = 0;   // sticky host-side error of a launch sequence (a TMA descriptor could not be built)
 };
 
 #define SB_T(E, call)                          \
@@ -145,7 +146,11 @@ static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, 
     for (int j = n_mats; j < 3; ++j) { a.W[j] = nullptr; a.n_end[j] = 0x7fffffff; }
     a.n_mats = n_mats; a.K = K; a.act = act; a.out = out; a.n_total = tot; a.r0 = r0; a.m = m;
     e.launches++;
-    if (e.gemm == 1 && !e.D.f32) return launch_gemm_tc(e.st, a, e.plans, e.W.status);
+    if (e.gemm == 1 && !e.D.f32) {
+        int s = launch_gemm_tc(e.st, a, e.plans, e.W.status);
+        if (s < 1) { e.err = SB_ERR_CUDA; return 1; }
+        return s;
+    }
     SB_T(e, launch_gemm_simt<T>(e.st, a));
     return 1;
 }
@@ -189,7 +194,10 @@ static void head(Exec& e, const void* lm_head, int r0, int m, float tau, float t
     HeadArgs a{lm_head, e.D.V, e.D.d, e.W.act_a, r0, m, 1.f / tau, threshold, conf, token, flag, logits_dbg,
                e.W.head_part, e.W.ticket};
     e.launches++;
-    if (e.gemm == 1 && !e.D.f32) { launch_head_tc(e.st, a, e.plans, e.W.status); return; }
+    if (e.gemm == 1 && !e.D.f32) {
+        if (!launch_head_tc(e.st, a, e.plans, e.W.status)) e.err = SB_ERR_CUDA;
+        return;
+    }
     SB_T(e, launch_head_simt<T>(e.st, a, 148 * 4));
 }
 
@@ -235,6 +243,7 @@ static int fetch_results(sb_ctx* c) {
         return SB_ERR_CUDA;
     if (cudaStreamSynchronize(c->e.st) != cudaSuccess) return SB_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return SB_ERR_CUDA;
+    if (c->e.err) return c->e.err;
     c->d2h += sizeof(int) * 41;
     if (c->mailbox[48] != 0) return SB_ERR_DEVICE_TIMEOUT;
     return SB_OK;
@@ -666,6 +675,7 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     head(e, lm_head, 0, m, tau_l, 2.f, reinterpret_cast<float*>(e.W.res), e.W.res + 8, e.W.res + 16, logits_dbg);
     cudaMemcpyAsync(conf, e.W.res, sizeof(float) * m, cudaMemcpyDeviceToDevice, e.st);
     cudaMemcpyAsync(token, e.W.res + 8, sizeof(int) * m, cudaMemcpyDeviceToDevice, e.st);
+    if (e.err) return e.err;
     return cuda_ok(cudaGetLastError());
 }
 
@@ -691,6 +701,7 @@ int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_
     e.plans = &plans;
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
     layer_step(e, *lw, k_cache, v_cache, 0, m, first_pos, nullptr);
+    if (e.err) return e.err;
     return cuda_ok(cudaGetLastError());
 }
 

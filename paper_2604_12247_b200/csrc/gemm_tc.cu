@@ -1,8 +1,492 @@
+// TMA + tcgen05 weight-streaming kernels for bf16 models (sm_100a).
+//
+//   out[row][n] = sum_k act[row][k] * W[n][k]        rows <= 8, W streamed from HBM exactly once
+//
+// The weight tile is the MMA's M operand (128 weight rows x 64 k per pipeline stage, staged by
+// TMA with the 128-byte swizzle); the activations are the N operand: 16 columns = the high and
+// the low bf16 halves of the 8 fp32 activation rows, so one kind::f16 MMA (M=128, N=16, K=16)
+// yields W.hi and W.lo side by side in TMEM and their sum is as accurate as an fp32 product.
+//
+// One persistent CTA per SM: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2-5 =
+// epilogue (tcgen05.ld, then either split-K partial stores or, for the LM head, the online
+// temperature-scaled softmax max/argmax of Eq. 2).  Work items are (row slab, k split) pairs
+// chosen on the host so that every CTA streams the same number of bytes whatever the number of
+// rows: the result of a row never depends on its companions.  Every wait is bounded: on expiry
+// the kernel raises a status word, drains and returns.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstring>
+
 #include "gemm_tc.cuh"
+
 namespace sb {
-struct TcPlan {};
-void TcPlanCache::clear() { for (auto& kv : plans) delete kv.second; plans.clear(); }
-bool tc_available() { return false; }
-int launch_gemm_tc(cudaStream_t, const GemmArgs&, TcPlanCache*, unsigned int*) { return 0; }
-void launch_head_tc(cudaStream_t, const HeadArgs&, TcPlanCache*, unsigned int*) {}
+
+constexpr int kStages = 6;
+constexpr int kBK = 64;                       // k elements per stage (128 bytes: one swizzle row)
+constexpr int kTileRows = 128;                // MMA M
+constexpr int kStageA = kTileRows * kBK * 2;  // 16 KB
+constexpr int kStageB = 16 * kBK * 2;         // 2 KB
+constexpr int kTcThreads = 192;
+constexpr int kSmemBytes = kStages * (kStageA + kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
+
+struct alignas(64) TcParams {
+    CUtensorMap tmA[3];
+    CUtensorMap tmB;
+    int n_mats;
+    int chunk_end[3];   // cumulative slab counts
+    int n_rows[3];      // rows of each matrix
+    int n_off[3];       // first output column of each matrix
+    int n_chunks, R, S, KB, n_items;
+    float* out;
+    int n_total;
+    int r0, m;
+    // LM-head mode
+    float inv_tau, threshold;
+    float* conf;
+    int* token;
+    int* exit_flag;
+    float* logits_dbg;
+    SoftTriple* part;
+    unsigned int* ticket;
+    unsigned int* status;
+};
+
+struct TcPlan {
+    TcParams p;
+    int grid;
+};
+
+void TcPlanCache::clear() {
+    for (auto& kv : plans) delete kv.second;
+    plans.clear();
 }
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag + status word) if the budget runs out
+// or another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
+                                          unsigned int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicExch(status, code);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(tm), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], "
+        "[%4], %5;" ::"r"(dst),
+        "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;              // leading byte offset (unused for swizzled K-major): 16 bytes
+    d |= (uint64_t)(1024 >> 4) << 32;    // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;              // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;              // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor: D = f32, A = B = bf16, both K-major, N = 16, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+
+struct ItemInfo {
+    int mat, row0, kb0, kb1;
+};
+__device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
+    int chunk = item % p.n_chunks, s = item / p.n_chunks;
+    int j = 0, base = 0;
+    while (j < p.n_mats - 1 && chunk >= p.chunk_end[j]) base = p.chunk_end[j++];
+    ItemInfo it;
+    it.mat = j;
+    it.row0 = (chunk - base) * p.R;
+    it.kb0 = (int)((long long)s * p.KB / p.S);
+    it.kb1 = (int)((long long)(s + 1) * p.KB / p.S);
+    return it;
+}
+
+template <bool kHead>
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile int abort_s;
+    __shared__ SoftTriple cta_part[4][kMaxW];
+    __shared__ bool is_last_s;
+
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
+    const uint32_t smA = tiles, smB = tiles + kStages * kStageA;
+    const uint32_t bars = smB + kStages * kStageB;             // 8-byte mbarriers
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * kStages + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * kStages + 2 + b); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // TMEM: 32 columns = two 16-column accumulators
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(32));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t stage_bytes = (uint32_t)p.R * (kBK * 2) + kStageB;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            for (int j = 0; j < p.n_mats; ++j) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA[j]) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
+            const uint64_t pol = policy_evict_first();
+            int stage = 0, phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+                ItemInfo it = decode_item(p, item);
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, &abort_s, p.status, 1u))) break;
+                    mbar_expect_tx(full_bar(stage), stage_bytes);
+                    tma_load_2d_hint(smA + stage * kStageA, &p.tmA[it.mat], kb * kBK, it.row0, full_bar(stage), pol);
+                    tma_load_2d(smB + stage * kStageB, &p.tmB, kb * kBK, 0, full_bar(stage));
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            int stage = 0, phase = 0, n_local = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++n_local) {
+                ItemInfo it = decode_item(p, item);
+                int buf = n_local & 1;
+                uint32_t use = (uint32_t)(n_local >> 1);   // how often this accumulator was used before
+                if (!(ok = mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, &abort_s, p.status, 2u))) break;
+                tc_fence_after();
+                uint32_t d_tmem = tmem_base + (uint32_t)buf * 16u;
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!(ok = mbar_wait(full_bar(stage), phase, &abort_s, p.status, 3u))) break;
+                    tc_fence_after();
+                    uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageB);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)   // +32 bytes per 16-element k step inside the swizzle row
+                        tc_mma(d_tmem, da + 2u * k, db + 2u * k, kIdesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
+                    tc_commit(empty_bar(stage));          // frees the stage once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+                if (ok) tc_commit(tfull_bar(buf));        // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (128 threads) ------------------------------
+        const int q = warp & 3;                            // TMEM lane quadrant this warp may read
+        const int row_in_tile = q * 32 + lane;
+        SoftTriple tr[kMaxW];
+        if (kHead) {
+#pragma unroll
+            for (int i = 0; i < kMaxW; ++i) tr[i] = soft_empty();
+        }
+        int n_local = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++n_local) {
+            ItemInfo it = decode_item(p, item);
+            int buf = n_local & 1;
+            uint32_t use = (uint32_t)(n_local >> 1);
+            ok = mbar_wait(tfull_bar(buf), use & 1u, &abort_s, p.status, 4u);
+            ok = __all_sync(0xffffffffu, ok);              // the TMEM load below needs the whole warp
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t v[16];
+            tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 16u, v);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator may be overwritten
+            int n = it.row0 + row_in_tile;
+            if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
+                int s = item / p.n_chunks;
+#pragma unroll
+                for (int i = 0; i < kMaxW; ++i) {
+                    if (i >= p.r0 && i < p.r0 + p.m) {
+                        float z = __uint_as_float(v[i]) + __uint_as_float(v[i + 8]);
+                        if (kHead) {
+                            soft_push(tr[i], z, n, p.inv_tau);
+                            if (p.logits_dbg) p.logits_dbg[(size_t)(i - p.r0) * p.n_total + n] = z;
+                        } else {
+                            p.out[((size_t)s * kMaxW + i) * p.n_total + p.n_off[it.mat] + n] = z;
+                        }
+                    }
+                }
+            }
+        }
+        if (kHead) {
+            // lanes -> warp: butterfly merge (both partners compute the same merged triple)
+#pragma unroll
+            for (int i = 0; i < kMaxW; ++i) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    SoftTriple other;
+                    other.m = __shfl_xor_sync(0xffffffffu, tr[i].m, o);
+                    other.idx = __shfl_xor_sync(0xffffffffu, tr[i].idx, o);
+                    other.s = __shfl_xor_sync(0xffffffffu, tr[i].s, o);
+                    tr[i] = soft_merge(tr[i], other, p.inv_tau);
+                }
+                if (lane == 0) cta_part[q][i] = tr[i];
+            }
+        }
+    }
+
+    if (abort_s) {   // a wait expired: give copies and MMAs still in flight time to land before leaving
+        unsigned long long t0 = clock64();
+        while (clock64() - t0 < 4000000ull) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32));
+    }
+    if (!kHead) return;
+
+    // CTA triples -> scratch; the last CTA to arrive merges all CTAs in index order (wait-free)
+    if (threadIdx.x < kMaxW) {
+        int i = threadIdx.x;
+        SoftTriple t = cta_part[0][i];
+        for (int w = 1; w < 4; ++w) t = soft_merge(t, cta_part[w][i], p.inv_tau);
+        p.part[(size_t)blockIdx.x * kMaxW + i] = t;
+        __threadfence();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned int prev = atomicAdd(p.ticket, 1u);
+        is_last_s = (prev == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last_s) return;
+    __threadfence();
+    if (threadIdx.x < kMaxW) {
+        int i = threadIdx.x;
+        if (i >= p.r0 && i < p.r0 + p.m) {
+            SoftTriple t = soft_empty();
+            for (unsigned int c = 0; c < gridDim.x; ++c) {
+                const volatile SoftTriple* src = p.part + (size_t)c * kMaxW + i;
+                SoftTriple qv{src->m, src->idx, src->s};
+                t = soft_merge(t, qv, p.inv_tau);
+            }
+            float conf = 1.f / t.s;
+            p.conf[i] = conf;
+            p.token[i] = t.idx;
+            p.exit_flag[i] = conf >= p.threshold ? 1 : 0;
+        }
+    }
+    if (threadIdx.x == 0) *p.ticket = 0u;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side: tensor maps and work decomposition
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+bool tc_available() { return true; }
+
+static bool make_map(CUtensorMap* tm, const void* base, int rows, int K, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    }
+    return n;
+}
+
+// Slab height R (multiple of 8 in [64,128]) and split count S that minimise what the busiest
+// CTA streams.  Depends on the shape only, never on the number of rows.
+static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out) {
+    double best = 1e300;
+    int bR = 128, bS = 1;
+    for (int S = 1; S <= max_split && S <= KB; ++S)
+        for (int R = 128; R >= 64; R -= 8) {
+            long long chunks = 0;
+            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + R - 1) / R;
+            long long items = chunks * S;
+            long long per = (items + G - 1) / G;
+            double cost = (double)per * R * ((KB + S - 1) / S) * (1.0 + 0.004 * S);   // mild preference for few splits
+            if (cost < best - 1e-9) { best = cost; bR = R; bS = S; }
+        }
+    *R_out = bR;
+    *S_out = bS;
+}
+
+static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_end, int n_mats, int K, const void* act,
+                        bool head) {
+    std::vector<uint64_t> key;
+    for (int j = 0; j < n_mats; ++j) { key.push_back((uint64_t)(uintptr_t)W[j]); key.push_back((uint64_t)n_end[j]); }
+    key.push_back((uint64_t)K);
+    key.push_back((uint64_t)(uintptr_t)act);
+    key.push_back(head ? 1 : 0);
+    auto it = cache->plans.find(key);
+    if (it != cache->plans.end()) return it->second;
+    TcPlan* pl = new TcPlan();
+    memset(&pl->p, 0, sizeof(pl->p));
+    TcParams& p = pl->p;
+    int G = sm_count();
+    p.n_mats = n_mats;
+    p.KB = (K + kBK - 1) / kBK;
+    int prev = 0;
+    for (int j = 0; j < n_mats; ++j) { p.n_rows[j] = n_end[j] - prev; p.n_off[j] = prev; prev = n_end[j]; }
+    choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
+    int chunks = 0;
+    for (int j = 0; j < 3; ++j) {
+        if (j < n_mats) chunks += (p.n_rows[j] + p.R - 1) / p.R;
+        p.chunk_end[j] = chunks;
+    }
+    p.n_chunks = chunks;
+    p.n_items = chunks * p.S;
+    pl->grid = p.n_items < G ? p.n_items : G;
+    bool ok = make_map(&p.tmB, act, 16, K, 16);
+    for (int j = 0; j < n_mats && ok; ++j) ok = make_map(&p.tmA[j], W[j], p.n_rows[j], K, p.R);
+    if (!ok) { delete pl; return nullptr; }
+    cache->plans[key] = pl;
+    return pl;
+}
+
+static bool g_attr_set[2] = {false, false};
+template <bool kHead> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
+    if (!g_attr_set[kHead]) {
+        cudaFuncSetAttribute(k_tc<kHead>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        g_attr_set[kHead] = true;
+    }
+    k_tc<kHead><<<pl->grid, kTcThreads, kSmemBytes, st>>>(p);
+}
+
+int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status) {
+    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false);
+    if (!pl) return -1;
+    TcParams p = pl->p;
+    p.out = a.out; p.n_total = a.n_total; p.r0 = a.r0; p.m = a.m; p.status = status;
+    launch<false>(st, pl, p);
+    return p.S;
+}
+
+bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status) {
+    const void* W[1] = {a.W};
+    int n_end[1] = {a.V};
+    TcPlan* pl = get_plan(cache, W, n_end, 1, a.K, a.act, true);
+    if (!pl) return false;
+    TcParams p = pl->p;
+    p.n_total = a.V; p.r0 = a.r0; p.m = a.m; p.status = status;
+    p.inv_tau = a.inv_tau; p.threshold = a.threshold; p.conf = a.conf; p.token = a.token; p.exit_flag = a.exit_flag;
+    p.logits_dbg = a.logits_dbg; p.part = a.part; p.ticket = a.ticket;
+    launch<true>(st, pl, p);
+    return true;
+}
+
+}  // namespace sb
