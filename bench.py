@@ -274,6 +274,90 @@ def product_arm(args, run: inputs.Run):
         dist.destroy_process_group()
 
 
+def micro_arm(args):
+    """Kernel micro-benchmarks (bf16, 7B-shaped layer): the verify pass of one layer for w rows over
+    a KV cache of S positions, and the exit-confidence kernel against LM heads of two vocabulary
+    sizes.  L2 is defeated by rotating over distinct weight copies totalling more than 1 GB."""
+    from paper_2604_12247_b200 import binding, build
+    build.build()
+    torch.cuda.set_device(0)
+    peak, peak_src = measured_peak()
+    s = inputs.scaled(inputs.LLAMA2_7B, n_layers=1)
+    out = {"mode": "micro", "peak_gbs": peak, "peak_source": peak_src, "iters": args.iters, "layer": [], "exit": []}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    cases = [c for c in args.micro_case.split(",") if c] if args.micro_case else None
+
+    def want(name):
+        return cases is None or name in cases
+
+    n_copies = 4
+    layers = None
+    for S in (512, 2048, 8192):
+        for w in (1, 2, 4, 6, 8):
+            name = f"layer:w={w}:S={S}"
+            if not want(name):
+                continue
+            if layers is None:
+                layers = [inputs.make_weights(s, 100 + i, device="cuda")["layers"][0] for i in range(n_copies)]
+                lws = [binding.layer_weights(lw) for lw in layers]
+            cfg = binding.make_config(s, S + 16, 64)
+            kvd = s.n_kv_heads * s.head_dim
+            n_pages = (S + 16 + 63) // 64
+            kc = torch.randn((n_pages, 64, kvd), device="cuda").to(torch.bfloat16)
+            vc = torch.randn((n_pages, 64, kvd), device="cuda").to(torch.bfloat16)
+            pt = torch.arange(n_pages, dtype=torch.int32, device="cuda")
+            sc = binding.KernelScratch(cfg)
+            h0 = torch.randn((w, s.d_model), device="cuda")
+            h = h0.clone()
+            for i in range(3):
+                binding.k_layer(cfg, lws[i % n_copies], h, kc, vc, pt, S, sc)
+            torch.cuda.synchronize()
+            times = []
+            for i in range(args.iters):
+                h.copy_(h0)
+                e0, e1 = ev(), ev()
+                e0.record()
+                binding.k_layer(cfg, lws[i % n_copies], h, kc, vc, pt, S, sc)
+                e1.record()
+                e1.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e3)
+            us = statistics.median(times)
+            nbytes = inputs.weight_bytes(s)["layer"] + (S + 2 * w) * kv_bytes_per_pos(s)
+            out["layer"].append({"w": w, "S": S, "us": us, "us_min": min(times), "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                                 "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS})
+    del layers
+    for V in (32000, 128256):
+        for m in (1, 4, 8):
+            name = f"exit:m={m}:V={V}"
+            if not want(name):
+                continue
+            sh = inputs.scaled(s, vocab=V)
+            cfg = binding.make_config(sh, 64, 64)
+            copies = 4 if V == 32000 else 2
+            heads = [(torch.randn((V, sh.d_model), device="cuda") * 0.08).to(torch.bfloat16) for _ in range(copies)]
+            gain = torch.ones(sh.d_model, device="cuda", dtype=torch.bfloat16)
+            sc = binding.KernelScratch(cfg)
+            h = torch.randn((m, sh.d_model), device="cuda")
+            for i in range(3):
+                binding.k_exit_confidence(cfg, h, gain, heads[i % copies], 1.4, sc)
+            torch.cuda.synchronize()
+            times = []
+            for i in range(args.iters):
+                e0, e1 = ev(), ev()
+                e0.record()
+                binding.k_exit_confidence(cfg, h, gain, heads[i % copies], 1.0 + 0.2 * (i % 6), sc)
+                e1.record()
+                e1.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e3)
+            us = statistics.median(times)
+            nbytes = V * sh.d_model * 2
+            out["exit"].append({"m": m, "V": V, "us": us, "us_min": min(times), "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                                "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
+                                "note": "includes the RMSNorm launch and two small device copies of the stateless entry point"})
+            del heads
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -283,12 +367,17 @@ def main():
     ap.add_argument("--workload", default="7b", choices=sorted(inputs.RUNS))
     ap.add_argument("--n-gen", type=int, default=None, help="override the number of generated tokens")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--micro", action="store_true", help="kernel micro-benchmarks instead of the generation benchmark")
+    ap.add_argument("--micro-case", default="", help="comma list, e.g. layer:w=4:S=512,exit:m=1:V=32000 (default: all)")
+    ap.add_argument("--iters", type=int, default=40)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     run = inputs.RUNS[args.workload]
     if args.n_gen:
         run = inputs.Run(run.shape, run.n_prompt, args.n_gen, run.d_max, run.w_max, run.tau, run.threshold, run.seed, run.damp_rho)
-    if args.impl == "reference":
+    if args.micro:
+        micro_arm(args)
+    elif args.impl == "reference":
         reference_arm(args, run)
     else:
         product_arm(args, run)

@@ -187,8 +187,14 @@ int sb_tau_schedule(float alpha, int32_t L, float* out);
 /* Eq. 5: analytic speed-up for acceptance rate a, draft width w, depth bound d_max. */
 double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
 
-/* Options: SB_OPT_GEMM 0 = CUDA-core streaming kernels, 1 = TMA + tcgen05 kernels (bf16 only). */
-enum { SB_OPT_GEMM = 1 };
+/* Options.
+ *   SB_OPT_GEMM      0 = CUDA-core streaming kernels, 1 = TMA + tcgen05 kernels (bf16 only).
+ *   SB_OPT_TRACE     (default option only) 1 = sb_k_layer times each of its launches with CUDA events
+ *                    and prints them to stderr; a profiling aid, off by default.
+ *   SB_OPT_TC_TUNING (default option only) stages * 16 + CTAs per SM of the tcgen05 kernels.
+ *   SB_OPT_PDL       (default option only) 1 (default) = launch kernels with programmatic dependent
+ *                    launch so that a kernel's prologue and weight prefetch overlap its predecessor. */
+enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);
 /* Process-wide default for contexts and stateless calls created afterwards. */
 int sb_set_default_option(int32_t key, int32_t value);

@@ -14,12 +14,50 @@
 namespace sb {
 
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
+static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
+
+struct Tracer {
+    static constexpr int kMax = 64;
+    cudaEvent_t ev[kMax];
+    const char* name[kMax];
+    int n = 0;
+    bool on = false;
+    cudaStream_t st;
+    void begin(cudaStream_t s) {
+        on = true; st = s; n = 0;
+        mark("start");
+    }
+    void mark(const char* what) {
+        if (!on || n >= kMax) return;
+        cudaEventCreate(&ev[n]);
+        cudaEventRecord(ev[n], st);
+        name[n++] = what;
+    }
+    void end() {
+        if (!on) return;
+        cudaEventSynchronize(ev[n - 1]);
+        float tot = 0.f;
+        cudaEventElapsedTime(&tot, ev[0], ev[n - 1]);
+        fprintf(stderr, "[sb trace] %d launches, %.1f us:", n - 1, tot * 1e3f);
+        for (int i = 1; i < n; ++i) {
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, ev[i - 1], ev[i]);
+            fprintf(stderr, " %s=%.1f", name[i], ms * 1e3f);
+        }
+        fprintf(stderr, "\n");
+        for (int i = 0; i < n; ++i) cudaEventDestroy(ev[i]);
+        on = false;
+    }
+};
+static Tracer g_tracer;
+#define SB_MARK(what) g_tracer.mark(what)
 
 struct Dims {
     int L, d, H, Hkv, hd, F, V, qd, kvd;
     int page, page_shift, n_pages, max_seq, chunk;
     float rope_base, eps;
     bool f32;
+    double inv_freq[64];
 };
 
 static int pick_gemm(bool f32) {
@@ -36,7 +74,7 @@ static bool make_dims(const sb_config* c, Dims* o) {
         return false;
     if (c->n_heads % c->n_kv_heads) return false;
     if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
-    if (c->d_model % 8 || c->d_ffn % 8) return false;
+    if (c->d_model % 8 || c->d_ffn % 8 || c->d_model > 8192) return false;
     if (c->dtype != SB_F32 && c->dtype != SB_BF16) return false;
     if (!is_pow2(c->kv_page) || c->kv_page < 16) return false;
     if (!(c->rope_base > 0.f) || !(c->rms_eps > 0.f)) return false;
@@ -51,6 +89,7 @@ static bool make_dims(const sb_config* c, Dims* o) {
     while (ch < 256 && ch * 64 < c->max_seq) ch <<= 1;
     o->chunk = ch;
     o->rope_base = c->rope_base; o->eps = c->rms_eps; o->f32 = c->dtype == SB_F32;
+    for (int i = 0; i < o->hd / 2; ++i) o->inv_freq[i] = std::pow((double)c->rope_base, -2.0 * i / o->hd);
     return true;
 }
 
@@ -164,26 +203,37 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     ensure_act(e, lw.attn_norm, r0, m);
     const void* wqkv[3] = {lw.wq, lw.wk, lw.wv};
     int nqkv[3] = {D.qd, D.kvd, D.kvd};
+    SB_MARK("norm");
     int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.act_a, W.p_qkv, r0, m);
+    SB_MARK("qkv");
     RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                pos0, r0, m, D.rope_base};
+                pos0, r0, m, D.rope_base, {}};
+    for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
     SB_T(e, launch_rope_append<T>(e.st, ra));
+    SB_MARK("rope");
     AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, W.act_o, D.H, D.Hkv, D.hd, D.page, D.page_shift,
                 pos0, r0, m, D.chunk};
     SB_T(e, launch_attention<T>(e.st, aa));
+    SB_MARK("attn");
     e.launches += 3;
     const void* wo[1] = {lw.wo};
     int no[1] = {D.d};
     int s_o = gemm(e, wo, no, 1, D.qd, W.act_o, W.p_o, r0, m);
+    SB_MARK("o");
     SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_o, s_o, D.d, (const T*)lw.mlp_norm, D.eps, W.act_a, r0, m));
+    SB_MARK("norm2");
     const void* wgu[2] = {lw.w_gate, lw.w_up};
     int ngu[2] = {D.F, D.F};
     int s_gu = gemm(e, wgu, ngu, 2, D.d, W.act_a, W.p_gu, r0, m);
+    SB_MARK("gateup");
     SB_T(e, launch_swiglu<T>(e.st, W.p_gu, s_gu, D.F, W.act_f, r0, m));
+    SB_MARK("swiglu");
     const void* wd[1] = {lw.w_down};
     int nd[1] = {D.d};
     int s_d = gemm(e, wd, nd, 1, D.F, W.act_f, W.p_down, r0, m);
+    SB_MARK("down");
     SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_down, s_d, D.d, (const T*)next_gain, D.eps, W.act_a, r0, m));
+    SB_MARK("resid");
     e.launches += 3;
     e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
 }
@@ -370,6 +420,9 @@ int sb_set_option(sb_ctx* c, int32_t key, int32_t value) {
 }
 
 int sb_set_default_option(int32_t key, int32_t value) {
+    if (key == SB_OPT_TRACE) { g_trace = value != 0; return SB_OK; }
+    if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
+    if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_GEMM && (value == 0 || value == 1 || value == -1)) {
         if (value == 1 && !tc_available()) return SB_ERR_UNSUPPORTED;
         g_default_gemm = value;
@@ -700,7 +753,9 @@ int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_
     TcPlanCache plans;
     e.plans = &plans;
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    if (g_trace) g_tracer.begin(e.st);
     layer_step(e, *lw, k_cache, v_cache, 0, m, first_pos, nullptr);
+    g_tracer.end();
     if (e.err) return e.err;
     return cuda_ok(cudaGetLastError());
 }

@@ -61,6 +61,8 @@ __device__ __forceinline__ void row_dots(const T* __restrict__ wrow, const typen
 template <typename T>
 __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs a) {
     using AT = typename Act<T>::type;
+    pdl_trigger();
+    pdl_wait();
     const AT* act = reinterpret_cast<const AT*>(a.act);
     int lane = threadIdx.x & 31;
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -80,7 +82,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs a) {
 }
 template <typename T> void launch_gemm_simt(cudaStream_t st, const GemmArgs& a) {
     int ctas = min((a.n_total + 7) / 8, 148 * 8);
-    k_gemm_simt<T><<<ctas, 256, 0, st>>>(a);
+    launch_k(k_gemm_simt<T>, dim3(ctas), dim3(256), 0, st, a);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -95,6 +97,8 @@ __global__ void __launch_bounds__(kHeadWarps * 32) k_head_simt(HeadArgs a) {
     using AT = typename Act<T>::type;
     __shared__ SoftTriple cta_part[kHeadWarps][kMaxW];
     __shared__ bool is_last;
+    pdl_trigger();
+    pdl_wait();
     const AT* act = reinterpret_cast<const AT*>(a.act);
     int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     int warp = blockIdx.x * kHeadWarps + wib;
@@ -134,25 +138,11 @@ __global__ void __launch_bounds__(kHeadWarps * 32) k_head_simt(HeadArgs a) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    if (threadIdx.x < kMaxW) {
-        int i = threadIdx.x;
-        if (i >= a.r0 && i < a.r0 + a.m) {
-            SoftTriple t = soft_empty();
-            for (unsigned int c = 0; c < gridDim.x; ++c) {
-                const volatile SoftTriple* p = a.part + (size_t)c * kMaxW + i;
-                SoftTriple q{p->m, p->idx, p->s};
-                t = soft_merge(t, q, a.inv_tau);
-            }
-            float conf = 1.f / t.s;   // the arg-max term contributes exp(0) = 1, so max softmax = 1 / sum
-            a.conf[i] = conf;
-            a.token[i] = t.idx;
-            a.exit_flag[i] = conf >= a.threshold ? 1 : 0;
-        }
-    }
+    soft_final_merge(a.part, (int)gridDim.x, a.r0, a.m, a.inv_tau, a.threshold, a.conf, a.token, a.exit_flag);
     if (threadIdx.x == 0) *a.ticket = 0u;   // ready for the next launch on this stream
 }
 template <typename T> void launch_head_simt(cudaStream_t st, const HeadArgs& a, int n_ctas) {
-    k_head_simt<T><<<n_ctas, kHeadWarps * 32, 0, st>>>(a);
+    launch_k(k_head_simt<T>, dim3(n_ctas), dim3(kHeadWarps * 32), 0, st, a);
 }
 
 template void launch_gemm_simt<float>(cudaStream_t, const GemmArgs&);

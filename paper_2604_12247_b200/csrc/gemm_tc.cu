@@ -22,13 +22,14 @@
 
 namespace sb {
 
-constexpr int kStages = 6;
+constexpr int kMaxStages = 12;                // pipeline depth is a launch parameter (tuned per use)
 constexpr int kBK = 64;                       // k elements per stage (128 bytes: one swizzle row)
 constexpr int kTileRows = 128;                // MMA M
 constexpr int kStageA = kTileRows * kBK * 2;  // 16 KB
 constexpr int kStageB = 16 * kBK * 2;         // 2 KB
 constexpr int kTcThreads = 192;
-constexpr int kSmemBytes = kStages * (kStageA + kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+static int g_stages = 6, g_ctas_per_sm = 1;   // defaults; see tc_set_tuning
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
 struct alignas(64) TcParams {
@@ -39,6 +40,7 @@ struct alignas(64) TcParams {
     int n_rows[3];      // rows of each matrix
     int n_off[3];       // first output column of each matrix
     int n_chunks, R, S, KB, n_items;
+    int stages;
     float* out;
     int n_total;
     int r0, m;
@@ -172,6 +174,24 @@ __device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
     return it;
 }
 
+// Position of a CTA in its sequence of (work item, k block) pipeline fills.
+struct WorkIter {
+    int item, i, kb;
+    ItemInfo it;
+    __device__ explicit WorkIter(const TcParams& p) : item((int)blockIdx.x), i(0), kb(0) {
+        if (valid_item(p)) { it = decode_item(p, item); kb = it.kb0; }
+        n_items = p.n_items;
+    }
+    int n_items;
+    __device__ bool valid_item(const TcParams& p) const { return item < p.n_items; }
+    __device__ bool valid() const { return item < n_items; }
+    __device__ void next(const TcParams& p) {
+        if (++kb < it.kb1) return;
+        item += (int)gridDim.x;
+        if (item < p.n_items) { it = decode_item(p, item); kb = it.kb0; }
+    }
+};
+
 template <bool kHead>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ TcParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -182,6 +202,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
+    const int kStages = p.stages;
     const uint32_t smA = tiles, smB = tiles + kStages * kStageA;
     const uint32_t bars = smB + kStages * kStageB;             // 8-byte mbarriers
     auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -190,6 +211,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
     auto tempty_bar = [&](int b) { return bars + 8u * (2 * kStages + 2 + b); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_trigger();
     if (threadIdx.x == 0) {
         abort_s = 0;
         for (int s = 0; s < kStages; ++s) {
@@ -214,25 +236,36 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
+        // The weight tiles of the first pipeline fill do not depend on the preceding kernel, so
+        // they are requested BEFORE the grid-dependency wait; the activation tiles (written by
+        // the preceding kernel) follow after it.
         if (lane == 0) {
             for (int j = 0; j < p.n_mats; ++j) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA[j]) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
             const uint64_t pol = policy_evict_first();
-            int stage = 0, phase = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-                ItemInfo it = decode_item(p, item);
-                for (int kb = it.kb0; kb < it.kb1; ++kb) {
-                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, &abort_s, p.status, 1u))) break;
-                    mbar_expect_tx(full_bar(stage), stage_bytes);
-                    tma_load_2d_hint(smA + stage * kStageA, &p.tmA[it.mat], kb * kBK, it.row0, full_bar(stage), pol);
-                    tma_load_2d(smB + stage * kStageB, &p.tmB, kb * kBK, 0, full_bar(stage));
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
-                }
+            WorkIter w(p), w0(p);
+            int n_pre = 0;
+            for (; w.valid() && n_pre < kStages; w.next(p), ++n_pre) {
+                mbar_expect_tx(full_bar(n_pre), stage_bytes);
+                tma_load_2d_hint(smA + n_pre * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(n_pre), pol);
             }
+            pdl_wait();
+            for (int j = 0; j < n_pre; ++j, w0.next(p))
+                tma_load_2d(smB + j * kStageB, &p.tmB, w0.kb * kBK, 0, full_bar(j));
+            int stage = n_pre % kStages, phase = (n_pre / kStages) & 1;
+            for (; w.valid(); w.next(p)) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_s, p.status, 1u)) break;
+                mbar_expect_tx(full_bar(stage), stage_bytes);
+                tma_load_2d_hint(smA + stage * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(stage), pol);
+                tma_load_2d(smB + stage * kStageB, &p.tmB, w.kb * kBK, 0, full_bar(stage));
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        } else {
+            pdl_wait();
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
+        pdl_wait();
         if (lane == 0) {
             int stage = 0, phase = 0, n_local = 0;
             bool ok = true;
@@ -258,6 +291,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
         }
     } else {
         // ------------------------------ epilogue (128 threads) ------------------------------
+        pdl_wait();
         const int q = warp & 3;                            // TMEM lane quadrant this warp may read
         const int row_in_tile = q * 32 + lane;
         SoftTriple tr[kMaxW];
@@ -342,21 +376,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
     __syncthreads();
     if (!is_last_s) return;
     __threadfence();
-    if (threadIdx.x < kMaxW) {
-        int i = threadIdx.x;
-        if (i >= p.r0 && i < p.r0 + p.m) {
-            SoftTriple t = soft_empty();
-            for (unsigned int c = 0; c < gridDim.x; ++c) {
-                const volatile SoftTriple* src = p.part + (size_t)c * kMaxW + i;
-                SoftTriple qv{src->m, src->idx, src->s};
-                t = soft_merge(t, qv, p.inv_tau);
-            }
-            float conf = 1.f / t.s;
-            p.conf[i] = conf;
-            p.token[i] = t.idx;
-            p.exit_flag[i] = conf >= p.threshold ? 1 : 0;
-        }
-    }
+    soft_final_merge(p.part, (int)gridDim.x, p.r0, p.m, p.inv_tau, p.threshold, p.conf, p.token, p.exit_flag);
     if (threadIdx.x == 0) *p.ticket = 0u;
 }
 
@@ -432,12 +452,14 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     key.push_back((uint64_t)K);
     key.push_back((uint64_t)(uintptr_t)act);
     key.push_back(head ? 1 : 0);
+    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm);
     auto it = cache->plans.find(key);
     if (it != cache->plans.end()) return it->second;
     TcPlan* pl = new TcPlan();
     memset(&pl->p, 0, sizeof(pl->p));
     TcParams& p = pl->p;
-    int G = sm_count();
+    int G = sm_count() * g_ctas_per_sm;
+    p.stages = g_stages;
     p.n_mats = n_mats;
     p.KB = (K + kBK - 1) / kBK;
     int prev = 0;
@@ -461,10 +483,18 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
 static bool g_attr_set[2] = {false, false};
 template <bool kHead> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
     if (!g_attr_set[kHead]) {
-        cudaFuncSetAttribute(k_tc<kHead>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaFuncSetAttribute(k_tc<kHead>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(kMaxStages));
         g_attr_set[kHead] = true;
     }
-    k_tc<kHead><<<pl->grid, kTcThreads, kSmemBytes, st>>>(p);
+    launch_k(k_tc<kHead>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages), st, p);
+}
+
+bool tc_set_tuning(int stages, int ctas_per_sm) {
+    if (stages < 2 || stages > kMaxStages || ctas_per_sm < 1 || ctas_per_sm > 2) return false;
+    if (ctas_per_sm * (smem_bytes(stages) + 2048) > 227 * 1024) return false;
+    g_stages = stages;
+    g_ctas_per_sm = ctas_per_sm;
+    return true;
 }
 
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status) {

@@ -19,6 +19,8 @@ struct TcPlanCache {
 };
 
 bool tc_available();
+// pipeline depth (2..12 stages of 18 KB) and persistent CTAs per SM (1..2) of the launches that follow
+bool tc_set_tuning(int stages, int ctas_per_sm);
 // returns the number of split-K partials written to a.out, or -1 if no TMA descriptor could be made
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status);
 bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status);

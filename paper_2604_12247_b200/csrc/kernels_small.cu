@@ -6,12 +6,16 @@
 
 namespace sb {
 
+bool g_use_pdl = true;
+
 // ------------------------------------------------------------------------------------------------
 // h[row0 + i] = embed[token_i]
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void k_embed(const T* __restrict__ embed, int d, const int* __restrict__ toks, int tok_scalar, int row0,
                         float* __restrict__ h) {
+    pdl_trigger();
+    pdl_wait();
     int i = blockIdx.x;
     int tok = toks ? toks[i] : tok_scalar;
     const T* src = embed + (size_t)tok * d;
@@ -20,7 +24,7 @@ __global__ void k_embed(const T* __restrict__ embed, int d, const int* __restric
 }
 template <typename T>
 void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, int tok_scalar, int row0, int m, float* h) {
-    k_embed<T><<<m, 256, 0, st>>>(embed, d, toks_dev, tok_scalar, row0, h);
+    launch_k(k_embed<T>, dim3(m), dim3(256), 0, st, embed, d, toks_dev, tok_scalar, row0, h);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -28,22 +32,35 @@ void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, i
 // act[row] = h[row] / sqrt(mean(h[row]^2) + eps) * gain      (if gain != null)
 // One CTA per row; the reduction order is fixed by the thread layout only.
 // ------------------------------------------------------------------------------------------------
-constexpr int kNormThreads = 512;
+constexpr int kNormThreads = 1024;
+constexpr int kNormVec = 2;   // float4 per thread: rows up to 1024 * 2 * 4 = 8192 wide
 template <typename T>
 __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__ h, const float* __restrict__ part,
                                                             int n_split, int d, const T* __restrict__ gain, float eps,
                                                             void* __restrict__ act, int r0) {
     __shared__ float red[kNormThreads / 32];
+    pdl_trigger();
+    pdl_wait();
     int row = r0 + blockIdx.x;
-    float* hr = h + (size_t)row * d;
+    float4* hr = reinterpret_cast<float4*>(h + (size_t)row * d);
+    const int nv = d >> 2;
+    float4 v[kNormVec];
     float ss = 0.f;
-    for (int k = threadIdx.x; k < d; k += kNormThreads) {
-        float v = hr[k];
-        if (part) {
-            for (int s = 0; s < n_split; ++s) v += part[((size_t)s * kMaxW + row) * d + k];
-            hr[k] = v;
+    // every load of a thread is independent: the hidden row and all partials are in flight at once
+#pragma unroll
+    for (int j = 0; j < kNormVec; ++j) {
+        int k4 = threadIdx.x + j * kNormThreads;
+        if (k4 < nv) {
+            v[j] = hr[k4];
+            if (part) {
+                for (int s = 0; s < n_split; ++s) {   // summed in split order
+                    float4 p = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)s * kMaxW + row) * d) + k4);
+                    v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
+                }
+                hr[k4] = v[j];
+            }
+            ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
         }
-        ss += v * v;
     }
     if (!gain) return;
     ss = warp_sum(ss);
@@ -55,12 +72,22 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
     float inv = rsqrtf(tot / (float)d + eps);
     using A = Act<T>;
     typename A::type* a = reinterpret_cast<typename A::type*>(act);
-    for (int k = threadIdx.x; k < d; k += kNormThreads) A::store(a, row, k, d, hr[k] * inv * to_f32(gain[k]));
+#pragma unroll
+    for (int j = 0; j < kNormVec; ++j) {
+        int k4 = threadIdx.x + j * kNormThreads;
+        if (k4 < nv) {
+            int k = k4 << 2;
+            A::store(a, row, k, d, v[j].x * inv * to_f32(gain[k]));
+            A::store(a, row, k + 1, d, v[j].y * inv * to_f32(gain[k + 1]));
+            A::store(a, row, k + 2, d, v[j].z * inv * to_f32(gain[k + 2]));
+            A::store(a, row, k + 3, d, v[j].w * inv * to_f32(gain[k + 3]));
+        }
+    }
 }
 template <typename T>
 void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d, const T* gain, float eps,
                        void* act, int r0, int m) {
-    k_resid_norm<T><<<m, kNormThreads, 0, st>>>(h, part, n_split, d, gain, eps, act, r0);
+    launch_k(k_resid_norm<T>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -70,6 +97,8 @@ void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void k_rope_append(RopeArgs a) {
+    pdl_trigger();
+    pdl_wait();
     int head = blockIdx.x;
     int row = a.r0 + blockIdx.y;
     int pos = a.pos0 + row;
@@ -85,10 +114,12 @@ __global__ void k_rope_append(RopeArgs a) {
     }
     bool is_v = head >= a.H + a.Hkv;
     if (!is_v) {
-        double inv_freq = pow((double)a.rope_base, -2.0 * (double)i / (double)a.hd);
-        double sn, cs;
-        sincos((double)pos * inv_freq, &sn, &cs);
-        float c = (float)cs, s = (float)sn;
+        // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
+        // the fp32 sincos sees a small argument
+        double ang = (double)pos * a.inv_freq[i];
+        ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+        float s, c;
+        sincosf((float)ang, &s, &c);
         float y0 = x0 * c - x1 * s, y1 = x1 * c + x0 * s;
         x0 = y0;
         x1 = y1;
@@ -108,7 +139,7 @@ __global__ void k_rope_append(RopeArgs a) {
 }
 template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a) {
     dim3 grid(a.H + 2 * a.Hkv, a.m);
-    k_rope_append<T><<<grid, a.hd / 2, 0, st>>>(a);
+    launch_k(k_rope_append<T>, grid, dim3(a.hd / 2), 0, st, a);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -124,6 +155,8 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     constexpr int HD = E * 32;
     __shared__ float q_s[kMaxW][HD];
     __shared__ float mrg[kAttnWarps][kMaxW][HD + 2];
+    pdl_trigger();
+    pdl_wait();
     int hq = blockIdx.x, c = blockIdx.y;
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int kvh = hq / (a.H / a.Hkv);
@@ -215,6 +248,8 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
 // grid = (H, m), block = hd: merge the chunk partials of one (row, head) in chunk order.
 template <typename T>
 __global__ void k_attn_combine(AttnArgs a) {
+    pdl_trigger();
+    pdl_wait();
     int hq = blockIdx.x, row = a.r0 + blockIdx.y, e = threadIdx.x;
     int hd = a.hd;
     int n_chunks = (a.pos0 + row) / a.chunk + 1;   // chunks that hold positions <= this row's own
@@ -237,11 +272,11 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) 
     int n_chunks = (a.pos0 + a.r0 + a.m - 1) / a.chunk + 1;
     dim3 grid(a.H, n_chunks);
     switch (a.hd) {
-        case 32: k_attn_partial<T, 1><<<grid, kAttnWarps * 32, 0, st>>>(a); break;
-        case 64: k_attn_partial<T, 2><<<grid, kAttnWarps * 32, 0, st>>>(a); break;
-        default: k_attn_partial<T, 4><<<grid, kAttnWarps * 32, 0, st>>>(a); break;
+        case 32: launch_k(k_attn_partial<T, 1>, grid, dim3(kAttnWarps * 32), 0, st, a); break;
+        case 64: launch_k(k_attn_partial<T, 2>, grid, dim3(kAttnWarps * 32), 0, st, a); break;
+        default: launch_k(k_attn_partial<T, 4>, grid, dim3(kAttnWarps * 32), 0, st, a); break;
     }
-    k_attn_combine<T><<<dim3(a.H, a.m), a.hd, 0, st>>>(a);
+    launch_k(k_attn_combine<T>, dim3(a.H, a.m), dim3(a.hd), 0, st, a);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -249,6 +284,8 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) 
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void k_swiglu(const float* __restrict__ part, int n_split, int F, void* __restrict__ act, int r0) {
+    pdl_trigger();
+    pdl_wait();
     int row = r0 + blockIdx.y;
     int f = blockIdx.x * blockDim.x + threadIdx.x;
     if (f >= F) return;
@@ -263,7 +300,7 @@ __global__ void k_swiglu(const float* __restrict__ part, int n_split, int F, voi
     A::store(reinterpret_cast<typename A::type*>(act), row, f, F, v);
 }
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m) {
-    k_swiglu<T><<<dim3((F + 255) / 256, m), 256, 0, st>>>(part, n_split, F, act, r0);
+    launch_k(k_swiglu<T>, dim3((F + 255) / 256, m), dim3(256), 0, st, part, n_split, F, act, r0);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -272,6 +309,8 @@ template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int
 // ------------------------------------------------------------------------------------------------
 struct Drafts8 { int v[kMaxW]; };
 __global__ void k_accept(const int* __restrict__ g, Drafts8 drafts, int w, int max_emit, int* __restrict__ result) {
+    pdl_trigger();
+    pdl_wait();
     if (threadIdx.x != 0) return;
     int acc = 0;
     while (acc < w && drafts.v[acc] >= 0 && g[acc] == drafts.v[acc]) ++acc;
@@ -284,7 +323,7 @@ __global__ void k_accept(const int* __restrict__ g, Drafts8 drafts, int w, int m
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result) {
     Drafts8 d;
     for (int i = 0; i < kMaxW; ++i) d.v[i] = drafts8[i];
-    k_accept<<<1, 32, 0, st>>>(g, d, w, max_emit, result);
+    launch_k(k_accept, dim3(1), dim3(32), 0, st, g, d, w, max_emit, result);
 }
 
 __global__ void k_init_pages(int* pt, int n) {

@@ -38,6 +38,27 @@ template <> struct Act<__nv_bfloat16> {
     }
 };
 
+// Programmatic dependent launch.  Every kernel of the library is launched with programmatic
+// stream serialisation: it may start while its predecessor is still running, lets its own
+// successor start early (pdl_trigger), and must execute pdl_wait -- EVERY thread, before any
+// early return -- before it touches memory the predecessor writes or reads.  Only loads of
+// weights (never written) may precede the wait.  Without the launch attribute both are no-ops.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+extern bool g_use_pdl;
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_use_pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T from_f32(float v);
@@ -73,6 +94,37 @@ __device__ __forceinline__ void soft_push(SoftTriple& t, float z, int idx, float
         t.idx = idx;
     } else {
         t.s += expf((z - t.m) * inv_t);
+    }
+}
+
+// Final merge of the per-CTA triples of an exit-confidence launch, run by the last CTA to arrive:
+// warp w takes rows w, w + n_warps, ...; lane l folds CTAs l, l+32, ... in that order, then the
+// lanes fold as a butterfly.  The tree is fixed by (n_ctas) alone, so the result is deterministic,
+// and all loads of a lane are independent (no latency chain).
+__device__ __forceinline__ void soft_final_merge(const SoftTriple* part, int n_ctas, int r0, int m, float inv_t,
+                                                 float threshold, float* conf, int* token, int* exit_flag) {
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    for (int i = r0 + warp; i < r0 + m; i += n_warps) {
+        SoftTriple t = soft_empty();
+        for (int c = lane; c < n_ctas; c += 32) {
+            const SoftTriple* p = part + (size_t)c * 8 + i;
+            SoftTriple q{__ldcg(&p->m), __ldcg(&p->idx), __ldcg(&p->s)};
+            t = soft_merge(t, q, inv_t);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            SoftTriple other;
+            other.m = __shfl_xor_sync(0xffffffffu, t.m, o);
+            other.idx = __shfl_xor_sync(0xffffffffu, t.idx, o);
+            other.s = __shfl_xor_sync(0xffffffffu, t.s, o);
+            t = soft_merge(t, other, inv_t);
+        }
+        if (lane == 0) {
+            float c = 1.f / t.s;   // the arg-max term contributes exp(0) = 1, so max softmax = 1 / sum
+            conf[i] = c;
+            token[i] = t.idx;
+            exit_flag[i] = c >= threshold ? 1 : 0;
+        }
     }
 }
 
@@ -128,6 +180,7 @@ struct RopeArgs {
     int H, Hkv, hd, page, page_shift;
     int pos0, r0, m;
     float rope_base;
+    double inv_freq[64];   // base^(-2i/hd), i < hd/2, computed on the host in fp64
 };
 
 // ---- launchers (kernels_small.cu) ----
