@@ -7,9 +7,11 @@
 // the low bf16 halves of the 8 fp32 activation rows, so one kind::f16 MMA (M=128, N=16, K=16)
 // yields W.hi and W.lo side by side in TMEM and their sum is as accurate as an fp32 product.
 //
-// One persistent CTA per SM: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2-5 =
-// epilogue (tcgen05.ld, then either split-K partial stores or, for the LM head, the online
-// temperature-scaled softmax max/argmax of Eq. 2).  Work items are (row slab, k split) pairs
+// One persistent CTA per SM: warps 0-3 = TMA producers (one issuing thread moves only ~20 B/clk
+// through TMA -- a 128-byte row every ~6.5 clocks -- so four of them take every fourth pipeline
+// fill to reach the HBM rate), warp 4 = MMA issuer (owns TMEM), warps 5-8 = epilogue (tcgen05.ld,
+// then either split-K partial stores or, for the LM head, the online temperature-scaled softmax
+// max/argmax of Eq. 2).  Work items are (row slab, k split) pairs
 // chosen on the host so that every CTA streams the same number of bytes whatever the number of
 // rows: the result of a row never depends on its companions.  Every wait is bounded: on expiry
 // the kernel raises a status word, drains and returns.
@@ -27,9 +29,12 @@ constexpr int kBK = 64;                       // k elements per stage (128 bytes
 constexpr int kTileRows = 128;                // MMA M
 constexpr int kStageA = kTileRows * kBK * 2;  // 16 KB
 constexpr int kStageB = 16 * kBK * 2;         // 2 KB
-constexpr int kTcThreads = 192;
+constexpr int kProducers = 4;                 // producer warps
+constexpr int kTcThreads = (kProducers + 5) * 32;
 static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
-static int g_stages = 6, g_ctas_per_sm = 1;   // defaults; see tc_set_tuning
+// Two CTAs per SM (each with its own producers, MMA issuer and TMEM accumulators) stream measurably
+// faster than one CTA with twice the pipeline depth.
+static int g_stages = 6, g_ctas_per_sm = 2;   // defaults; see tc_set_tuning
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
 struct alignas(64) TcParams {
@@ -97,6 +102,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = clock64();
     for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicExch(status, code);
+            return false;
+        }
+    }
+}
+// Same, for waits that are expected to last long (an epilogue warp waiting for a whole work
+// item): backs off with nanosleep so that the polling does not compete with the producers.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  unsigned int* status, unsigned int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = clock64();
+    for (;;) {
+        __nanosleep(200);
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) {
@@ -176,9 +198,9 @@ __device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
 
 // Position of a CTA in its sequence of (work item, k block) pipeline fills.
 struct WorkIter {
-    int item, i, kb;
+    int item, kb;
     ItemInfo it;
-    __device__ explicit WorkIter(const TcParams& p) : item((int)blockIdx.x), i(0), kb(0) {
+    __device__ explicit WorkIter(const TcParams& p) : item((int)blockIdx.x), kb(0) {
         if (valid_item(p)) { it = decode_item(p, item); kb = it.kb0; }
         n_items = p.n_items;
     }
@@ -186,6 +208,7 @@ struct WorkIter {
     __device__ bool valid_item(const TcParams& p) const { return item < p.n_items; }
     __device__ bool valid() const { return item < n_items; }
     __device__ void next(const TcParams& p) {
+        if (item >= n_items) return;
         if (++kb < it.kb1) return;
         item += (int)gridDim.x;
         if (item < p.n_items) { it = decode_item(p, item); kb = it.kb0; }
@@ -193,7 +216,7 @@ struct WorkIter {
 };
 
 template <bool kHead>
-__global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ TcParams p) {
+__global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_s;
@@ -224,7 +247,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {   // TMEM: 32 columns = two 16-column accumulators
+    if (warp == kProducers) {   // TMEM: 32 columns = two 16-column accumulators
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(32));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
@@ -234,36 +257,43 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
     const uint32_t tmem_base = tmem_base_s;
     const uint32_t stage_bytes = (uint32_t)p.R * (kBK * 2) + kStageB;
 
-    if (warp == 0) {
-        // ------------------------------ TMA producer ------------------------------
-        // The weight tiles of the first pipeline fill do not depend on the preceding kernel, so
-        // they are requested BEFORE the grid-dependency wait; the activation tiles (written by
-        // the preceding kernel) follow after it.
+    if (warp < kProducers) {
+        // ------------------------------ TMA producers ------------------------------
+        // Producer j owns pipeline fills j, j + kProducers, ...  The weight tiles of the first
+        // pipeline fill do not depend on the preceding kernel, so they are requested BEFORE the
+        // grid-dependency wait; the activation tiles (written by that kernel) follow after it.
         if (lane == 0) {
-            for (int j = 0; j < p.n_mats; ++j) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA[j]) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
+            if (warp == 0) {
+                for (int j = 0; j < p.n_mats; ++j) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA[j]) : "memory");
+                asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
+            }
             const uint64_t pol = policy_evict_first();
             WorkIter w(p), w0(p);
-            int n_pre = 0;
-            for (; w.valid() && n_pre < kStages; w.next(p), ++n_pre) {
-                mbar_expect_tx(full_bar(n_pre), stage_bytes);
-                tma_load_2d_hint(smA + n_pre * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(n_pre), pol);
+            for (int j = 0; j < warp; ++j) { w.next(p); w0.next(p); }
+            int fill = warp;
+            for (; w.valid() && fill < kStages; fill += kProducers) {
+                mbar_expect_tx(full_bar(fill), stage_bytes);
+                tma_load_2d_hint(smA + fill * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(fill), pol);
+                for (int j = 0; j < kProducers; ++j) w.next(p);
             }
             pdl_wait();
-            for (int j = 0; j < n_pre; ++j, w0.next(p))
-                tma_load_2d(smB + j * kStageB, &p.tmB, w0.kb * kBK, 0, full_bar(j));
-            int stage = n_pre % kStages, phase = (n_pre / kStages) & 1;
-            for (; w.valid(); w.next(p)) {
-                if (!mbar_wait(empty_bar(stage), phase ^ 1, &abort_s, p.status, 1u)) break;
+            for (int f0 = warp; f0 < fill; f0 += kProducers) {
+                tma_load_2d(smB + f0 * kStageB, &p.tmB, w0.kb * kBK, 0, full_bar(f0));
+                for (int j = 0; j < kProducers; ++j) w0.next(p);
+            }
+            for (; w.valid(); fill += kProducers) {
+                int stage = fill % kStages;
+                uint32_t phase = (uint32_t)(fill / kStages) & 1u;
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_s, p.status, 1u)) break;
                 mbar_expect_tx(full_bar(stage), stage_bytes);
                 tma_load_2d_hint(smA + stage * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(stage), pol);
                 tma_load_2d(smB + stage * kStageB, &p.tmB, w.kb * kBK, 0, full_bar(stage));
-                if (++stage == kStages) { stage = 0; phase ^= 1; }
+                for (int j = 0; j < kProducers; ++j) w.next(p);
             }
         } else {
             pdl_wait();
         }
-    } else if (warp == 1) {
+    } else if (warp == kProducers) {
         // ------------------------------ MMA issuer ------------------------------
         pdl_wait();
         if (lane == 0) {
@@ -305,8 +335,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
             ItemInfo it = decode_item(p, item);
             int buf = n_local & 1;
             uint32_t use = (uint32_t)(n_local >> 1);
-            ok = mbar_wait(tfull_bar(buf), use & 1u, &abort_s, p.status, 4u);
-            ok = __all_sync(0xffffffffu, ok);              // the TMEM load below needs the whole warp
+            if (lane == 0) ok = mbar_wait_relaxed(tfull_bar(buf), use & 1u, &abort_s, p.status, 4u);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;   // one lane polls; the TMEM load needs the whole warp
             if (!ok) break;
             tc_fence_after();
             uint32_t v[16];
@@ -354,7 +384,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc(const __grid_constant__ Tc
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kProducers) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32));
     }
@@ -490,7 +520,9 @@ template <bool kHead> static void launch(cudaStream_t st, const TcPlan* pl, cons
 }
 
 bool tc_set_tuning(int stages, int ctas_per_sm) {
-    if (stages < 2 || stages > kMaxStages || ctas_per_sm < 1 || ctas_per_sm > 2) return false;
+    // stages >= producers: a producer's parity wait on a stage's "empty" barrier is only sound if no
+    // peer can lag two phases behind, which in-order consumption guarantees when stages >= producers
+    if (stages < kProducers || stages > kMaxStages || ctas_per_sm < 1 || ctas_per_sm > 2) return false;
     if (ctas_per_sm * (smem_bytes(stages) + 2048) > 227 * 1024) return false;
     g_stages = stages;
     g_ctas_per_sm = ctas_per_sm;
