@@ -89,6 +89,18 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def aggregate_replicas(dec_ms: float, call_ms: float, steps: int, dec_tokens: int, gen_tokens: int, world: int,
+                       device: str = "cuda"):
+    """Replica aggregation: every rank decodes its own sequence; the job's time is the slowest rank's
+    (max over ranks), its throughput the tokens of all ranks over that time.  Returns (value, e2e)."""
+    t = torch.tensor([dec_ms, call_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dec_max, call_max = t.tolist()
+    return world * steps * dec_tokens / (dec_max / 1e3), world * steps * gen_tokens / (call_max / 1e3), dec_max, call_max
+
+
 def kv_bytes_per_pos(s: inputs.Shape) -> int:
     return 2 * s.n_kv_heads * s.head_dim * (4 if s.dtype == "f32" else 2)
 
@@ -207,12 +219,7 @@ def product_arm(args, run: inputs.Run):
 
     dec_tok = run.n_gen - 1                          # the first token comes out of prefill
     dec_ms = sum(st.us_decode_dev for st in stats) / 1e3
-    t = torch.tensor([dec_ms, sum(call_ms)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dec_ms_max, call_ms_max = t.tolist()
-    value = world * args.steps * dec_tok / (dec_ms_max / 1e3)
-    e2e = world * args.steps * run.n_gen / (call_ms_max / 1e3)
+    value, e2e, dec_ms_max, call_ms_max = aggregate_replicas(dec_ms, sum(call_ms), args.steps, dec_tok, run.n_gen, world)
     ar_ms = sum(st.us_decode_dev for st in ar_stats) / 1e3
     ar_value = args.steps * dec_tok / (ar_ms / 1e3)
 
