@@ -172,6 +172,27 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
                          float tau_l, float* conf, int32_t* token, float* logits_dbg, void* scratch,
                          size_t scratch_bytes, void* cuda_stream);
 
+/* The same exit-confidence computation for callers that cannot allocate device memory (the paper has
+ * no counterpart; this is a convenience of the library).  Some users of this kernel run where
+ * cudaMalloc is off limits -- inside a serving loop whose memory was handed out once at start-up,
+ * under a framework that owns the caching allocator and forbids foreign allocations, or in a
+ * latency-critical path where an allocation's implicit synchronisation is unacceptable -- and they
+ * have no spare buffer to lend as scratch.  This variant takes none: its scratch is a fixed 1 MiB
+ * array in device memory that every GPU holding the library keeps from load to exit.
+ *   - Inputs and outputs are still the caller's: h device fp32 [m, d], final_norm / lm_head device
+ *     in cfg->dtype, conf device fp32 [m], token device int32 [m]; work runs on cuda_stream.
+ *   - Limit: the rows, their normalised copy and the per-CTA partial results must fit the array,
+ *     which holds for d_model <= 8192; a larger model is refused with SB_ERR_CAPACITY.  Other
+ *     errors as sb_k_exit_confidence (SB_ERR_ARG for bad pointers, m outside 1..8, tau_l <= 0).
+ *   - The call allocates nothing on the device: no cudaMalloc / cudaFree, no allocating library
+ *     routine.  The first call on each device looks up the array's device address (a short
+ *     host-side query); make that first call before any stream capture starts.
+ *   - All calls on one device share the array and it keeps the previous call's contents; the call
+ *     itself resets the words that must start at zero.  Two calls whose GPU work overlaps (different
+ *     streams, or different host threads) race on it: serialise them. */
+int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, const void* final_norm,
+                                const void* lm_head, float tau_l, float* conf, int32_t* token, void* cuda_stream);
+
 /* One decoder layer for m rows at positions first_pos .. first_pos+m-1 (the verify pass of one
  * layer, Section 3.3): h device fp32 [m, d] in/out.  k_cache / v_cache: device, cfg->dtype,
  * [n_pages, kv_page, n_kv_heads*head_dim]; page_table device int32 [ceil(max_seq / kv_page)]

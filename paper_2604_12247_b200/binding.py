@@ -64,7 +64,8 @@ class SBError(RuntimeError):
 
 EXPORTS = ("sb_workspace_bytes", "sb_create", "sb_destroy", "sb_load_weights", "sb_reset", "sb_get_state",
            "sb_read_hidden", "sb_prefill", "sb_draft_push", "sb_draft_advance", "sb_exit_confidence", "sb_verify",
-           "sb_generate", "sb_generate_ar", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_layer",
+           "sb_generate", "sb_generate_ar", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
+           "sb_k_layer",
            "sb_tau_schedule", "sb_model_speedup", "sb_set_option", "sb_set_default_option", "sb_strerror")
 
 _lib = None
@@ -98,6 +99,7 @@ def lib():
                                   C.POINTER(i32)]
         L.sb_generate_ar.argtypes = [vp, vp, i32, i32, vp, C.POINTER(i32), C.POINTER(Stats)]
         L.sb_k_exit_confidence.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp, vp, C.c_size_t, vp]
+        L.sb_k_exit_confidence_static.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp]
         L.sb_k_layer.argtypes = [C.POINTER(Config), C.POINTER(LayerWeights), vp, i32, vp, vp, vp, i32, vp, C.c_size_t, vp]
         L.sb_tau_schedule.argtypes = [f32, i32, vp]
         L.sb_model_speedup.restype = C.c_double
@@ -269,6 +271,23 @@ def k_exit_confidence(cfg: Config, h: torch.Tensor, final_norm: torch.Tensor, lm
                                       C.c_void_p(scratch.ptr), scratch.nbytes, _stream_handle(stream)),
            "sb_k_exit_confidence")
     return (conf, tok, logits) if want_logits else (conf, tok)
+
+
+def k_exit_confidence_static(cfg: Config, h: torch.Tensor, final_norm: torch.Tensor, lm_head: torch.Tensor, tau_l: float,
+                             stream=None):
+    """Exit confidence for callers that may not allocate device memory and have no scratch to lend:
+    the library's own fixed device array serves as scratch (d_model <= 8192).  Calls on one device
+    share that array, so do not let two of them overlap on the GPU.  The output tensors made here
+    are the binding's convenience; the C entry point itself allocates nothing.
+    Returns (conf [m] fp32, token [m] int32) as CUDA tensors."""
+    m = h.shape[0]
+    assert h.is_cuda and h.dtype == torch.float32 and h.is_contiguous()
+    conf = torch.empty(m, dtype=torch.float32, device="cuda")
+    tok = torch.empty(m, dtype=torch.int32, device="cuda")
+    _check(lib().sb_k_exit_confidence_static(C.byref(cfg), h.data_ptr(), m, final_norm.data_ptr(), lm_head.data_ptr(),
+                                             tau_l, conf.data_ptr(), tok.data_ptr(), _stream_handle(stream)),
+           "sb_k_exit_confidence_static")
+    return conf, tok
 
 
 def k_layer(cfg: Config, lw: dict, h: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,

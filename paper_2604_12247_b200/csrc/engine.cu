@@ -315,6 +315,50 @@ static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats*
     return m;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Scratch of sb_k_exit_confidence_static: a fixed array in device memory that exists as soon as the
+// library is loaded on a GPU, so the call needs no allocation from anybody.  Shared by all calls.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = size_t(1) << 20;   // 1 MiB
+constexpr int kStaticMaxDModel = 8192;                    // widest model whose rows fit it
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// what the exit-confidence call keeps in scratch: hidden rows, the normalised operand, the per-CTA
+// softmax triples, the ticket, the result block and the status word
+static size_t carve_exit_only(const Dims& D, char* base, Work* w) {
+    Carver c{base};
+    Work tmp;
+    Work& W = w ? *w : tmp;
+    size_t es = D.f32 ? 4 : 2, act_rows = D.f32 ? 8 : 16;
+    c.take(W.h, sizeof(float) * kMaxW * D.d);
+    c.take(W.act_a, es * act_rows * D.d);
+    c.take(W.head_part, sizeof(SoftTriple) * kHeadMaxCtas * kMaxW);
+    c.take(W.ticket, 64);
+    c.take(W.res, sizeof(int) * 64);
+    c.take(W.status, 64);
+    return (c.off + 1023) & ~size_t(1023);
+}
+
+// Device address of the static scratch on the current device.  In host code the array's name is
+// only a host-side handle, never a device address: the address comes from cudaGetSymbolAddress,
+// asked once per device with that device current.
+static int static_scratch_ptr(char** out) {
+    constexpr int kMaxDev = 64;
+    static char* ptrs[kMaxDev] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return SB_ERR_CUDA;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return SB_ERR_CUDA;
+        }
+        ptrs[dev] = static_cast<char*>(p);
+    }
+    *out = ptrs[dev];
+    return SB_OK;
+}
+
 extern "C" {
 
 size_t sb_workspace_bytes(const sb_config* cfg) {
@@ -726,6 +770,37 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     cudaMemcpyAsync(e.W.h, h, sizeof(float) * m * D.d, cudaMemcpyDeviceToDevice, e.st);
     ensure_act(e, final_norm, 0, m);
     head(e, lm_head, 0, m, tau_l, 2.f, reinterpret_cast<float*>(e.W.res), e.W.res + 8, e.W.res + 16, logits_dbg);
+    cudaMemcpyAsync(conf, e.W.res, sizeof(float) * m, cudaMemcpyDeviceToDevice, e.st);
+    cudaMemcpyAsync(token, e.W.res + 8, sizeof(int) * m, cudaMemcpyDeviceToDevice, e.st);
+    if (e.err) return e.err;
+    return cuda_ok(cudaGetLastError());
+}
+
+int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, const void* final_norm,
+                                const void* lm_head, float tau_l, float* conf, int32_t* token, void* stream) {
+    Dims D;
+    if (cfg && cfg->d_model > kStaticMaxDModel) return SB_ERR_CAPACITY;   // would not fit the fixed array
+    if (!make_dims(cfg, &D) || !h || !final_norm || !lm_head || !conf || !token) return SB_ERR_ARG;
+    if (m < 1 || m > SB_MAX_W || !(tau_l > 0.f)) return SB_ERR_ARG;
+    if ((uintptr_t)lm_head & 15) return SB_ERR_ARG;
+    if (carve_exit_only(D, nullptr, nullptr) > kStaticScratchBytes) return SB_ERR_CAPACITY;
+    char* base = nullptr;
+    int rc = static_scratch_ptr(&base);   // first call on a device looks the address up
+    if (rc) return rc;
+    Exec e;
+    e.D = D;
+    e.st = (cudaStream_t)stream;
+    e.W = Work{};
+    carve_exit_only(D, base, &e.W);
+    e.gemm = pick_gemm(D.f32);
+    TcPlanCache plans;
+    e.plans = &plans;
+    // the array keeps whatever the previous call left: the ticket and the status word must start at zero
+    cudaMemsetAsync(e.W.ticket, 0, 64, e.st);
+    cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    cudaMemcpyAsync(e.W.h, h, sizeof(float) * m * D.d, cudaMemcpyDeviceToDevice, e.st);
+    ensure_act(e, final_norm, 0, m);
+    head(e, lm_head, 0, m, tau_l, 2.f, reinterpret_cast<float*>(e.W.res), e.W.res + 8, e.W.res + 16, nullptr);
     cudaMemcpyAsync(conf, e.W.res, sizeof(float) * m, cudaMemcpyDeviceToDevice, e.st);
     cudaMemcpyAsync(token, e.W.res + 8, sizeof(int) * m, cudaMemcpyDeviceToDevice, e.st);
     if (e.err) return e.err;
