@@ -85,9 +85,7 @@ static bool make_dims(const sb_config* c, Dims* o) {
     o->max_seq = c->max_seq;
     o->n_pages = (c->max_seq + o->page - 1) / o->page;
     // split-KV chunk: fixed per context so that a row's attention never depends on its companions
-    int ch = 32;
-    while (ch < 256 && ch * 64 < c->max_seq) ch <<= 1;
-    o->chunk = ch;
+    o->chunk = 128;   // = the attention kernel's chunk: 4 warps x 32 positions
     o->rope_base = c->rope_base; o->eps = c->rms_eps; o->f32 = c->dtype == SB_F32;
     for (int i = 0; i < o->hd / 2; ++i) o->inv_freq[i] = std::pow((double)c->rope_base, -2.0 * i / o->hd);
     return true;

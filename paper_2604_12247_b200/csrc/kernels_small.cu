@@ -143,100 +143,199 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 }
 
 // ------------------------------------------------------------------------------------------------
-// Decode attention, split over the KV length in chunks whose boundaries depend on absolute
-// positions only.  grid = (H, n_chunks); 4 warps; warp v of a CTA takes tokens base+v, base+v+4, ...
-// A lane owns hd/32 contiguous channels; q.k is reduced with warp shuffles; the running
-// (max, sum, out) of every row lives in registers.  Per-(chunk,row,head) partials go to scratch
-// and k_attn_combine merges them in chunk order.
+// Decode attention over the paged KV cache, split over the KV length into chunks of 128 positions
+// whose boundaries depend on absolute positions only (so a row's result never depends on its
+// companions).  grid = (Hkv, n_chunks), 4 warps; warp v owns positions base + 32 v .. + 31.
+//   1. each warp stages its 32 K rows and 32 V rows in shared memory once (128-bit loads); they
+//      serve every query head of the KV group and every row: K and V leave HBM once per layer;
+//   2. q.k with one position per lane (no reduction per dot product); the softmax max and sum
+//      over the 32 positions are warp-shuffle reductions;
+//   3. P.V with one channel group per lane, probabilities broadcast from shared memory.
+// (row, query head) pairs are processed eight at a time.  Per-warp partials (max, sum, out) are
+// merged in warp order into one partial per (chunk, row, head); k_attn_combine merges the chunks.
 // ------------------------------------------------------------------------------------------------
 constexpr int kAttnWarps = 4;
-template <typename T, int E>   // E = hd / 32
+constexpr int kAttnChunk = 128;
+constexpr int kPairGroup = 8;
+
+template <typename T> __device__ __forceinline__ void unpack16(const uint4& u, float (&f)[16 / sizeof(T)]);
+template <> __device__ __forceinline__ void unpack16<float>(const uint4& u, float (&f)[4]) {
+    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+}
+template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& u, float (&f)[8]) {
+    const uint32_t r[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = __uint_as_float(r[j] << 16);
+        f[2 * j + 1] = __uint_as_float(r[j] & 0xffff0000u);
+    }
+}
+
+template <typename T, int HD>
 __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
-    constexpr int HD = E * 32;
-    __shared__ float q_s[kMaxW][HD];
-    __shared__ float mrg[kAttnWarps][kMaxW][HD + 2];
+    constexpr int E = HD / 32;                       // channels per lane in P.V
+    constexpr int EPP = 16 / (int)sizeof(T);         // elements per 16-byte piece
+    constexpr int PPR = HD / EPP;                    // pieces per K/V row
+    constexpr int ROWB = HD * (int)sizeof(T) + 16;   // padded row pitch: lane-per-row 16-byte reads are conflict-free
+    extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
     pdl_wait();
-    int hq = blockIdx.x, c = blockIdx.y;
-    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int kvh = hq / (a.H / a.Hkv);
-    int kvd = a.Hkv * HD, qd = a.H * HD;
-    int t_begin = c * a.chunk;
-    int pos_last = a.pos0 + a.r0 + a.m - 1;
-    int t_end = min(t_begin + a.chunk, pos_last + 1);
-    for (int idx = threadIdx.x; idx < a.m * HD; idx += blockDim.x) {
-        int i = idx / HD, e = idx - i * HD;
-        q_s[i][e] = a.q[(size_t)(a.r0 + i) * qd + hq * HD + e];
+    const int kvh = blockIdx.x, c = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
+    constexpr int p_lo = 0;
+    const int kvd = a.Hkv * HD, qd = a.H * HD;
+    float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD]
+    unsigned char* kv_s = smem + (size_t)P * HD * 4;                                // per warp: K[32], V[32]
+    unsigned char* K_w = kv_s + (size_t)warp * 64 * ROWB;
+    unsigned char* V_w = K_w + 32 * ROWB;
+    float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + warp * kPairGroup * 32;   // [8][32]
+    float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + kAttnWarps * kPairGroup * 32;   // [4][P][HD+2]
+
+    for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
+        int p = idx / HD, e = idx - p * HD;
+        int i = (p_lo + p) / G, g = (p_lo + p) - i * G;
+        q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
     }
-    __syncthreads();
-    const float scale = rsqrtf((float)HD);
-    float mx[kMaxW], l[kMaxW], o[kMaxW][E];
-#pragma unroll
-    for (int i = 0; i < kMaxW; ++i) {
-        mx[i] = -INFINITY;
-        l[i] = 0.f;
-#pragma unroll
-        for (int e = 0; e < E; ++e) o[i][e] = 0.f;
+    const int pos_last = a.pos0 + a.r0 + a.m - 1;
+    const int tbase = c * kAttnChunk + warp * 32;
+    const int my_t = tbase + lane;
+    // stage this warp's K and V rows (positions beyond the last row's own are never read: zero them)
+    size_t my_off = 0;
+    if (my_t <= pos_last) {
+        int page = a.page_table[my_t >> a.page_shift];
+        my_off = ((size_t)page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
     }
     const T* kc = reinterpret_cast<const T*>(a.k_cache);
     const T* vc = reinterpret_cast<const T*>(a.v_cache);
-    for (int t = t_begin + warp; t < t_end; t += kAttnWarps) {
-        int page = a.page_table[t >> a.page_shift];
-        size_t off = ((size_t)page * a.page + (t & (a.page - 1))) * kvd + kvh * HD + lane * E;
-        float kf[E], vf[E];
+    // asynchronous 16-byte copies straight into shared memory: all 2 * PPR copies of a lane are in
+    // flight at once (a source size of 0 zero-fills the rows beyond the last position)
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            kf[e] = to_f32(kc[off + e]);
-            vf[e] = to_f32(vc[off + e]);
-        }
+    for (int j = lane; j < 32 * PPR; j += 32) {
+        int tk = j / PPR, piece = j - tk * PPR;
+        size_t off = __shfl_sync(0xffffffffu, my_off, tk);
+        unsigned int nbytes = (tbase + tk <= pos_last) ? 16u : 0u;
+        unsigned int kd = (unsigned int)__cvta_generic_to_shared(K_w + tk * ROWB + piece * 16);
+        unsigned int vd = (unsigned int)__cvta_generic_to_shared(V_w + tk * ROWB + piece * 16);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(kd), "l"(reinterpret_cast<const uint4*>(kc + off) + piece), "r"(nbytes) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(vd), "l"(reinterpret_cast<const uint4*>(vc + off) + piece), "r"(nbytes) : "memory");
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncthreads();   // q_s complete, own tiles complete
+
+    const float scale = rsqrtf((float)HD);
+    for (int pg = 0; pg < P; pg += kPairGroup) {
+        // ---- scores: lane = position ----
+        float sc[kPairGroup];
 #pragma unroll
-        for (int i = 0; i < kMaxW; ++i) {
-            if (i < a.m && t <= a.pos0 + a.r0 + i) {   // causal: row i sees positions <= its own
-                float s = 0.f;
+        for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = 0.f;
+#pragma unroll 2
+        for (int piece = 0; piece < PPR; ++piece) {
+            float kf[EPP];
+            unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB + piece * 16), kf);
 #pragma unroll
-                for (int e = 0; e < E; ++e) s += q_s[i][lane * E + e] * kf[e];
-                s = warp_sum(s) * scale;
-                float nm = fmaxf(mx[i], s);
-                float corr = expf(mx[i] - nm);   // exp(-inf) = 0 on the first token
-                float p = expf(s - nm);
-                l[i] = l[i] * corr + p;
+            for (int pp = 0; pp < kPairGroup; ++pp) {
+                if (pg + pp < P) {
+                    const float4* qv = reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP);
 #pragma unroll
-                for (int e = 0; e < E; ++e) o[i][e] = o[i][e] * corr + p * vf[e];
-                mx[i] = nm;
+                    for (int v4 = 0; v4 < EPP / 4; ++v4) {
+                        float4 qq = qv[v4];
+                        sc[pp] = fmaf(qq.x, kf[4 * v4], sc[pp]);
+                        sc[pp] = fmaf(qq.y, kf[4 * v4 + 1], sc[pp]);
+                        sc[pp] = fmaf(qq.z, kf[4 * v4 + 2], sc[pp]);
+                        sc[pp] = fmaf(qq.w, kf[4 * v4 + 3], sc[pp]);
+                    }
+                }
             }
         }
-    }
+        // ---- softmax pieces of this warp's 32 positions (warp-shuffle max and sum) ----
+        float mx[kPairGroup], ls[kPairGroup];
 #pragma unroll
-    for (int i = 0; i < kMaxW; ++i) {
-        if (i < a.m) {
+        for (int pp = 0; pp < kPairGroup; ++pp) {
+            mx[pp] = -INFINITY;
+            ls[pp] = 0.f;
+            float pt = 0.f;
+            if (pg + pp < P) {
+                int i = (p_lo + pg + pp) / G;
+                bool on = my_t <= a.pos0 + a.r0 + i;     // causal: a row sees positions <= its own
+                float s = on ? sc[pp] * scale : -INFINITY;
+                float m = s;
 #pragma unroll
-            for (int e = 0; e < E; ++e) mrg[warp][i][lane * E + e] = o[i][e];
-            if (lane == 0) {
-                mrg[warp][i][HD] = mx[i];
-                mrg[warp][i][HD + 1] = l[i];
+                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                if (m > -INFINITY) {
+                    pt = on ? expf(s - m) : 0.f;
+                    mx[pp] = m;
+                    ls[pp] = warp_sum(pt);
+                }
+            }
+            P_w[pp * 32 + lane] = pt;
+        }
+        __syncwarp();
+        // ---- out = sum_t p_t V_t: lane = channels lane*E .. lane*E+E-1 ----
+        float o[kPairGroup][E];
+#pragma unroll
+        for (int pp = 0; pp < kPairGroup; ++pp)
+#pragma unroll
+            for (int e = 0; e < E; ++e) o[pp][e] = 0.f;
+#pragma unroll 2
+        for (int t4 = 0; t4 < 8; ++t4) {
+            float vf[4][E];
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {
+                const T* vp = reinterpret_cast<const T*>(V_w + (t4 * 4 + tt) * ROWB) + lane * E;
+#pragma unroll
+                for (int e = 0; e < E; ++e) vf[tt][e] = to_f32(vp[e]);
+            }
+#pragma unroll
+            for (int pp = 0; pp < kPairGroup; ++pp) {
+                if (pg + pp < P) {
+                    float4 p4 = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        o[pp][e] = fmaf(p4.x, vf[0][e], o[pp][e]);
+                        o[pp][e] = fmaf(p4.y, vf[1][e], o[pp][e]);
+                        o[pp][e] = fmaf(p4.z, vf[2][e], o[pp][e]);
+                        o[pp][e] = fmaf(p4.w, vf[3][e], o[pp][e]);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int pp = 0; pp < kPairGroup; ++pp) {
+            if (pg + pp < P) {
+                float* dst = mrg + ((size_t)warp * P + pg + pp) * (HD + 2);
+#pragma unroll
+                for (int e = 0; e < E; ++e) dst[lane * E + e] = o[pp][e];
+                if (lane == 0) {
+                    dst[HD] = mx[pp];
+                    dst[HD + 1] = ls[pp];
+                }
             }
         }
     }
     __syncthreads();
-    // merge the four warps in warp order; thread -> (row, channel)
-    for (int idx = threadIdx.x; idx < a.m * HD; idx += blockDim.x) {
-        int i = idx / HD, e = idx - i * HD;
+    // merge the four warps in warp order; thread -> (pair, channel)
+    for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
+        int p = idx / HD, e = idx - p * HD;
+        int i = (p_lo + p) / G, g = (p_lo + p) - i * G;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, mrg[w][i][HD]);
+        for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, mrg[((size_t)w * P + p) * (HD + 2) + HD]);
         float L = 0.f, O = 0.f;
         if (M > -INFINITY) {
 #pragma unroll
             for (int w = 0; w < kAttnWarps; ++w) {
-                float mw = mrg[w][i][HD];
+                const float* src = mrg + ((size_t)w * P + p) * (HD + 2);
+                float mw = src[HD];
                 if (mw > -INFINITY) {
                     float f = expf(mw - M);
-                    L += mrg[w][i][HD + 1] * f;
-                    O += mrg[w][i][e] * f;
+                    L += src[HD + 1] * f;
+                    O += src[e] * f;
                 }
             }
         }
-        float* dst = a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + hq) * (HD + 2);
+        float* dst = a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
         dst[e] = O;
         if (e == 0) {
             dst[HD] = M;
@@ -252,29 +351,43 @@ __global__ void k_attn_combine(AttnArgs a) {
     pdl_wait();
     int hq = blockIdx.x, row = a.r0 + blockIdx.y, e = threadIdx.x;
     int hd = a.hd;
-    int n_chunks = (a.pos0 + row) / a.chunk + 1;   // chunks that hold positions <= this row's own
+    int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own
     float M = -INFINITY, L = 0.f, O = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
+#pragma unroll 8
+    for (int c = 0; c < n_chunks; ++c) {               // loads of different chunks are independent
         const float* src = a.part + (((size_t)c * kMaxW + row) * a.H + hq) * (hd + 2);
-        float mc = src[hd];
+        float mc = __ldcg(src + hd), lc = __ldcg(src + hd + 1), oc = __ldcg(src + e);
         if (mc == -INFINITY) continue;
         float nm = fmaxf(M, mc);
         float f0 = expf(M - nm), f1 = expf(mc - nm);
-        L = L * f0 + src[hd + 1] * f1;
-        O = O * f0 + src[e] * f1;
+        L = L * f0 + lc * f1;
+        O = O * f0 + oc * f1;
         M = nm;
     }
     using A = Act<T>;
     A::store(reinterpret_cast<typename A::type*>(a.act_out), row, hq * hd + e, a.H * hd, O / L);
 }
 
+template <typename T, int HD> static void launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid) {
+    const int P = a.m * (a.H / a.Hkv);
+    const int rowb = HD * (int)sizeof(T) + 16;
+    size_t smem = (size_t)P * HD * 4 + (size_t)kAttnWarps * 64 * rowb + (size_t)kAttnWarps * kPairGroup * 32 * 4 +
+                  (size_t)kAttnWarps * P * (HD + 2) * 4;
+    static size_t configured = 0;
+    if (smem > configured) {
+        cudaFuncSetAttribute(k_attn_partial<T, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
+        configured = 200 * 1024;
+    }
+    launch_k(k_attn_partial<T, HD>, grid, dim3(kAttnWarps * 32), smem, st, a);
+}
+
 template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) {
-    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / a.chunk + 1;
-    dim3 grid(a.H, n_chunks);
+    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
+    dim3 grid(a.Hkv, n_chunks);
     switch (a.hd) {
-        case 32: launch_k(k_attn_partial<T, 1>, grid, dim3(kAttnWarps * 32), 0, st, a); break;
-        case 64: launch_k(k_attn_partial<T, 2>, grid, dim3(kAttnWarps * 32), 0, st, a); break;
-        default: launch_k(k_attn_partial<T, 4>, grid, dim3(kAttnWarps * 32), 0, st, a); break;
+        case 32: launch_attn_partial<T, 32>(st, a, grid); break;
+        case 64: launch_attn_partial<T, 64>(st, a, grid); break;
+        default: launch_attn_partial<T, 128>(st, a, grid); break;
     }
     launch_k(k_attn_combine<T>, dim3(a.H, a.m), dim3(a.hd), 0, st, a);
 }
