@@ -214,8 +214,10 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                    and prints them to stderr; a profiling aid, off by default.
  *   SB_OPT_TC_TUNING (default option only) stages * 16 + CTAs per SM of the tcgen05 kernels.
  *   SB_OPT_PDL       (default option only) 1 (default) = launch kernels with programmatic dependent
- *                    launch so that a kernel's prologue and weight prefetch overlap its predecessor. */
-enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4 };
+ *                    launch so that a kernel's prologue and weight prefetch overlap its predecessor.
+ *   SB_OPT_L2_PREFETCH_KB (default option only) KB of weight tiles per CTA that a tcgen05 kernel prefetches
+ *                    into L2 while it still waits for its predecessor (default 128, 0 = off). */
+enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH_KB = 5 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);
 /* Process-wide default for contexts and stateless calls created afterwards. */
 int sb_set_default_option(int32_t key, int32_t value);

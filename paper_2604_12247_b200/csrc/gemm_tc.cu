@@ -34,7 +34,8 @@ constexpr int kTcThreads = (kProducers + 5) * 32;
 static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
 // Two CTAs per SM (each with its own producers, MMA issuer and TMEM accumulators) stream measurably
 // faster than one CTA with twice the pipeline depth.
-static int g_stages = 6, g_ctas_per_sm = 2;   // defaults; see tc_set_tuning
+static int g_stages = 6, g_ctas_per_sm = 2;
+static int g_l2_prefetch_kb = 128;   // per CTA, see tc_set_l2_prefetch   // defaults; see tc_set_tuning
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
 struct alignas(64) TcParams {
@@ -46,6 +47,7 @@ struct alignas(64) TcParams {
     int n_off[3];       // first output column of each matrix
     int n_chunks, R, S, KB, n_items;
     int stages;
+    int l2_fills;       // pipeline fills per producer that are prefetched into L2 while waiting for the predecessor
     float* out;
     int n_total;
     int r0, m;
@@ -276,6 +278,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 tma_load_2d_hint(smA + fill * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(fill), pol);
                 for (int j = 0; j < kProducers; ++j) w.next(p);
             }
+            // Still waiting for the predecessor kernel: HBM would sit idle.  Ask TMA to bring the next
+            // weight tiles of this producer into L2 (no shared memory, no barrier involved), so that
+            // the pipeline later refills from L2 instead of HBM.
+            {
+                WorkIter wl = w;
+                for (int j = 0; j < p.l2_fills && wl.valid(); ++j) {
+                    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(&p.tmA[wl.it.mat]),
+                                 "r"(wl.kb * kBK), "r"(wl.it.row0)
+                                 : "memory");
+                    for (int k = 0; k < kProducers; ++k) wl.next(p);
+                }
+            }
             pdl_wait();
             for (int f0 = warp; f0 < fill; f0 += kProducers) {
                 tma_load_2d(smB + f0 * kStageB, &p.tmB, w0.kb * kBK, 0, full_bar(f0));
@@ -482,7 +496,7 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     key.push_back((uint64_t)K);
     key.push_back((uint64_t)(uintptr_t)act);
     key.push_back(head ? 1 : 0);
-    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm);
+    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_l2_prefetch_kb << 16));
     auto it = cache->plans.find(key);
     if (it != cache->plans.end()) return it->second;
     TcPlan* pl = new TcPlan();
@@ -490,11 +504,13 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     TcParams& p = pl->p;
     int G = sm_count() * g_ctas_per_sm;
     p.stages = g_stages;
+    p.l2_fills = 0;   // set below once the slab height is known
     p.n_mats = n_mats;
     p.KB = (K + kBK - 1) / kBK;
     int prev = 0;
     for (int j = 0; j < n_mats; ++j) { p.n_rows[j] = n_end[j] - prev; p.n_off[j] = prev; prev = n_end[j]; }
     choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
+    p.l2_fills = (g_l2_prefetch_kb * 1024) / (p.R * kBK * 2) / kProducers;
     int chunks = 0;
     for (int j = 0; j < 3; ++j) {
         if (j < n_mats) chunks += (p.n_rows[j] + p.R - 1) / p.R;
@@ -517,6 +533,12 @@ template <bool kHead> static void launch(cudaStream_t st, const TcPlan* pl, cons
         g_attr_set[kHead] = true;
     }
     launch_k(k_tc<kHead>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages), st, p);
+}
+
+bool tc_set_l2_prefetch(int kb_per_cta) {
+    if (kb_per_cta < 0 || kb_per_cta > 4096) return false;
+    g_l2_prefetch_kb = kb_per_cta;
+    return true;
 }
 
 bool tc_set_tuning(int stages, int ctas_per_sm) {

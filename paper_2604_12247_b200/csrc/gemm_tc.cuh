@@ -9,7 +9,7 @@
 
 namespace sb {
 
-constexpr int kMaxSplit = 8;   // most split-K partials a GEMM may leave for its consumer
+constexpr int kMaxSplit = kMaxSplitK;   // most split-K partials a GEMM may leave for its consumer
 
 struct TcPlan;                 // tensor maps + work decomposition of one GEMM call shape
 struct TcPlanCache {
@@ -21,6 +21,8 @@ struct TcPlanCache {
 bool tc_available();
 // pipeline depth (2..12 stages of 18 KB) and persistent CTAs per SM (1..2) of the launches that follow
 bool tc_set_tuning(int stages, int ctas_per_sm);
+// KB of weight tiles per CTA that the producers prefetch into L2 while their kernel still waits for its predecessor
+bool tc_set_l2_prefetch(int kb_per_cta);
 // returns the number of split-K partials written to a.out, or -1 if no TMA descriptor could be made
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status);
 bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status);

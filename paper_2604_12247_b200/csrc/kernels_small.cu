@@ -53,10 +53,8 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
         if (k4 < nv) {
             v[j] = hr[k4];
             if (part) {
-                for (int s = 0; s < n_split; ++s) {   // summed in split order
-                    float4 p = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)s * kMaxW + row) * d) + k4);
-                    v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
-                }
+                float4 p = sum_splits4(reinterpret_cast<const float4*>(part + (size_t)row * d) + k4, (size_t)kMaxW * d / 4, n_split);
+                v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
                 hr[k4] = v[j];
             }
             ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
@@ -106,12 +104,9 @@ __global__ void k_rope_append(RopeArgs a) {
     int i = threadIdx.x;
     int qd = a.H * a.hd, kvd = a.Hkv * a.hd, ntot = qd + 2 * kvd;
     int col = head * a.hd;   // q heads, then k heads, then v heads are contiguous in the GEMM output
-    float x0 = 0.f, x1 = 0.f;
-    for (int s = 0; s < a.n_split; ++s) {
-        const float* p = a.qkv + ((size_t)s * kMaxW + row) * ntot + col;
-        x0 += p[i];
-        x1 += p[i + half];
-    }
+    const float* p0 = a.qkv + (size_t)row * ntot + col + i;
+    float x0 = sum_splits(p0, (size_t)kMaxW * ntot, a.n_split);
+    float x1 = sum_splits(p0 + half, (size_t)kMaxW * ntot, a.n_split);
     bool is_v = head >= a.H + a.Hkv;
     if (!is_v) {
         // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
@@ -402,12 +397,9 @@ __global__ void k_swiglu(const float* __restrict__ part, int n_split, int F, voi
     int row = r0 + blockIdx.y;
     int f = blockIdx.x * blockDim.x + threadIdx.x;
     if (f >= F) return;
-    float g = 0.f, u = 0.f;
-    for (int s = 0; s < n_split; ++s) {
-        const float* p = part + ((size_t)s * kMaxW + row) * (2 * (size_t)F);
-        g += p[f];
-        u += p[F + f];
-    }
+    const float* p0 = part + (size_t)row * (2 * (size_t)F) + f;
+    float g = sum_splits(p0, (size_t)kMaxW * 2 * F, n_split);
+    float u = sum_splits(p0 + F, (size_t)kMaxW * 2 * F, n_split);
     float v = g / (1.f + expf(-g)) * u;
     using A = Act<T>;
     A::store(reinterpret_cast<typename A::type*>(act), row, f, F, v);

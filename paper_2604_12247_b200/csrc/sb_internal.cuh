@@ -65,6 +65,30 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+constexpr int kMaxSplitK = 8;   // most split-K partials a GEMM leaves for its consumer (= kMaxSplit of the tcgen05 kernels)
+
+// Sum of the split-K partials of one output element, in split order.  All loads are issued before
+// the first add (fixed trip count, unused splits predicated off and contributing an exact 0), so a
+// consumer pays one L2 round trip instead of one per split.
+__device__ __forceinline__ float sum_splits(const float* __restrict__ first, size_t split_stride, int n_split) {
+    float v[kMaxSplitK];
+#pragma unroll
+    for (int s = 0; s < kMaxSplitK; ++s) v[s] = s < n_split ? __ldcg(first + (size_t)s * split_stride) : 0.f;
+    float acc = v[0];
+#pragma unroll
+    for (int s = 1; s < kMaxSplitK; ++s) acc += v[s];
+    return acc;
+}
+__device__ __forceinline__ float4 sum_splits4(const float4* __restrict__ first, size_t split_stride4, int n_split) {
+    float4 v[kMaxSplitK];
+#pragma unroll
+    for (int s = 0; s < kMaxSplitK; ++s) v[s] = s < n_split ? __ldcg(first + (size_t)s * split_stride4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc = v[0];
+#pragma unroll
+    for (int s = 1; s < kMaxSplitK; ++s) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
+    return acc;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
