@@ -39,6 +39,16 @@ METRIC = "batch-1 decode tokens/s (SpecBound, 7B shape)"
 NOMINAL_HBM_GBS = 8000.0
 
 
+def captured_traffic(key: str):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu capture
+    summaries, or None if there is none for this kernel."""
+    p = ROOT / "profiles" / "traffic.json"
+    try:
+        return json.loads(p.read_text()).get(key)
+    except Exception:
+        return None
+
+
 def measured_peak():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -142,9 +152,9 @@ def reference_arm(args, run: inputs.Run):
     vals, secs = [], []
     desc = None
     for _ in range(args.steps):
-        desc, dt = cpu_oracle_sample(run, w, 2, 3)
+        desc, dt = cpu_oracle_sample(run, w, 4, 28)   # 31 forward passes per step: about 10 s
         vals.append(desc["value"]); secs.append(dt)
-    v = sum(4 for _ in vals) / sum(secs)     # 4 forward passes per step
+    v = sum(31 for _ in vals) / sum(secs)    # 31 forward passes per step
     desc["value"] = v
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak",
@@ -240,13 +250,14 @@ def product_arm(args, run: inputs.Run):
                 "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "peak_source": peak_src, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
                 "bytes_per_launch": uni_bytes / max(uni_steps, 1), "us_per_launch": uni_us / max(uni_steps, 1),
-                "launches": uni_steps, "traffic": None}
+                "launches": uni_steps, "traffic": captured_traffic(f"layer_pass:{s.name}")}
     probes, probe_us = S("probes"), S("us_probe_kernels")
     ach_p = probes * wb["head"] / (probe_us * 1e-6) / 1e9 if probe_us > 0 else 0.0
     roofline_exit = {"kernel": "exit-confidence kernel (final RMSNorm'd row x LM head, fused temperature softmax max/argmax)",
                      "bound": "hbm", "achieved": ach_p, "peak": peak, "unit": "GB/s", "frac": ach_p / peak,
                      "frac_of_nominal_8TBs": ach_p / NOMINAL_HBM_GBS, "bytes_per_launch": wb["head"],
-                     "us_per_launch": probe_us / max(probes, 1), "launches": probes, "traffic": None}
+                     "us_per_launch": probe_us / max(probes, 1), "launches": probes,
+                     "traffic": captured_traffic(f"exit_confidence:{s.name}")}
     st0 = stats[-1]
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -274,7 +285,7 @@ def product_arm(args, run: inputs.Run):
         from oracle import oracle
         oracle.build()
         wc = inputs.weights_to(w, "cpu")
-        line["cpu_baseline"], _ = cpu_oracle_sample(run, wc, 2, 4)
+        line["cpu_baseline"], _ = cpu_oracle_sample(run, wc, 4, 40)   # 43 forward passes: about 10-30 s of CPU work
     print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
@@ -373,6 +384,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(inputs.RUNS))
     ap.add_argument("--n-gen", type=int, default=None, help="override the number of generated tokens")
+    ap.add_argument("--n-prompt", type=int, default=None, help="override the prompt length (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", action="store_true", help="kernel micro-benchmarks instead of the generation benchmark")
     ap.add_argument("--micro-case", default="", help="comma list, e.g. layer:w=4:S=512,exit:m=1:V=32000 (default: all)")
@@ -380,8 +392,9 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     run = inputs.RUNS[args.workload]
-    if args.n_gen:
-        run = inputs.Run(run.shape, run.n_prompt, args.n_gen, run.d_max, run.w_max, run.tau, run.threshold, run.seed, run.damp_rho)
+    if args.n_gen or args.n_prompt:
+        run = inputs.Run(run.shape, args.n_prompt or run.n_prompt, args.n_gen or run.n_gen, run.d_max, run.w_max, run.tau,
+                         run.threshold, run.seed, run.damp_rho)
     if args.micro:
         micro_arm(args)
     elif args.impl == "reference":
