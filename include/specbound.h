@@ -115,6 +115,11 @@ int sb_load_weights(sb_ctx* ctx, const sb_weights* w);
 /* Forget the sequence: n = 0, no pending token, no rows in flight.  KV pages stay allocated. */
 int sb_reset(sb_ctx* ctx);
 int sb_get_state(sb_ctx* ctx, sb_state* out);
+/* Self-test of the bounded device-side waits: launches one small kernel that waits, for at most
+ * about budget_ms (1..1000) milliseconds, on a barrier that nothing completes.  Returns
+ * SB_ERR_DEVICE_TIMEOUT when the wait gave up and the kernel returned normally (the expected
+ * outcome); the CUDA context stays usable, the status is cleared by the next sb_reset. */
+int sb_selftest_wait_timeout(sb_ctx* ctx, int32_t budget_ms);
 /* Copy the cached hidden state of in-flight row `row` (fp32 [d_model]) to host memory. */
 int sb_read_hidden(sb_ctx* ctx, int32_t row, float* host_out);
 

@@ -63,6 +63,7 @@ class SBError(RuntimeError):
 
 
 EXPORTS = ("sb_workspace_bytes", "sb_create", "sb_destroy", "sb_load_weights", "sb_reset", "sb_get_state",
+           "sb_selftest_wait_timeout",
            "sb_read_hidden", "sb_prefill", "sb_draft_push", "sb_draft_advance", "sb_exit_confidence", "sb_verify",
            "sb_generate", "sb_generate_ar", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
            "sb_k_layer",
@@ -89,6 +90,7 @@ def lib():
         L.sb_load_weights.argtypes = [vp, C.POINTER(Weights)]
         L.sb_reset.argtypes = [vp]
         L.sb_get_state.argtypes = [vp, C.POINTER(State)]
+        L.sb_selftest_wait_timeout.argtypes = [vp, i32]
         L.sb_read_hidden.argtypes = [vp, i32, vp]
         L.sb_prefill.argtypes = [vp, vp, i32, C.POINTER(i32)]
         L.sb_draft_push.argtypes = [vp, i32]
@@ -185,6 +187,10 @@ class Context:
 
     def reset(self):
         _check(lib().sb_reset(self.h), "sb_reset")
+
+    def selftest_wait_timeout(self, budget_ms: int = 20) -> int:
+        """Returns the status of a kernel whose bounded wait is made to run out (expected: -5)."""
+        return lib().sb_selftest_wait_timeout(self.h, budget_ms)
 
     def state(self) -> State:
         s = State()

@@ -432,7 +432,23 @@ int sb_reset(sb_ctx* c) {
     if (!c) return SB_ERR_ARG;
     c->n = 0; c->pending = -1; c->rows = 0;
     c->e.act_gain = nullptr;
+    // a sticky host error or an expired device wait of an earlier call is forgotten with the sequence
+    c->e.err = 0;
+    if (cudaMemsetAsync(c->e.W.status, 0, 64, c->e.st) != cudaSuccess) return SB_ERR_CUDA;
     return SB_OK;
+}
+
+int sb_selftest_wait_timeout(sb_ctx* c, int32_t budget_ms) {
+    if (!c || budget_ms < 1 || budget_ms > 1000) return SB_ERR_ARG;
+    // the kernel reports through the context's own status word and the last word of the result block
+    unsigned int* flag = reinterpret_cast<unsigned int*>(c->e.W.res) + 63;
+    cudaMemsetAsync(flag, 0, sizeof(unsigned int), c->e.st);
+    launch_wait_selftest(c->e.st, c->e.W.status, (unsigned long long)budget_ms * 2000000ull, flag);
+    int rc = fetch_results(c);   // SB_ERR_DEVICE_TIMEOUT when the wait gave up, as it must
+    unsigned int f = 0;
+    if (cudaMemcpy(&f, flag, sizeof(f), cudaMemcpyDeviceToHost) != cudaSuccess) return SB_ERR_CUDA;
+    if (rc == SB_ERR_DEVICE_TIMEOUT && f != 2u) return SB_ERR_STATE;
+    return rc;
 }
 
 int sb_get_state(sb_ctx* c, sb_state* out) {

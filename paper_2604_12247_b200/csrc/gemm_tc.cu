@@ -100,13 +100,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the abort flag + status word) if the budget runs out
 // or another role of this CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
-                                          unsigned int code) {
+                                          unsigned int code, unsigned long long budget = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > budget) {
             *abort_flag = 1;
             atomicExch(status, code);
             return false;
@@ -539,6 +539,26 @@ bool tc_set_l2_prefetch(int kb_per_cta) {
     if (kb_per_cta < 0 || kb_per_cta > 4096) return false;
     g_l2_prefetch_kb = kb_per_cta;
     return true;
+}
+
+// Self-test of the bounded wait: one CTA waits on an mbarrier that nothing ever completes, with a
+// small cycle budget.  The wait must give up, raise the status word and let the kernel return.
+__global__ void k_wait_selftest(unsigned int* status, unsigned long long budget_cycles, unsigned int* waited_flag) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ volatile int abort_s;
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool ok = mbar_wait(smem_u32(&bar), 0, &abort_s, status, 9u, budget_cycles);
+        *waited_flag = ok ? 1u : 2u;
+    }
+}
+void launch_wait_selftest(cudaStream_t st, unsigned int* status, unsigned long long budget_cycles, unsigned int* waited_flag) {
+    k_wait_selftest<<<1, 32, 0, st>>>(status, budget_cycles, waited_flag);
 }
 
 bool tc_set_tuning(int stages, int ctas_per_sm) {

@@ -19,6 +19,8 @@ struct TcPlanCache {
 };
 
 bool tc_available();
+// one CTA waits (bounded by budget_cycles) on a barrier nothing completes; status receives code 9, waited_flag 2
+void launch_wait_selftest(cudaStream_t st, unsigned int* status, unsigned long long budget_cycles, unsigned int* waited_flag);
 // pipeline depth (2..12 stages of 18 KB) and persistent CTAs per SM (1..2) of the launches that follow
 bool tc_set_tuning(int stages, int ctas_per_sm);
 // KB of weight tiles per CTA that the producers prefetch into L2 while their kernel still waits for its predecessor

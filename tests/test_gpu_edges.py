@@ -98,3 +98,22 @@ def test_context_reuse_across_sequences(tiny_damped_weights):
         assert np.array_equal(ctx.generate(pr, n_gen, 2, 4, (1.5, 1.0), 0.3)["tokens"], ref)
         assert np.array_equal(ctx.generate_ar(pr, n_gen)["tokens"], ref)
     ctx.close()
+
+
+def test_bounded_device_wait_runs_out_and_context_survives(tiny_damped_weights):
+    """Failure detection without a GPU fault: a wait on a barrier that nothing completes gives up
+    after its budget, the kernel returns, the call reports SB_ERR_DEVICE_TIMEOUT, later calls keep
+    reporting it until sb_reset, and the context then works as before."""
+    run = inputs.RUNS["tiny-damped"]
+    pr = inputs.make_prompt(run.shape, 6, 4).numpy()
+    ctx, _ = gpu_ctx(run.shape, tiny_damped_weights, 48)
+    ref = ctx.generate_ar(pr, 6)["tokens"]
+    assert ctx.selftest_wait_timeout(20) == -5
+    ctx.draft_push(1)                                # launches only; the next call that reads a result sees the status
+    ctx.draft_advance(1)
+    with pytest.raises(binding.SBError) as e:        # the status word is sticky until the sequence is reset
+        ctx.exit_confidence(1, 1.0, 0.5)
+    assert e.value.status == -5
+    ctx.reset()
+    assert np.array_equal(ctx.generate_ar(pr, 6)["tokens"], ref)
+    ctx.close()
