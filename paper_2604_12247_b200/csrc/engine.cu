@@ -16,6 +16,14 @@ namespace sb {
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
 static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
 
+// TMA descriptors of the stateless entry points: keyed by (pointers, shapes), so they stay valid for as
+// long as the key matches; kept across calls because encoding them costs more host time than the launch.
+static TcPlanCache& stateless_plans() {
+    static TcPlanCache cache;
+    if (cache.plans.size() > 512) cache.clear();
+    return cache;
+}
+
 struct Tracer {
     static constexpr int kMax = 64;
     cudaEvent_t ev[kMax];
@@ -778,8 +786,7 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     e.st = (cudaStream_t)stream;
     carve(D, (char*)scratch, false, &e.W);
     e.gemm = pick_gemm(D.f32);
-    TcPlanCache plans;
-    e.plans = &plans;
+    e.plans = &stateless_plans();
     cudaMemsetAsync(e.W.ticket, 0, 64, e.st);
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
     cudaMemcpyAsync(e.W.h, h, sizeof(float) * m * D.d, cudaMemcpyDeviceToDevice, e.st);
@@ -808,8 +815,7 @@ int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, 
     e.W = Work{};
     carve_exit_only(D, base, &e.W);
     e.gemm = pick_gemm(D.f32);
-    TcPlanCache plans;
-    e.plans = &plans;
+    e.plans = &stateless_plans();
     // the array keeps whatever the previous call left: the ticket and the status word must start at zero
     cudaMemsetAsync(e.W.ticket, 0, 64, e.st);
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
@@ -840,8 +846,7 @@ int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_
     e.W.page_table = const_cast<int*>(page_table);
     e.W.h = reinterpret_cast<float*>(h);   // rows 0..m-1 of the caller's buffer are the hidden cache
     e.gemm = pick_gemm(D.f32);
-    TcPlanCache plans;
-    e.plans = &plans;
+    e.plans = &stateless_plans();
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
     if (g_trace) g_tracer.begin(e.st);
     layer_step(e, *lw, k_cache, v_cache, 0, m, first_pos, nullptr);

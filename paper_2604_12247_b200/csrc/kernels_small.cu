@@ -44,14 +44,15 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
     int row = r0 + blockIdx.x;
     float4* hr = reinterpret_cast<float4*>(h + (size_t)row * d);
     const int nv = d >> 2;
-    float4 v[kNormVec];
+    float4 v[kNormVec], g4[kNormVec];
     float ss = 0.f;
-    // every load of a thread is independent: the hidden row and all partials are in flight at once
+    // every load of a thread is independent: the hidden row, all partials and the gains are in flight at once
 #pragma unroll
     for (int j = 0; j < kNormVec; ++j) {
         int k4 = threadIdx.x + j * kNormThreads;
         if (k4 < nv) {
             v[j] = hr[k4];
+            if (gain) g4[j] = load_gain4(gain, k4 << 2);
             if (part) {
                 float4 p = sum_splits4(reinterpret_cast<const float4*>(part + (size_t)row * d) + k4, (size_t)kMaxW * d / 4, n_split);
                 v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
@@ -73,13 +74,9 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
 #pragma unroll
     for (int j = 0; j < kNormVec; ++j) {
         int k4 = threadIdx.x + j * kNormThreads;
-        if (k4 < nv) {
-            int k = k4 << 2;
-            A::store(a, row, k, d, v[j].x * inv * to_f32(gain[k]));
-            A::store(a, row, k + 1, d, v[j].y * inv * to_f32(gain[k + 1]));
-            A::store(a, row, k + 2, d, v[j].z * inv * to_f32(gain[k + 2]));
-            A::store(a, row, k + 3, d, v[j].w * inv * to_f32(gain[k + 3]));
-        }
+        if (k4 < nv)
+            A::store4(a, row, k4 << 2, d, make_float4(v[j].x * inv * g4[j].x, v[j].y * inv * g4[j].y, v[j].z * inv * g4[j].z,
+                                                     v[j].w * inv * g4[j].w));
     }
 }
 template <typename T>
@@ -151,7 +148,7 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 // ------------------------------------------------------------------------------------------------
 constexpr int kAttnWarps = 4;
 constexpr int kAttnChunk = 128;
-constexpr int kPairGroup = 8;
+constexpr int kMaxPairGroup = 8;
 
 template <typename T> __device__ __forceinline__ void unpack16(const uint4& u, float (&f)[16 / sizeof(T)]);
 template <> __device__ __forceinline__ void unpack16<float>(const uint4& u, float (&f)[4]) {
@@ -166,8 +163,11 @@ template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4&
     }
 }
 
-template <typename T, int HD>
+// PG = (row, query head) pairs handled per sweep over the staged tile: the largest of 8, 4, 2, 1 that
+// divides the pair count, so that the inner loops carry no run-time predicates.
+template <typename T, int HD, int PG>
 __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
+    constexpr int kPairGroup = PG;
     constexpr int E = HD / 32;                       // channels per lane in P.V
     constexpr int EPP = 16 / (int)sizeof(T);         // elements per 16-byte piece
     constexpr int PPR = HD / EPP;                    // pieces per K/V row
@@ -178,18 +178,17 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     const int kvh = blockIdx.x, c = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
-    constexpr int p_lo = 0;
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD]
     unsigned char* kv_s = smem + (size_t)P * HD * 4;                                // per warp: K[32], V[32]
     unsigned char* K_w = kv_s + (size_t)warp * 64 * ROWB;
     unsigned char* V_w = K_w + 32 * ROWB;
-    float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + warp * kPairGroup * 32;   // [8][32]
-    float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + kAttnWarps * kPairGroup * 32;   // [4][P][HD+2]
+    float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + warp * kMaxPairGroup * 32;   // [PG][32]
+    float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + kAttnWarps * kMaxPairGroup * 32;   // [4][P][HD+2]
 
     for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
         int p = idx / HD, e = idx - p * HD;
-        int i = (p_lo + p) / G, g = (p_lo + p) - i * G;
+        int i = p / G, g = p - i * G;
         q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
     }
     const int pos_last = a.pos0 + a.r0 + a.m - 1;
@@ -230,16 +229,14 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
             unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB + piece * 16), kf);
 #pragma unroll
             for (int pp = 0; pp < kPairGroup; ++pp) {
-                if (pg + pp < P) {
-                    const float4* qv = reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP);
+                const float4* qv = reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP);
 #pragma unroll
-                    for (int v4 = 0; v4 < EPP / 4; ++v4) {
-                        float4 qq = qv[v4];
-                        sc[pp] = fmaf(qq.x, kf[4 * v4], sc[pp]);
-                        sc[pp] = fmaf(qq.y, kf[4 * v4 + 1], sc[pp]);
-                        sc[pp] = fmaf(qq.z, kf[4 * v4 + 2], sc[pp]);
-                        sc[pp] = fmaf(qq.w, kf[4 * v4 + 3], sc[pp]);
-                    }
+                for (int v4 = 0; v4 < EPP / 4; ++v4) {
+                    float4 qq = qv[v4];
+                    sc[pp] = fmaf(qq.x, kf[4 * v4], sc[pp]);
+                    sc[pp] = fmaf(qq.y, kf[4 * v4 + 1], sc[pp]);
+                    sc[pp] = fmaf(qq.z, kf[4 * v4 + 2], sc[pp]);
+                    sc[pp] = fmaf(qq.w, kf[4 * v4 + 3], sc[pp]);
                 }
             }
         }
@@ -250,18 +247,16 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
             mx[pp] = -INFINITY;
             ls[pp] = 0.f;
             float pt = 0.f;
-            if (pg + pp < P) {
-                int i = (p_lo + pg + pp) / G;
-                bool on = my_t <= a.pos0 + a.r0 + i;     // causal: a row sees positions <= its own
-                float s = on ? sc[pp] * scale : -INFINITY;
-                float m = s;
+            int i = (pg + pp) / G;
+            bool on = my_t <= a.pos0 + a.r0 + i;         // causal: a row sees positions <= its own
+            float s = on ? sc[pp] * scale : -INFINITY;
+            float m = s;
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                if (m > -INFINITY) {
-                    pt = on ? expf(s - m) : 0.f;
-                    mx[pp] = m;
-                    ls[pp] = warp_sum(pt);
-                }
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            if (m > -INFINITY) {
+                pt = on ? expf(s - m) : 0.f;
+                mx[pp] = m;
+                ls[pp] = warp_sum(pt);
             }
             P_w[pp * 32 + lane] = pt;
         }
@@ -283,29 +278,25 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
             }
 #pragma unroll
             for (int pp = 0; pp < kPairGroup; ++pp) {
-                if (pg + pp < P) {
-                    float4 p4 = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
+                float4 p4 = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) {
-                        o[pp][e] = fmaf(p4.x, vf[0][e], o[pp][e]);
-                        o[pp][e] = fmaf(p4.y, vf[1][e], o[pp][e]);
-                        o[pp][e] = fmaf(p4.z, vf[2][e], o[pp][e]);
-                        o[pp][e] = fmaf(p4.w, vf[3][e], o[pp][e]);
-                    }
+                for (int e = 0; e < E; ++e) {
+                    o[pp][e] = fmaf(p4.x, vf[0][e], o[pp][e]);
+                    o[pp][e] = fmaf(p4.y, vf[1][e], o[pp][e]);
+                    o[pp][e] = fmaf(p4.z, vf[2][e], o[pp][e]);
+                    o[pp][e] = fmaf(p4.w, vf[3][e], o[pp][e]);
                 }
             }
         }
         __syncwarp();
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
-            if (pg + pp < P) {
-                float* dst = mrg + ((size_t)warp * P + pg + pp) * (HD + 2);
+            float* dst = mrg + ((size_t)warp * P + pg + pp) * (HD + 2);
 #pragma unroll
-                for (int e = 0; e < E; ++e) dst[lane * E + e] = o[pp][e];
-                if (lane == 0) {
-                    dst[HD] = mx[pp];
-                    dst[HD + 1] = ls[pp];
-                }
+            for (int e = 0; e < E; ++e) dst[lane * E + e] = o[pp][e];
+            if (lane == 0) {
+                dst[HD] = mx[pp];
+                dst[HD + 1] = ls[pp];
             }
         }
     }
@@ -313,7 +304,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     // merge the four warps in warp order; thread -> (pair, channel)
     for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
         int p = idx / HD, e = idx - p * HD;
-        int i = (p_lo + p) / G, g = (p_lo + p) - i * G;
+        int i = p / G, g = p - i * G;
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, mrg[((size_t)w * P + p) * (HD + 2) + HD]);
@@ -363,17 +354,23 @@ __global__ void k_attn_combine(AttnArgs a) {
     A::store(reinterpret_cast<typename A::type*>(a.act_out), row, hq * hd + e, a.H * hd, O / L);
 }
 
+template <typename T, int HD, int PG> static void launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem) {
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(k_attn_partial<T, HD, PG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
+        configured = true;
+    }
+    launch_k(k_attn_partial<T, HD, PG>, grid, dim3(kAttnWarps * 32), smem, st, a);
+}
 template <typename T, int HD> static void launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid) {
     const int P = a.m * (a.H / a.Hkv);
     const int rowb = HD * (int)sizeof(T) + 16;
-    size_t smem = (size_t)P * HD * 4 + (size_t)kAttnWarps * 64 * rowb + (size_t)kAttnWarps * kPairGroup * 32 * 4 +
+    size_t smem = (size_t)P * HD * 4 + (size_t)kAttnWarps * 64 * rowb + (size_t)kAttnWarps * kMaxPairGroup * 32 * 4 +
                   (size_t)kAttnWarps * P * (HD + 2) * 4;
-    static size_t configured = 0;
-    if (smem > configured) {
-        cudaFuncSetAttribute(k_attn_partial<T, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
-        configured = 200 * 1024;
-    }
-    launch_k(k_attn_partial<T, HD>, grid, dim3(kAttnWarps * 32), smem, st, a);
+    if (P % 8 == 0) launch_attn_pg<T, HD, 8>(st, a, grid, smem);
+    else if (P % 4 == 0) launch_attn_pg<T, HD, 4>(st, a, grid, smem);
+    else if (P % 2 == 0) launch_attn_pg<T, HD, 2>(st, a, grid, smem);
+    else launch_attn_pg<T, HD, 1>(st, a, grid, smem);
 }
 
 template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) {

@@ -24,7 +24,18 @@ template <> struct Act<float> {
     static constexpr int rows = 8;
     __device__ static void store(float* a, int row, int k, int K, float v) { a[(size_t)row * K + k] = v; }
     __device__ static float load(const float* a, int row, int k, int K) { return a[(size_t)row * K + k]; }
+    __device__ static void store4(float* a, int row, int k, int K, float4 v) {
+        *reinterpret_cast<float4*>(a + (size_t)row * K + k) = v;
+    }
 };
+
+// four consecutive gains as floats (k a multiple of 4)
+__device__ __forceinline__ float4 load_gain4(const float* g, int k) { return *reinterpret_cast<const float4*>(g + k); }
+__device__ __forceinline__ float4 load_gain4(const __nv_bfloat16* g, int k) {
+    uint2 u = *reinterpret_cast<const uint2*>(g + k);
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xffff0000u));
+}
 template <> struct Act<__nv_bfloat16> {
     using type = __nv_bfloat16;
     static constexpr int rows = 16;
@@ -35,6 +46,21 @@ template <> struct Act<__nv_bfloat16> {
     }
     __device__ static float load(const __nv_bfloat16* a, int row, int k, int K) {
         return __bfloat162float(a[(size_t)row * K + k]) + __bfloat162float(a[(size_t)(row + 8) * K + k]);
+    }
+    // four consecutive values (k a multiple of 4): one 8-byte store for the high halves, one for the low halves
+    __device__ static void store4(__nv_bfloat16* a, int row, int k, int K, float4 v) {
+        __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y), h2 = __float2bfloat16_rn(v.z),
+                      h3 = __float2bfloat16_rn(v.w);
+        __nv_bfloat162 hi01 = __halves2bfloat162(h0, h1), hi23 = __halves2bfloat162(h2, h3);
+        __nv_bfloat162 lo01 = __halves2bfloat162(__float2bfloat16_rn(v.x - __bfloat162float(h0)),
+                                                 __float2bfloat16_rn(v.y - __bfloat162float(h1)));
+        __nv_bfloat162 lo23 = __halves2bfloat162(__float2bfloat16_rn(v.z - __bfloat162float(h2)),
+                                                 __float2bfloat16_rn(v.w - __bfloat162float(h3)));
+        uint2 hp, lp;
+        hp.x = *reinterpret_cast<unsigned int*>(&hi01); hp.y = *reinterpret_cast<unsigned int*>(&hi23);
+        lp.x = *reinterpret_cast<unsigned int*>(&lo01); lp.y = *reinterpret_cast<unsigned int*>(&lo23);
+        *reinterpret_cast<uint2*>(a + (size_t)row * K + k) = hp;
+        *reinterpret_cast<uint2*>(a + (size_t)(row + 8) * K + k) = lp;
     }
 };
 
@@ -56,6 +82,16 @@ inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_use_pdl ? 1 : 0;
+    // every kernel asks for the same (maximal) shared-memory carve-out: an SM never has to drain to
+    // change its L1/shared split between two kernels of the chain
+    static void* seen[32];
+    static int n_seen = 0;
+    bool known = false;
+    for (int i = 0; i < n_seen; ++i) known |= seen[i] == (void*)kernel;
+    if (!known) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (n_seen < 32) seen[n_seen++] = (void*)kernel;
+    }
     cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
