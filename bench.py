@@ -389,12 +389,20 @@ def main():
     ap.add_argument("--micro", action="store_true", help="kernel micro-benchmarks instead of the generation benchmark")
     ap.add_argument("--micro-case", default="", help="comma list, e.g. layer:w=4:S=512,exit:m=1:V=32000 (default: all)")
     ap.add_argument("--iters", type=int, default=40)
+    ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
+                    help="library option set before the run (sb_set_default_option), e.g. 6=10; for tuning sweeps")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     run = inputs.RUNS[args.workload]
     if args.n_gen or args.n_prompt:
         run = inputs.Run(run.shape, args.n_prompt or run.n_prompt, args.n_gen or run.n_gen, run.d_max, run.w_max, run.tau,
                          run.threshold, run.seed, run.damp_rho)
+    if args.tune and args.impl == "ours":
+        from paper_2604_12247_b200 import binding, build
+        build.build()
+        for kv in args.tune:
+            k, v = kv.split("=")
+            assert binding.lib().sb_set_default_option(int(k), int(v)) == 0, kv
     if args.micro:
         micro_arm(args)
     elif args.impl == "reference":

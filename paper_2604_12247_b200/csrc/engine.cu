@@ -488,6 +488,7 @@ int sb_set_option(sb_ctx* c, int32_t key, int32_t value) {
 int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_TRACE) { g_trace = value != 0; return SB_OK; }
     if (key == SB_OPT_L2_PREFETCH_KB) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
+    if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_GEMM && (value == 0 || value == 1 || value == -1)) {

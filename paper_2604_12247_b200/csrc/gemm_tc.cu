@@ -35,6 +35,7 @@ static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /
 // Two CTAs per SM (each with its own producers, MMA issuer and TMEM accumulators) stream measurably
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;
+static int g_split_penalty_pm = 10;  // cost of one more k split, per mille of the streaming time (see choose_split)
 static int g_l2_prefetch_kb = 128;   // per CTA, see tc_set_l2_prefetch   // defaults; see tc_set_tuning
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
@@ -482,7 +483,7 @@ static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, i
             for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + R - 1) / R;
             long long items = chunks * S;
             long long per = (items + G - 1) / G;
-            double cost = (double)per * R * ((KB + S - 1) / S) * (1.0 + 0.004 * S);   // mild preference for few splits
+            double cost = (double)per * R * ((KB + S - 1) / S) * (1.0 + 0.001 * g_split_penalty_pm * S);   // each split adds partial traffic and consumer loads
             if (cost < best - 1e-9) { best = cost; bR = R; bS = S; }
         }
     *R_out = bR;
@@ -496,7 +497,7 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     key.push_back((uint64_t)K);
     key.push_back((uint64_t)(uintptr_t)act);
     key.push_back(head ? 1 : 0);
-    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_l2_prefetch_kb << 16));
+    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_l2_prefetch_kb << 16) + ((uint64_t)g_split_penalty_pm << 40));
     auto it = cache->plans.find(key);
     if (it != cache->plans.end()) return it->second;
     TcPlan* pl = new TcPlan();
@@ -533,6 +534,12 @@ template <bool kHead> static void launch(cudaStream_t st, const TcPlan* pl, cons
         g_attr_set[kHead] = true;
     }
     launch_k(k_tc<kHead>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages), st, p);
+}
+
+bool tc_set_split_penalty(int per_mille) {
+    if (per_mille < 0 || per_mille > 1000) return false;
+    g_split_penalty_pm = per_mille;
+    return true;
 }
 
 bool tc_set_l2_prefetch(int kb_per_cta) {

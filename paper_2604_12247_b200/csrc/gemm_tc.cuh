@@ -25,6 +25,8 @@ void launch_wait_selftest(cudaStream_t st, unsigned int* status, unsigned long l
 bool tc_set_tuning(int stages, int ctas_per_sm);
 // KB of weight tiles per CTA that the producers prefetch into L2 while their kernel still waits for its predecessor
 bool tc_set_l2_prefetch(int kb_per_cta);
+// cost the host's work decomposition charges for each additional k split, per mille of the streaming time
+bool tc_set_split_penalty(int per_mille);
 // returns the number of split-K partials written to a.out, or -1 if no TMA descriptor could be made
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status);
 bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status);
