@@ -221,7 +221,7 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *   SB_OPT_PDL       (default option only) 1 (default) = launch kernels with programmatic dependent
  *                    launch so that a kernel's prologue and weight prefetch overlap its predecessor.
  *   SB_OPT_L2_PREFETCH_KB (default option only) KB of weight tiles per CTA that a tcgen05 kernel prefetches
- *                    into L2 while it still waits for its predecessor (default 128, 0 = off).
+ *                    into L2 while it still waits for its predecessor (default 0 = off).
  *   SB_OPT_SPLIT_PENALTY (default option only) what the work decomposition charges per additional k split,
  *                    in per mille of the streaming time (more splits balance the CTAs better but cost
  *                    partial-sum traffic and consumer loads). */

@@ -36,7 +36,7 @@ static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;
 static int g_split_penalty_pm = 10;  // cost of one more k split, per mille of the streaming time (see choose_split)
-static int g_l2_prefetch_kb = 128;   // per CTA, see tc_set_l2_prefetch   // defaults; see tc_set_tuning
+static int g_l2_prefetch_kb = 0;     // per CTA, see tc_set_l2_prefetch (off: inside the decode loop it slowed the layer pass by 2 %)
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
 struct alignas(64) TcParams {
