@@ -339,16 +339,27 @@ __global__ void k_attn_combine(AttnArgs a) {
     int hd = a.hd;
     int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own
     float M = -INFINITY, L = 0.f, O = 0.f;
-#pragma unroll 8
-    for (int c = 0; c < n_chunks; ++c) {               // loads of different chunks are independent
-        const float* src = a.part + (((size_t)c * kMaxW + row) * a.H + hq) * (hd + 2);
-        float mc = __ldcg(src + hd), lc = __ldcg(src + hd + 1), oc = __ldcg(src + e);
-        if (mc == -INFINITY) continue;
-        float nm = fmaxf(M, mc);
-        float f0 = expf(M - nm), f1 = expf(mc - nm);
-        L = L * f0 + lc * f1;
-        O = O * f0 + oc * f1;
-        M = nm;
+    constexpr int kBatch = 8;   // chunks whose partials are loaded together (one L2 round trip per batch)
+    for (int c0 = 0; c0 < n_chunks; c0 += kBatch) {
+        float mc[kBatch], lc[kBatch], oc[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const bool ok = c0 + u < n_chunks;
+            const float* src = a.part + (((size_t)(ok ? c0 + u : 0) * kMaxW + row) * a.H + hq) * (hd + 2);
+            mc[u] = ok ? __ldcg(src + hd) : -INFINITY;
+            lc[u] = ok ? __ldcg(src + hd + 1) : 0.f;
+            oc[u] = ok ? __ldcg(src + e) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            if (mc[u] > -INFINITY) {
+                float nm = fmaxf(M, mc[u]);
+                float f0 = expf(M - nm), f1 = expf(mc[u] - nm);
+                L = L * f0 + lc[u] * f1;
+                O = O * f0 + oc[u] * f1;
+                M = nm;
+            }
+        }
     }
     using A = Act<T>;
     A::store(reinterpret_cast<typename A::type*>(a.act_out), row, hq * hd + e, a.H * hd, O / L);
