@@ -220,13 +220,19 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *   SB_OPT_TC_TUNING (default option only) stages * 16 + CTAs per SM of the tcgen05 kernels.
  *   SB_OPT_PDL       (default option only) 1 (default) = launch kernels with programmatic dependent
  *                    launch so that a kernel's prologue and weight prefetch overlap its predecessor.
- *   SB_OPT_L2_PREFETCH_KB (default option only) KB of weight tiles per CTA that a tcgen05 kernel prefetches
- *                    into L2 while it still waits for its predecessor (default 0 = off).
+ *   SB_OPT_L2_PREFETCH (default option only) n > 0: while the output projection waits for the attention
+ *                    kernels (HBM idle), it prefetches every n-th k block of the layer's gate/up weights
+ *                    into L2; 0 = off.  Default 5.  Needs SB_OPT_FUSE = 1.
  *   SB_OPT_SPLIT_PENALTY (default option only) what the work decomposition charges per additional k split,
  *                    in per mille of the streaming time (more splits balance the CTAs better but cost
- *                    partial-sum traffic and consumer loads). */
-enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH_KB = 5,
-       SB_OPT_SPLIT_PENALTY = 6 };
+ *                    partial-sum traffic and consumer loads).
+ *   SB_OPT_FUSE      (default option only) 1 (default) = the tcgen05 gate/up GEMM pairs gate and up rows in
+ *                    one tile and its epilogue writes SwiGLU as the down projection's operand; 0 = SwiGLU is
+ *                    a kernel of its own.  The fused GEMM is never split along k, so its sums may round
+ *                    differently from the separate kernels' (fp32 rounding level); each setting by itself
+ *                    is deterministic and row-invariant. */
+enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,
+       SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);
 /* Process-wide default for contexts and stateless calls created afterwards. */
 int sb_set_default_option(int32_t key, int32_t value);

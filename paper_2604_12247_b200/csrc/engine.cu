@@ -14,6 +14,7 @@
 namespace sb {
 
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
+static int g_fuse = 1;            // bit 0: SwiGLU in the epilogue of the tcgen05 gate/up GEMM instead of a kernel of its own
 static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
 
 // TMA descriptors of the stateless entry points: keyed by (pointers, shapes), so they stay valid for as
@@ -184,8 +185,13 @@ static void ensure_act(Exec& e, const void* gain, int r0, int m) {
 }
 
 // out = act x W^T for up to three matrices; returns the number of split-K partials written
-static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, const void* act, float* out, int r0, int m) {
+static bool tc_path(const Exec& e) { return e.gemm == 1 && !e.D.f32; }
+struct NextGemm { const void* W[2] = {nullptr, nullptr}; int rows = 0, K = 0; const void* act = nullptr; };
+static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, const void* act, float* out, int r0, int m,
+                void* swiglu_out = nullptr, const NextGemm& next = NextGemm()) {
     GemmArgs a{};
+    a.swiglu_out = swiglu_out;
+    a.next_W[0] = next.W[0]; a.next_W[1] = next.W[1]; a.next_rows = next.rows; a.next_K = next.K; a.next_act = next.act;
     int tot = 0;
     for (int j = 0; j < n_mats; ++j) { a.W[j] = W[j]; tot += N[j]; a.n_end[j] = tot; }
     for (int j = n_mats; j < 3; ++j) { a.W[j] = nullptr; a.n_end[j] = 0x7fffffff; }
@@ -224,23 +230,33 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     e.launches += 3;
     const void* wo[1] = {lw.wo};
     int no[1] = {D.d};
-    int s_o = gemm(e, wo, no, 1, D.qd, W.act_o, W.p_o, r0, m);
+    // the output projection waits through the whole attention chain with HBM idle: it announces the
+    // gate/up GEMM so that part of those weights is already in L2 when their turn comes
+    NextGemm nx;
+    if (tc_path(e) && (g_fuse & 1)) { nx.W[0] = lw.w_gate; nx.W[1] = lw.w_up; nx.rows = D.F; nx.K = D.d; nx.act = W.act_a; }
+    int s_o = gemm(e, wo, no, 1, D.qd, W.act_o, W.p_o, r0, m, nullptr, nx);
     SB_MARK("o");
     SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_o, s_o, D.d, (const T*)lw.mlp_norm, D.eps, W.act_a, r0, m));
     SB_MARK("norm2");
     const void* wgu[2] = {lw.w_gate, lw.w_up};
     int ngu[2] = {D.F, D.F};
-    int s_gu = gemm(e, wgu, ngu, 2, D.d, W.act_a, W.p_gu, r0, m);
-    SB_MARK("gateup");
-    SB_T(e, launch_swiglu<T>(e.st, W.p_gu, s_gu, D.F, W.act_f, r0, m));
-    SB_MARK("swiglu");
+    if (tc_path(e) && (g_fuse & 1)) {   // SwiGLU in the gate/up GEMM's epilogue: act_f comes straight out of it
+        gemm(e, wgu, ngu, 2, D.d, W.act_a, W.p_gu, r0, m, W.act_f);
+        SB_MARK("gateup");
+    } else {
+        int s_gu = gemm(e, wgu, ngu, 2, D.d, W.act_a, W.p_gu, r0, m);
+        SB_MARK("gateup");
+        SB_T(e, launch_swiglu<T>(e.st, W.p_gu, s_gu, D.F, W.act_f, r0, m));
+        e.launches++;
+        SB_MARK("swiglu");
+    }
     const void* wd[1] = {lw.w_down};
     int nd[1] = {D.d};
     int s_d = gemm(e, wd, nd, 1, D.F, W.act_f, W.p_down, r0, m);
     SB_MARK("down");
     SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_down, s_d, D.d, (const T*)next_gain, D.eps, W.act_a, r0, m));
     SB_MARK("resid");
-    e.launches += 3;
+    e.launches += 2;
     e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
 }
 
@@ -487,9 +503,10 @@ int sb_set_option(sb_ctx* c, int32_t key, int32_t value) {
 
 int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_TRACE) { g_trace = value != 0; return SB_OK; }
-    if (key == SB_OPT_L2_PREFETCH_KB) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
+    if (key == SB_OPT_L2_PREFETCH) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
+    if (key == SB_OPT_FUSE) { if (value < 0 || value > 1) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_GEMM && (value == 0 || value == 1 || value == -1)) {
         if (value == 1 && !tc_available()) return SB_ERR_UNSUPPORTED;

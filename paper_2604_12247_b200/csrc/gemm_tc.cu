@@ -36,7 +36,7 @@ static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;
 static int g_split_penalty_pm = 10;  // cost of one more k split, per mille of the streaming time (see choose_split)
-static int g_l2_prefetch_kb = 0;     // per CTA, see tc_set_l2_prefetch (off: inside the decode loop it slowed the layer pass by 2 %)
+static int g_l2_next_every = 5;      // see tc_set_l2_prefetch: every n-th k block of the announced GEMM goes to L2 early (0 = off)
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
 struct alignas(64) TcParams {
@@ -48,10 +48,15 @@ struct alignas(64) TcParams {
     int n_off[3];       // first output column of each matrix
     int n_chunks, R, S, KB, n_items;
     int stages;
-    int l2_fills;       // pipeline fills per producer that are prefetched into L2 while waiting for the predecessor
+    // L2 prefetch on behalf of a later (pair mode) GEMM whose weights this kernel's idle wait can hide
+    CUtensorMap tmN[2];
+    int next_half, next_chunks, next_KB, next_every;   // next_every = 0: none
     float* out;
     int n_total;
     int r0, m;
+    // gate/up pair mode: every work item is half gate rows (tile rows 0 ..), half up rows (tile rows 64 ..)
+    int pair_half;              // rows of each kind per item (<= 64)
+    __nv_bfloat16* swiglu_out;  // [16][n_rows[0]]: high halves in rows 0-7, low halves in rows 8-15
     // LM-head mode
     float inv_tau, threshold;
     float* conf;
@@ -189,6 +194,7 @@ struct ItemInfo {
 };
 __device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
     int chunk = item % p.n_chunks, s = item / p.n_chunks;
+    if (p.pair_half) return ItemInfo{0, chunk * p.pair_half, 0, p.KB};   // never split along k
     int j = 0, base = 0;
     while (j < p.n_mats - 1 && chunk >= p.chunk_end[j]) base = p.chunk_end[j++];
     ItemInfo it;
@@ -218,13 +224,14 @@ struct WorkIter {
     }
 };
 
-template <bool kHead>
+template <bool kHead, bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_s;
     __shared__ SoftTriple cta_part[4][kMaxW];
     __shared__ bool is_last_s;
+    __shared__ float up_s[kPair ? kMaxW * 64 : 1];   // pair mode: the up projections of an item, [row][column in item]
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
@@ -271,25 +278,37 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
             }
             const uint64_t pol = policy_evict_first();
+            // weight tile(s) of one pipeline fill; pair mode: gate rows to tile rows 0 .., up rows to tile rows 64 ..
+            auto load_a = [&](int st, const WorkIter& wi) {
+                if (kPair) {
+                    tma_load_2d_hint(smA + st * kStageA, &p.tmA[0], wi.kb * kBK, wi.it.row0, full_bar(st), pol);
+                    tma_load_2d_hint(smA + st * kStageA + 64 * kBK * 2, &p.tmA[1], wi.kb * kBK, wi.it.row0, full_bar(st), pol);
+                } else {
+                    tma_load_2d_hint(smA + st * kStageA, &p.tmA[wi.it.mat], wi.kb * kBK, wi.it.row0, full_bar(st), pol);
+                }
+            };
             WorkIter w(p), w0(p);
             for (int j = 0; j < warp; ++j) { w.next(p); w0.next(p); }
             int fill = warp;
             for (; w.valid() && fill < kStages; fill += kProducers) {
                 mbar_expect_tx(full_bar(fill), stage_bytes);
-                tma_load_2d_hint(smA + fill * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(fill), pol);
+                load_a(fill, w);
                 for (int j = 0; j < kProducers; ++j) w.next(p);
             }
-            // Still waiting for the predecessor kernel: HBM would sit idle.  Ask TMA to bring the next
-            // weight tiles of this producer into L2 (no shared memory, no barrier involved), so that
-            // the pipeline later refills from L2 instead of HBM.
-            {
-                WorkIter wl = w;
-                for (int j = 0; j < p.l2_fills && wl.valid(); ++j) {
-                    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(&p.tmA[wl.it.mat]),
-                                 "r"(wl.kb * kBK), "r"(wl.it.row0)
-                                 : "memory");
-                    for (int k = 0; k < kProducers; ++k) wl.next(p);
-                }
+            // Still waiting for the predecessor kernel, and so will the kernels after this one: HBM would
+            // sit idle.  Ask TMA to bring every next_every-th k block of the weights of a GEMM that runs
+            // later into L2 (no shared memory, no barrier involved), so that it then streams from L2 and
+            // HBM side by side.
+            if (p.next_every > 0) {
+                for (int c = blockIdx.x; c < p.next_chunks; c += gridDim.x)
+                    for (int kb = warp * p.next_every; kb < p.next_KB; kb += kProducers * p.next_every) {
+                        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(&p.tmN[0]), "r"(kb * kBK),
+                                     "r"(c * p.next_half)
+                                     : "memory");
+                        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(&p.tmN[1]), "r"(kb * kBK),
+                                     "r"(c * p.next_half)
+                                     : "memory");
+                    }
             }
             pdl_wait();
             for (int f0 = warp; f0 < fill; f0 += kProducers) {
@@ -301,7 +320,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 uint32_t phase = (uint32_t)(fill / kStages) & 1u;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_s, p.status, 1u)) break;
                 mbar_expect_tx(full_bar(stage), stage_bytes);
-                tma_load_2d_hint(smA + stage * kStageA, &p.tmA[w.it.mat], w.kb * kBK, w.it.row0, full_bar(stage), pol);
+                load_a(stage, w);
                 tma_load_2d(smB + stage * kStageB, &p.tmB, w.kb * kBK, 0, full_bar(stage));
                 for (int j = 0; j < kProducers; ++j) w.next(p);
             }
@@ -359,6 +378,34 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator may be overwritten
+            if (kPair) {
+                // warps 2-3 hold the up projections (tile rows 64 ..): hand them to the thread that holds the
+                // gate projection of the same column, which writes silu(gate) * up as the next GEMM's operand
+                float z[kMaxW];
+#pragma unroll
+                for (int i = 0; i < kMaxW; ++i) z[i] = __uint_as_float(v[i]) + __uint_as_float(v[i + 8]);
+                if (q >= 2) {
+#pragma unroll
+                    for (int i = 0; i < kMaxW; ++i) up_s[i * 64 + (row_in_tile - 64)] = z[i];
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int col = it.row0 + row_in_tile;
+                if (q < 2 && row_in_tile < p.pair_half && col < p.n_rows[0]) {
+                    const size_t F = (size_t)p.n_rows[0];
+#pragma unroll
+                    for (int i = 0; i < kMaxW; ++i) {
+                        if (i >= p.r0 && i < p.r0 + p.m) {
+                            const float g = z[i], u = up_s[i * 64 + row_in_tile];
+                            const float val = g / (1.f + expf(-g)) * u;
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+                            p.swiglu_out[(size_t)i * F + col] = hi;
+                            p.swiglu_out[(size_t)(i + 8) * F + col] = __float2bfloat16_rn(val - __bfloat162float(hi));
+                        }
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");   // up_s may be overwritten by the next item
+                continue;
+            }
             int n = it.row0 + row_in_tile;
             if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
                 int s = item / p.n_chunks;
@@ -490,14 +537,26 @@ static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, i
     *S_out = bS;
 }
 
+// Pair mode: rows of each kind per item (multiple of 8 in [32,64]) that minimise what the busiest CTA streams.
+static int choose_pair_half(int n_rows, int G) {
+    double best = 1e300;
+    int bh = 64;
+    for (int h = 64; h >= 32; h -= 8) {
+        long long items = (n_rows + h - 1) / h;
+        double cost = (double)((items + G - 1) / G) * h;
+        if (cost < best - 1e-9) { best = cost; bh = h; }
+    }
+    return bh;
+}
+
 static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_end, int n_mats, int K, const void* act,
-                        bool head) {
+                        bool head, bool pair = false) {
     std::vector<uint64_t> key;
     for (int j = 0; j < n_mats; ++j) { key.push_back((uint64_t)(uintptr_t)W[j]); key.push_back((uint64_t)n_end[j]); }
     key.push_back((uint64_t)K);
     key.push_back((uint64_t)(uintptr_t)act);
-    key.push_back(head ? 1 : 0);
-    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_l2_prefetch_kb << 16) + ((uint64_t)g_split_penalty_pm << 40));
+    key.push_back((head ? 1 : 0) + (pair ? 2 : 0));
+    key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_split_penalty_pm << 40));
     auto it = cache->plans.find(key);
     if (it != cache->plans.end()) return it->second;
     TcPlan* pl = new TcPlan();
@@ -505,35 +564,41 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     TcParams& p = pl->p;
     int G = sm_count() * g_ctas_per_sm;
     p.stages = g_stages;
-    p.l2_fills = 0;   // set below once the slab height is known
     p.n_mats = n_mats;
     p.KB = (K + kBK - 1) / kBK;
     int prev = 0;
     for (int j = 0; j < n_mats; ++j) { p.n_rows[j] = n_end[j] - prev; p.n_off[j] = prev; prev = n_end[j]; }
-    choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
-    p.l2_fills = (g_l2_prefetch_kb * 1024) / (p.R * kBK * 2) / kProducers;
     int chunks = 0;
-    for (int j = 0; j < 3; ++j) {
-        if (j < n_mats) chunks += (p.n_rows[j] + p.R - 1) / p.R;
-        p.chunk_end[j] = chunks;
+    if (pair) {
+        p.pair_half = choose_pair_half(p.n_rows[0], G);
+        p.R = 2 * p.pair_half;
+        p.S = 1;
+        chunks = (p.n_rows[0] + p.pair_half - 1) / p.pair_half;
+        for (int j = 0; j < 3; ++j) p.chunk_end[j] = chunks;
+    } else {
+        choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
+        for (int j = 0; j < 3; ++j) {
+            if (j < n_mats) chunks += (p.n_rows[j] + p.R - 1) / p.R;
+            p.chunk_end[j] = chunks;
+        }
     }
     p.n_chunks = chunks;
     p.n_items = chunks * p.S;
     pl->grid = p.n_items < G ? p.n_items : G;
     bool ok = make_map(&p.tmB, act, 16, K, 16);
-    for (int j = 0; j < n_mats && ok; ++j) ok = make_map(&p.tmA[j], W[j], p.n_rows[j], K, p.R);
+    for (int j = 0; j < n_mats && ok; ++j) ok = make_map(&p.tmA[j], W[j], p.n_rows[j], K, pair ? p.pair_half : p.R);
     if (!ok) { delete pl; return nullptr; }
     cache->plans[key] = pl;
     return pl;
 }
 
-static bool g_attr_set[2] = {false, false};
-template <bool kHead> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
-    if (!g_attr_set[kHead]) {
-        cudaFuncSetAttribute(k_tc<kHead>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(kMaxStages));
-        g_attr_set[kHead] = true;
+template <bool kHead, bool kPair> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_tc<kHead, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(kMaxStages));
+        attr_set = true;
     }
-    launch_k(k_tc<kHead>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages), st, p);
+    launch_k(k_tc<kHead, kPair>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages), st, p);
 }
 
 bool tc_set_split_penalty(int per_mille) {
@@ -542,9 +607,9 @@ bool tc_set_split_penalty(int per_mille) {
     return true;
 }
 
-bool tc_set_l2_prefetch(int kb_per_cta) {
-    if (kb_per_cta < 0 || kb_per_cta > 4096) return false;
-    g_l2_prefetch_kb = kb_per_cta;
+bool tc_set_l2_prefetch(int every) {
+    if (every < 0 || every > 64) return false;
+    g_l2_next_every = every;
     return true;
 }
 
@@ -579,11 +644,28 @@ bool tc_set_tuning(int stages, int ctas_per_sm) {
 }
 
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status) {
-    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false);
+    const bool pair = a.swiglu_out != nullptr;
+    if (pair && (a.n_mats != 2 || a.n_end[1] != 2 * a.n_end[0])) return -1;
+    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false, pair);
     if (!pl) return -1;
     TcParams p = pl->p;
     p.out = a.out; p.n_total = a.n_total; p.r0 = a.r0; p.m = a.m; p.status = status;
-    launch<false>(st, pl, p);
+    if (a.next_W[0] && g_l2_next_every > 0) {   // announce a later pair-mode GEMM: same plan that GEMM will use
+        const void* nW[2] = {a.next_W[0], a.next_W[1]};
+        int n_end[2] = {a.next_rows, 2 * a.next_rows};
+        TcPlan* nx = get_plan(cache, nW, n_end, 2, a.next_K, a.next_act, false, true);
+        if (nx) {
+            p.tmN[0] = nx->p.tmA[0]; p.tmN[1] = nx->p.tmA[1];
+            p.next_half = nx->p.pair_half; p.next_chunks = nx->p.n_chunks; p.next_KB = nx->p.KB;
+            p.next_every = g_l2_next_every;
+        }
+    }
+    if (pair) {
+        p.swiglu_out = reinterpret_cast<__nv_bfloat16*>(a.swiglu_out);
+        launch<false, true>(st, pl, p);
+    } else {
+        launch<false, false>(st, pl, p);
+    }
     return p.S;
 }
 
@@ -596,7 +678,7 @@ bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsi
     p.n_total = a.V; p.r0 = a.r0; p.m = a.m; p.status = status;
     p.inv_tau = a.inv_tau; p.threshold = a.threshold; p.conf = a.conf; p.token = a.token; p.exit_flag = a.exit_flag;
     p.logits_dbg = a.logits_dbg; p.part = a.part; p.ticket = a.ticket;
-    launch<true>(st, pl, p);
+    launch<true, false>(st, pl, p);
     return true;
 }
 

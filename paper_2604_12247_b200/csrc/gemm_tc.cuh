@@ -23,8 +23,9 @@ bool tc_available();
 void launch_wait_selftest(cudaStream_t st, unsigned int* status, unsigned long long budget_cycles, unsigned int* waited_flag);
 // pipeline depth (2..12 stages of 18 KB) and persistent CTAs per SM (1..2) of the launches that follow
 bool tc_set_tuning(int stages, int ctas_per_sm);
-// KB of weight tiles per CTA that the producers prefetch into L2 while their kernel still waits for its predecessor
-bool tc_set_l2_prefetch(int kb_per_cta);
+// a GEMM that announces a later pair-mode GEMM (GemmArgs::next_*) prefetches every n-th k block of that GEMM's
+// weights into L2 while it waits for its own predecessor; 0 = never
+bool tc_set_l2_prefetch(int every);
 // cost the host's work decomposition charges for each additional k split, per mille of the streaming time
 bool tc_set_split_penalty(int per_mille);
 // returns the number of split-K partials written to a.out, or -1 if no TMA descriptor could be made

@@ -200,6 +200,15 @@ struct GemmArgs {          // out[s][row][n] = sum_k act[row][k] * W[n][k]   for
     float* out;            // [n_split][8][n_total]
     int n_total;
     int r0, m;
+    // tcgen05 kernel only, two matrices (gate, up) of equal shape: if set, nothing is written to out;
+    // the kernel stores SwiGLU(gate, up) = silu(act.gate) * (act.up) as an Act<T> operand [.][n_end[0]] here
+    void* swiglu_out;
+    // tcgen05 kernel only: a later GEMM of the same stream that will run with swiglu_out set (its two
+    // matrices, rows of each, K, activation operand).  This launch may prefetch part of those weights
+    // into L2 while it waits for its predecessor.  Null = nothing announced.
+    const void* next_W[2];
+    int next_rows, next_K;
+    const void* next_act;
 };
 
 struct HeadArgs {          // exit-confidence / final-head kernel
