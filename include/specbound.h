@@ -226,11 +226,15 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *   SB_OPT_SPLIT_PENALTY (default option only) what the work decomposition charges per additional k split,
  *                    in per mille of the streaming time (more splits balance the CTAs better but cost
  *                    partial-sum traffic and consumer loads).
- *   SB_OPT_FUSE      (default option only) 1 (default) = the tcgen05 gate/up GEMM pairs gate and up rows in
- *                    one tile and its epilogue writes SwiGLU as the down projection's operand; 0 = SwiGLU is
- *                    a kernel of its own.  The fused GEMM is never split along k, so its sums may round
- *                    differently from the separate kernels' (fp32 rounding level); each setting by itself
- *                    is deterministic and row-invariant. */
+ *   SB_OPT_FUSE      (default option only) bit mask, default 3.
+ *                    1: the tcgen05 gate/up GEMM pairs gate and up rows in one tile and its epilogue writes
+ *                       SwiGLU as the down projection's operand (otherwise SwiGLU is a kernel of its own).
+ *                       The fused GEMM is never split along k, so its sums may round differently from the
+ *                       separate kernels' (fp32 rounding level).
+ *                    2: RoPE, KV-cache append, attention and the merge of its 128-position chunks run as one
+ *                       launch (chunk CTAs of a KV head form a thread-block cluster; up to 8 chunks, longer
+ *                       contexts use the separate kernels).  Bit-identical to the separate kernels.
+ *                    Each setting by itself is deterministic and row-invariant. */
 enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,
        SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);

@@ -14,7 +14,7 @@
 namespace sb {
 
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
-static int g_fuse = 1;            // bit 0: SwiGLU in the epilogue of the tcgen05 gate/up GEMM instead of a kernel of its own
+static int g_fuse = 3;            // bit 0: SwiGLU in the epilogue of the tcgen05 gate/up GEMM; bit 1: RoPE + append + attention + chunk merge in one launch
 static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
 
 // TMA descriptors of the stateless entry points: keyed by (pointers, shapes), so they stay valid for as
@@ -218,16 +218,24 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     SB_MARK("norm");
     int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.act_a, W.p_qkv, r0, m);
     SB_MARK("qkv");
-    RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                pos0, r0, m, D.rope_base, {}};
-    for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
-    SB_T(e, launch_rope_append<T>(e.st, ra));
-    SB_MARK("rope");
     AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, W.act_o, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                pos0, r0, m, D.chunk};
-    SB_T(e, launch_attention<T>(e.st, aa));
-    SB_MARK("attn");
-    e.launches += 3;
+                pos0, r0, m, D.chunk, W.p_qkv, s_qkv, {}};
+    for (int i = 0; i < D.hd / 2; ++i) aa.inv_freq[i] = D.inv_freq[i];
+    bool fused = false;
+    if (g_fuse & 2) SB_T(e, fused = launch_attention_fused<T>(e.st, aa));   // RoPE + append + attention + merge in one launch
+    if (fused) {
+        e.launches += 1;
+        SB_MARK("attn");
+    } else {
+        RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
+                    pos0, r0, m, D.rope_base, {}};
+        for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
+        SB_T(e, launch_rope_append<T>(e.st, ra));
+        SB_MARK("rope");
+        SB_T(e, launch_attention<T>(e.st, aa));
+        SB_MARK("attn");
+        e.launches += 3;
+    }
     const void* wo[1] = {lw.wo};
     int no[1] = {D.d};
     // the output projection waits through the whole attention chain with HBM idle: it announces the
@@ -506,7 +514,7 @@ int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_L2_PREFETCH) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
-    if (key == SB_OPT_FUSE) { if (value < 0 || value > 1) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
+    if (key == SB_OPT_FUSE) { if (value < 0 || value > 3) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_GEMM && (value == 0 || value == 1 || value == -1)) {
         if (value == 1 && !tc_available()) return SB_ERR_UNSUPPORTED;

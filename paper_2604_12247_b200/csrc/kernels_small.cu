@@ -90,6 +90,19 @@ void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split
 // write q (fp32) and append k, v to the paged cache in the storage dtype.
 // grid = (H + 2 Hkv, m), block = hd/2 threads (one rotation pair each).
 // ------------------------------------------------------------------------------------------------
+// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head by the angle pos * inv_freq[i]
+__device__ __forceinline__ void rope_rotate(const double* inv_freq, int pos, int i, float& x0, float& x1) {
+    // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
+    // the fp32 sincos sees a small argument
+    double ang = (double)pos * inv_freq[i];
+    ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+    float s, c;
+    sincosf((float)ang, &s, &c);
+    float y0 = x0 * c - x1 * s, y1 = x1 * c + x0 * s;
+    x0 = y0;
+    x1 = y1;
+}
+
 template <typename T>
 __global__ void k_rope_append(RopeArgs a) {
     pdl_trigger();
@@ -105,17 +118,7 @@ __global__ void k_rope_append(RopeArgs a) {
     float x0 = sum_splits(p0, (size_t)kMaxW * ntot, a.n_split);
     float x1 = sum_splits(p0 + half, (size_t)kMaxW * ntot, a.n_split);
     bool is_v = head >= a.H + a.Hkv;
-    if (!is_v) {
-        // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
-        // the fp32 sincos sees a small argument
-        double ang = (double)pos * a.inv_freq[i];
-        ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
-        float s, c;
-        sincosf((float)ang, &s, &c);
-        float y0 = x0 * c - x1 * s, y1 = x1 * c + x0 * s;
-        x0 = y0;
-        x1 = y1;
-    }
+    if (!is_v) rope_rotate(a.inv_freq, pos, i, x0, x1);
     if (head < a.H) {
         float* q = a.q + (size_t)row * qd + col;
         q[i] = x0;
@@ -165,7 +168,18 @@ template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4&
 
 // PG = (row, query head) pairs handled per sweep over the staged tile: the largest of 8, 4, 2, 1 that
 // divides the pair count, so that the inner loops carry no run-time predicates.
-template <typename T, int HD, int PG>
+//
+// kFused: the kernel also does what precedes and follows it.  q is summed from the QKV split-K
+// partials and rotated here (every chunk CTA redoes it: a few hundred values); the CTA whose chunk
+// holds the new positions sums, rotates and rounds their K and V, appends them to the cache and puts
+// them straight into its staged tile; the chunk CTAs of a KV head form one thread-block cluster
+// (grid.y = cluster size = number of chunks <= 8) and CTA 0 of the cluster merges the chunk partials,
+// read from the other CTAs' shared memory, in chunk order.  Same arithmetic in the same order as
+// k_rope_append + k_attn_partial<.., false> + k_attn_combine: bit-identical results.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+template <typename T, int HD, int PG, bool kFused>
 __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     constexpr int kPairGroup = PG;
     constexpr int E = HD / 32;                       // channels per lane in P.V
@@ -185,18 +199,56 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     unsigned char* V_w = K_w + 32 * ROWB;
     float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + warp * kMaxPairGroup * 32;   // [PG][32]
     float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + kAttnWarps * kMaxPairGroup * 32;   // [4][P][HD+2]
+    float* out_s = mrg + (size_t)kAttnWarps * P * (HD + 2);   // kFused: this chunk's merged partial [P][HD+2]
 
-    for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
-        int p = idx / HD, e = idx - p * HD;
-        int i = p / G, g = p - i * G;
-        q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
-    }
     const int pos_last = a.pos0 + a.r0 + a.m - 1;
+    const int pos_new0 = kFused ? a.pos0 + a.r0 : pos_last + 1;   // first position whose K,V this launch creates
     const int tbase = c * kAttnChunk + warp * 32;
     const int my_t = tbase + lane;
+    if (kFused) {
+        constexpr int half = HD / 2;
+        const int ntot = qd + 2 * kvd;
+        const size_t sstride = (size_t)kMaxW * ntot;
+        for (int idx = threadIdx.x; idx < P * half; idx += blockDim.x) {
+            int p = idx / half, e2 = idx - p * half;
+            int i = p / G, g = p - i * G;
+            const float* p0 = a.qkv + (size_t)(a.r0 + i) * ntot + (kvh * G + g) * HD + e2;
+            float x0 = sum_splits(p0, sstride, a.n_split), x1 = sum_splits(p0 + half, sstride, a.n_split);
+            rope_rotate(a.inv_freq, a.pos0 + a.r0 + i, e2, x0, x1);
+            q_s[p * HD + e2] = x0;
+            q_s[p * HD + e2 + half] = x1;
+        }
+        // new positions that fall into this chunk: K (rotated) and V, rounded to the storage type, to the
+        // cache and into the staged tile of the warp that owns the position
+        const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
+        for (int idx = threadIdx.x; idx < (hi - lo + 1) * HD; idx += blockDim.x) {
+            int tp = lo + idx / HD, it = idx % HD;
+            bool is_v = it >= half;
+            int e2 = is_v ? it - half : it;
+            const float* p0 = a.qkv + (size_t)(tp - a.pos0) * ntot + qd + (is_v ? kvd : 0) + kvh * HD + e2;
+            float x0 = sum_splits(p0, sstride, a.n_split), x1 = sum_splits(p0 + half, sstride, a.n_split);
+            if (!is_v) rope_rotate(a.inv_freq, tp, e2, x0, x1);
+            const T y0 = from_f32<T>(x0), y1 = from_f32<T>(x1);
+            T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
+            int page = a.page_table[tp >> a.page_shift];
+            T* dst = cache + ((size_t)page * a.page + (tp & (a.page - 1))) * kvd + (size_t)kvh * HD;
+            dst[e2] = y0;
+            dst[e2 + half] = y1;
+            int tl = tp - c * kAttnChunk;
+            T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
+            srow[e2] = y0;
+            srow[e2 + half] = y1;
+        }
+    } else {
+        for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
+            int p = idx / HD, e = idx - p * HD;
+            int i = p / G, g = p - i * G;
+            q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
+        }
+    }
     // stage this warp's K and V rows (positions beyond the last row's own are never read: zero them)
     size_t my_off = 0;
-    if (my_t <= pos_last) {
+    if (my_t < pos_new0 || (!kFused && my_t <= pos_last)) {
         int page = a.page_table[my_t >> a.page_shift];
         my_off = ((size_t)page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
     }
@@ -209,6 +261,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         int tk = j / PPR, piece = j - tk * PPR;
         size_t off = __shfl_sync(0xffffffffu, my_off, tk);
         unsigned int nbytes = (tbase + tk <= pos_last) ? 16u : 0u;
+        if (kFused && tbase + tk >= pos_new0 && tbase + tk <= pos_last) continue;   // written above
         unsigned int kd = (unsigned int)__cvta_generic_to_shared(K_w + tk * ROWB + piece * 16);
         unsigned int vd = (unsigned int)__cvta_generic_to_shared(V_w + tk * ROWB + piece * 16);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(kd), "l"(reinterpret_cast<const uint4*>(kc + off) + piece), "r"(nbytes) : "memory");
@@ -321,13 +374,55 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
                 }
             }
         }
-        float* dst = a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
+        float* dst = kFused ? out_s + (size_t)p * (HD + 2)
+                            : a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
         dst[e] = O;
         if (e == 0) {
             dst[HD] = M;
             dst[HD + 1] = L;
         }
     }
+    if (!kFused) return;
+    // ---- chunk merge across the cluster (one CTA per chunk of this KV head) ----
+    __syncthreads();
+    cluster_sync_all();   // every chunk's partial is in its CTA's out_s
+    if (c == 0) {
+        const uint32_t out_local = (uint32_t)__cvta_generic_to_shared(out_s);
+        constexpr int kBatch = 8;
+        for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
+            int p = idx / HD, e = idx - p * HD;
+            int i = p / G, g = p - i * G;
+            int row = a.r0 + i;
+            int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own (<= cluster size)
+            float M = -INFINITY, L = 0.f, O = 0.f;
+            float mc[kBatch], lc[kBatch], oc[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                mc[u] = -INFINITY; lc[u] = 0.f; oc[u] = 0.f;
+                if (u < n_chunks) {
+                    uint32_t base;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(base) : "r"(out_local + (uint32_t)(p * (HD + 2)) * 4u), "r"(u));
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mc[u]) : "r"(base + (uint32_t)HD * 4u) : "memory");
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(lc[u]) : "r"(base + (uint32_t)(HD + 1) * 4u) : "memory");
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(oc[u]) : "r"(base + (uint32_t)e * 4u) : "memory");
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                if (mc[u] > -INFINITY) {
+                    float nm = fmaxf(M, mc[u]);
+                    float f0 = expf(M - nm), f1 = expf(mc[u] - nm);
+                    L = L * f0 + lc[u] * f1;
+                    O = O * f0 + oc[u] * f1;
+                    M = nm;
+                }
+            }
+            using A = Act<T>;
+            A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (kvh * G + g) * HD + e, a.H * HD, O / L);
+        }
+    }
+    __syncthreads();
+    cluster_sync_all();   // the other CTAs' shared memory stays alive until CTA 0 has read it
 }
 
 // grid = (H, m), block = hd: merge the chunk partials of one (row, head) in chunk order.
@@ -365,34 +460,68 @@ __global__ void k_attn_combine(AttnArgs a) {
     A::store(reinterpret_cast<typename A::type*>(a.act_out), row, hq * hd + e, a.H * hd, O / L);
 }
 
-template <typename T, int HD, int PG> static void launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem) {
+static size_t attn_smem(int P, int HD, size_t elt, bool fused) {
+    const int rowb = HD * (int)elt + 16;
+    return (size_t)P * HD * 4 + (size_t)kAttnWarps * 64 * rowb + (size_t)kAttnWarps * kMaxPairGroup * 32 * 4 +
+           (size_t)kAttnWarps * P * (HD + 2) * 4 + (fused ? (size_t)P * (HD + 2) * 4 : 0);
+}
+// cluster_y = 0: plain launch; > 0: the fused kernel as clusters of that many chunk CTAs.  Returns false if the
+// device cannot co-schedule such a cluster (nothing is launched then).
+template <typename T, int HD, int PG, bool kFused>
+static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem, int cluster_y) {
+    auto kernel = k_attn_partial<T, HD, PG, kFused>;
     static bool configured = false;
     if (!configured) {
-        cudaFuncSetAttribute(k_attn_partial<T, HD, PG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
         configured = true;
     }
-    launch_k(k_attn_partial<T, HD, PG>, grid, dim3(kAttnWarps * 32), smem, st, a);
+    if (kFused && cluster_y > 1) {
+        static int fits[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // per cluster size: 0 unknown, 1 yes, -1 no
+        if (fits[cluster_y] == 0) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = grid; cfg.blockDim = dim3(kAttnWarps * 32); cfg.dynamicSmemBytes = 200 * 1024;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = (unsigned)cluster_y; at[0].val.clusterDim.z = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+            fits[cluster_y] = n > 0 ? 1 : -1;
+        }
+        if (fits[cluster_y] < 0) return false;
+    }
+    return launch_kc(kernel, grid, dim3(kAttnWarps * 32), smem, st, kFused ? cluster_y : 1, a) == cudaSuccess;
 }
-template <typename T, int HD> static void launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid) {
+template <typename T, int HD, bool kFused>
+static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
     const int P = a.m * (a.H / a.Hkv);
-    const int rowb = HD * (int)sizeof(T) + 16;
-    size_t smem = (size_t)P * HD * 4 + (size_t)kAttnWarps * 64 * rowb + (size_t)kAttnWarps * kMaxPairGroup * 32 * 4 +
-                  (size_t)kAttnWarps * P * (HD + 2) * 4;
-    if (P % 8 == 0) launch_attn_pg<T, HD, 8>(st, a, grid, smem);
-    else if (P % 4 == 0) launch_attn_pg<T, HD, 4>(st, a, grid, smem);
-    else if (P % 2 == 0) launch_attn_pg<T, HD, 2>(st, a, grid, smem);
-    else launch_attn_pg<T, HD, 1>(st, a, grid, smem);
+    size_t smem = attn_smem(P, HD, sizeof(T), kFused);
+    if (P % 8 == 0) return launch_attn_pg<T, HD, 8, kFused>(st, a, grid, smem, cluster_y);
+    if (P % 4 == 0) return launch_attn_pg<T, HD, 4, kFused>(st, a, grid, smem, cluster_y);
+    if (P % 2 == 0) return launch_attn_pg<T, HD, 2, kFused>(st, a, grid, smem, cluster_y);
+    return launch_attn_pg<T, HD, 1, kFused>(st, a, grid, smem, cluster_y);
 }
 
 template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) {
     int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
     dim3 grid(a.Hkv, n_chunks);
     switch (a.hd) {
-        case 32: launch_attn_partial<T, 32>(st, a, grid); break;
-        case 64: launch_attn_partial<T, 64>(st, a, grid); break;
-        default: launch_attn_partial<T, 128>(st, a, grid); break;
+        case 32: launch_attn_partial<T, 32, false>(st, a, grid, 0); break;
+        case 64: launch_attn_partial<T, 64, false>(st, a, grid, 0); break;
+        default: launch_attn_partial<T, 128, false>(st, a, grid, 0); break;
     }
     launch_k(k_attn_combine<T>, dim3(a.H, a.m), dim3(a.hd), 0, st, a);
+}
+
+template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a) {
+    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
+    if (n_chunks > 8) return false;   // portable cluster size
+    dim3 grid(a.Hkv, n_chunks);
+    switch (a.hd) {
+        case 32: return launch_attn_partial<T, 32, true>(st, a, grid, n_chunks);
+        case 64: return launch_attn_partial<T, 64, true>(st, a, grid, n_chunks);
+        default: return launch_attn_partial<T, 128, true>(st, a, grid, n_chunks);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -453,6 +582,7 @@ void launch_init_pages(cudaStream_t st, int* page_table, int n_pages) {
     template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int); \
     template void launch_rope_append<T>(cudaStream_t, const RopeArgs&);                                             \
     template void launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
+    template bool launch_attention_fused<T>(cudaStream_t, const AttnArgs&);                                         \
     template void launch_swiglu<T>(cudaStream_t, const float*, int, int, void*, int, int);
 SB_INST(float)
 SB_INST(__nv_bfloat16)

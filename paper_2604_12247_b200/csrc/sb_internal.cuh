@@ -73,15 +73,28 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 extern bool g_use_pdl;
+// cluster.y > 1 launches thread-block clusters of that many CTAs along y (grid.y must be a multiple of it)
 template <typename... KArgs, typename... Args>
-inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+inline cudaError_t launch_kc(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,
+                             Args&&... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (g_use_pdl) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    if (cluster_y > 1) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 1;
+        attr[n_attr].val.clusterDim.y = (unsigned)cluster_y;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = g_use_pdl ? 1 : 0;
+    cfg.numAttrs = n_attr;
     // every kernel asks for the same (maximal) shared-memory carve-out: an SM never has to drain to
     // change its L1/shared split between two kernels of the chain
     static void* seen[32];
@@ -92,7 +105,11 @@ inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
         cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
         if (n_seen < 32) seen[n_seen++] = (void*)kernel;
     }
-    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    (void)launch_kc(kernel, grid, block, smem, st, 1, static_cast<Args&&>(args)...);
 }
 
 __device__ __forceinline__ float to_f32(float v) { return v; }
@@ -237,6 +254,10 @@ struct AttnArgs {
     int pos0;              // position of row 0
     int r0, m;
     int chunk;             // tokens per split (fixed per context)
+    // fused variant only (RoPE, cache append and chunk merge inside the attention kernel)
+    const float* qkv;      // QKV split-K partials [n_split][8][qd + 2 kvd]
+    int n_split;
+    double inv_freq[64];   // as in RopeArgs
 };
 
 struct RopeArgs {
@@ -259,6 +280,10 @@ template <typename T> void launch_resid_norm(cudaStream_t st, float* h, const fl
                                              const T* gain, float eps, void* act, int r0, int m);
 template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a);
 template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
+// RoPE + cache append + attention + chunk merge in one launch (a.qkv, a.n_split, a.inv_freq set; a.q unused).
+// Returns false without launching when the shape is not covered (more than 8 chunks of 128 positions, or the
+// device cannot co-schedule the cluster): the caller then runs launch_rope_append + launch_attention.
+template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result);
 void launch_init_pages(cudaStream_t st, int* page_table, int n_pages);

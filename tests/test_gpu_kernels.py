@@ -212,27 +212,31 @@ def test_layer_rows_do_not_depend_on_companions(shape):
 
 @pytest.mark.parametrize("shape", [LAYER_BF16, LAYER_HD128], ids=lambda s: s.name)
 def test_layer_under_fusion_and_prefetch_options(shape):
-    """The L2 prefetch of later weights (SB_OPT_L2_PREFETCH) is pure scheduling: bit-identical results.
-    SwiGLU in the gate/up GEMM's epilogue (SB_OPT_FUSE) runs that GEMM without a k split, so it may sum
-    in another order than the separate kernels: equal to fp32 rounding, not bit for bit."""
+    """The L2 prefetch of later weights (SB_OPT_L2_PREFETCH) and the one-launch attention (SB_OPT_FUSE
+    bit 1: RoPE, cache append, attention and chunk merge in one kernel) do the same arithmetic in the same
+    order as the separate kernels: bit-identical results.  SwiGLU in the gate/up GEMM's epilogue
+    (SB_OPT_FUSE bit 0) runs that GEMM without a k split, so it may sum in another order than the separate
+    kernels: equal to fp32 rounding, not bit for bit."""
     w = inputs.make_weights(shape, 24, std=0.05)
-    page, max_seq = 16, 160
+    page, max_seq = 16, 1100
     kvd = shape.n_kv_heads * shape.head_dim
     k_hist, v_hist = inputs.make_kv(max_seq, kvd, 33, shape.dtype)
     lib = binding.lib()
     outs = {}
+    # (rows, first position): one chunk, a round that straddles a chunk boundary, 8 chunks, 9 chunks (separate kernels)
+    cases = ((1, 0), (5, 40), (8, 124), (8, 130), (3, 1000), (4, 1022), (2, 1090))
     try:
-        for fuse, prefetch in ((1, 5), (1, 0), (1, 1), (0, 0)):
+        for fuse, prefetch in ((3, 5), (3, 0), (3, 1), (1, 5), (0, 0)):
             assert lib.sb_set_default_option(7, fuse) == 0 and lib.sb_set_default_option(5, prefetch) == 0
             outs[fuse, prefetch] = [run_layer(shape, w, inputs.make_hidden(m, shape.d_model, 3 + m), k_hist, v_hist, pos,
-                                              max_seq, page, 1) for m, pos in ((1, 0), (5, 40), (8, 130))]
+                                              max_seq, page, 1) for m, pos in cases]
     finally:
-        lib.sb_set_default_option(7, 1)
+        lib.sb_set_default_option(7, 3)
         lib.sb_set_default_option(5, 5)
-    for key in ((1, 0), (1, 1)):
-        for a, b in zip(outs[1, 5], outs[key]):
+    for key in ((3, 0), (3, 1), (1, 5)):
+        for a, b in zip(outs[3, 5], outs[key]):
             assert all(np.array_equal(x, y) for x, y in zip(a, b)), key
-    for a, b in zip(outs[1, 5], outs[0, 0]):
+    for a, b in zip(outs[3, 5], outs[0, 0]):
         assert np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])          # cache rows come before the MLP
         assert np.abs(a[0] - b[0]).max() <= 1e-5 * np.abs(b[0]).max()
 
