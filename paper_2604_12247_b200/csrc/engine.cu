@@ -113,6 +113,7 @@ struct Work {
     int* res;              // result block: conf[8] | token[8] | flag[8] | accept[10] (32-bit words)
     int* toks;             // [max_seq + 8] device token log
     unsigned int* status;  // device status word of the bounded waits
+    float2* rope_tab;      // contexts only: cos/sin of the RoPE angles [n_pages * page][hd/2]
     void* k_cache;         // [L][n_pages][page][kvd]
     void* v_cache;
 };
@@ -149,8 +150,10 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     c.take(W.ticket, 64);
     c.take(W.res, sizeof(int) * 64);
     c.take(W.status, 64);
+    W.rope_tab = nullptr;
     if (with_state) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
+        c.take(W.rope_tab, sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2));
         size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
         c.take(W.k_cache, kv);
         c.take(W.v_cache, kv);
@@ -219,7 +222,7 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.act_a, W.p_qkv, r0, m);
     SB_MARK("qkv");
     AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, W.act_o, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                pos0, r0, m, D.chunk, W.p_qkv, s_qkv, {}};
+                pos0, r0, m, D.chunk, W.p_qkv, s_qkv, W.rope_tab, W.status, {}};
     for (int i = 0; i < D.hd / 2; ++i) aa.inv_freq[i] = D.inv_freq[i];
     bool fused = false;
     if (g_fuse & 2) SB_T(e, fused = launch_attention_fused<T>(e.st, aa));   // RoPE + append + attention + merge in one launch
@@ -228,7 +231,7 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
         SB_MARK("attn");
     } else {
         RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                    pos0, r0, m, D.rope_base, {}};
+                    pos0, r0, m, D.rope_base, W.rope_tab, {}};
         for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
         SB_T(e, launch_rope_append<T>(e.st, ra));
         SB_MARK("rope");
@@ -422,6 +425,7 @@ int sb_create(const sb_config* cfg, void* workspace, size_t bytes, void* stream,
     }
     for (auto& ev : c->ev) cudaEventCreate(&ev);
     launch_init_pages(c->e.st, c->e.W.page_table, D.n_pages);
+    launch_rope_table(c->e.st, c->e.W.rope_tab, D.n_pages * D.page, D.hd / 2, D.inv_freq);
     cudaMemsetAsync(c->e.W.ticket, 0, 64, c->e.st);
     cudaMemsetAsync(c->e.W.status, 0, 64, c->e.st);
     cudaMemsetAsync(c->e.W.res, 0, sizeof(int) * 64, c->e.st);

@@ -90,17 +90,36 @@ void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split
 // write q (fp32) and append k, v to the paged cache in the storage dtype.
 // grid = (H + 2 Hkv, m), block = hd/2 threads (one rotation pair each).
 // ------------------------------------------------------------------------------------------------
-// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head by the angle pos * inv_freq[i]
-__device__ __forceinline__ void rope_rotate(const double* inv_freq, int pos, int i, float& x0, float& x1) {
+// cos and sin of the angle pos * inv_freq[i]
+__device__ __forceinline__ float2 rope_cos_sin(const double* inv_freq, int pos, int i) {
     // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
     // the fp32 sincos sees a small argument
     double ang = (double)pos * inv_freq[i];
     ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
     float s, c;
     sincosf((float)ang, &s, &c);
-    float y0 = x0 * c - x1 * s, y1 = x1 * c + x0 * s;
+    return make_float2(c, s);
+}
+// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head by the angle pos * inv_freq[i]; tab (nullable)
+// = rope_cos_sin tabulated as [position][hd/2] by k_rope_table: the same values, one load instead of the math
+__device__ __forceinline__ void rope_rotate(const double* inv_freq, const float2* __restrict__ tab, int half, int pos, int i,
+                                            float& x0, float& x1) {
+    const float2 cs = tab ? __ldg(tab + (size_t)pos * half + i) : rope_cos_sin(inv_freq, pos, i);
+    // explicit roundings: the compiler must not contract these into fused multiply-adds differently at
+    // different call sites (the separate and the fused kernels have to agree bit for bit)
+    float y0 = __fsub_rn(__fmul_rn(x0, cs.x), __fmul_rn(x1, cs.y)), y1 = __fadd_rn(__fmul_rn(x1, cs.x), __fmul_rn(x0, cs.y));
     x0 = y0;
     x1 = y1;
+}
+struct RopeFreq { double inv_freq[64]; };
+__global__ void k_rope_table(float2* tab, int n_pos, int half, RopeFreq f) {
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < n_pos * half) tab[idx] = rope_cos_sin(f.inv_freq, idx / half, idx % half);
+}
+void launch_rope_table(cudaStream_t st, float2* tab, int n_pos, int half, const double* inv_freq) {
+    RopeFreq f{};
+    for (int i = 0; i < half; ++i) f.inv_freq[i] = inv_freq[i];
+    k_rope_table<<<(n_pos * half + 255) / 256, 256, 0, st>>>(tab, n_pos, half, f);
 }
 
 template <typename T>
@@ -118,7 +137,7 @@ __global__ void k_rope_append(RopeArgs a) {
     float x0 = sum_splits(p0, (size_t)kMaxW * ntot, a.n_split);
     float x1 = sum_splits(p0 + half, (size_t)kMaxW * ntot, a.n_split);
     bool is_v = head >= a.H + a.Hkv;
-    if (!is_v) rope_rotate(a.inv_freq, pos, i, x0, x1);
+    if (!is_v) rope_rotate(a.inv_freq, a.rope_tab, half, pos, i, x0, x1);
     if (head < a.H) {
         float* q = a.q + (size_t)row * qd + col;
         q[i] = x0;
@@ -149,8 +168,10 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 // (row, query head) pairs are processed eight at a time.  Per-warp partials (max, sum, out) are
 // merged in warp order into one partial per (chunk, row, head); k_attn_combine merges the chunks.
 // ------------------------------------------------------------------------------------------------
-constexpr int kAttnWarps = 4;
+constexpr int kPosWarps = 4;                  // 32-position blocks per chunk
+constexpr int kAttnWarps = 2 * kPosWarps;     // two warps per block: each takes half of the (row, query head) pairs
 constexpr int kAttnChunk = 128;
+constexpr unsigned long long kStageWaitCycles = 2000000000ull;   // bound of the wait for the staging copies (~1 s)
 constexpr int kMaxPairGroup = 8;
 
 template <typename T> __device__ __forceinline__ void unpack16(const uint4& u, float (&f)[16 / sizeof(T)]);
@@ -173,8 +194,8 @@ template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4&
 // partials and rotated here (every chunk CTA redoes it: a few hundred values); the CTA whose chunk
 // holds the new positions sums, rotates and rounds their K and V, appends them to the cache and puts
 // them straight into its staged tile; the chunk CTAs of a KV head form one thread-block cluster
-// (grid.y = cluster size = number of chunks <= 8) and CTA 0 of the cluster merges the chunk partials,
-// read from the other CTAs' shared memory, in chunk order.  Same arithmetic in the same order as
+// (grid.y = cluster size = number of chunks <= 8) and merge the chunk partials, read from one another's
+// shared memory, in chunk order (each CTA takes a share of the outputs).  Same arithmetic in the same order as
 // k_rope_append + k_attn_partial<.., false> + k_attn_combine: bit-identical results.
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -188,56 +209,113 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     constexpr int ROWB = HD * (int)sizeof(T) + 16;   // padded row pitch: lane-per-row 16-byte reads are conflict-free
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
-    pdl_wait();
     const int kvh = blockIdx.x, c = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD]
     unsigned char* kv_s = smem + (size_t)P * HD * 4;                                // per warp: K[32], V[32]
-    unsigned char* K_w = kv_s + (size_t)warp * 64 * ROWB;
+    const int v = warp & (kPosWarps - 1), hsel = warp / kPosWarps;   // position block; which half of the pairs
+    unsigned char* K_w = kv_s + (size_t)v * 64 * ROWB;
     unsigned char* V_w = K_w + 32 * ROWB;
-    float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + warp * kMaxPairGroup * 32;   // [PG][32]
-    float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kAttnWarps * 64 * ROWB) + kAttnWarps * kMaxPairGroup * 32;   // [4][P][HD+2]
-    float* out_s = mrg + (size_t)kAttnWarps * P * (HD + 2);   // kFused: this chunk's merged partial [P][HD+2]
+    float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kPosWarps * 64 * ROWB) + warp * kMaxPairGroup * 32;   // [PG][32]
+    float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kPosWarps * 64 * ROWB) + kAttnWarps * kMaxPairGroup * 32;   // [4][P][HD+2]
+    float* out_s = mrg + (size_t)kPosWarps * P * (HD + 2);   // kFused: this chunk's merged partial [P][HD+2]
+    __shared__ __align__(8) unsigned long long stage_bar[kPosWarps];
+    if (threadIdx.x < kPosWarps) mbar_init(smem_u32(&stage_bar[threadIdx.x]), 2);   // one arrival per warp of the block
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 
     const int pos_last = a.pos0 + a.r0 + a.m - 1;
     const int pos_new0 = kFused ? a.pos0 + a.r0 : pos_last + 1;   // first position whose K,V this launch creates
-    const int tbase = c * kAttnChunk + warp * 32;
+    const int tbase = c * kAttnChunk + v * 32;
     const int my_t = tbase + lane;
+    // The page table is set up when the context is created (or, for the stateless call, before the call)
+    // and no kernel of a launch sequence writes it: like the weights it may be read before the wait.
+    int my_page = 0;
+    if (my_t < pos_new0) my_page = a.page_table[my_t >> a.page_shift];
+    pdl_wait();
+    __syncthreads();   // barriers initialised
+    // 1. stage the block's K rows (first warp of the block) or V rows (second warp): one TMA copy per row of an
+    //    earlier launch; rows beyond the last position are zeroed (their probabilities are 0, but 0 * garbage
+    //    must stay 0); rows this launch creates are written in step 2
+    {
+        constexpr uint32_t kRowBytes = HD * (uint32_t)sizeof(T);
+        const bool old_row = my_t < pos_new0;
+        const uint32_t bar = smem_u32(&stage_bar[v]);
+        const unsigned n_old = __popc(__ballot_sync(0xffffffffu, old_row));
+        if (lane == 0) mbar_expect_tx(bar, n_old * kRowBytes);
+        __syncwarp();
+        unsigned char* row = (hsel ? V_w : K_w) + lane * ROWB;
+        if (old_row) {
+            const T* src = reinterpret_cast<const T*>(hsel ? a.v_cache : a.k_cache) +
+                           ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+            bulk_load(smem_u32(row), src, kRowBytes, bar);
+        } else if (my_t > pos_last) {
+#pragma unroll
+            for (int j = 0; j < (int)kRowBytes / 16; ++j) reinterpret_cast<uint4*>(row)[j] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    // 2. while those copies fly: q, and (fused) the new positions' K and V
     if (kFused) {
         constexpr int half = HD / 2;
+        constexpr int kBatch = 4;   // work items whose partial sums are requested together
         const int ntot = qd + 2 * kvd;
         const size_t sstride = (size_t)kMaxW * ntot;
-        for (int idx = threadIdx.x; idx < P * half; idx += blockDim.x) {
-            int p = idx / half, e2 = idx - p * half;
-            int i = p / G, g = p - i * G;
-            const float* p0 = a.qkv + (size_t)(a.r0 + i) * ntot + (kvh * G + g) * HD + e2;
-            float x0 = sum_splits(p0, sstride, a.n_split), x1 = sum_splits(p0 + half, sstride, a.n_split);
-            rope_rotate(a.inv_freq, a.pos0 + a.r0 + i, e2, x0, x1);
-            q_s[p * HD + e2] = x0;
-            q_s[p * HD + e2 + half] = x1;
-        }
-        // new positions that fall into this chunk: K (rotated) and V, rounded to the storage type, to the
-        // cache and into the staged tile of the warp that owns the position
+        // work items: P * half rotation pairs of q, then, for each new position of this chunk, half rotation pairs
+        // of K and half element pairs of V (rounded to the storage type, written to the cache and into the staged
+        // tile of the warp that owns the position)
         const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
-        for (int idx = threadIdx.x; idx < (hi - lo + 1) * HD; idx += blockDim.x) {
-            int tp = lo + idx / HD, it = idx % HD;
+        const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
+        auto src_of = [&](int idx) -> const float* {
+            if (idx < n_q) {
+                int p = idx / half, e2 = idx - p * half;
+                int i = p / G, g = p - i * G;
+                return a.qkv + (size_t)(a.r0 + i) * ntot + (kvh * G + g) * HD + e2;
+            }
+            int j = idx - n_q;
+            int tp = lo + j / HD, it = j % HD;
             bool is_v = it >= half;
-            int e2 = is_v ? it - half : it;
-            const float* p0 = a.qkv + (size_t)(tp - a.pos0) * ntot + qd + (is_v ? kvd : 0) + kvh * HD + e2;
-            float x0 = sum_splits(p0, sstride, a.n_split), x1 = sum_splits(p0 + half, sstride, a.n_split);
-            if (!is_v) rope_rotate(a.inv_freq, tp, e2, x0, x1);
-            const T y0 = from_f32<T>(x0), y1 = from_f32<T>(x1);
-            T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
-            int page = a.page_table[tp >> a.page_shift];
-            T* dst = cache + ((size_t)page * a.page + (tp & (a.page - 1))) * kvd + (size_t)kvh * HD;
-            dst[e2] = y0;
-            dst[e2 + half] = y1;
-            int tl = tp - c * kAttnChunk;
-            T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
-            srow[e2] = y0;
-            srow[e2 + half] = y1;
+            return a.qkv + (size_t)(tp - a.pos0) * ntot + qd + (is_v ? kvd : 0) + kvh * HD + (is_v ? it - half : it);
+        };
+        for (int base = threadIdx.x; base < n_items; base += kBatch * blockDim.x) {
+            float x0[kBatch], x1[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                int idx = base + u * blockDim.x;
+                x0[u] = x1[u] = 0.f;
+                if (idx < n_items) {
+                    const float* p0 = src_of(idx);
+                    x0[u] = sum_splits(p0, sstride, a.n_split);
+                    x1[u] = sum_splits(p0 + half, sstride, a.n_split);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                int idx = base + u * blockDim.x;
+                if (idx >= n_items) continue;
+                if (idx < n_q) {
+                    int p = idx / half, e2 = idx - p * half;
+                    rope_rotate(a.inv_freq, a.rope_tab, half, a.pos0 + a.r0 + p / G, e2, x0[u], x1[u]);
+                    q_s[p * HD + e2] = x0[u];
+                    q_s[p * HD + e2 + half] = x1[u];
+                } else {
+                    int j = idx - n_q;
+                    int tp = lo + j / HD, it = j % HD;
+                    bool is_v = it >= half;
+                    int e2 = is_v ? it - half : it;
+                    if (!is_v) rope_rotate(a.inv_freq, a.rope_tab, half, tp, e2, x0[u], x1[u]);
+                    const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
+                    T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
+                    int page = a.page_table[tp >> a.page_shift];
+                    T* dst = cache + ((size_t)page * a.page + (tp & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                    dst[e2] = y0;
+                    dst[e2 + half] = y1;
+                    int tl = tp - c * kAttnChunk;
+                    T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
+                    srow[e2] = y0;
+                    srow[e2 + half] = y1;
+                }
+            }
         }
     } else {
         for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
@@ -246,32 +324,23 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
             q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
         }
     }
-    // stage this warp's K and V rows (positions beyond the last row's own are never read: zero them)
-    size_t my_off = 0;
-    if (my_t < pos_new0 || (!kFused && my_t <= pos_last)) {
-        int page = a.page_table[my_t >> a.page_shift];
-        my_off = ((size_t)page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+    {   // bounded wait for this block's copies
+        const uint32_t bar = smem_u32(&stage_bar[v]);
+        if (!mbar_try_wait(bar, 0)) {
+            const unsigned long long t0 = clock64();
+            while (!mbar_try_wait(bar, 0)) {
+                if (clock64() - t0 > kStageWaitCycles) {
+                    if (a.status) atomicExch(a.status, 5u);
+                    break;
+                }
+            }
+        }
     }
-    const T* kc = reinterpret_cast<const T*>(a.k_cache);
-    const T* vc = reinterpret_cast<const T*>(a.v_cache);
-    // asynchronous 16-byte copies straight into shared memory: all 2 * PPR copies of a lane are in
-    // flight at once (a source size of 0 zero-fills the rows beyond the last position)
-#pragma unroll
-    for (int j = lane; j < 32 * PPR; j += 32) {
-        int tk = j / PPR, piece = j - tk * PPR;
-        size_t off = __shfl_sync(0xffffffffu, my_off, tk);
-        unsigned int nbytes = (tbase + tk <= pos_last) ? 16u : 0u;
-        if (kFused && tbase + tk >= pos_new0 && tbase + tk <= pos_last) continue;   // written above
-        unsigned int kd = (unsigned int)__cvta_generic_to_shared(K_w + tk * ROWB + piece * 16);
-        unsigned int vd = (unsigned int)__cvta_generic_to_shared(V_w + tk * ROWB + piece * 16);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(kd), "l"(reinterpret_cast<const uint4*>(kc + off) + piece), "r"(nbytes) : "memory");
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(vd), "l"(reinterpret_cast<const uint4*>(vc + off) + piece), "r"(nbytes) : "memory");
-    }
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    __syncthreads();   // q_s complete, own tiles complete
+    __syncthreads();   // q_s, the rows of step 2 and both warps' tiles are complete
 
     const float scale = rsqrtf((float)HD);
-    for (int pg = 0; pg < P; pg += kPairGroup) {
+    const int P0 = (P + 1) / 2;   // pairs [0, P0) go to the first warp of a block, [P0, P) to the second
+    for (int pg = hsel ? P0 : 0; pg < (hsel ? P : P0); pg += kPairGroup) {
         // ---- scores: lane = position ----
         float sc[kPairGroup];
 #pragma unroll
@@ -344,7 +413,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         __syncwarp();
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
-            float* dst = mrg + ((size_t)warp * P + pg + pp) * (HD + 2);
+            float* dst = mrg + ((size_t)v * P + pg + pp) * (HD + 2);
 #pragma unroll
             for (int e = 0; e < E; ++e) dst[lane * E + e] = o[pp][e];
             if (lane == 0) {
@@ -360,11 +429,11 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         int i = p / G, g = p - i * G;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, mrg[((size_t)w * P + p) * (HD + 2) + HD]);
+        for (int w = 0; w < kPosWarps; ++w) M = fmaxf(M, mrg[((size_t)w * P + p) * (HD + 2) + HD]);
         float L = 0.f, O = 0.f;
         if (M > -INFINITY) {
 #pragma unroll
-            for (int w = 0; w < kAttnWarps; ++w) {
+            for (int w = 0; w < kPosWarps; ++w) {
                 const float* src = mrg + ((size_t)w * P + p) * (HD + 2);
                 float mw = src[HD];
                 if (mw > -INFINITY) {
@@ -386,10 +455,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     // ---- chunk merge across the cluster (one CTA per chunk of this KV head) ----
     __syncthreads();
     cluster_sync_all();   // every chunk's partial is in its CTA's out_s
-    if (c == 0) {
+    {   // every CTA of the cluster merges its share of the (pair, channel) outputs
         const uint32_t out_local = (uint32_t)__cvta_generic_to_shared(out_s);
         constexpr int kBatch = 8;
-        for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
+        for (int idx = c * blockDim.x + threadIdx.x; idx < P * HD; idx += gridDim.y * blockDim.x) {
             int p = idx / HD, e = idx - p * HD;
             int i = p / G, g = p - i * G;
             int row = a.r0 + i;
@@ -422,7 +491,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         }
     }
     __syncthreads();
-    cluster_sync_all();   // the other CTAs' shared memory stays alive until CTA 0 has read it
+    cluster_sync_all();   // a CTA's shared memory stays alive until its peers have read it
 }
 
 // grid = (H, m), block = hd: merge the chunk partials of one (row, head) in chunk order.
@@ -462,8 +531,8 @@ __global__ void k_attn_combine(AttnArgs a) {
 
 static size_t attn_smem(int P, int HD, size_t elt, bool fused) {
     const int rowb = HD * (int)elt + 16;
-    return (size_t)P * HD * 4 + (size_t)kAttnWarps * 64 * rowb + (size_t)kAttnWarps * kMaxPairGroup * 32 * 4 +
-           (size_t)kAttnWarps * P * (HD + 2) * 4 + (fused ? (size_t)P * (HD + 2) * 4 : 0);
+    return (size_t)P * HD * 4 + (size_t)kPosWarps * 64 * rowb + (size_t)kAttnWarps * kMaxPairGroup * 32 * 4 +
+           (size_t)kPosWarps * P * (HD + 2) * 4 + (fused ? (size_t)P * (HD + 2) * 4 : 0);
 }
 // cluster_y = 0: plain launch; > 0: the fused kernel as clusters of that many chunk CTAs.  Returns false if the
 // device cannot co-schedule such a cluster (nothing is launched then).
@@ -496,9 +565,12 @@ template <typename T, int HD, bool kFused>
 static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
     const int P = a.m * (a.H / a.Hkv);
     size_t smem = attn_smem(P, HD, sizeof(T), kFused);
-    if (P % 8 == 0) return launch_attn_pg<T, HD, 8, kFused>(st, a, grid, smem, cluster_y);
-    if (P % 4 == 0) return launch_attn_pg<T, HD, 4, kFused>(st, a, grid, smem, cluster_y);
-    if (P % 2 == 0) return launch_attn_pg<T, HD, 2, kFused>(st, a, grid, smem, cluster_y);
+    // pairs per sweep: the largest of 8, 4, 2, 1 that divides what each of a block's two warps gets
+    const int P0 = (P + 1) / 2, P1 = P - P0;
+    auto divides = [&](int g) { return P0 % g == 0 && P1 % g == 0; };
+    if (divides(8)) return launch_attn_pg<T, HD, 8, kFused>(st, a, grid, smem, cluster_y);
+    if (divides(4)) return launch_attn_pg<T, HD, 4, kFused>(st, a, grid, smem, cluster_y);
+    if (divides(2)) return launch_attn_pg<T, HD, 2, kFused>(st, a, grid, smem, cluster_y);
     return launch_attn_pg<T, HD, 1, kFused>(st, a, grid, smem, cluster_y);
 }
 

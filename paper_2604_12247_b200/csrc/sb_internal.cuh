@@ -72,6 +72,37 @@ template <> struct Act<__nv_bfloat16> {
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// ---- shared-memory barriers (mbarrier) used by the TMA pipelines ----
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// plain (untiled) TMA copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from global to this
+// CTA's shared memory, completing on an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+                 "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 extern bool g_use_pdl;
 // cluster.y > 1 launches thread-block clusters of that many CTAs along y (grid.y must be a multiple of it)
 template <typename... KArgs, typename... Args>
@@ -257,6 +288,8 @@ struct AttnArgs {
     // fused variant only (RoPE, cache append and chunk merge inside the attention kernel)
     const float* qkv;      // QKV split-K partials [n_split][8][qd + 2 kvd]
     int n_split;
+    const float2* rope_tab;   // nullable: cos/sin [position][hd/2] (launch_rope_table)
+    unsigned int* status;     // device status word: a staging copy that never completes raises code 5 here
     double inv_freq[64];   // as in RopeArgs
 };
 
@@ -270,6 +303,7 @@ struct RopeArgs {
     int H, Hkv, hd, page, page_shift;
     int pos0, r0, m;
     float rope_base;
+    const float2* rope_tab;   // nullable: cos/sin [position][hd/2] (launch_rope_table)
     double inv_freq[64];   // base^(-2i/hd), i < hd/2, computed on the host in fp64
 };
 
@@ -279,6 +313,8 @@ template <typename T> void launch_embed(cudaStream_t st, const T* embed, int d, 
 template <typename T> void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d,
                                              const T* gain, float eps, void* act, int r0, int m);
 template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a);
+// cos/sin of pos * inv_freq[i] for pos < n_pos, i < half, as [pos][half]
+void launch_rope_table(cudaStream_t st, float2* tab, int n_pos, int half, const double* inv_freq);
 template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
 // RoPE + cache append + attention + chunk merge in one launch (a.qkv, a.n_split, a.inv_freq set; a.q unused).
 // Returns false without launching when the shape is not covered (more than 8 chunks of 128 positions, or the
