@@ -100,11 +100,13 @@ __device__ __forceinline__ float2 rope_cos_sin(const double* inv_freq, int pos, 
     sincosf((float)ang, &s, &c);
     return make_float2(c, s);
 }
-// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head by the angle pos * inv_freq[i]; tab (nullable)
-// = rope_cos_sin tabulated as [position][hd/2] by k_rope_table: the same values, one load instead of the math
-__device__ __forceinline__ void rope_rotate(const double* inv_freq, const float2* __restrict__ tab, int half, int pos, int i,
-                                            float& x0, float& x1) {
-    const float2 cs = tab ? __ldg(tab + (size_t)pos * half + i) : rope_cos_sin(inv_freq, pos, i);
+// cos/sin of the angle of rotation pair i at position pos; tab (nullable) = rope_cos_sin tabulated as
+// [position][hd/2] by k_rope_table: the same values, one load instead of the math
+__device__ __forceinline__ float2 rope_fetch(const double* inv_freq, const float2* __restrict__ tab, int half, int pos, int i) {
+    return tab ? __ldg(tab + (size_t)pos * half + i) : rope_cos_sin(inv_freq, pos, i);
+}
+// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head
+__device__ __forceinline__ void rope_apply(float2 cs, float& x0, float& x1) {
     // explicit roundings: the compiler must not contract these into fused multiply-adds differently at
     // different call sites (the separate and the fused kernels have to agree bit for bit)
     float y0 = __fsub_rn(__fmul_rn(x0, cs.x), __fmul_rn(x1, cs.y)), y1 = __fadd_rn(__fmul_rn(x1, cs.x), __fmul_rn(x0, cs.y));
@@ -137,7 +139,7 @@ __global__ void k_rope_append(RopeArgs a) {
     float x0 = sum_splits(p0, (size_t)kMaxW * ntot, a.n_split);
     float x1 = sum_splits(p0 + half, (size_t)kMaxW * ntot, a.n_split);
     bool is_v = head >= a.H + a.Hkv;
-    if (!is_v) rope_rotate(a.inv_freq, a.rope_tab, half, pos, i, x0, x1);
+    if (!is_v) rope_apply(rope_fetch(a.inv_freq, a.rope_tab, half, pos, i), x0, x1);
     if (head < a.H) {
         float* q = a.q + (size_t)row * qd + col;
         q[i] = x0;
@@ -266,54 +268,56 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         // tile of the warp that owns the position)
         const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
         const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
-        auto src_of = [&](int idx) -> const float* {
+        struct Item { int kind, pos, e2, p; };   // kind 0: q pair of (row, head) pair p; 1: K pair; 2: V pair of position pos
+        auto item_of = [&](int idx) -> Item {
             if (idx < n_q) {
-                int p = idx / half, e2 = idx - p * half;
-                int i = p / G, g = p - i * G;
-                return a.qkv + (size_t)(a.r0 + i) * ntot + (kvh * G + g) * HD + e2;
+                int p = idx / half;
+                return Item{0, a.pos0 + a.r0 + p / G, idx - p * half, p};
             }
-            int j = idx - n_q;
-            int tp = lo + j / HD, it = j % HD;
-            bool is_v = it >= half;
-            return a.qkv + (size_t)(tp - a.pos0) * ntot + qd + (is_v ? kvd : 0) + kvh * HD + (is_v ? it - half : it);
+            int j = idx - n_q, it = j % HD;
+            return Item{it >= half ? 2 : 1, lo + j / HD, it >= half ? it - half : it, 0};
         };
         for (int base = threadIdx.x; base < n_items; base += kBatch * blockDim.x) {
+            // everything a thread's items need from memory is requested before the first value is used
             float x0[kBatch], x1[kBatch];
+            float2 cs[kBatch];
+            int page[kBatch];
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 int idx = base + u * blockDim.x;
                 x0[u] = x1[u] = 0.f;
+                cs[u] = make_float2(1.f, 0.f);
+                page[u] = 0;
                 if (idx < n_items) {
-                    const float* p0 = src_of(idx);
+                    const Item it = item_of(idx);
+                    const float* p0 = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
+                                      (it.kind == 0 ? (kvh * G + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
                     x0[u] = sum_splits(p0, sstride, a.n_split);
                     x1[u] = sum_splits(p0 + half, sstride, a.n_split);
+                    if (it.kind != 2) cs[u] = rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2);
+                    if (it.kind != 0) page[u] = a.page_table[it.pos >> a.page_shift];
                 }
             }
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 int idx = base + u * blockDim.x;
                 if (idx >= n_items) continue;
-                if (idx < n_q) {
-                    int p = idx / half, e2 = idx - p * half;
-                    rope_rotate(a.inv_freq, a.rope_tab, half, a.pos0 + a.r0 + p / G, e2, x0[u], x1[u]);
-                    q_s[p * HD + e2] = x0[u];
-                    q_s[p * HD + e2 + half] = x1[u];
+                const Item it = item_of(idx);
+                if (it.kind != 2) rope_apply(cs[u], x0[u], x1[u]);
+                if (it.kind == 0) {
+                    q_s[it.p * HD + it.e2] = x0[u];
+                    q_s[it.p * HD + it.e2 + half] = x1[u];
                 } else {
-                    int j = idx - n_q;
-                    int tp = lo + j / HD, it = j % HD;
-                    bool is_v = it >= half;
-                    int e2 = is_v ? it - half : it;
-                    if (!is_v) rope_rotate(a.inv_freq, a.rope_tab, half, tp, e2, x0[u], x1[u]);
+                    const bool is_v = it.kind == 2;
                     const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
                     T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
-                    int page = a.page_table[tp >> a.page_shift];
-                    T* dst = cache + ((size_t)page * a.page + (tp & (a.page - 1))) * kvd + (size_t)kvh * HD;
-                    dst[e2] = y0;
-                    dst[e2 + half] = y1;
-                    int tl = tp - c * kAttnChunk;
+                    T* dst = cache + ((size_t)page[u] * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                    dst[it.e2] = y0;
+                    dst[it.e2 + half] = y1;
+                    int tl = it.pos - c * kAttnChunk;
                     T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
-                    srow[e2] = y0;
-                    srow[e2 + half] = y1;
+                    srow[it.e2] = y0;
+                    srow[it.e2 + half] = y1;
                 }
             }
         }
