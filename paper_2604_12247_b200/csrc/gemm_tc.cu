@@ -167,6 +167,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // instruction descriptor: D = f32, A = B = bf16, both K-major, N = 16, M = 128
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
 
+// The four epilogue warps agree on whether to go on: each has waited (bounded) for the accumulator on its
+// own, and a named barrier that one of them skipped would hang the others.  ok_s is [2][4], alternating per call.
+__device__ __forceinline__ bool epi_vote(bool ok, volatile int* ok_s, int n_call, int q, int lane) {
+    volatile int* slot = ok_s + (n_call & 1) * 4;
+    if (lane == 0) slot[q] = ok ? 1 : 0;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    return (slot[0] & slot[1] & slot[2] & slot[3]) != 0;
+}
+
 struct ItemInfo {
     int mat, row0, kb0, kb1;
 };
@@ -210,6 +219,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
     __shared__ SoftTriple cta_part[4][kMaxW];
     __shared__ bool is_last_s;
     __shared__ float up_s[kPair ? kMaxW * 64 : 1];   // pair mode: the up projections of an item, [row][column in item]
+    __shared__ volatile int ok_s[8];
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
@@ -349,6 +359,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             uint32_t use = (uint32_t)(n_local >> 1);
             if (lane == 0) ok = mbar_wait_relaxed(tfull_bar(buf), use & 1u, &abort_s, p.status, 4u);
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;   // one lane polls; the TMEM load needs the whole warp
+            if (kPair) ok = epi_vote(ok, ok_s, n_local, q, lane);   // the pair epilogue synchronises the four warps
             if (!ok) break;
             tc_fence_after();
             uint32_t v[16];
