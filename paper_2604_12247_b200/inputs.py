@@ -86,6 +86,12 @@ RUNS: Dict[str, Run] = {
     "tiny-damped": Run(scaled(TINY, name="tiny-damped", head_scale=16.0), 16, 32, 2, 4, (1.5, 1.0), 0.3, seed=0,
                        damp_rho=0.2),
     "7b": Run(LLAMA2_7B, 512, 512, 6, 4, tau_linear(6, 2.0, 1.0), 0.6, seed=0),
+    # addition, the synthetic stand-in for trained exit heads: W_o and W_down of layer l scaled by
+    # max(0.3^(l-1), 0.01) and a sharper head (x8), so that a confident shallow prediction usually is the
+    # full model's token; the paper's own hyper-parameters: d_max 10, w_max 8, Eq. 1 with alpha 0.2,
+    # confidence threshold 0.55
+    "7b-damped": Run(scaled(LLAMA2_7B, name="llama2-7b-shape-damped", head_scale=8.0), 512, 512, 10, 8,
+                     tuple(1.0 + 0.2 * (1.0 - l / 32.0) for l in range(1, 11)), 0.55, seed=0, damp_rho=0.3),
     "l3-8b": Run(LLAMA3_8B, 1024, 2048, 8, 6, tau_linear(8, 2.0, 1.0), 0.5, seed=0),
     "13b": Run(LLAMA_13B, 2048, 1024, 8, 4, tau_linear(8, 2.0, 1.0), 0.6, seed=0),
 }

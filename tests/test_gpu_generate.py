@@ -257,3 +257,33 @@ def test_7b_shape_run_matches_oracle_on_sampled_positions():
     assert worst_kernel < CONF_TOL
     assert worst_drift < 1e-2 and worst_hidden < HIDDEN_TOL["bf16"]
     ctx.close()
+
+
+def test_7b_damped_run_accepts_drafts_and_equals_ar():
+    """The labelled addition `7b-damped` (damped deep layers: the stand-in for trained exit heads) is what
+    exercises long rounds and accepted drafts at the bench shape: speculative decoding must still be
+    bit-identical to autoregressive decoding, emit more than one token per round on average, and every token
+    must be the oracle's top-1 or within the logit tolerance of it (teacher-forced)."""
+    run = inputs.RUNS["7b-damped"]
+    shape = run.shape
+    wg = inputs.make_weights(shape, run.seed, device="cuda", damp_rho=run.damp_rho)
+    pr = inputs.make_prompt(shape, 24, run.seed).numpy()
+    n_gen, max_seq = 40, 96
+    ctx = binding.Context(shape, wg, max_seq, kv_page=64)
+    ar = ctx.generate_ar(pr, n_gen)["tokens"]
+    sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, run.tau, run.threshold, trace=True)
+    assert np.array_equal(sp["tokens"], ar)
+    rounds = sp["rounds"]
+    emitted = sum(r.emitted for r in rounds)
+    assert emitted == n_gen - 1
+    assert all(1 <= r.w <= run.w_max and r.D <= run.d_max and 1 <= r.emitted <= r.w for r in rounds)
+    print(f"\n[7b-damped] {len(rounds)} rounds, mean width {np.mean([r.w for r in rounds]):.2f}, "
+          f"emitted per round {emitted / len(rounds):.2f}, widest {max(r.w for r in rounds)}")
+    assert emitted / len(rounds) > 1.5 and max(r.emitted for r in rounds) >= 3
+    wc = inputs.weights_to(wg, "cpu")
+    n_chk = 12   # oracle cost: one teacher-forced pass over prompt + n_chk tokens
+    toks = np.concatenate([pr, ar[:n_chk]]).astype(np.int32)
+    top1, top2, margin, deficit = oracle.Oracle(shape, wc, max_seq).teacher_forced(toks, len(pr))
+    assert deficit.min() > -LOGIT_TOL["bf16"]
+    assert all(margin[i] < 2 * LOGIT_TOL["bf16"] for i in range(n_chk) if top1[i] != ar[i])
+    ctx.close()
