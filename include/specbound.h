@@ -63,6 +63,12 @@ typedef struct { /* device pointers */
 typedef struct {
     const void *embed /*[V,d]*/, *final_norm /*[d]*/, *lm_head /*[V,d]*/; /* device */
     const sb_layer_weights* layers;                                      /* HOST array [n_layers] */
+    /* Section 3.2 trains one lightweight LM head per layer for the exit test.  Both tables are nullable HOST
+     * arrays [n_layers] of DEVICE pointers, copied by sb_load_weights: exit_head[l-1] ([V,d]) replaces lm_head
+     * and exit_norm[l-1] ([d]) replaces final_norm in the exit test after layer l; a NULL table or entry means
+     * the shared one.  The final head of the verify pass is always lm_head / final_norm. */
+    const void* const* exit_head;
+    const void* const* exit_norm;
 } sb_weights;
 
 typedef struct {

@@ -70,6 +70,8 @@ def lib():
         L.orc_speedup.argtypes = [C.c_int, C.c_double, C.c_int, C.c_int]
         L.orc_exit_confidence.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_confidence.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_void_p]
+        L.orc_set_exit_head.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_exit_confidence_at.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p]
         L.orc_set_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_get_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_layer_forward.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int]
@@ -141,6 +143,14 @@ class Oracle:
         self.h = lib().orc_create(C.byref(self.cfg), C.byref(self._w))
         if not self.h:
             raise MemoryError("oracle KV cache allocation failed")
+        self._want = want
+        self._exit_keep = {}
+        heads, norms = weights.get("exit_head"), weights.get("exit_norm")   # optional per-layer exit heads / norm gains
+        for l in range(1, shape.n_layers + 1):
+            eh = heads[l - 1] if heads else None
+            en = norms[l - 1] if norms else None
+            if eh is not None or en is not None:
+                self.set_exit_head(l, eh, en)
 
     def close(self):
         if self.h:
@@ -153,7 +163,21 @@ class Oracle:
         except Exception:
             pass
 
+    def set_exit_head(self, layer: int, head: Optional[torch.Tensor], norm: Optional[torch.Tensor] = None):
+        """Head [vocab, d_model] (and norm gain [d_model]) of the exit test after `layer`; None = the shared ones."""
+        for t in (head, norm):
+            assert t is None or (t.device.type == "cpu" and t.dtype == self._want and t.is_contiguous())
+        self._exit_keep[layer] = (head, norm)
+        lib().orc_set_exit_head(self.h, layer, head.data_ptr() if head is not None else None,
+                                norm.data_ptr() if norm is not None else None)
+
     # ---- single operations ------------------------------------------------
+    def exit_confidence_at(self, layer: int, h, T: float):
+        h = np.ascontiguousarray(h, dtype=np.float64)
+        conf, tok = C.c_double(), C.c_int32()
+        lib().orc_exit_confidence_at(self.h, layer, _ptr(h), T, C.byref(conf), C.byref(tok))
+        return conf.value, tok.value
+
     def exit_confidence(self, h, T: float, want_logits: bool = False):
         h = np.ascontiguousarray(h, dtype=np.float64)
         conf, tok = C.c_double(), C.c_int32()

@@ -72,6 +72,10 @@ typedef struct orc_ctx {
     orc_weights w;
     orc_layer* layers;
     double *K, *V; /* [n_layers][max_seq][n_kv_heads*head_dim] */
+    /* Section 3.2: the exit test after layer l may use a head of its own ("lightweight LM heads"):
+     * exit_head[l-1] / exit_norm[l-1], NULL = the shared LM head / final norm gain */
+    const void** exit_head;
+    const void** exit_norm;
 } orc_ctx;
 
 /* ---------------------------------------------------------------- helpers */
@@ -203,6 +207,17 @@ static void head_logits(const orc_ctx* o, const double* h, double* z) {
     free(x);
 }
 
+/* logits of the exit test after layer `layer` (1-based): that layer's own head if one was set */
+static void exit_logits(const orc_ctx* o, int layer, const double* h, double* z) {
+    int d = o->c.d_model;
+    const void* head = o->exit_head[layer - 1] ? o->exit_head[layer - 1] : o->w.lm_head;
+    const void* gain = o->exit_norm[layer - 1] ? o->exit_norm[layer - 1] : o->w.final_norm;
+    double* x = malloc(sizeof(double) * d);
+    rmsnorm(h, gain, o->c.wdtype, d, o->c.rms_eps, x);
+    matvec(head, o->c.wdtype, o->c.vocab, d, x, z);
+    free(x);
+}
+
 static int argmax_first(const double* z, int n) {
     int t = 0;
     for (int v = 1; v < n; ++v) if (z[v] > z[t]) t = v; /* ties: lowest index */
@@ -229,13 +244,31 @@ orc_ctx* orc_create(const orc_config* cfg, const orc_weights* w) {
     size_t n = (size_t)cfg->n_layers * cfg->max_seq * cfg->n_kv_heads * cfg->head_dim;
     o->K = calloc(n, sizeof(double));
     o->V = calloc(n, sizeof(double));
-    if (!o->K || !o->V) { free(o->K); free(o->V); free(o->layers); free(o); return NULL; }
+    o->exit_head = calloc(cfg->n_layers, sizeof(void*));
+    o->exit_norm = calloc(cfg->n_layers, sizeof(void*));
+    if (!o->K || !o->V) { free(o->K); free(o->V); free(o->layers); free(o->exit_head); free(o->exit_norm); free(o); return NULL; }
     return o;
 }
 
 void orc_destroy(orc_ctx* o) {
     if (!o) return;
-    free(o->K); free(o->V); free(o->layers); free(o);
+    free(o->K); free(o->V); free(o->layers); free(o->exit_head); free(o->exit_norm); free(o);
+}
+
+/* Head ([vocab, d_model], storage dtype) and norm gain ([d_model]) of the exit test after `layer`; NULL = shared. */
+void orc_set_exit_head(orc_ctx* o, int layer, const void* head, const void* norm) {
+    o->exit_head[layer - 1] = head;
+    o->exit_norm[layer - 1] = norm;
+}
+
+/* Exit test of Section 3.2 after layer `layer` on one hidden state, with that layer's head. */
+void orc_exit_confidence_at(orc_ctx* o, int layer, const double* h, double T, double* conf, int32_t* token) {
+    double* z = malloc(sizeof(double) * o->c.vocab);
+    int t;
+    exit_logits(o, layer, h, z);
+    confidence_from_logits(z, o->c.vocab, T, conf, &t);
+    *token = t;
+    free(z);
 }
 
 /* Section 3.2, Eq. 1: T_l = 1 + alpha (1 - l/L), l = 1..L, out[l-1] */
@@ -484,7 +517,7 @@ int orc_specbound_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int 
                 for (int i = r0; i <= r; ++i) { depth[i] = l; R.layers_done[i]++; }
                 R.layer_steps++;
                 double p; int t;
-                head_logits(o, h + (size_t)r * d, z);
+                exit_logits(o, l, h + (size_t)r * d, z);
                 confidence_from_logits(z, V, tau[l - 1], &p, &t);
                 R.probes++;
                 R.conf[r] = p;

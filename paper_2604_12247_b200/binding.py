@@ -33,7 +33,8 @@ class LayerWeights(C.Structure):
 
 class Weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p),
-                ("layers", C.POINTER(LayerWeights))]
+                ("layers", C.POINTER(LayerWeights)), ("exit_head", C.POINTER(C.c_void_p)),
+                ("exit_norm", C.POINTER(C.c_void_p))]
 
 
 class Stats(C.Structure):
@@ -168,8 +169,15 @@ class Context:
         _check(lib().sb_create(C.byref(self.cfg), C.c_void_p(base), nbytes, _stream_handle(stream), C.byref(h)), "sb_create")
         self.h = h
         self._layers = (LayerWeights * shape.n_layers)(*[layer_weights(lw) for lw in weights["layers"]])
+        def table(key):   # optional per-layer exit heads / norm gains: list of tensors or None entries
+            items = weights.get(key)
+            if not items:
+                return None
+            assert len(items) == shape.n_layers
+            return (C.c_void_p * shape.n_layers)(*[t.data_ptr() if t is not None else None for t in items])
+        self._exit_head, self._exit_norm = table("exit_head"), table("exit_norm")
         self._w = Weights(weights["embed"].data_ptr(), weights["final_norm"].data_ptr(), weights["lm_head"].data_ptr(),
-                          self._layers)
+                          self._layers, self._exit_head, self._exit_norm)
         _check(lib().sb_load_weights(self.h, C.byref(self._w)), "sb_load_weights")
         if gemm is not None:
             _check(lib().sb_set_option(self.h, OPT_GEMM, gemm), "sb_set_option")

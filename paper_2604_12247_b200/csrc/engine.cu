@@ -293,6 +293,10 @@ struct sb_ctx {
     Exec e;
     sb_weights w;
     sb_layer_weights layers[SB_MAX_LAYERS];
+    const void* exit_head[SB_MAX_LAYERS];   // per-layer exit heads / norm gains, null = shared (copied from sb_weights)
+    const void* exit_norm[SB_MAX_LAYERS];
+    const void* head_of(int layer) const { return exit_head[layer - 1] ? exit_head[layer - 1] : w.lm_head; }
+    const void* norm_of(int layer) const { return exit_norm[layer - 1] ? exit_norm[layer - 1] : w.final_norm; }
     bool loaded = false;
     int* mailbox = nullptr;   // pinned host
     int n = 0, pending = -1, rows = 0;
@@ -456,9 +460,20 @@ int sb_load_weights(sb_ctx* c, const sb_weights* w) {
         for (const void* p : ps)
             if (bad(p)) return SB_ERR_ARG;
     }
+    for (int l = 0; l < c->e.D.L; ++l) {
+        const void* eh = w->exit_head ? w->exit_head[l] : nullptr;
+        const void* en = w->exit_norm ? w->exit_norm[l] : nullptr;
+        if (((uintptr_t)eh & 15) || ((uintptr_t)en & 15)) return SB_ERR_ARG;
+    }
     c->w = *w;
-    for (int l = 0; l < c->e.D.L; ++l) c->layers[l] = w->layers[l];
+    for (int l = 0; l < c->e.D.L; ++l) {
+        c->layers[l] = w->layers[l];
+        c->exit_head[l] = w->exit_head ? w->exit_head[l] : nullptr;
+        c->exit_norm[l] = w->exit_norm ? w->exit_norm[l] : nullptr;
+    }
     c->w.layers = c->layers;
+    c->w.exit_head = c->exit_head;
+    c->w.exit_norm = c->exit_norm;
     c->plans.clear();
     c->loaded = true;
     return SB_OK;
@@ -585,16 +600,16 @@ int sb_draft_advance(sb_ctx* c, int32_t to_layer) {
     if (!c) return SB_ERR_ARG;
     if (!c->loaded || c->rows < 1) return SB_ERR_STATE;
     if (to_layer < 1 || to_layer > c->e.D.L) return SB_ERR_ARG;
-    for (int l = 1; l <= to_layer; ++l) advance_suffix(c, l, c->w.final_norm, nullptr);
+    for (int l = 1; l <= to_layer; ++l) advance_suffix(c, l, c->norm_of(l), nullptr);
     return cuda_ok(cudaGetLastError());
 }
 
 static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf, int32_t* token, int32_t* flag,
                  sb_stats* st = nullptr) {
     int r = c->rows - 1;
-    ensure_act(c->e, c->w.final_norm, r, 1);
+    ensure_act(c->e, c->norm_of(layer), r, 1);
     cudaEventRecord(c->ev[5], c->e.st);
-    head(c->e, c->w.lm_head, r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
+    head(c->e, c->head_of(layer), r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
     cudaEventRecord(c->ev[6], c->e.st);
     int rc = fetch_results(c);
     if (rc) return rc;
@@ -711,7 +726,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
             int r = c->rows - 1;
             bool exited = false;
             for (int l = 1; l <= d_max; ++l) {
-                advance_suffix(c, l, c->w.final_norm, st);
+                advance_suffix(c, l, c->norm_of(l), st);
                 float conf; int tok, flag;
                 if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag, st))) return rc;
                 st->probes++;

@@ -171,8 +171,33 @@ def make_kv(n_pos: int, kv_dim: int, seed: int, dtype: str) -> tuple:
     return k, v
 
 
+def add_exit_heads(w: dict, s: Shape, seed: int = 0, noise: float = 0.5) -> dict:
+    """Synthetic per-layer exit heads (stand-ins for the lightweight heads Section 3.2 trains): for every layer a
+    head = shared LM head + ``noise`` x an independent draw of the same scale, and a norm gain around 1.  Adds
+    ``exit_head`` / ``exit_norm`` (lists of n_layers tensors) to ``w`` in place and returns it."""
+    dev = w["lm_head"].device
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed + 1000)
+    dt = torch_dtype(s.dtype)
+    heads, norms = [], []
+    base = w["lm_head"].float()
+    for _ in range(s.n_layers):
+        n = torch.empty_like(base).normal_(0.0, 0.02 * s.head_scale, generator=g)
+        heads.append((base + noise * n).to(dt).contiguous())
+        gn = torch.empty(s.d_model, dtype=torch.float32, device=dev).normal_(0.0, 0.1, generator=g)
+        norms.append((1.0 + gn).to(dt).contiguous())
+    w["exit_head"], w["exit_norm"] = heads, norms
+    return w
+
+
 def weights_to(w: dict, device: str) -> dict:
-    out = {k: (v.to(device) if isinstance(v, torch.Tensor) else v) for k, v in w.items() if k != "layers"}
+    def move(v):
+        if isinstance(v, torch.Tensor):
+            return v.to(device)
+        if isinstance(v, list):
+            return [move(x) for x in v]
+        return v
+    out = {k: move(v) for k, v in w.items() if k != "layers"}
     out["layers"] = [{k: v.to(device) for k, v in lw.items()} for lw in w["layers"]]
     return out
 

@@ -55,6 +55,42 @@ def test_tiny_run_matches_oracle_tokens_and_trace(which, tiny_weights, tiny_damp
     ctx.close()
 
 
+def test_per_layer_exit_heads_match_oracle_trace():
+    """Section 3.2's per-layer exit heads (pointer tables exit_head / exit_norm): the exit test after layer l
+    uses that layer's head and norm gain, the verify pass the shared head.  Tokens stay those of plain
+    autoregressive decoding; exit layers, drafts and confidences follow the oracle run with the same heads,
+    and differ from the run with the shared head (the tables are really used)."""
+    run = inputs.RUNS["tiny-damped"]
+    w = inputs.add_exit_heads(inputs.make_weights(run.shape, run.seed, damp_rho=run.damp_rho), run.shape, seed=3)
+    pr = inputs.make_prompt(run.shape, run.n_prompt, run.seed).numpy()
+    max_seq = run.n_prompt + run.n_gen + run.w_max + 1
+    orc_ar = oracle.Oracle(run.shape, w, max_seq).ar_generate(pr, run.n_gen)
+    orc_sp, orc_rounds = oracle.Oracle(run.shape, w, max_seq).specbound_generate(
+        pr, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold)
+    assert np.array_equal(orc_sp, orc_ar)
+    ctx, _ = gpu_ctx(run.shape, w, max_seq)
+    sp = ctx.generate(pr, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold, trace=True)
+    assert np.array_equal(sp["tokens"], orc_ar)
+    compare_traces(sp["rounds"], orc_rounds)
+    # the probe primitive with a per-layer head, against the oracle on the same hidden state
+    ctx.reset()
+    first = ctx.prefill(pr)
+    ctx.draft_push(first)
+    for l in (1, 2):
+        ctx.draft_advance(l)
+        conf, tok, _ = ctx.exit_confidence(l, run.tau[l - 1], run.threshold)
+        o = oracle.Oracle(run.shape, w, max_seq)
+        p_ref, t_ref = o.exit_confidence_at(l, ctx.read_hidden(0).astype(np.float64), run.tau[l - 1])
+        assert tok == t_ref and abs(conf - p_ref) < CONF_TOL
+        p_shared, _ = o.exit_confidence(ctx.read_hidden(0).astype(np.float64), run.tau[l - 1])
+        assert abs(p_shared - p_ref) > 10 * CONF_TOL
+    ctx.close()
+    shared = {k: v for k, v in w.items() if k not in ("exit_head", "exit_norm")}
+    _, shared_rounds = oracle.Oracle(run.shape, shared, max_seq).specbound_generate(
+        pr, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold)
+    assert [list(r.conf[:r.w]) for r in shared_rounds] != [list(r.conf[:r.w]) for r in orc_rounds]
+
+
 def test_tiny_hyper_parameter_grid_equals_ar(tiny_damped_weights):
     run = inputs.RUNS["tiny-damped"]
     pr = inputs.make_prompt(run.shape, run.n_prompt, run.seed).numpy()

@@ -79,6 +79,27 @@ def test_layers_and_head_match_torch_library(shape):
         assert t == int(ref.argmax()) and p == pytest.approx(float(ref.max()), rel=1e-10)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_per_layer_exit_head_matches_torch_library(dtype):
+    """Exit test with a layer's own head and norm gain (Section 3.2): equals torch's rms_norm -> linear ->
+    softmax(z / T).max() with THAT layer's tensors, and falls back to the shared head where none is set."""
+    shape = inputs.scaled(GQA, name="gqa-heads", dtype=dtype)
+    w = inputs.add_exit_heads(perturbed_gains(inputs.make_weights(shape, 5)), shape, seed=2)
+    w["exit_head"][1] = None      # layer 2 keeps the shared head but has its own norm gain
+    o = oracle.Oracle(shape, w, 8)
+    h = torch.randn(shape.d_model, dtype=torch.float64, generator=torch.Generator().manual_seed(4))
+    for l in range(1, shape.n_layers + 1):
+        head = w["exit_head"][l - 1] if w["exit_head"][l - 1] is not None else w["lm_head"]
+        gain = w["exit_norm"][l - 1]
+        x = torch.nn.functional.rms_norm(h, (shape.d_model,), gain.double(), shape.rms_eps)
+        ref = torch.softmax(torch.nn.functional.linear(x, head.double()) / 1.7, dim=0)
+        p, t = o.exit_confidence_at(l, h.numpy(), 1.7)
+        assert t == int(ref.argmax()) and p == pytest.approx(float(ref.max()), rel=1e-10)
+    o.set_exit_head(1, None, None)
+    p_shared, t_shared = o.exit_confidence(h.numpy(), 1.7)
+    assert o.exit_confidence_at(1, h.numpy(), 1.7) == (p_shared, t_shared)
+
+
 def test_rope_properties():
     """Position 0 is the identity; q.k after rotation depends only on the position difference."""
     shape = inputs.scaled(GQA, n_layers=1)
