@@ -228,7 +228,7 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                    launch so that a kernel's prologue and weight prefetch overlap its predecessor.
  *   SB_OPT_L2_PREFETCH (default option only) n > 0: while the output projection waits for the attention
  *                    kernels (HBM idle), it prefetches every n-th k block of the layer's gate/up weights
- *                    into L2; 0 = off.  Default 5.  Needs SB_OPT_FUSE = 1.
+ *                    into L2; 0 = off.  Default 4.  Needs bit 0 of SB_OPT_FUSE.
  *   SB_OPT_SPLIT_PENALTY (default option only) what the work decomposition charges per additional k split,
  *                    in per mille of the streaming time (more splits balance the CTAs better but cost
  *                    partial-sum traffic and consumer loads).

@@ -36,7 +36,7 @@ static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;
 static int g_split_penalty_pm = 10;  // cost of one more k split, per mille of the streaming time (see choose_split)
-static int g_l2_next_every = 5;      // see tc_set_l2_prefetch: every n-th k block of the announced GEMM goes to L2 early (0 = off)
+static int g_l2_next_every = 4;      // see tc_set_l2_prefetch: every n-th k block of the announced GEMM goes to L2 early (0 = off)
 constexpr unsigned long long kWaitCycles = 3000000000ull;   // ~1.5 s at 2 GHz
 
 struct alignas(64) TcParams {
