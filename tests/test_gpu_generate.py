@@ -323,3 +323,33 @@ def test_7b_damped_run_accepts_drafts_and_equals_ar():
     assert deficit.min() > -LOGIT_TOL["bf16"]
     assert all(margin[i] < 2 * LOGIT_TOL["bf16"] for i in range(n_chk) if top1[i] != ar[i])
     ctx.close()
+
+
+@pytest.mark.parametrize("which", ["l3-8b", "13b"])
+def test_large_config_tokens_match_oracle(which):
+    """Contract configs 3 (Llama-3-8B shape: GQA 32/8 heads, vocabulary 128256) and 4 (13B shape: 40 layers,
+    d = 5120) in the launch configuration bench.py uses, on a sequence short enough for the oracle:
+    speculative == autoregressive bit for bit on the GPU, and every token is the oracle's top-1 or within the
+    logit tolerance of it (teacher-forced)."""
+    run = inputs.RUNS[which]
+    shape = run.shape
+    wg = inputs.make_weights(shape, run.seed, device="cuda")
+    pr = inputs.make_prompt(shape, 12, run.seed).numpy()
+    n_gen, max_seq = 8, 48
+    ctx = binding.Context(shape, wg, max_seq, kv_page=64)
+    ar = ctx.generate_ar(pr, n_gen)["tokens"]
+    sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, run.tau, run.threshold, trace=True)
+    assert np.array_equal(sp["tokens"], ar)
+    for r in sp["rounds"]:
+        assert 1 <= r.w <= run.w_max and r.D <= run.d_max and 1 <= r.emitted <= r.w
+    ctx.close()
+    wc = inputs.weights_to(wg, "cpu")
+    del wg
+    torch.cuda.empty_cache()
+    toks = np.concatenate([pr, ar]).astype(np.int32)
+    top1, top2, margin, deficit = oracle.Oracle(shape, wc, max_seq).teacher_forced(toks, len(pr))
+    n_off = int((top1 != ar).sum())
+    print(f"\n[{which}] GPU tokens that are not the oracle's top-1: {n_off} of {n_gen}; worst deficit {deficit.min():.2e}; "
+          f"smallest top-2 margin {margin.min():.3f}")
+    assert deficit.min() > -LOGIT_TOL["bf16"]
+    assert all(margin[i] < 2 * LOGIT_TOL["bf16"] for i in range(n_gen) if top1[i] != ar[i])
