@@ -218,13 +218,14 @@ def test_layer_under_fusion_and_prefetch_options(shape):
     (SB_OPT_FUSE bit 0) runs that GEMM without a k split, so it may sum in another order than the separate
     kernels: equal to fp32 rounding, not bit for bit."""
     w = inputs.make_weights(shape, 24, std=0.05)
-    page, max_seq = 16, 1100
+    page, max_seq = 16, 2200
     kvd = shape.n_kv_heads * shape.head_dim
     k_hist, v_hist = inputs.make_kv(max_seq, kvd, 33, shape.dtype)
     lib = binding.lib()
     outs = {}
-    # (rows, first position): one chunk, a round that straddles a chunk boundary, 8 chunks, 9 chunks (separate kernels)
-    cases = ((1, 0), (5, 40), (8, 124), (8, 130), (3, 1000), (4, 1022), (2, 1090))
+    # (rows, first position): one chunk, a round that straddles a chunk boundary, 8 chunks, a round whose last rows
+    # need a 9th chunk, 9 and 17 chunks (separate kernels either way)
+    cases = ((1, 0), (5, 40), (8, 124), (8, 130), (3, 1000), (4, 1022), (2, 1090), (3, 2100))
     try:
         for fuse, prefetch in ((3, 4), (3, 0), (3, 1), (1, 4), (0, 0)):
             assert lib.sb_set_default_option(7, fuse) == 0 and lib.sb_set_default_option(5, prefetch) == 0
