@@ -149,7 +149,8 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     c.take(W.head_part, sizeof(SoftTriple) * kHeadMaxCtas * kMaxW);
     c.take(W.ticket, 64);
     c.take(W.res, sizeof(int) * 64);
-    c.take(W.status, 64);
+    // the status word sits inside the result block (word 48), so that one copy brings results and status to the host
+    W.status = reinterpret_cast<unsigned int*>(W.res + 48);
     W.rope_tab = nullptr;
     if (with_state) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
@@ -321,17 +322,15 @@ struct sb_ctx {
 
 static int cuda_ok(cudaError_t err) { return err == cudaSuccess ? SB_OK : SB_ERR_CUDA; }
 
-// copy the 40-word result block to the pinned mailbox and wait for it; also surfaces launch errors
+// copy the result block (40 words + the status word at 48) to the pinned mailbox and wait for it; also surfaces launch errors
 // and expired device waits
 static int fetch_results(sb_ctx* c) {
-    if (cudaMemcpyAsync(c->mailbox, c->e.W.res, sizeof(int) * 40, cudaMemcpyDeviceToHost, c->e.st) != cudaSuccess)
-        return SB_ERR_CUDA;
-    if (cudaMemcpyAsync(c->mailbox + 48, c->e.W.status, sizeof(int), cudaMemcpyDeviceToHost, c->e.st) != cudaSuccess)
+    if (cudaMemcpyAsync(c->mailbox, c->e.W.res, sizeof(int) * 49, cudaMemcpyDeviceToHost, c->e.st) != cudaSuccess)
         return SB_ERR_CUDA;
     if (cudaStreamSynchronize(c->e.st) != cudaSuccess) return SB_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return SB_ERR_CUDA;
     if (c->e.err) return c->e.err;
-    c->d2h += sizeof(int) * 41;
+    c->d2h += sizeof(int) * 49;
     if (c->mailbox[48] != 0) return SB_ERR_DEVICE_TIMEOUT;
     return SB_OK;
 }

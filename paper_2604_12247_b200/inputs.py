@@ -173,7 +173,7 @@ def make_kv(n_pos: int, kv_dim: int, seed: int, dtype: str) -> tuple:
 
 def add_exit_heads(w: dict, s: Shape, seed: int = 0, noise: float = 0.5) -> dict:
     """Synthetic per-layer exit heads (stand-ins for the lightweight heads Section 3.2 trains): for every layer a
-    head = shared LM head + ``noise`` x an independent draw of the same scale, and a norm gain around 1.  Adds
+    head = shared LM head + ``noise`` x an independent draw of the same scale, and a norm gain close to 1.  Adds
     ``exit_head`` / ``exit_norm`` (lists of n_layers tensors) to ``w`` in place and returns it."""
     dev = w["lm_head"].device
     g = torch.Generator(device=dev)
