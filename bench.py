@@ -292,6 +292,48 @@ def product_arm(args, run: inputs.Run):
         dist.destroy_process_group()
 
 
+def sweep_arm(args, run: inputs.Run):
+    """Hyper-parameter sweep in the spirit of the paper's ablations (Section 4.4: confidence threshold, depth bound
+    d_max, width bound w_max), on the synthetic workload given by --workload: for every point the decode tokens/s
+    of SpecBound, the speed-up over autoregressive decoding with the same kernels, tokens emitted per round, and
+    what Eq. 5 predicts from the measured per-draft acceptance rate (Eq. 5 has no term for the exit probes, which
+    cost a read of the LM head each on this GPU).  One JSON line with all points."""
+    from paper_2604_12247_b200 import binding, build
+    build.build()
+    torch.cuda.set_device(0)
+    s = run.shape
+    w = inputs.make_weights(s, run.seed, device="cuda", damp_rho=run.damp_rho)
+    n_prompt, n_gen = min(run.n_prompt, 256), min(run.n_gen, 256)
+    pr = inputs.make_prompt(s, n_prompt, run.seed).numpy()
+    ctx = binding.Context(s, w, n_prompt + n_gen + 16, kv_page=16)
+    ar = None
+    for _ in range(2):
+        ar = ctx.generate_ar(pr, n_gen)
+    ar_tps = (n_gen - 1) / (ar["stats"].us_decode_dev * 1e-6)
+    alpha = (run.tau[0] - 1.0) / (1.0 - 1.0 / s.n_layers) if run.tau[0] > 1.0 else 0.0   # Eq. 1 strength of the workload's schedule
+    points = []
+    depths = [d for d in (1, 2, 4, 6, 8, 10, 12) if d < s.n_layers]
+    grid = [(d, wm, th) for d in depths for wm in (2, 4, 8) for th in (run.threshold,)]
+    grid += [(run.d_max, run.w_max, th) for th in (0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9) if th != run.threshold]
+    for d_max, w_max, thr in grid:
+        tau = [1.0 + alpha * (1.0 - l / s.n_layers) for l in range(1, d_max + 1)] if alpha > 0 else list(inputs.tau_linear(d_max, 2.0, 1.0))
+        ctx.generate(pr, n_gen, d_max, w_max, tau, thr)   # warm-up (descriptor cache)
+        sp = ctx.generate(pr, n_gen, d_max, w_max, tau, thr)
+        st = sp["stats"]
+        equal = bool((sp["tokens"] == ar["tokens"]).all())
+        tps = (n_gen - 1) / (st.us_decode_dev * 1e-6)
+        drafts = sum(st.exit_hist[1:])                      # rows that produced a draft
+        acc = st.accepted_drafts / drafts if drafts else 0.0
+        points.append({"d_max": d_max, "w_max": w_max, "threshold": thr, "tokens_per_s": tps, "speedup_vs_ar": tps / ar_tps,
+                       "tokens_equal_ar": equal, "rounds": st.rounds, "emitted_per_round": st.emitted / max(st.rounds, 1),
+                       "mean_width": st.rows / max(st.rounds, 1), "draft_acceptance": acc,
+                       "eq5_speedup_at_that_acceptance": binding.model_speedup(s.n_layers, min(acc, 0.999), w_max, d_max),
+                       "probes": st.probes})
+    ctx.close()
+    print(json.dumps({"mode": "sweep", "workload": workload_config(run, "single GPU")["workload"], "prompt_tokens": n_prompt,
+                      "generated_tokens": n_gen, "ar_tokens_per_s": ar_tps, "points": points}), flush=True)
+
+
 def micro_arm(args):
     """Kernel micro-benchmarks (bf16, 7B-shaped layer): the verify pass of one layer for w rows over
     a KV cache of S positions, and the exit-confidence kernel against LM heads of two vocabulary
@@ -387,6 +429,7 @@ def main():
     ap.add_argument("--n-prompt", type=int, default=None, help="override the prompt length (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", action="store_true", help="kernel micro-benchmarks instead of the generation benchmark")
+    ap.add_argument("--sweep", action="store_true", help="d_max x w_max and threshold sweep on --workload (one JSON line)")
     ap.add_argument("--micro-case", default="", help="comma list, e.g. layer:w=4:S=512,exit:m=1:V=32000 (default: all)")
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
@@ -403,7 +446,9 @@ def main():
         for kv in args.tune:
             k, v = kv.split("=")
             assert binding.lib().sb_set_default_option(int(k), int(v)) == 0, kv
-    if args.micro:
+    if args.sweep:
+        sweep_arm(args, run)
+    elif args.micro:
         micro_arm(args)
     elif args.impl == "reference":
         reference_arm(args, run)

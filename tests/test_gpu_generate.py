@@ -353,3 +353,19 @@ def test_large_config_tokens_match_oracle(which):
           f"smallest top-2 margin {margin.min():.3f}")
     assert deficit.min() > -LOGIT_TOL["bf16"]
     assert all(margin[i] < 2 * LOGIT_TOL["bf16"] for i in range(n_gen) if top1[i] != ar[i])
+
+
+def test_bench_sweep_mode_on_tiny(capsys):
+    """bench.py --sweep (depth bound x width bound and threshold sweep): every point decodes the same tokens as
+    autoregressive decoding and reports its statistics."""
+    import argparse
+    import json
+    import bench
+    bench.sweep_arm(argparse.Namespace(), inputs.RUNS["tiny-damped"])
+    line = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
+    pts = line["points"]
+    assert line["mode"] == "sweep" and len(pts) >= 9
+    assert all(p["tokens_equal_ar"] for p in pts)
+    assert {p["d_max"] for p in pts} == {1, 2} and {p["w_max"] for p in pts} == {2, 4, 8}
+    assert all(1.0 <= p["emitted_per_round"] <= p["w_max"] and 0.0 <= p["draft_acceptance"] <= 1.0 for p in pts)
+    assert max(p["emitted_per_round"] for p in pts) > 1.5
