@@ -161,14 +161,16 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 // ------------------------------------------------------------------------------------------------
 // Decode attention over the paged KV cache, split over the KV length into chunks of 128 positions
 // whose boundaries depend on absolute positions only (so a row's result never depends on its
-// companions).  grid = (Hkv, n_chunks), 4 warps; warp v owns positions base + 32 v .. + 31.
-//   1. each warp stages its 32 K rows and 32 V rows in shared memory once (128-bit loads); they
-//      serve every query head of the KV group and every row: K and V leave HBM once per layer;
+// companions).  grid = (Hkv, n_chunks), 8 warps: two per 32-position block (positions base + 32 v .. + 31), each
+// taking half of the (row, query head) pairs.
+//   1. the block's 32 K rows (first warp) and 32 V rows (second warp) are staged in shared memory once, one TMA
+//      row copy each on the block's mbarrier; they serve every query head of the KV group and every row: K and V
+//      leave HBM once per layer;
 //   2. q.k with one position per lane (no reduction per dot product); the softmax max and sum
 //      over the 32 positions are warp-shuffle reductions;
 //   3. P.V with one channel group per lane, probabilities broadcast from shared memory.
-// (row, query head) pairs are processed eight at a time.  Per-warp partials (max, sum, out) are
-// merged in warp order into one partial per (chunk, row, head); k_attn_combine merges the chunks.
+// A warp sweeps its pairs PG at a time.  Per-block partials (max, sum, out) are merged in block order into one
+// partial per (chunk, row, head); the chunks are merged by k_attn_combine or, in the fused kernel, by the cluster.
 // ------------------------------------------------------------------------------------------------
 constexpr int kPosWarps = 4;                  // 32-position blocks per chunk
 constexpr int kAttnWarps = 2 * kPosWarps;     // two warps per block: each takes half of the (row, query head) pairs
