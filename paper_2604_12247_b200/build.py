@@ -44,7 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     objs = [objdir / (s.stem + ".o") for s in sources()]
     if force or jobs or _stale(LIB, objs):
         tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-        subprocess.check_call([NVCC, "-shared", "-o", str(tmp), *map(str, objs), "-lcudart"])
+        subprocess.check_call([NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp), *map(str, objs), "-lcudart"])
         os.replace(tmp, LIB)
     return LIB
 
