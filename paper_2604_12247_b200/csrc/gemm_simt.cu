@@ -140,6 +140,7 @@ __global__ void __launch_bounds__(kHeadWarps * 32) k_head_simt(HeadArgs a) {
     __threadfence();
     soft_final_merge(a.part, (int)gridDim.x, a.r0, a.m, a.inv_tau, a.threshold, a.conf, a.token, a.exit_flag);
     if (threadIdx.x == 0) *a.ticket = 0u;   // ready for the next launch on this stream
+    publish_results(a.mirror);
 }
 template <typename T> void launch_head_simt(cudaStream_t st, const HeadArgs& a, int n_ctas) {
     launch_k(k_head_simt<T>, dim3(n_ctas), dim3(kHeadWarps * 32), 0, st, a);

@@ -66,6 +66,7 @@ struct alignas(64) TcParams {
     SoftTriple* part;
     unsigned int* ticket;
     unsigned int* status;
+    Mirror mirror;
 };
 
 struct TcPlan {
@@ -459,6 +460,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
     __threadfence();
     soft_final_merge(p.part, (int)gridDim.x, p.r0, p.m, p.inv_tau, p.threshold, p.conf, p.token, p.exit_flag);
     if (threadIdx.x == 0) *p.ticket = 0u;
+    publish_results(p.mirror);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -666,7 +668,7 @@ bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsi
     TcParams p = pl->p;
     p.n_total = a.V; p.r0 = a.r0; p.m = a.m; p.status = status;
     p.inv_tau = a.inv_tau; p.threshold = a.threshold; p.conf = a.conf; p.token = a.token; p.exit_flag = a.exit_flag;
-    p.logits_dbg = a.logits_dbg; p.part = a.part; p.ticket = a.ticket;
+    p.logits_dbg = a.logits_dbg; p.part = a.part; p.ticket = a.ticket; p.mirror = a.mirror;
     launch<true, false>(st, pl, p);
     return true;
 }

@@ -628,22 +628,24 @@ template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int
 // model's own token.  result = {n_emit, n_accepted_drafts, g[0..7]}
 // ------------------------------------------------------------------------------------------------
 struct Drafts8 { int v[kMaxW]; };
-__global__ void k_accept(const int* __restrict__ g, Drafts8 drafts, int w, int max_emit, int* __restrict__ result) {
+__global__ void k_accept(const int* __restrict__ g, Drafts8 drafts, int w, int max_emit, int* __restrict__ result, Mirror mirror) {
     pdl_trigger();
     pdl_wait();
-    if (threadIdx.x != 0) return;
-    int acc = 0;
-    while (acc < w && drafts.v[acc] >= 0 && g[acc] == drafts.v[acc]) ++acc;
-    int emit = acc < w ? acc + 1 : w;
-    if (emit > max_emit) emit = max_emit;
-    result[0] = emit;
-    result[1] = acc;
-    for (int i = 0; i < kMaxW; ++i) result[2 + i] = i < w ? g[i] : -1;
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        while (acc < w && drafts.v[acc] >= 0 && g[acc] == drafts.v[acc]) ++acc;
+        int emit = acc < w ? acc + 1 : w;
+        if (emit > max_emit) emit = max_emit;
+        result[0] = emit;
+        result[1] = acc;
+        for (int i = 0; i < kMaxW; ++i) result[2 + i] = i < w ? g[i] : -1;
+    }
+    publish_results(mirror);
 }
-void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result) {
+void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror) {
     Drafts8 d;
     for (int i = 0; i < kMaxW; ++i) d.v[i] = drafts8[i];
-    launch_k(k_accept, dim3(1), dim3(32), 0, st, g, d, w, max_emit, result);
+    launch_k(k_accept, dim3(1), dim3(64), 0, st, g, d, w, max_emit, result, mirror);
 }
 
 __global__ void k_init_pages(int* pt, int n) {

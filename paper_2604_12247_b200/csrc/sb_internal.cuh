@@ -236,6 +236,24 @@ __device__ __forceinline__ void soft_final_merge(const SoftTriple* part, int n_c
     }
 }
 
+// Result mirror: the kernel that produces what the host waits for (exit decision, acceptance) also copies the
+// 49-word result block (results + status word) into host memory mapped into the device's address space and then
+// writes a sequence number; the host polls that word instead of paying a copy and a stream synchronisation.
+// Called by every thread of ONE CTA after its own writes to `res`; mirror may be null.
+struct Mirror {
+    int* host;            // device address of the mapped 64-word host block, or null
+    const int* res;       // the device result block
+    unsigned int seq;     // value for word 63
+};
+__device__ __forceinline__ void publish_results(const Mirror& m) {
+    if (!m.host) return;
+    __syncthreads();                                   // the CTA's writes to res
+    if (threadIdx.x < 49) reinterpret_cast<volatile int*>(m.host)[threadIdx.x] = __ldcg(m.res + threadIdx.x);
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) reinterpret_cast<volatile unsigned int*>(m.host)[63] = m.seq;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Launch arguments
 // ---------------------------------------------------------------------------------------------
@@ -272,6 +290,7 @@ struct HeadArgs {          // exit-confidence / final-head kernel
     float* logits_dbg;     // nullable [m][V] (row r0 first)
     SoftTriple* part;      // scratch [kHeadMaxCtas][8]
     unsigned int* ticket;  // scratch counter, zero between launches (the kernel re-zeroes it)
+    Mirror mirror;         // host.host = null: results stay on the device
 };
 
 struct AttnArgs {
@@ -321,7 +340,7 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
 // device cannot co-schedule the cluster): the caller then runs launch_rope_append + launch_attention.
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
-void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result);
+void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror);
 void launch_init_pages(cudaStream_t st, int* page_table, int n_pages);
 
 // ---- launchers (gemm_simt.cu) ----
