@@ -242,9 +242,12 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                    2: RoPE, KV-cache append, attention and the merge of its 128-position chunks run as one
  *                       launch (chunk CTAs of a KV head form a thread-block cluster; up to 8 chunks, longer
  *                       contexts use the separate kernels).  Bit-identical to the separate kernels.
- *                    Each setting by itself is deterministic and row-invariant. */
+ *                    Each setting by itself is deterministic and row-invariant.
+ *   SB_OPT_QKV_AHEAD (default option only) 1 (default) = while sb_generate waits for an exit decision it already
+ *                    issues the RMSNorm and QKV GEMM of the layer step that follows if the row does not exit
+ *                    (they write scratch only; on an exit they are discarded).  Results do not depend on it. */
 enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,
-       SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7 };
+       SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7, SB_OPT_QKV_AHEAD = 8 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);
 /* Process-wide default for contexts and stateless calls created afterwards. */
 int sb_set_default_option(int32_t key, int32_t value);

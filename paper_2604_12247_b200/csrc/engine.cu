@@ -15,6 +15,7 @@ namespace sb {
 
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
 static int g_fuse = 3;            // bit 0: SwiGLU in the epilogue of the tcgen05 gate/up GEMM; bit 1: RoPE + append + attention + chunk merge in one launch
+static int g_qkv_ahead = 1;       // draft loop: issue the next layer step's norm + QKV GEMM while waiting for the exit decision
 static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
 
 // TMA descriptors of the stateless entry points: keyed by (pointers, shapes), so they stay valid for as
@@ -212,16 +213,26 @@ static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, 
 
 // One decoder layer for rows r0 .. r0+m-1 (row i sits at position pos0 + i).  Ends by adding the
 // MLP output to the hidden rows and, if next_gain is given, leaving their RMSNorm in act_a.
-static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int r0, int m, int pos0,
-                       const void* next_gain) {
+// The first two launches of a layer step: RMSNorm of the rows with the layer's attention gain (if the operand does
+// not hold it already) and the QKV GEMM.  They read the hidden rows and write scratch only, so the draft loop may
+// issue them ahead of time (qkv_ahead) while the host still waits for an exit decision.  Returns the split count.
+static int layer_qkv(Exec& e, const sb_layer_weights& lw, int r0, int m) {
     const Dims& D = e.D;
-    Work& W = e.W;
     ensure_act(e, lw.attn_norm, r0, m);
     const void* wqkv[3] = {lw.wq, lw.wk, lw.wv};
     int nqkv[3] = {D.qd, D.kvd, D.kvd};
     SB_MARK("norm");
-    int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.act_a, W.p_qkv, r0, m);
+    int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, e.W.act_a, e.W.p_qkv, r0, m);
     SB_MARK("qkv");
+    return s_qkv;
+}
+
+// s_qkv_ahead > 0: layer_qkv was already issued for exactly these rows of this layer, with that split count
+static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int r0, int m, int pos0,
+                       const void* next_gain, int s_qkv_ahead = 0) {
+    const Dims& D = e.D;
+    Work& W = e.W;
+    const int s_qkv = s_qkv_ahead > 0 ? s_qkv_ahead : layer_qkv(e, lw, r0, m);
     AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, W.act_o, D.H, D.Hkv, D.hd, D.page, D.page_shift,
                 pos0, r0, m, D.chunk, W.p_qkv, s_qkv, W.rope_tab, W.status, {}};
     for (int i = 0; i < D.hd / 2; ++i) aa.inv_freq[i] = D.inv_freq[i];
@@ -302,6 +313,8 @@ struct sb_ctx {
     int* mailbox = nullptr;      // pinned host memory, mapped into the device's address space
     int* mailbox_dev = nullptr;  // its device address (null: the device cannot map host memory; results are copied)
     unsigned int seq = 0;        // sequence number of the last mirrored result block
+    struct { int layer = 0, r0 = 0, m = 0, s_qkv = 0; } ahead;   // QKV issued ahead for the next layer step (layer 0: none)
+    int64_t probes_at[SB_MAX_LAYERS + 1] = {}, exits_at[SB_MAX_LAYERS + 1] = {};   // per layer, of the current sb_generate call
     int64_t probes_issued = 0;
     int n = 0, pending = -1, rows = 0;
     int depth[SB_MAX_W];
@@ -363,7 +376,10 @@ static int wait_results(sb_ctx* c, const Mirror& m) {
 }
 
 static void run_layer(sb_ctx* c, int layer, int r0, int m, const void* next_gain) {
-    layer_step(c->e, c->layers[layer - 1], c->kc(layer), c->vc(layer), r0, m, c->n, next_gain);
+    // a QKV issued ahead is good for the very next layer step only (the scratch it wrote is reused by every step)
+    const int s_ahead = (c->ahead.layer == layer && c->ahead.r0 == r0 && c->ahead.m == m) ? c->ahead.s_qkv : 0;
+    c->ahead.layer = 0;
+    layer_step(c->e, c->layers[layer - 1], c->kc(layer), c->vc(layer), r0, m, c->n, next_gain, s_ahead);
     for (int i = r0; i < r0 + m; ++i) c->depth[i] = layer;
 }
 
@@ -563,6 +579,7 @@ int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_TRACE) { g_trace = value != 0; return SB_OK; }
     if (key == SB_OPT_L2_PREFETCH) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
+    if (key == SB_OPT_QKV_AHEAD) { g_qkv_ahead = value != 0; return SB_OK; }
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
     if (key == SB_OPT_FUSE) { if (value < 0 || value > 3) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;
@@ -636,8 +653,23 @@ int sb_draft_advance(sb_ctx* c, int32_t to_layer) {
     return cuda_ok(cudaGetLastError());
 }
 
+// While the host waits for the exit decision after layer `layer`, the GPU would idle: issue the norm + QKV GEMM of
+// the layer step that follows if the row does not exit (rows of the trailing run at depth `layer`).  If it exits,
+// the work is discarded: nothing but scratch was written.
+static void qkv_ahead(sb_ctx* c, int layer) {
+    if (!g_qkv_ahead || layer >= c->e.D.L) return;
+    // not where rows usually exit (the work would be thrown away more often than used)
+    if (c->probes_at[layer] >= 8 && 3 * c->exits_at[layer] > c->probes_at[layer]) return;
+    int r0 = c->rows;
+    while (r0 > 0 && c->depth[r0 - 1] == layer) --r0;
+    const int m = c->rows - r0;
+    if (m < 1) return;
+    c->ahead.s_qkv = layer_qkv(c->e, c->layers[layer], r0, m);   // layers[layer] = layer number layer + 1
+    c->ahead.layer = layer + 1; c->ahead.r0 = r0; c->ahead.m = m;
+}
+
 static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf, int32_t* token, int32_t* flag,
-                 sb_stats* st = nullptr) {
+                 sb_stats* st = nullptr, bool more_layers = false) {
     int r = c->rows - 1;
     ensure_act(c->e, c->norm_of(layer), r, 1);
     // One probe in eight is bracketed by events (which needs the copy + synchronise path and keeps the kernel from
@@ -647,6 +679,7 @@ static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf
         cudaEventRecord(c->ev[5], c->e.st);
         head(c->e, c->head_of(layer), r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
         cudaEventRecord(c->ev[6], c->e.st);
+        if (more_layers) qkv_ahead(c, layer);
         int rc = fetch_results(c);
         if (rc) return rc;
         float ms = 0.f;
@@ -654,6 +687,7 @@ static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf
     } else {
         const Mirror mir = next_mirror(c);
         head(c->e, c->head_of(layer), r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr, mir);
+        if (more_layers) qkv_ahead(c, layer);
         int rc = wait_results(c, mir);
         if (rc) return rc;
     }
@@ -740,6 +774,8 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
     sb_stats local;
     sb_stats* st = stats ? stats : &local;
     memset(st, 0, sizeof(*st));
+    memset(c->probes_at, 0, sizeof(c->probes_at));
+    memset(c->exits_at, 0, sizeof(c->exits_at));
     Exec& e = c->e;
     int64_t launches0 = e.launches, h2d0 = c->h2d, d2h0 = c->d2h;
     sb_reset(c);
@@ -767,8 +803,10 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
             for (int l = 1; l <= d_max; ++l) {
                 advance_suffix(c, l, c->norm_of(l), st);
                 float conf; int tok, flag;
-                if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag, st))) return rc;
+                if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag, st, l < d_max))) return rc;
                 st->probes++;
+                c->probes_at[l]++;
+                if (flag) c->exits_at[l]++;
                 R.conf[r] = conf;
                 if (flag) { drafts[r] = tok; R.exit_layer[r] = l; exited = true; break; }
             }
