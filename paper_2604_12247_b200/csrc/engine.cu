@@ -714,6 +714,7 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     int D = 0;
     for (int i = 0; i < w; ++i) D = c->depth[i] > D ? c->depth[i] : D;
     for (int l = 1; l <= D; ++l) advance_suffix(c, l, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm, st);
+    c->ahead.layer = 0;   // the unified pass is timed as a whole: it never starts from work issued ahead of its window
     cudaEventRecord(c->ev[3], e.st);
     for (int l = D + 1; l <= e.D.L; ++l) {
         run_layer(c, l, 0, w, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
