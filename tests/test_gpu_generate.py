@@ -369,3 +369,26 @@ def test_bench_sweep_mode_on_tiny(capsys):
     assert {p["d_max"] for p in pts} == {1, 2} and {p["w_max"] for p in pts} == {2, 4, 8}
     assert all(1.0 <= p["emitted_per_round"] <= p["w_max"] and 0.0 <= p["draft_acceptance"] <= 1.0 for p in pts)
     assert max(p["emitted_per_round"] for p in pts) > 1.5
+
+
+def test_host_side_options_do_not_change_results(tiny_damped_weights):
+    """Work issued ahead while the host waits for an exit decision (SB_OPT_QKV_AHEAD) and programmatic dependent
+    launch (SB_OPT_PDL) are scheduling choices: tokens, rounds, exit layers and confidences are bit-identical."""
+    run = inputs.RUNS["tiny-damped"]
+    pr = inputs.make_prompt(run.shape, run.n_prompt, run.seed).numpy()
+    max_seq = run.n_prompt + run.n_gen + run.w_max + 1
+    lib = binding.lib()
+    results = []
+    try:
+        for ahead, pdl in ((1, 1), (0, 1), (1, 0), (0, 0)):
+            assert lib.sb_set_default_option(8, ahead) == 0 and lib.sb_set_default_option(4, pdl) == 0
+            for shape, w in ((run.shape, tiny_damped_weights),):
+                ctx, _ = gpu_ctx(shape, w, max_seq)
+                sp = ctx.generate(pr, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold, trace=True)
+                results.append((sp["tokens"].copy(), [(r.w, r.D, r.emitted, list(r.exit_layer), list(r.conf)) for r in sp["rounds"]]))
+                ctx.close()
+    finally:
+        lib.sb_set_default_option(8, 1)
+        lib.sb_set_default_option(4, 1)
+    for tokens, rounds in results[1:]:
+        assert np.array_equal(tokens, results[0][0]) and rounds == results[0][1]
