@@ -148,10 +148,11 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     int max_chunks = (D.max_seq + kMaxW + D.chunk - 1) / D.chunk + 1;
     c.take(W.attn_part, sizeof(float) * (size_t)max_chunks * kMaxW * D.H * (D.hd + 2));
     c.take(W.head_part, sizeof(SoftTriple) * kHeadMaxCtas * kMaxW);
-    c.take(W.ticket, 64);
     c.take(W.res, sizeof(int) * 64);
-    // the status word sits inside the result block (word 48), so that one copy brings results and status to the host
+    // the status word sits inside the result block (word 48), so that one copy brings results and status to the host;
+    // the exit kernel's ticket follows (word 56): one 64-byte clear resets both
     W.status = reinterpret_cast<unsigned int*>(W.res + 48);
+    W.ticket = reinterpret_cast<unsigned int*>(W.res + 56);
     W.rope_tab = nullptr;
     if (with_state) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
@@ -412,9 +413,9 @@ static size_t carve_exit_only(const Dims& D, char* base, Work* w) {
     c.take(W.h, sizeof(float) * kMaxW * D.d);
     c.take(W.act_a, es * act_rows * D.d);
     c.take(W.head_part, sizeof(SoftTriple) * kHeadMaxCtas * kMaxW);
-    c.take(W.ticket, 64);
     c.take(W.res, sizeof(int) * 64);
-    c.take(W.status, 64);
+    W.status = reinterpret_cast<unsigned int*>(W.res + 48);   // status word and ticket inside the result block, as in carve()
+    W.ticket = reinterpret_cast<unsigned int*>(W.res + 56);
     return (c.off + 1023) & ~size_t(1023);
 }
 
@@ -477,9 +478,7 @@ int sb_create(const sb_config* cfg, void* workspace, size_t bytes, void* stream,
     for (auto& ev : c->ev) cudaEventCreate(&ev);
     launch_init_pages(c->e.st, c->e.W.page_table, D.n_pages);
     launch_rope_table(c->e.st, c->e.W.rope_tab, D.n_pages * D.page, D.hd / 2, D.inv_freq);
-    cudaMemsetAsync(c->e.W.ticket, 0, 64, c->e.st);
-    cudaMemsetAsync(c->e.W.status, 0, 64, c->e.st);
-    cudaMemsetAsync(c->e.W.res, 0, sizeof(int) * 64, c->e.st);
+    cudaMemsetAsync(c->e.W.res, 0, sizeof(int) * 64, c->e.st);   // results, status word (48) and ticket (56)
     if (cudaStreamSynchronize(c->e.st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
         sb_destroy(c);
         return SB_ERR_CUDA;
@@ -902,7 +901,7 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     Dims D;
     if (!make_dims(cfg, &D) || !h || !final_norm || !lm_head || !conf || !token || !scratch) return SB_ERR_ARG;
     if (m < 1 || m > SB_MAX_W || !(tau_l > 0.f)) return SB_ERR_ARG;
-    if (((uintptr_t)scratch & 1023) || ((uintptr_t)lm_head & 15)) return SB_ERR_ARG;
+    if (((uintptr_t)scratch & 1023) || ((uintptr_t)lm_head & 15) || ((uintptr_t)h & 15)) return SB_ERR_ARG;
     if (scratch_bytes < carve(D, nullptr, false, nullptr)) return SB_ERR_CAPACITY;
     Exec e;
     e.D = D;
@@ -910,13 +909,12 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     carve(D, (char*)scratch, false, &e.W);
     e.gemm = pick_gemm(D.f32);
     e.plans = &stateless_plans();
-    cudaMemsetAsync(e.W.ticket, 0, 64, e.st);
+    // the kernels read the caller's rows and write the caller's outputs directly: the call is one 64-byte clear
+    // (status word + ticket), the RMSNorm and the exit-confidence kernel
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
-    cudaMemcpyAsync(e.W.h, h, sizeof(float) * m * D.d, cudaMemcpyDeviceToDevice, e.st);
+    e.W.h = const_cast<float*>(reinterpret_cast<const float*>(h));
     ensure_act(e, final_norm, 0, m);
-    head(e, lm_head, 0, m, tau_l, 2.f, reinterpret_cast<float*>(e.W.res), e.W.res + 8, e.W.res + 16, logits_dbg);
-    cudaMemcpyAsync(conf, e.W.res, sizeof(float) * m, cudaMemcpyDeviceToDevice, e.st);
-    cudaMemcpyAsync(token, e.W.res + 8, sizeof(int) * m, cudaMemcpyDeviceToDevice, e.st);
+    head(e, lm_head, 0, m, tau_l, 2.f, conf, token, e.W.res + 16, logits_dbg);
     if (e.err) return e.err;
     return cuda_ok(cudaGetLastError());
 }
@@ -927,7 +925,7 @@ int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, 
     if (cfg && cfg->d_model > kStaticMaxDModel) return SB_ERR_CAPACITY;   // would not fit the fixed array
     if (!make_dims(cfg, &D) || !h || !final_norm || !lm_head || !conf || !token) return SB_ERR_ARG;
     if (m < 1 || m > SB_MAX_W || !(tau_l > 0.f)) return SB_ERR_ARG;
-    if ((uintptr_t)lm_head & 15) return SB_ERR_ARG;
+    if (((uintptr_t)lm_head & 15) || ((uintptr_t)h & 15)) return SB_ERR_ARG;
     if (carve_exit_only(D, nullptr, nullptr) > kStaticScratchBytes) return SB_ERR_CAPACITY;
     char* base = nullptr;
     int rc = static_scratch_ptr(&base);   // first call on a device looks the address up
@@ -939,14 +937,11 @@ int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, 
     carve_exit_only(D, base, &e.W);
     e.gemm = pick_gemm(D.f32);
     e.plans = &stateless_plans();
-    // the array keeps whatever the previous call left: the ticket and the status word must start at zero
-    cudaMemsetAsync(e.W.ticket, 0, 64, e.st);
+    // the array keeps whatever the previous call left: the status word and the ticket must start at zero
     cudaMemsetAsync(e.W.status, 0, 64, e.st);
-    cudaMemcpyAsync(e.W.h, h, sizeof(float) * m * D.d, cudaMemcpyDeviceToDevice, e.st);
+    e.W.h = const_cast<float*>(reinterpret_cast<const float*>(h));
     ensure_act(e, final_norm, 0, m);
-    head(e, lm_head, 0, m, tau_l, 2.f, reinterpret_cast<float*>(e.W.res), e.W.res + 8, e.W.res + 16, nullptr);
-    cudaMemcpyAsync(conf, e.W.res, sizeof(float) * m, cudaMemcpyDeviceToDevice, e.st);
-    cudaMemcpyAsync(token, e.W.res + 8, sizeof(int) * m, cudaMemcpyDeviceToDevice, e.st);
+    head(e, lm_head, 0, m, tau_l, 2.f, conf, token, e.W.res + 16, nullptr);
     if (e.err) return e.err;
     return cuda_ok(cudaGetLastError());
 }
