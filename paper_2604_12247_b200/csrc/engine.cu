@@ -174,6 +174,7 @@ struct Exec {   // everything a launch sequence needs
     const void* act_gain = nullptr;
     int act_r0 = 0, act_m = 0;
     TcPlanCache* plans = nullptr;
+    unsigned int* clear_next = nullptr;   // 16 words that the next RMSNorm launch of ensure_act zeroes (stateless calls)
     int err = 0;   // sticky host-side error of a launch sequence (a TMA descriptor could not be built)
 };
 
@@ -185,7 +186,8 @@ struct Exec {   // everything a launch sequence needs
 
 static void ensure_act(Exec& e, const void* gain, int r0, int m) {
     if (e.act_gain == gain && r0 >= e.act_r0 && r0 + m <= e.act_r0 + e.act_m) return;
-    SB_T(e, launch_resid_norm<T>(e.st, e.W.h, nullptr, 0, e.D.d, (const T*)gain, e.D.eps, e.W.act_a, r0, m));
+    SB_T(e, launch_resid_norm<T>(e.st, e.W.h, nullptr, 0, e.D.d, (const T*)gain, e.D.eps, e.W.act_a, r0, m, e.clear_next));
+    e.clear_next = nullptr;
     e.launches++;
     e.act_gain = gain; e.act_r0 = r0; e.act_m = m;
 }
@@ -909,9 +911,9 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     carve(D, (char*)scratch, false, &e.W);
     e.gemm = pick_gemm(D.f32);
     e.plans = &stateless_plans();
-    // the kernels read the caller's rows and write the caller's outputs directly: the call is one 64-byte clear
-    // (status word + ticket), the RMSNorm and the exit-confidence kernel
-    cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    // the kernels read the caller's rows and write the caller's outputs directly: the call is the RMSNorm (which also
+    // clears the status word and the ticket) and the exit-confidence kernel
+    e.clear_next = e.W.status;
     e.W.h = const_cast<float*>(reinterpret_cast<const float*>(h));
     ensure_act(e, final_norm, 0, m);
     head(e, lm_head, 0, m, tau_l, 2.f, conf, token, e.W.res + 16, logits_dbg);
@@ -937,8 +939,9 @@ int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, 
     carve_exit_only(D, base, &e.W);
     e.gemm = pick_gemm(D.f32);
     e.plans = &stateless_plans();
-    // the array keeps whatever the previous call left: the status word and the ticket must start at zero
-    cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    // the array keeps whatever the previous call left: the status word and the ticket must start at zero (the RMSNorm
+    // launch clears them)
+    e.clear_next = e.W.status;
     e.W.h = const_cast<float*>(reinterpret_cast<const float*>(h));
     ensure_act(e, final_norm, 0, m);
     head(e, lm_head, 0, m, tau_l, 2.f, conf, token, e.W.res + 16, nullptr);

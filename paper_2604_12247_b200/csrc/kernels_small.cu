@@ -37,10 +37,12 @@ constexpr int kNormVec = 2;   // float4 per thread: rows up to 1024 * 2 * 4 = 81
 template <typename T>
 __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__ h, const float* __restrict__ part,
                                                             int n_split, int d, const T* __restrict__ gain, float eps,
-                                                            void* __restrict__ act, int r0) {
+                                                            void* __restrict__ act, int r0, unsigned int* __restrict__ clear16) {
     __shared__ float red[kNormThreads / 32];
     pdl_trigger();
     pdl_wait();
+    // optional: zero 16 words for the kernels that follow (the stateless calls' status word and ticket)
+    if (clear16 && blockIdx.x == 0 && threadIdx.x < 16) clear16[threadIdx.x] = 0u;
     int row = r0 + blockIdx.x;
     float4* hr = reinterpret_cast<float4*>(h + (size_t)row * d);
     const int nv = d >> 2;
@@ -81,8 +83,8 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
 }
 template <typename T>
 void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d, const T* gain, float eps,
-                       void* act, int r0, int m) {
-    launch_k(k_resid_norm<T>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0);
+                       void* act, int r0, int m, unsigned int* clear16) {
+    launch_k(k_resid_norm<T>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -659,7 +661,7 @@ void launch_init_pages(cudaStream_t st, int* page_table, int n_pages) {
 // explicit instantiations
 #define SB_INST(T)                                                                                                  \
     template void launch_embed<T>(cudaStream_t, const T*, int, const int*, int, int, int, float*);                  \
-    template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int); \
+    template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int, unsigned int*); \
     template void launch_rope_append<T>(cudaStream_t, const RopeArgs&);                                             \
     template void launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
     template bool launch_attention_fused<T>(cudaStream_t, const AttnArgs&);                                         \
