@@ -262,7 +262,7 @@ def product_arm(args, run: inputs.Run):
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dec_ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 storage, f32 accumulate" if s.dtype == "bf16" else "f32", "data": "synthetic",
+        "dtype": "f32", "storage_dtype": s.dtype, "data": "synthetic",
         "config": workload_config(run, f"replicas x{world}" if world > 1 else "single GPU"),
         "ar_tokens_per_s": ar_value, "speedup_vs_ar": (value / world) / ar_value,
         "tokens_equal_ar": tokens_equal,
