@@ -72,6 +72,12 @@ def lib():
         L.orc_confidence.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_void_p]
         L.orc_set_exit_head.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_exit_confidence_at.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_double, C.c_void_p, C.c_void_p]
+        L.orc_mix64.restype = C.c_uint64
+        L.orc_mix64.argtypes = [C.c_uint64, C.c_int64]
+        L.orc_uniform.restype = C.c_double
+        L.orc_uniform.argtypes = [C.c_uint64, C.c_int64]
+        L.orc_sample_token.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p]
+        L.orc_set_sampling.argtypes = [C.c_void_p, C.c_double, C.c_uint64]
         L.orc_set_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_get_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_layer_forward.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int]
@@ -107,6 +113,24 @@ def expected_accepted(a, w):
 
 def speedup(L, a, w, d_max):
     return lib().orc_speedup(L, a, w, d_max)
+
+
+def mix64(seed: int, pos: int) -> int:
+    """Counter-based 64-bit hash behind the sampling uniforms (splitmix64 output function)."""
+    return int(lib().orc_mix64(seed, pos))
+
+
+def uniform(seed: int, pos: int) -> float:
+    """u(seed, pos) in (0, 1): the uniform number that decides the token at sequence position pos."""
+    return float(lib().orc_uniform(seed, pos))
+
+
+def sample_token(z: np.ndarray, temperature: float, u: float):
+    """Inverse-CDF sample of softmax(z / temperature) in vocabulary order -> (token, slack)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    slack = C.c_double()
+    t = lib().orc_sample_token(_ptr(z), z.size, float(temperature), float(u), C.byref(slack))
+    return int(t), float(slack.value)
 
 
 def confidence(z: np.ndarray, T: float):
@@ -162,6 +186,10 @@ class Oracle:
             self.close()
         except Exception:
             pass
+
+    def set_sampling(self, temperature: float, seed: int = 0):
+        """Sampling decoding (Section 4.3): temperature 0 restores greedy decoding."""
+        lib().orc_set_sampling(self.h, float(temperature), int(seed))
 
     def set_exit_head(self, layer: int, head: Optional[torch.Tensor], norm: Optional[torch.Tensor] = None):
         """Head [vocab, d_model] (and norm gain [d_model]) of the exit test after `layer`; None = the shared ones."""

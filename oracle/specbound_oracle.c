@@ -24,6 +24,16 @@
  * cases, torch CPU library routines for each decoder block, no-cache brute
  * force, speculative == autoregressive over a hyper-parameter grid, and the two
  * worked scenarios of Section 3.3 / the appendix with scripted exits.
+ * Sampling decoding (Section 4.3 "decoding strategies", Table 2): the paper names
+ * temperature sampling but prints no acceptance rule.  The reading taken here:
+ * the token at sequence position p is the inverse-CDF sample, in vocabulary
+ * order, of softmax(z / T_s) at the uniform number u(seed, p) of a counter-based
+ * generator; verification recomputes that token for every draft row and accepts
+ * a draft iff it equals it.  Autoregressive sampling with the same (seed, T_s)
+ * DEFINES the correct output; the speculative loop must reproduce it token for
+ * token, which makes it lossless sample by sample and hence in distribution.
+ * Pins: published splitmix64 outputs, stratified-u counts against a library
+ * softmax, the T_s -> 0 limit (greedy), speculative == autoregressive over a grid.
  * Not pinned by the paper: the confidence VALUES on random weights (the paper
  * prints none) -- "parity unpinned" for those beyond the library cross-check.
  */
@@ -76,6 +86,9 @@ typedef struct orc_ctx {
      * exit_head[l-1] / exit_norm[l-1], NULL = the shared LM head / final norm gain */
     const void** exit_head;
     const void** exit_norm;
+    /* sampling decoding (Section 4.3, decoding strategies): temperature 0 = greedy */
+    double sample_temperature;
+    uint64_t sample_seed;
 } orc_ctx;
 
 /* ---------------------------------------------------------------- helpers */
@@ -224,6 +237,59 @@ static int argmax_first(const double* z, int n) {
     return t;
 }
 
+/* ---- sampling decoding (Section 4.3, decoding strategies; Table 2) ---- */
+
+/* Counter-based uniform number in (0,1): the splitmix64 output function applied to
+ * seed + (pos+1) * golden-ratio increment, i.e. for seed 0 the (pos+1)-th output of
+ * the published splitmix64 stream; top 53 bits, centred in their cell. */
+uint64_t orc_mix64(uint64_t seed, int64_t pos) {
+    uint64_t x = seed + 0x9E3779B97F4A7C15ull * (uint64_t)(pos + 1);
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+double orc_uniform(uint64_t seed, int64_t pos) {
+    return ((double)(orc_mix64(seed, pos) >> 11) + 0.5) * (1.0 / 9007199254740992.0);
+}
+
+/* Inverse-CDF sample of softmax(z / temperature) in vocabulary order: the first token v
+ * whose cumulative un-normalised mass reaches u * total.  slack (nullable) receives the
+ * distance from u to the nearer edge of the chosen token's CDF interval. */
+int orc_sample_token(const double* z, int V, double temperature, double u, double* slack) {
+    double m = z[0];
+    for (int v = 1; v < V; ++v) if (z[v] > m) m = z[v];
+    double total = 0.0;
+    for (int v = 0; v < V; ++v) total += exp((z[v] - m) / temperature);
+    double target = u * total, run = 0.0;
+    int pick = -1;
+    double lo = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double e = exp((z[v] - m) / temperature);
+        if (e > 0.0) pick = v;                      /* rounding guard: last token with mass */
+        if (run + e >= target) { pick = v; lo = run; run += e; break; }
+        run += e;
+        lo = run;
+    }
+    if (slack) {
+        double a = target - lo, b = run - target;
+        *slack = (a < b ? a : b) / total;
+    }
+    return pick;
+}
+
+
+/* The decoding rule at the last layer: greedy top-1, or (temperature > 0) the inverse-CDF
+ * sample at u(seed, pos), pos = sequence position of the token being produced. */
+static int next_token(const orc_ctx* o, const double* z, int pos, double* slack) {
+    if (o->sample_temperature > 0.0)
+        return orc_sample_token(z, o->c.vocab, o->sample_temperature, orc_uniform(o->sample_seed, pos), slack);
+    return argmax_first(z, o->c.vocab);
+}
+void orc_set_sampling(orc_ctx* o, double temperature, uint64_t seed) {
+    o->sample_temperature = temperature > 0.0 ? temperature : 0.0;
+    o->sample_seed = seed;
+}
+
 /* Eq. 2: p = max softmax(z / T) = 1 / sum_v exp((z_v - z_max)/T); token = argmax z */
 static void confidence_from_logits(const double* z, int V, double T, double* conf, int* token) {
     int t = argmax_first(z, V);
@@ -332,8 +398,8 @@ void orc_embed(orc_ctx* o, int tok, double* h) { embed_row(o, tok, h); }
 
 void orc_final_logits(orc_ctx* o, const double* h, double* z) { head_logits(o, h, z); }
 
-/* Full-depth forward of one token at `pos` using the cache; returns greedy token,
- * optionally the logits. */
+/* Full-depth forward of one token at `pos` using the cache; returns the token the decoding
+ * rule produces for position pos + 1 (greedy unless sampling is set), optionally the logits. */
 static int full_step(orc_ctx* o, int tok, int pos, double* z_out) {
     int d = o->c.d_model, V = o->c.vocab;
     double* h = malloc(sizeof(double) * d);
@@ -341,7 +407,7 @@ static int full_step(orc_ctx* o, int tok, int pos, double* z_out) {
     embed_row(o, tok, h);
     for (int l = 1; l <= o->c.n_layers; ++l) layer_row(o, l, h, pos);
     head_logits(o, h, z);
-    int t = argmax_first(z, V);
+    int t = next_token(o, z, pos + 1, NULL);
     if (!z_out) free(z);
     free(h);
     return t;
@@ -354,8 +420,9 @@ int orc_prefill(orc_ctx* o, const int32_t* prompt, int n_prompt) {
     return t;
 }
 
-/* Plain greedy autoregressive decoding: the definition of the correct output.
- * margins (nullable) receives top1 - top2 of the final logits behind each token. */
+/* Plain autoregressive decoding (greedy, or sampling when set): the definition of the correct
+ * output.  margins (nullable) receives top1 - top2 of the final logits behind each token; under
+ * sampling, the distance from u to the nearer edge of the chosen token's CDF interval. */
 int orc_ar_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int n_gen, int32_t* out, double* margins) {
     if (n_prompt < 1 || n_prompt + n_gen > o->c.max_seq) return -1;
     int V = o->c.vocab;
@@ -366,7 +433,9 @@ int orc_ar_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int n_gen, 
         tok = full_step(o, in, p, z);
         if (p >= n_prompt - 1) {
             out[p - n_prompt + 1] = tok;
-            if (margins) {
+            if (margins && o->sample_temperature > 0.0) {
+                next_token(o, z, p + 1, &margins[p - n_prompt + 1]);   /* CDF slack instead of a logit margin */
+            } else if (margins) {
                 double second = -INFINITY;
                 for (int v = 0; v < V; ++v) if (v != tok && z[v] > second) second = z[v];
                 margins[p - n_prompt + 1] = z[tok] - second;
@@ -446,7 +515,7 @@ int orc_bruteforce_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int
             }
         }
         head_logits(o, X + (size_t)(n - 1) * d, z);
-        toks[n] = out[gi] = argmax_first(z, V);
+        toks[n] = out[gi] = next_token(o, z, n, NULL);
     }
     free(toks); free(X); free(A); free(Q); free(Kl); free(Vl); free(O); free(G); free(U); free(P); free(sc); free(z);
     return n_gen;
@@ -462,7 +531,8 @@ int orc_teacher_forced(orc_ctx* o, const int32_t* tokens, int n_total, int from,
     double* z = malloc(sizeof(double) * V);
     for (int p = 0; p < n_total - 1; ++p) {
         if (p < from - 1) { full_step(o, tokens[p], p, z); continue; }
-        int t1 = full_step(o, tokens[p], p, z);
+        full_step(o, tokens[p], p, z);
+        int t1 = argmax_first(z, V);
         int t2 = -1;
         for (int v = 0; v < V; ++v) if (v != t1 && (t2 < 0 || z[v] > z[t2])) t2 = v;
         int k = p - (from - 1);
@@ -546,7 +616,7 @@ int orc_specbound_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int 
         }
         for (int i = 0; i < w; ++i) {
             head_logits(o, h + (size_t)i * d, z);
-            R.g[i] = argmax_first(z, V);
+            R.g[i] = next_token(o, z, n + i + 1, NULL);   /* row i holds position n+i and predicts n+i+1 */
         }
         /* greedy acceptance: the longest prefix of drafts the full model reproduces, then the
          * model's own token at the first row that had no draft or a wrong one */
