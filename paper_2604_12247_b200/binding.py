@@ -66,7 +66,7 @@ class SBError(RuntimeError):
 EXPORTS = ("sb_workspace_bytes", "sb_create", "sb_destroy", "sb_load_weights", "sb_reset", "sb_get_state",
            "sb_selftest_wait_timeout",
            "sb_read_hidden", "sb_prefill", "sb_draft_push", "sb_draft_advance", "sb_exit_confidence", "sb_verify",
-           "sb_generate", "sb_generate_ar", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
+           "sb_generate", "sb_generate_ar", "sb_set_sampling", "sb_sample_uniform", "sb_k_sample", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
            "sb_k_layer",
            "sb_tau_schedule", "sb_model_speedup", "sb_set_option", "sb_set_default_option", "sb_strerror")
 
@@ -101,6 +101,10 @@ def lib():
         L.sb_generate.argtypes = [vp, vp, i32, i32, i32, i32, vp, f32, vp, C.POINTER(i32), C.POINTER(Stats), vp, i32,
                                   C.POINTER(i32)]
         L.sb_generate_ar.argtypes = [vp, vp, i32, i32, vp, C.POINTER(i32), C.POINTER(Stats)]
+        L.sb_set_sampling.argtypes = [vp, f32, C.c_uint64]
+        L.sb_sample_uniform.argtypes = [C.c_uint64, C.c_int64]
+        L.sb_sample_uniform.restype = C.c_double
+        L.sb_k_sample.argtypes = [vp, i32, i32, f32, C.c_uint64, C.c_int64, vp, vp]
         L.sb_k_exit_confidence.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp, vp, C.c_size_t, vp]
         L.sb_k_exit_confidence_static.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp]
         L.sb_k_layer.argtypes = [C.POINTER(Config), C.POINTER(LayerWeights), vp, i32, vp, vp, vp, i32, vp, C.c_size_t, vp]
@@ -145,6 +149,11 @@ def tau_schedule(alpha: float, L: int) -> np.ndarray:
 
 def model_speedup(L: int, a: float, w: int, d_max: int) -> float:
     return lib().sb_model_speedup(L, a, w, d_max)
+
+
+def sample_uniform(seed: int, pos: int) -> float:
+    """sb_sample_uniform: the uniform number that decides the token at sequence position pos."""
+    return float(lib().sb_sample_uniform(int(seed), int(pos)))
 
 
 def set_default_gemm(value: int):
@@ -251,6 +260,10 @@ class Context:
             res["rounds"] = [rounds[i] for i in range(nr.value)]
         return res
 
+    def set_sampling(self, temperature: float, seed: int = 0):
+        """sb_set_sampling: temperature 0 restores greedy decoding."""
+        _check(lib().sb_set_sampling(self.h, float(temperature), int(seed)), "sb_set_sampling")
+
     def generate_ar(self, prompt: Sequence[int], n_gen: int):
         pr = np.ascontiguousarray(prompt, dtype=np.int32)
         out = np.zeros(n_gen, dtype=np.int32)
@@ -285,6 +298,15 @@ def k_exit_confidence(cfg: Config, h: torch.Tensor, final_norm: torch.Tensor, lm
                                       C.c_void_p(scratch.ptr), scratch.nbytes, _stream_handle(stream)),
            "sb_k_exit_confidence")
     return (conf, tok, logits) if want_logits else (conf, tok)
+
+
+def k_sample(logits: torch.Tensor, temperature: float, seed: int, pos0: int, stream=None) -> torch.Tensor:
+    """sb_k_sample on a [m, vocab] fp32 device tensor -> int32 tokens [m] (device)."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
+    tok = torch.empty(logits.shape[0], dtype=torch.int32, device=logits.device)
+    _check(lib().sb_k_sample(logits.data_ptr(), logits.shape[0], logits.shape[1], float(temperature), int(seed), int(pos0),
+                             tok.data_ptr(), _stream_handle(stream)), "sb_k_sample")
+    return tok
 
 
 def k_exit_confidence_static(cfg: Config, h: torch.Tensor, final_norm: torch.Tensor, lm_head: torch.Tensor, tau_l: float,

@@ -115,6 +115,7 @@ struct Work {
     int* toks;             // [max_seq + 8] device token log
     unsigned int* status;  // device status word of the bounded waits
     float2* rope_tab;      // contexts only: cos/sin of the RoPE angles [n_pages * page][hd/2]
+    float* logits;         // contexts only: [8][V] final logits of the rows being sampled (sampling decoding)
     void* k_cache;         // [L][n_pages][page][kvd]
     void* v_cache;
 };
@@ -154,8 +155,10 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     W.status = reinterpret_cast<unsigned int*>(W.res + 48);
     W.ticket = reinterpret_cast<unsigned int*>(W.res + 56);
     W.rope_tab = nullptr;
+    W.logits = nullptr;
     if (with_state) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
+        c.take(W.logits, sizeof(float) * (size_t)kMaxW * D.V);
         c.take(W.rope_tab, sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2));
         size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
         c.take(W.k_cache, kv);
@@ -321,6 +324,8 @@ struct sb_ctx {
     int64_t probes_issued = 0;
     int n = 0, pending = -1, rows = 0;
     int depth[SB_MAX_W];
+    float sample_temperature = 0.f;      // sampling decoding (Section 4.3): 0 = greedy
+    unsigned long long sample_seed = 0;
     cudaEvent_t ev[9];   // 0 draft start, 1 verify start, 2 round end, 3/4 unified pass, 5/6 probe kernel, 7/8 decode phase
     int64_t h2d = 0, d2h = 0;
     TcPlanCache plans;
@@ -387,6 +392,23 @@ static void run_layer(sb_ctx* c, int layer, int r0, int m, const void* next_gain
 }
 
 // run layer `layer` on the trailing rows whose depth is layer-1; returns rows advanced
+// The decoding rule at the last layer for rows [r0, r0+m) (their final-norm activation is in place): greedy top-1
+// from the fused head kernel, or, under sampling decoding (Section 4.3), the head kernel writes the logits and the
+// sampling kernel draws token[r0 + j] at the uniform number of sequence position pos0 + j.  `mir` is published by
+// whichever kernel runs last.
+static void final_tokens(sb_ctx* c, int r0, int m, long long pos0, int* token, const Mirror& mir) {
+    Exec& e = c->e;
+    if (c->sample_temperature <= 0.f) {
+        head(e, c->w.lm_head, r0, m, 1.f, 2.f, c->conf_d(), token, c->flag_d(), nullptr, mir);
+        return;
+    }
+    head(e, c->w.lm_head, r0, m, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), e.W.logits);
+    SampleArgs a{e.W.logits, e.D.V, r0, m, (double)c->sample_temperature, c->sample_seed, pos0, token,
+                 reinterpret_cast<unsigned int*>(e.W.res + 57), mir};
+    launch_sample(e.st, a);
+    e.launches++;
+}
+
 static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats* st) {
     int r0 = c->rows;
     while (r0 > 0 && c->depth[r0 - 1] == layer - 1) --r0;
@@ -403,7 +425,7 @@ static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats*
 // ---------------------------------------------------------------------------------------------
 constexpr size_t kStaticScratchBytes = size_t(1) << 20;   // 1 MiB
 constexpr int kStaticMaxDModel = 8192;                    // widest model whose rows fit it
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes + 256];   // + the sampling kernel's counter word
 
 // what the exit-confidence call keeps in scratch: hidden rows, the normalised operand, the per-CTA
 // softmax triples, the ticket, the result block and the status word
@@ -592,6 +614,16 @@ int sb_set_default_option(int32_t key, int32_t value) {
     return SB_ERR_ARG;
 }
 
+int sb_set_sampling(sb_ctx* c, float temperature, uint64_t seed) {
+    if (!c || temperature != temperature || temperature < 0.f) return SB_ERR_ARG;
+    if (temperature > 0.f && c->e.D.V > kSampleMaxVocab) return SB_ERR_CAPACITY;
+    c->sample_temperature = temperature;
+    c->sample_seed = seed;
+    return SB_OK;
+}
+
+double sb_sample_uniform(uint64_t seed, int64_t pos) { return sample_uniform(seed, pos); }
+
 static int check_tokens(const sb_ctx* c, const int32_t* t, int n) {
     for (int i = 0; i < n; ++i)
         if (t[i] < 0 || t[i] >= c->e.D.V) return SB_ERR_ARG;
@@ -624,7 +656,7 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
     c->n = n_prompt;
     ensure_act(e, c->w.final_norm, m - 1, 1);
     const Mirror mir = next_mirror(c);
-    head(e, c->w.lm_head, m - 1, 1, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), nullptr, mir);
+    final_tokens(c, m - 1, 1, n_prompt, c->token_d(), mir);
     int rc = wait_results(c, mir);
     if (rc) return rc;
     c->pending = c->mailbox[8 + (m - 1)];
@@ -723,7 +755,7 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     }
     cudaEventRecord(c->ev[4], e.st);
     ensure_act(e, c->w.final_norm, 0, w);
-    head(e, c->w.lm_head, 0, w, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
+    final_tokens(c, 0, w, (long long)c->n + 1, c->token_d(), Mirror{nullptr, nullptr, 0u});   // row i holds position n + i
     int d8[kMaxW];
     for (int i = 0; i < kMaxW; ++i) d8[i] = i < w ? drafts[i] : -1;
     const Mirror mir = next_mirror(c);
@@ -872,7 +904,7 @@ int sb_generate_ar(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n
         e.act_gain = nullptr;
         for (int l = 1; l <= e.D.L; ++l)
             layer_step(e, c->layers[l - 1], c->kc(l), c->vc(l), 0, 1, c->n, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
-        head(e, c->w.lm_head, 0, 1, 1.f, 2.f, c->conf_d(), log + i, c->flag_d(), nullptr);
+        final_tokens(c, 0, 1, (long long)c->n + 1, log + i, Mirror{nullptr, nullptr, 0u});
         c->n += 1;
         st->layer_steps += e.D.L; st->layer_row_steps += e.D.L; st->rounds++; st->rows++;
     }
@@ -918,6 +950,21 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     ensure_act(e, final_norm, 0, m);
     head(e, lm_head, 0, m, tau_l, 2.f, conf, token, e.W.res + 16, logits_dbg);
     if (e.err) return e.err;
+    return cuda_ok(cudaGetLastError());
+}
+
+// Sampling kernel alone: tokens of m rows of device logits.  Its completion counter is the word behind the static
+// scratch (zero at load, left at zero by every launch).
+int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, uint64_t seed, int64_t pos0,
+                int32_t* token, void* stream) {
+    if (!logits || !token || m < 1 || m > SB_MAX_W || vocab < 1 || !(temperature > 0.f)) return SB_ERR_ARG;
+    if (vocab > kSampleMaxVocab) return SB_ERR_CAPACITY;
+    char* base = nullptr;
+    int rc = static_scratch_ptr(&base);
+    if (rc) return rc;
+    SampleArgs a{logits, vocab, 0, m, (double)temperature, seed, pos0, token,
+                 reinterpret_cast<unsigned int*>(base + kStaticScratchBytes), Mirror{nullptr, nullptr, 0u}};
+    launch_sample((cudaStream_t)stream, a);
     return cuda_ok(cudaGetLastError());
 }
 

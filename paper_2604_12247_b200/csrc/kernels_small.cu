@@ -650,6 +650,103 @@ void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int
     launch_k(k_accept, dim3(1), dim3(64), 0, st, g, d, w, max_emit, result, mirror);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Sampling decoding (Section 4.3, decoding strategies): token = inverse CDF, in vocabulary order, of
+// softmax(z / temperature) at the uniform number of the token's sequence position.  One CTA per row.
+// The vocabulary is cut into cells of 128 consecutive tokens; a warp sums a cell (coalesced loads, fixed
+// shuffle tree, fp64), the CTA scans the cell sums in order, and the one thread whose cells straddle
+// u * total walks its cell token by token.  The exponentials and sums are fp64 (a few thousand per thread at
+// most), so that for equal logits the token can differ from an fp64 reference only by summation order.
+// Everything is a pure function of (logits, u): deterministic.
+// ------------------------------------------------------------------------------------------------
+constexpr int kSampleThreads = 1024;
+constexpr int kSampleCell = 128;
+constexpr int kSampleMaxCells = kSampleMaxVocab / kSampleCell;
+
+__global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ double s_cell[kSampleMaxCells];
+    __shared__ double s_warp[32];
+    __shared__ float s_maxw[32];
+    __shared__ int s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int V = a.V, row = blockIdx.x;
+    const float* __restrict__ z = a.logits + (size_t)row * V;
+
+    float mx = -INFINITY;
+    for (int v = tid; v < V; v += kSampleThreads) mx = fmaxf(mx, __ldcg(z + v));
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) s_maxw[warp] = mx;
+    __syncthreads();
+    mx = s_maxw[0];
+    for (int i = 1; i < 32; ++i) mx = fmaxf(mx, s_maxw[i]);
+
+    const int n_cells = (V + kSampleCell - 1) / kSampleCell;
+    for (int c = warp; c < n_cells; c += 32) {
+        double s = 0.0;
+#pragma unroll
+        for (int j = 0; j < kSampleCell / 32; ++j) {
+            int v = c * kSampleCell + j * 32 + lane;
+            if (v < V) s += exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+        }
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) s_cell[c] = s;
+    }
+    __syncthreads();
+
+    // exclusive scan of the cell sums in vocabulary order: thread t owns cells [t*per, (t+1)*per)
+    const int per = (n_cells + kSampleThreads - 1) / kSampleThreads;
+    const int c0 = tid * per, c1 = min(c0 + per, n_cells);
+    double mine = 0.0;
+    for (int c = c0; c < c1; ++c) mine += s_cell[c];
+    double incl = mine;
+    for (int o = 1; o < 32; o <<= 1) {
+        double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    double before = 0.0, total = 0.0;
+    for (int i = 0; i < 32; ++i) {
+        if (i < warp) before += s_warp[i];
+        total += s_warp[i];
+    }
+    // [lower, upper] of consecutive threads tile [0, total] exactly: lower is the previous thread's upper, computed by
+    // the same additions, so exactly one thread sees lower < target <= upper
+    double lower = __shfl_up_sync(0xffffffffu, incl, 1);
+    lower = lane == 0 ? before : before + lower;
+    const double upper = before + incl;
+    const double target = sample_uniform(a.seed, a.pos0 + row) * total;
+    if (lower < target && target <= upper) {
+        double run = lower;
+        int c = c0;
+        while (c < c1 - 1 && run + s_cell[c] < target) run += s_cell[c++];
+        const int v0 = c * kSampleCell, v1 = min(v0 + kSampleCell, V);
+        int pick = -1;
+        for (int v = v0; v < v1; ++v) {
+            double e = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+            if (e > 0.0) pick = v;                     // last token with mass, if the walk falls an ulp short
+            run += e;
+            if (run >= target) break;
+        }
+        if (pick < 0) pick = v0;
+        a.token[a.r0 + row] = pick;
+        __threadfence();
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        s_last = atomicInc(a.counter, gridDim.x - 1) == gridDim.x - 1;   // wraps back to zero
+        __threadfence();
+    }
+    __syncthreads();
+    if (s_last) publish_results(a.mirror);
+}
+void launch_sample(cudaStream_t st, const SampleArgs& a) {
+    launch_k(k_sample, dim3(a.m), dim3(kSampleThreads), 0, st, a);
+}
+
 __global__ void k_init_pages(int* pt, int n) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) pt[i] = i;

@@ -254,6 +254,30 @@ __device__ __forceinline__ void publish_results(const Mirror& m) {
     if (threadIdx.x == 0) reinterpret_cast<volatile unsigned int*>(m.host)[63] = m.seq;
 }
 
+// ---- sampling decoding (Section 4.3, decoding strategies; Table 2) ----
+// Counter-based uniform number that decides the token at sequence position `pos`: the splitmix64 output
+// function of seed + (pos + 1) * golden-ratio increment, top 53 bits centred in their cell, in (0, 1).
+__host__ __device__ inline unsigned long long sample_hash(unsigned long long seed, long long pos) {
+    unsigned long long x = seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(pos + 1);
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+__host__ __device__ inline double sample_uniform(unsigned long long seed, long long pos) {
+    return ((double)(sample_hash(seed, pos) >> 11) + 0.5) * (1.0 / 9007199254740992.0);
+}
+constexpr int kSampleMaxVocab = 262144;
+struct SampleArgs {
+    const float* logits;       // [m][V] final logits, row r0 first
+    int V, r0, m;
+    double temperature;        // sampling temperature T_s > 0
+    unsigned long long seed;
+    long long pos0;            // sequence position of the token that row r0 produces (row r0 + j: pos0 + j)
+    int* token;                // token[r0 + j] receives the sample
+    unsigned int* counter;     // one zero-initialised word; left at zero
+    Mirror mirror;             // published by the CTA that finishes last; may be null
+};
+
 // ---------------------------------------------------------------------------------------------
 // Launch arguments
 // ---------------------------------------------------------------------------------------------
@@ -342,6 +366,7 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror);
+void launch_sample(cudaStream_t st, const SampleArgs& a);
 void launch_init_pages(cudaStream_t st, int* page_table, int n_pages);
 
 // ---- launchers (gemm_simt.cu) ----

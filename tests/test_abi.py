@@ -51,3 +51,12 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "nope.so")
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_sampling_uniforms_equal_the_oracles_generator(lib):
+    """Host function of the library (no GPU): both sides implement the same counter-based generator."""
+    from oracle import oracle
+    from paper_2604_12247_b200 import binding
+    for seed in (0, 1, 2 ** 63 + 12345, 2 ** 64 - 1):
+        for pos in (0, 1, 511, 1023, 10 ** 9):
+            assert binding.sample_uniform(seed, pos) == oracle.uniform(seed, pos)
