@@ -329,9 +329,28 @@ def sweep_arm(args, run: inputs.Run):
                        "mean_width": st.rows / max(st.rounds, 1), "draft_acceptance": acc,
                        "eq5_speedup_at_that_acceptance": binding.model_speedup(s.n_layers, min(acc, 0.999), w_max, d_max),
                        "probes": st.probes})
+    # decoding strategies (Section 4.3, Table 2): greedy and temperature sampling at the workload's own setting;
+    # under sampling the baseline is autoregressive sampling with the same temperature and seed
+    strategies = []
+    tau = list(run.tau[:run.d_max])
+    for name, temp in (("greedy", 0.0), ("temperature 0.3", 0.3), ("temperature 1.0", 1.0)):
+        ctx.set_sampling(temp, run.seed)
+        for _ in range(2):
+            a = ctx.generate_ar(pr, n_gen)
+            sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, tau, run.threshold)
+        a_tps = (n_gen - 1) / (a["stats"].us_decode_dev * 1e-6)
+        tps = (n_gen - 1) / (sp["stats"].us_decode_dev * 1e-6)
+        st = sp["stats"]
+        drafts = sum(st.exit_hist[1:])
+        strategies.append({"strategy": name, "ar_tokens_per_s": a_tps, "tokens_per_s": tps, "speedup_vs_ar": tps / a_tps,
+                           "tokens_equal_ar": bool((sp["tokens"] == a["tokens"]).all()),
+                           "emitted_per_round": st.emitted / max(st.rounds, 1),
+                           "draft_acceptance": st.accepted_drafts / drafts if drafts else 0.0})
+    ctx.set_sampling(0.0, 0)
     ctx.close()
     print(json.dumps({"mode": "sweep", "workload": workload_config(run, "single GPU")["workload"], "prompt_tokens": n_prompt,
-                      "generated_tokens": n_gen, "ar_tokens_per_s": ar_tps, "points": points}), flush=True)
+                      "generated_tokens": n_gen, "ar_tokens_per_s": ar_tps, "points": points,
+                      "decoding_strategies": strategies}), flush=True)
 
 
 def micro_arm(args):

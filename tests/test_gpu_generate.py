@@ -369,6 +369,9 @@ def test_bench_sweep_mode_on_tiny(capsys):
     assert {p["d_max"] for p in pts} == {1, 2} and {p["w_max"] for p in pts} == {2, 4, 8}
     assert all(1.0 <= p["emitted_per_round"] <= p["w_max"] and 0.0 <= p["draft_acceptance"] <= 1.0 for p in pts)
     assert max(p["emitted_per_round"] for p in pts) > 1.5
+    strat = line["decoding_strategies"]
+    assert [x["strategy"] for x in strat] == ["greedy", "temperature 0.3", "temperature 1.0"]
+    assert all(x["tokens_equal_ar"] and x["tokens_per_s"] > 0 and x["ar_tokens_per_s"] > 0 for x in strat)
 
 
 def test_host_side_options_do_not_change_results(tiny_damped_weights):
