@@ -76,8 +76,10 @@ def lib():
         L.orc_mix64.argtypes = [C.c_uint64, C.c_int64]
         L.orc_uniform.restype = C.c_double
         L.orc_uniform.argtypes = [C.c_uint64, C.c_int64]
-        L.orc_sample_token.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p]
-        L.orc_set_sampling.argtypes = [C.c_void_p, C.c_double, C.c_uint64]
+        L.orc_sample_token.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_double, C.c_void_p]
+        L.orc_nucleus_threshold.restype = C.c_double
+        L.orc_nucleus_threshold.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double]
+        L.orc_set_sampling.argtypes = [C.c_void_p, C.c_double, C.c_double, C.c_uint64]
         L.orc_set_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_get_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_layer_forward.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int]
@@ -125,12 +127,19 @@ def uniform(seed: int, pos: int) -> float:
     return float(lib().orc_uniform(seed, pos))
 
 
-def sample_token(z: np.ndarray, temperature: float, u: float):
-    """Inverse-CDF sample of softmax(z / temperature) in vocabulary order -> (token, slack)."""
+def sample_token(z: np.ndarray, temperature: float, u: float, top_p: float = 1.0):
+    """Inverse-CDF sample, in vocabulary order, of softmax(z / temperature) restricted to its top-p nucleus
+    -> (token, slack)."""
     z = np.ascontiguousarray(z, dtype=np.float64)
     slack = C.c_double()
-    t = lib().orc_sample_token(_ptr(z), z.size, float(temperature), float(u), C.byref(slack))
+    t = lib().orc_sample_token(_ptr(z), z.size, float(temperature), float(top_p), float(u), C.byref(slack))
     return int(t), float(slack.value)
+
+
+def nucleus_threshold(z: np.ndarray, temperature: float, top_p: float) -> float:
+    """Smallest logit inside the top-p nucleus of softmax(z / temperature) (-inf for top_p >= 1)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    return float(lib().orc_nucleus_threshold(_ptr(z), z.size, float(temperature), float(top_p)))
 
 
 def confidence(z: np.ndarray, T: float):
@@ -187,9 +196,9 @@ class Oracle:
         except Exception:
             pass
 
-    def set_sampling(self, temperature: float, seed: int = 0):
-        """Sampling decoding (Section 4.3): temperature 0 restores greedy decoding."""
-        lib().orc_set_sampling(self.h, float(temperature), int(seed))
+    def set_sampling(self, temperature: float, seed: int = 0, top_p: float = 1.0):
+        """Sampling decoding (Section 4.3): temperature 0 restores greedy decoding; top_p < 1 = nucleus sampling."""
+        lib().orc_set_sampling(self.h, float(temperature), float(top_p), int(seed))
 
     def set_exit_head(self, layer: int, head: Optional[torch.Tensor], norm: Optional[torch.Tensor] = None):
         """Head [vocab, d_model] (and norm gain [d_model]) of the exit test after `layer`; None = the shared ones."""

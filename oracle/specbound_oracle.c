@@ -27,8 +27,8 @@
  * Sampling decoding (Section 4.3 "decoding strategies", Table 2): the paper names
  * temperature sampling but prints no acceptance rule.  The reading taken here:
  * the token at sequence position p is the inverse-CDF sample, in vocabulary
- * order, of softmax(z / T_s) at the uniform number u(seed, p) of a counter-based
- * generator; verification recomputes that token for every draft row and accepts
+ * order, of softmax(z / T_s) -- restricted to its top-p nucleus when top_p < 1 --
+ * at the uniform number u(seed, p) of a counter-based generator; verification recomputes that token for every draft row and accepts
  * a draft iff it equals it.  Autoregressive sampling with the same (seed, T_s)
  * DEFINES the correct output; the speculative loop must reproduce it token for
  * token, which makes it lossless sample by sample and hence in distribution.
@@ -87,7 +87,7 @@ typedef struct orc_ctx {
     const void** exit_head;
     const void** exit_norm;
     /* sampling decoding (Section 4.3, decoding strategies): temperature 0 = greedy */
-    double sample_temperature;
+    double sample_temperature, sample_top_p;
     uint64_t sample_seed;
 } orc_ctx;
 
@@ -252,18 +252,51 @@ double orc_uniform(uint64_t seed, int64_t pos) {
     return ((double)(orc_mix64(seed, pos) >> 11) + 0.5) * (1.0 / 9007199254740992.0);
 }
 
-/* Inverse-CDF sample of softmax(z / temperature) in vocabulary order: the first token v
- * whose cumulative un-normalised mass reaches u * total.  slack (nullable) receives the
- * distance from u to the nearer edge of the chosen token's CDF interval. */
-int orc_sample_token(const double* z, int V, double temperature, double u, double* slack) {
+/* Nucleus of top-p sampling, as a logit threshold: the largest logit value z* such that the tokens
+ * with z_v >= z* hold at least top_p of the mass of softmax(z / temperature).  The nucleus is
+ * {v : z_v >= z*}: tokens in descending order of probability until top_p is reached, equal logits
+ * entering together.  top_p >= 1: -infinity (every token). */
+static const double* g_sort_key;
+static int by_logit_desc(const void* a, const void* b) {
+    double x = g_sort_key[*(const int*)a], y = g_sort_key[*(const int*)b];
+    if (x != y) return x > y ? -1 : 1;
+    return *(const int*)a - *(const int*)b;
+}
+double orc_nucleus_threshold(const double* z, int V, double temperature, double top_p) {
+    if (!(top_p < 1.0)) return -INFINITY;
     double m = z[0];
     for (int v = 1; v < V; ++v) if (z[v] > m) m = z[v];
     double total = 0.0;
     for (int v = 0; v < V; ++v) total += exp((z[v] - m) / temperature);
+    int* idx = malloc(sizeof(int) * V);
+    for (int v = 0; v < V; ++v) idx[v] = v;
+    g_sort_key = z;
+    qsort(idx, V, sizeof(int), by_logit_desc);
+    double acc = 0.0, zstar = z[idx[V - 1]];
+    for (int k = 0; k < V; ++k) {
+        acc += exp((z[idx[k]] - m) / temperature);
+        int group_ends = k == V - 1 || z[idx[k + 1]] != z[idx[k]];
+        if (group_ends && acc >= top_p * total) { zstar = z[idx[k]]; break; }
+    }
+    free(idx);
+    return zstar;
+}
+
+/* Inverse-CDF sample, in vocabulary order, of softmax(z / temperature) restricted to the top-p
+ * nucleus (top_p >= 1: all tokens) and renormalised: the first nucleus token whose cumulative
+ * un-normalised mass reaches u * (mass of the nucleus).  slack (nullable) receives the distance
+ * from u to the nearer edge of the chosen token's CDF interval. */
+int orc_sample_token(const double* z, int V, double temperature, double top_p, double u, double* slack) {
+    double m = z[0];
+    for (int v = 1; v < V; ++v) if (z[v] > m) m = z[v];
+    double zstar = orc_nucleus_threshold(z, V, temperature, top_p);
+    double total = 0.0;
+    for (int v = 0; v < V; ++v) if (z[v] >= zstar) total += exp((z[v] - m) / temperature);
     double target = u * total, run = 0.0;
     int pick = -1;
     double lo = 0.0;
     for (int v = 0; v < V; ++v) {
+        if (!(z[v] >= zstar)) continue;
         double e = exp((z[v] - m) / temperature);
         if (e > 0.0) pick = v;                      /* rounding guard: last token with mass */
         if (run + e >= target) { pick = v; lo = run; run += e; break; }
@@ -282,11 +315,12 @@ int orc_sample_token(const double* z, int V, double temperature, double u, doubl
  * sample at u(seed, pos), pos = sequence position of the token being produced. */
 static int next_token(const orc_ctx* o, const double* z, int pos, double* slack) {
     if (o->sample_temperature > 0.0)
-        return orc_sample_token(z, o->c.vocab, o->sample_temperature, orc_uniform(o->sample_seed, pos), slack);
+        return orc_sample_token(z, o->c.vocab, o->sample_temperature, o->sample_top_p, orc_uniform(o->sample_seed, pos), slack);
     return argmax_first(z, o->c.vocab);
 }
-void orc_set_sampling(orc_ctx* o, double temperature, uint64_t seed) {
+void orc_set_sampling(orc_ctx* o, double temperature, double top_p, uint64_t seed) {
     o->sample_temperature = temperature > 0.0 ? temperature : 0.0;
+    o->sample_top_p = top_p > 0.0 && top_p < 1.0 ? top_p : 1.0;
     o->sample_seed = seed;
 }
 

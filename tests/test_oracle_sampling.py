@@ -11,7 +11,10 @@ softmax(z / T_s) at a counter-based uniform u(seed, p); a draft is accepted iff 
 * sampling really is autoregressive sampling from the model: each generated token equals the
   sampler applied to logits recomputed by the no-cache brute-force path,
 * speculative == autoregressive, token for token, over a (d_max, w_max, threshold, T_s) grid,
-* the empirical frequency of the first generated token over many seeds against its softmax.
+* the empirical frequency of the first generated token over many seeds against its softmax,
+* top-p: the nucleus against a library sort + cumulative sum, ties entering together, the
+  renormalised counts inside the nucleus, the top_p -> 1 and top_p -> 0 limits, and
+  speculative == autoregressive under nucleus sampling.
 """
 import itertools
 
@@ -182,3 +185,61 @@ def test_first_token_frequency_over_seeds_follows_softmax(tiny):
         (p[~big] * N).sum(), 1e-9)
     dof = int(big.sum())
     assert chi2 < dof + 5 * np.sqrt(2 * dof), (chi2, dof)
+
+
+@pytest.mark.parametrize("temperature,top_p", [(1.0, 0.9), (0.5, 0.5), (2.0, 0.99), (1.0, 0.05)])
+def test_nucleus_matches_library_sort_and_cumsum(temperature, top_p):
+    g = torch.Generator().manual_seed(13)
+    z = (torch.randn(61, generator=g, dtype=torch.float64) * 2).numpy()
+    p = torch.softmax(torch.from_numpy(z) / temperature, 0)
+    ps, order = torch.sort(p, descending=True)
+    k = int(torch.nonzero(torch.cumsum(ps, 0) >= top_p)[0]) + 1        # tokens in the nucleus (no ties in random data)
+    members = set(order[:k].tolist())
+    zstar = oracle.nucleus_threshold(z, temperature, top_p)
+    assert {v for v in range(z.size) if z[v] >= zstar} == members
+    assert float(p[list(members)].sum()) >= top_p > float(p[list(members)].sum()) - float(ps[k - 1])   # minimal
+    # stratified counts follow the renormalised probabilities inside the nucleus, nothing falls outside
+    q = np.where(z >= zstar, p.numpy(), 0.0)
+    q /= q.sum()
+    N = 8000
+    counts = np.zeros(z.size)
+    for i in range(N):
+        counts[oracle.sample_token(z, temperature, (i + 0.5) / N, top_p)[0]] += 1
+    assert np.abs(counts - q * N).max() <= 1.0 + 1e-6
+    assert counts[[v for v in range(z.size) if v not in members]].sum() == 0
+
+
+def test_nucleus_ties_and_limits():
+    z = np.array([1.0, 0.0, 1.0, -3.0, 1.0, 0.0])
+    # the three tied maxima hold 3e / (3e + 2 + e^-3) = 0.80 of the mass and enter together
+    assert oracle.nucleus_threshold(z, 1.0, 0.05) == 1.0
+    assert oracle.nucleus_threshold(z, 1.0, 0.79) == 1.0
+    assert oracle.nucleus_threshold(z, 1.0, 0.81) == 0.0            # then both zeros together
+    assert oracle.nucleus_threshold(z, 1.0, 0.9999) == -3.0
+    assert oracle.nucleus_threshold(z, 1.0, 1.0) == -np.inf
+    assert {oracle.sample_token(z, 1.0, u, 0.5)[0] for u in np.linspace(0.001, 0.999, 50)} == {0, 2, 4}
+    # thirds of the unit interval map to the three maxima in vocabulary order
+    assert [oracle.sample_token(z, 1.0, u, 0.5)[0] for u in (0.2, 0.5, 0.9)] == [0, 2, 4]
+    g = torch.Generator().manual_seed(2)
+    r = torch.randn(40, generator=g, dtype=torch.float64).numpy()
+    for u in (0.01, 0.4, 0.8, 0.99):
+        assert oracle.sample_token(r, 0.8, u, 1.0) == oracle.sample_token(r, 0.8, u)       # top_p = 1: no restriction
+        assert oracle.sample_token(r, 0.8, u, 1e-9)[0] == int(np.argmax(r))               # top_p -> 0: the top-1 alone
+
+
+def test_speculative_equals_autoregressive_under_nucleus_sampling(tiny_damped_weights):
+    run = inputs.RUNS["tiny-damped"]
+    w = tiny_damped_weights
+    pr = inputs.make_prompt(run.shape, run.n_prompt, run.seed).numpy()
+    n_gen = 20
+    a = oracle.Oracle(run.shape, w, 64)
+    a.set_sampling(1.0, 5, top_p=0.9)
+    ar = a.ar_generate(pr, n_gen)
+    plain = oracle.Oracle(run.shape, w, 64)
+    plain.set_sampling(1.0, 5)
+    assert not np.array_equal(ar, plain.ar_generate(pr, n_gen))       # the nucleus changes the sampled sequence
+    for d_max, w_max, thr in ((1, 8, 0.0), (2, 4, 0.25), (3, 3, 2.0)):
+        o = oracle.Oracle(run.shape, w, 64)
+        o.set_sampling(1.0, 5, top_p=0.9)
+        out, _ = o.specbound_generate(pr, n_gen, d_max, w_max, inputs.tau_linear(d_max, 1.5, 1.0), thr)
+        assert np.array_equal(out, ar), (d_max, w_max, thr)
