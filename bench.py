@@ -329,12 +329,13 @@ def sweep_arm(args, run: inputs.Run):
                        "mean_width": st.rows / max(st.rounds, 1), "draft_acceptance": acc,
                        "eq5_speedup_at_that_acceptance": binding.model_speedup(s.n_layers, min(acc, 0.999), w_max, d_max),
                        "probes": st.probes})
-    # decoding strategies (Section 4.3, Table 2): greedy and temperature sampling at the workload's own setting;
+    # decoding strategies (Section 4.3, Table 2): greedy, temperature and top-p sampling at the workload's own setting;
     # under sampling the baseline is autoregressive sampling with the same temperature and seed
     strategies = []
     tau = list(run.tau[:run.d_max])
-    for name, temp in (("greedy", 0.0), ("temperature 0.3", 0.3), ("temperature 1.0", 1.0)):
-        ctx.set_sampling(temp, run.seed)
+    for name, temp, top_p in (("greedy", 0.0, 1.0), ("temperature 0.3", 0.3, 1.0), ("temperature 1.0", 1.0, 1.0),
+                              ("top-p 0.9", 1.0, 0.9)):
+        ctx.set_sampling(temp, run.seed, top_p)
         for _ in range(2):
             a = ctx.generate_ar(pr, n_gen)
             sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, tau, run.threshold)

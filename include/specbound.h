@@ -173,19 +173,23 @@ int sb_generate_ar(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t
                    int32_t* n_out, sb_stats* stats);
 
 /* Sampling decoding (Section 4.3, "decoding strategies"; Table 2 -- the paper names temperature
- * sampling but gives no acceptance rule; this is the rule implemented).  With temperature > 0,
- * every place above that takes the full model's greedy token (sb_prefill, sb_verify, sb_generate,
- * sb_generate_ar) instead takes the inverse-CDF sample, in vocabulary order, of
- * softmax(final logits / temperature) at u = sb_sample_uniform(seed, p), p = the sequence position
- * of the token being produced (the prompt occupies 0 .. n_prompt-1): the first token v whose
- * cumulative probability reaches u.  Drafts stay the shallow layers' top-1 tokens under the
- * annealed threshold; a draft is accepted iff it equals the sampled token of its row, so
- * sb_generate returns exactly what sb_generate_ar returns for the same (temperature, seed):
- * lossless sample by sample.  The final logits of the <= SB_MAX_W rows go through a [8][vocab]
- * fp32 buffer of the workspace; the exit tests never write logits.  temperature 0 (the default)
- * restores greedy decoding.  Errors: SB_ERR_ARG (negative or NaN temperature), SB_ERR_CAPACITY
- * (vocab > 262144 with temperature > 0). */
-int sb_set_sampling(sb_ctx* ctx, float temperature, uint64_t seed);
+ * and top-p sampling but gives no acceptance rule; this is the rule implemented).  With
+ * temperature > 0, every place above that takes the full model's greedy token (sb_prefill,
+ * sb_verify, sb_generate, sb_generate_ar) instead takes the inverse-CDF sample, in vocabulary
+ * order, of softmax(final logits / temperature) at u = sb_sample_uniform(seed, p), p = the
+ * sequence position of the token being produced (the prompt occupies 0 .. n_prompt-1): the first
+ * token v whose cumulative probability reaches u.  top_p in (0, 1) restricts the distribution to
+ * its nucleus first and renormalises: the tokens with logit >= z*, z* the largest logit whose
+ * upper set holds at least top_p of the mass (tokens in descending probability until top_p is
+ * reached; equal logits enter together); top_p = 1 keeps every token.  Drafts stay the shallow
+ * layers' top-1 tokens under the annealed threshold; a draft is accepted iff it equals the
+ * sampled token of its row, so sb_generate returns exactly what sb_generate_ar returns for the
+ * same (temperature, top_p, seed): lossless sample by sample.  The final logits of the
+ * <= SB_MAX_W rows go through a [8][vocab] fp32 buffer of the workspace; the exit tests never
+ * write logits.  temperature 0 (the default) restores greedy decoding.  Errors: SB_ERR_ARG
+ * (negative or NaN temperature, top_p outside (0, 1]), SB_ERR_CAPACITY (vocab > 262144 with
+ * temperature > 0). */
+int sb_set_sampling(sb_ctx* ctx, float temperature, float top_p, uint64_t seed);
 
 /* The counter-based uniform number in (0, 1) behind sb_set_sampling: the splitmix64 output function
  * of seed + (pos + 1) * 0x9E3779B97F4A7C15, top 53 bits, centred in their cell.  Host function. */
@@ -197,11 +201,12 @@ double sb_sample_uniform(uint64_t seed, int64_t pos);
 size_t sb_k_scratch_bytes(const sb_config* cfg);
 
 /* Sampling kernel alone (the rule of sb_set_sampling): token[j] (device) = inverse-CDF sample of
- * softmax(logits[j][:] / temperature) at sb_sample_uniform(seed, pos0 + j), for m <= SB_MAX_W rows
- * of device fp32 logits [m][vocab].  Asynchronous on `stream`.  Errors: SB_ERR_ARG (null pointer,
- * m outside [1, SB_MAX_W], temperature <= 0), SB_ERR_CAPACITY (vocab > 262144). */
-int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, uint64_t seed, int64_t pos0,
-                int32_t* token, void* stream);
+ * the top_p nucleus of softmax(logits[j][:] / temperature) at sb_sample_uniform(seed, pos0 + j),
+ * for m <= SB_MAX_W rows of device fp32 logits [m][vocab].  Asynchronous on `stream`.  Errors:
+ * SB_ERR_ARG (null pointer, m outside [1, SB_MAX_W], temperature <= 0, top_p outside (0, 1]),
+ * SB_ERR_CAPACITY (vocab > 262144). */
+int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, float top_p, uint64_t seed,
+                int64_t pos0, int32_t* token, void* stream);
 
 /* Exit-confidence kernel on m rows of hidden states (Section 3.2, Eq. 2):
  * h device fp32 [m, d]; final_norm / lm_head device in cfg->dtype; tau_l > 0.

@@ -101,10 +101,10 @@ def lib():
         L.sb_generate.argtypes = [vp, vp, i32, i32, i32, i32, vp, f32, vp, C.POINTER(i32), C.POINTER(Stats), vp, i32,
                                   C.POINTER(i32)]
         L.sb_generate_ar.argtypes = [vp, vp, i32, i32, vp, C.POINTER(i32), C.POINTER(Stats)]
-        L.sb_set_sampling.argtypes = [vp, f32, C.c_uint64]
+        L.sb_set_sampling.argtypes = [vp, f32, f32, C.c_uint64]
         L.sb_sample_uniform.argtypes = [C.c_uint64, C.c_int64]
         L.sb_sample_uniform.restype = C.c_double
-        L.sb_k_sample.argtypes = [vp, i32, i32, f32, C.c_uint64, C.c_int64, vp, vp]
+        L.sb_k_sample.argtypes = [vp, i32, i32, f32, f32, C.c_uint64, C.c_int64, vp, vp]
         L.sb_k_exit_confidence.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp, vp, C.c_size_t, vp]
         L.sb_k_exit_confidence_static.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp]
         L.sb_k_layer.argtypes = [C.POINTER(Config), C.POINTER(LayerWeights), vp, i32, vp, vp, vp, i32, vp, C.c_size_t, vp]
@@ -260,9 +260,9 @@ class Context:
             res["rounds"] = [rounds[i] for i in range(nr.value)]
         return res
 
-    def set_sampling(self, temperature: float, seed: int = 0):
-        """sb_set_sampling: temperature 0 restores greedy decoding."""
-        _check(lib().sb_set_sampling(self.h, float(temperature), int(seed)), "sb_set_sampling")
+    def set_sampling(self, temperature: float, seed: int = 0, top_p: float = 1.0):
+        """sb_set_sampling: temperature 0 restores greedy decoding; top_p < 1 = nucleus sampling."""
+        _check(lib().sb_set_sampling(self.h, float(temperature), float(top_p), int(seed)), "sb_set_sampling")
 
     def generate_ar(self, prompt: Sequence[int], n_gen: int):
         pr = np.ascontiguousarray(prompt, dtype=np.int32)
@@ -300,11 +300,11 @@ def k_exit_confidence(cfg: Config, h: torch.Tensor, final_norm: torch.Tensor, lm
     return (conf, tok, logits) if want_logits else (conf, tok)
 
 
-def k_sample(logits: torch.Tensor, temperature: float, seed: int, pos0: int, stream=None) -> torch.Tensor:
+def k_sample(logits: torch.Tensor, temperature: float, seed: int, pos0: int, top_p: float = 1.0, stream=None) -> torch.Tensor:
     """sb_k_sample on a [m, vocab] fp32 device tensor -> int32 tokens [m] (device)."""
     assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
     tok = torch.empty(logits.shape[0], dtype=torch.int32, device=logits.device)
-    _check(lib().sb_k_sample(logits.data_ptr(), logits.shape[0], logits.shape[1], float(temperature), int(seed), int(pos0),
+    _check(lib().sb_k_sample(logits.data_ptr(), logits.shape[0], logits.shape[1], float(temperature), float(top_p), int(seed), int(pos0),
                              tok.data_ptr(), _stream_handle(stream)), "sb_k_sample")
     return tok
 

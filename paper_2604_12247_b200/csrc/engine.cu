@@ -325,6 +325,7 @@ struct sb_ctx {
     int n = 0, pending = -1, rows = 0;
     int depth[SB_MAX_W];
     float sample_temperature = 0.f;      // sampling decoding (Section 4.3): 0 = greedy
+    float sample_top_p = 1.f;            // nucleus mass; 1 = the whole vocabulary
     unsigned long long sample_seed = 0;
     cudaEvent_t ev[9];   // 0 draft start, 1 verify start, 2 round end, 3/4 unified pass, 5/6 probe kernel, 7/8 decode phase
     int64_t h2d = 0, d2h = 0;
@@ -403,7 +404,7 @@ static void final_tokens(sb_ctx* c, int r0, int m, long long pos0, int* token, c
         return;
     }
     head(e, c->w.lm_head, r0, m, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), e.W.logits);
-    SampleArgs a{e.W.logits, e.D.V, r0, m, (double)c->sample_temperature, c->sample_seed, pos0, token,
+    SampleArgs a{e.W.logits, e.D.V, r0, m, (double)c->sample_temperature, (double)c->sample_top_p, c->sample_seed, pos0, token,
                  reinterpret_cast<unsigned int*>(e.W.res + 57), mir};
     launch_sample(e.st, a);
     e.launches++;
@@ -614,10 +615,11 @@ int sb_set_default_option(int32_t key, int32_t value) {
     return SB_ERR_ARG;
 }
 
-int sb_set_sampling(sb_ctx* c, float temperature, uint64_t seed) {
-    if (!c || temperature != temperature || temperature < 0.f) return SB_ERR_ARG;
+int sb_set_sampling(sb_ctx* c, float temperature, float top_p, uint64_t seed) {
+    if (!c || temperature != temperature || temperature < 0.f || !(top_p > 0.f) || top_p > 1.f) return SB_ERR_ARG;
     if (temperature > 0.f && c->e.D.V > kSampleMaxVocab) return SB_ERR_CAPACITY;
     c->sample_temperature = temperature;
+    c->sample_top_p = top_p;
     c->sample_seed = seed;
     return SB_OK;
 }
@@ -955,14 +957,15 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
 
 // Sampling kernel alone: tokens of m rows of device logits.  Its completion counter is the word behind the static
 // scratch (zero at load, left at zero by every launch).
-int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, uint64_t seed, int64_t pos0,
+int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, float top_p, uint64_t seed, int64_t pos0,
                 int32_t* token, void* stream) {
     if (!logits || !token || m < 1 || m > SB_MAX_W || vocab < 1 || !(temperature > 0.f)) return SB_ERR_ARG;
+    if (!(top_p > 0.f) || top_p > 1.f) return SB_ERR_ARG;
     if (vocab > kSampleMaxVocab) return SB_ERR_CAPACITY;
     char* base = nullptr;
     int rc = static_scratch_ptr(&base);
     if (rc) return rc;
-    SampleArgs a{logits, vocab, 0, m, (double)temperature, seed, pos0, token,
+    SampleArgs a{logits, vocab, 0, m, (double)temperature, (double)top_p, seed, pos0, token,
                  reinterpret_cast<unsigned int*>(base + kStaticScratchBytes), Mirror{nullptr, nullptr, 0u}};
     launch_sample((cudaStream_t)stream, a);
     return cuda_ok(cudaGetLastError());

@@ -652,20 +652,41 @@ void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int
 
 // ------------------------------------------------------------------------------------------------
 // Sampling decoding (Section 4.3, decoding strategies): token = inverse CDF, in vocabulary order, of
-// softmax(z / temperature) at the uniform number of the token's sequence position.  One CTA per row.
-// The vocabulary is cut into cells of 128 consecutive tokens; a warp sums a cell (coalesced loads, fixed
-// shuffle tree, fp64), the CTA scans the cell sums in order, and the one thread whose cells straddle
-// u * total walks its cell token by token.  The exponentials and sums are fp64 (a few thousand per thread at
-// most), so that for equal logits the token can differ from an fp64 reference only by summation order.
+// softmax(z / temperature), restricted to its top-p nucleus when top_p < 1, at the uniform number of the
+// token's sequence position.  One CTA per row.
+//
+// Nucleus: {v : z_v >= z*}, z* the largest logit whose upper set holds top_p of the mass (equal logits enter
+// together).  z* is found by a radix select over the order-preserving 32-bit keys of the logits, 11 + 11 + 10
+// bits from the top: each pass histograms the MASS of the tokens whose key matches the digits chosen so far and
+// walks the buckets downwards until the mass wanted is reached.  Masses are 2^40 fixed-point integers, so the
+// histogram's atomic additions are exact and order-free, and the result is a pure function of the logits; lanes of
+// a warp that hit the same bucket are merged first (match + three 14-bit integer reductions), so equal logits cost
+// one atomic per warp, not 32.
+//
+// CDF walk: the vocabulary is cut into cells of 128 consecutive tokens; a warp sums a cell (coalesced loads, fixed
+// shuffle tree, fp64), the CTA scans the cell sums in order, and the one thread whose cells straddle u * total
+// walks its cell token by token.  The exponentials and sums are fp64 (a few thousand per thread at most), so that
+// for equal logits the token can differ from an fp64 reference only by summation order.
 // Everything is a pure function of (logits, u): deterministic.
 // ------------------------------------------------------------------------------------------------
 constexpr int kSampleThreads = 1024;
 constexpr int kSampleCell = 128;
 constexpr int kSampleMaxCells = kSampleMaxVocab / kSampleCell;
 
+constexpr int kSelectBuckets = 2048;
+
+// larger logit <-> larger key; -0 and +0 share a key
+__device__ __forceinline__ unsigned int order_key(float z) {
+    const unsigned int b = __float_as_uint(z + 0.0f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
 __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     pdl_trigger();
     pdl_wait();
+    __shared__ unsigned long long s_hist[kSelectBuckets];
+    __shared__ unsigned long long s_above;
+    __shared__ unsigned int s_digit;
     __shared__ double s_cell[kSampleMaxCells];
     __shared__ double s_warp[32];
     __shared__ float s_maxw[32];
@@ -682,13 +703,79 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     mx = s_maxw[0];
     for (int i = 1; i < 32; ++i) mx = fmaxf(mx, s_maxw[i]);
 
+    // ---- top-p: key of the smallest logit inside the nucleus (0: every token) ----
+    unsigned int kstar = 0;
+    if (a.top_p < 1.0) {
+        unsigned int prefix = 0;
+        unsigned long long above = 0, target = 0;   // mass of the keys above the current range; mass wanted
+        int shift = 32;
+        for (int pass = 0; pass < 3; ++pass) {
+            const int bits = pass < 2 ? 11 : 10;
+            shift -= bits;
+            const unsigned int nb = 1u << bits;
+            for (int i = tid; i < kSelectBuckets; i += kSampleThreads) s_hist[i] = 0ull;
+            __syncthreads();
+            for (int v0 = 0; v0 < V; v0 += kSampleThreads) {
+                const int v = v0 + tid;
+                unsigned int digit = 0xffffffffu;
+                unsigned long long q = 0ull;
+                if (v < V) {
+                    const float zv = __ldcg(z + v);
+                    const unsigned int k = order_key(zv);
+                    if (pass == 0 || (k >> (shift + bits)) == prefix) {
+                        digit = (k >> shift) & (nb - 1);
+                        q = __double2ull_rn(exp(((double)zv - (double)mx) / a.temperature) * 1099511627776.0);   // 2^40
+                    }
+                }
+                const unsigned int peers = __match_any_sync(0xffffffffu, digit);
+                const unsigned int p0 = __reduce_add_sync(peers, (unsigned int)(q & 0x3fffull));
+                const unsigned int p1 = __reduce_add_sync(peers, (unsigned int)((q >> 14) & 0x3fffull));
+                const unsigned int p2 = __reduce_add_sync(peers, (unsigned int)(q >> 28));
+                if (digit != 0xffffffffu && lane == __ffs(peers) - 1)
+                    atomicAdd(&s_hist[digit], (unsigned long long)p0 + ((unsigned long long)p1 << 14) + ((unsigned long long)p2 << 28));
+            }
+            __syncthreads();
+            if (warp == 0) {   // walk the buckets from the top: lane l owns the l-th run of nb/32 buckets below the top
+                const int per = nb >> 5;
+                unsigned long long mine = 0ull;
+                for (int j = 0; j < per; ++j) mine += s_hist[nb - 1 - (lane * per + j)];
+                unsigned long long incl = mine;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                if (pass == 0) {
+                    const unsigned long long total_q = __shfl_sync(0xffffffffu, incl, 31);
+                    target = (unsigned long long)ceil(a.top_p * (double)total_q);
+                    target = target < 1ull ? 1ull : (target > total_q ? total_q : target);
+                }
+                const unsigned long long need = target - above, excl = incl - mine;
+                if (excl < need && need <= incl) {   // exactly one lane: the range holds at least `need`, and need >= 1
+                    unsigned long long run = excl;
+                    for (int j = 0; j < per; ++j) {
+                        const int b = nb - 1 - (lane * per + j);
+                        if (run + s_hist[b] >= need) { s_digit = b; s_above = above + run; break; }
+                        run += s_hist[b];
+                    }
+                }
+            }
+            __syncthreads();
+            above = s_above;
+            prefix = (prefix << bits) | s_digit;
+        }
+        kstar = prefix;
+    }
+
     const int n_cells = (V + kSampleCell - 1) / kSampleCell;
     for (int c = warp; c < n_cells; c += 32) {
         double s = 0.0;
 #pragma unroll
         for (int j = 0; j < kSampleCell / 32; ++j) {
             int v = c * kSampleCell + j * 32 + lane;
-            if (v < V) s += exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+            if (v < V) {
+                const float zv = __ldcg(z + v);
+                if (order_key(zv) >= kstar) s += exp(((double)zv - (double)mx) / a.temperature);
+            }
         }
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (lane == 0) s_cell[c] = s;
@@ -725,7 +812,9 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
         const int v0 = c * kSampleCell, v1 = min(v0 + kSampleCell, V);
         int pick = -1;
         for (int v = v0; v < v1; ++v) {
-            double e = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+            const float zv = __ldcg(z + v);
+            if (order_key(zv) < kstar) continue;       // outside the nucleus
+            double e = exp(((double)zv - (double)mx) / a.temperature);
             if (e > 0.0) pick = v;                     // last token with mass, if the walk falls an ulp short
             run += e;
             if (run >= target) break;

@@ -271,6 +271,7 @@ struct SampleArgs {
     const float* logits;       // [m][V] final logits, row r0 first
     int V, r0, m;
     double temperature;        // sampling temperature T_s > 0
+    double top_p;              // nucleus mass; >= 1: the whole vocabulary
     unsigned long long seed;
     long long pos0;            // sequence position of the token that row r0 produces (row r0 + j: pos0 + j)
     int* token;                // token[r0 + j] receives the sample

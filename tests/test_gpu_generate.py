@@ -370,7 +370,7 @@ def test_bench_sweep_mode_on_tiny(capsys):
     assert all(1.0 <= p["emitted_per_round"] <= p["w_max"] and 0.0 <= p["draft_acceptance"] <= 1.0 for p in pts)
     assert max(p["emitted_per_round"] for p in pts) > 1.5
     strat = line["decoding_strategies"]
-    assert [x["strategy"] for x in strat] == ["greedy", "temperature 0.3", "temperature 1.0"]
+    assert [x["strategy"] for x in strat] == ["greedy", "temperature 0.3", "temperature 1.0", "top-p 0.9"]
     assert all(x["tokens_equal_ar"] and x["tokens_per_s"] > 0 and x["ar_tokens_per_s"] > 0 for x in strat)
 
 

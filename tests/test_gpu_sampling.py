@@ -24,12 +24,12 @@ SMALL_BF16 = inputs.scaled(inputs.LLAMA3_8B, name="small-bf16", n_layers=4, d_mo
                            head_dim=64, d_ffn=1408, vocab=2048, head_scale=16.0)
 
 
-def _compare_with_oracle_samples(logits_cpu: np.ndarray, temperature, seed, pos0, gpu_tokens, edge_tol):
+def _compare_with_oracle_samples(logits_cpu: np.ndarray, temperature, seed, pos0, gpu_tokens, edge_tol, top_p=1.0):
     """Row by row: equal tokens, or the oracle's uniform number lies within edge_tol of the edge between the two."""
     n_edge = 0
     for j, z in enumerate(logits_cpu):
         u = oracle.uniform(seed, pos0 + j)
-        t, slack = oracle.sample_token(z.astype(np.float64), temperature, u)
+        t, slack = oracle.sample_token(z.astype(np.float64), temperature, u, top_p)
         if t != gpu_tokens[j]:
             assert abs(int(gpu_tokens[j]) - t) >= 1 and slack < edge_tol, (j, t, int(gpu_tokens[j]), slack)
             # the GPU's token must be the neighbour across that edge (skipping tokens without mass)
@@ -64,6 +64,35 @@ def test_sampling_kernel_matches_oracle(vocab, temperature):
     assert one[0] == tok[5]
 
 
+@pytest.mark.parametrize("vocab", [1, 7, 128, 1000, 32000, 128256, 262144])
+@pytest.mark.parametrize("temperature,top_p", [(1.0, 0.9), (0.3, 0.9), (1.0, 0.5), (2.0, 0.999), (1.0, 1e-6)])
+def test_nucleus_sampling_kernel_matches_oracle(vocab, temperature, top_p):
+    """top-p: the radix select must land on the oracle's logit threshold -- random rows, a peaked row, a flat row
+    (every token tied: the whole vocabulary is the nucleus), rows with few distinct values (ties at the threshold
+    enter together), signed zeros, half the vocabulary without mass."""
+    g = torch.Generator().manual_seed(1000 + vocab)
+    m = 8
+    z = torch.randn(m, vocab, generator=g) * 2.5
+    z[1] *= 4.0
+    z[2] = 0.0
+    if vocab > 4:
+        z[3, : vocab // 2] = -200.0
+        z[4] = torch.randint(-3, 4, (vocab,), generator=g).float()            # 7 distinct values, massive ties
+        z[5] = torch.where(torch.rand(vocab, generator=g) < 0.5, 0.0, -0.0)   # +0 and -0 are one value
+        z[6] = torch.round(z[6] * 4) / 4                                      # ties on a grid, negative and positive
+    seed, pos0 = 31, 77
+    temperature, top_p = f32(temperature), f32(top_p)
+    tok = binding.k_sample(z.cuda(), temperature, seed, pos0, top_p=top_p).cpu().numpy()
+    assert ((tok >= 0) & (tok < vocab)).all()
+    for j in range(m):   # every token lies inside the oracle's nucleus
+        zs = oracle.nucleus_threshold(z[j].double().numpy(), temperature, top_p)
+        assert float(z[j, tok[j]]) >= zs, (j, tok[j], zs)
+    assert _compare_with_oracle_samples(z.numpy(), temperature, seed, pos0, tok, edge_tol=1e-9, top_p=top_p) == 0
+    assert np.array_equal(binding.k_sample(z.cuda(), temperature, seed, pos0, top_p=top_p).cpu().numpy(), tok)
+    if top_p < 1e-3:     # the nucleus is the set of maxima
+        assert all(float(z[j, tok[j]]) == float(z[j].max()) for j in range(m))
+
+
 def test_sampling_kernel_frequencies_follow_softmax():
     g = torch.Generator().manual_seed(1)
     V, T, N = 200, 0.9, 4000
@@ -85,6 +114,11 @@ def test_sampling_argument_errors(tiny_weights):
     for bad in (-1.0, float("nan")):
         with pytest.raises(binding.SBError):
             ctx.set_sampling(bad, 0)
+    for bad_p in (0.0, -0.5, 1.5, float("nan")):
+        with pytest.raises(binding.SBError):
+            ctx.set_sampling(1.0, 0, top_p=bad_p)
+        with pytest.raises(binding.SBError):
+            binding.k_sample(torch.zeros(2, 10, device="cuda"), 1.0, 0, 0, top_p=bad_p)
     z = torch.zeros(2, 10, device="cuda")
     with pytest.raises(binding.SBError):
         binding.k_sample(z, 0.0, 0, 0)
@@ -102,11 +136,11 @@ def test_tiny_sampled_generation_matches_oracle_and_ar(which, tiny_weights, tiny
     ctx, _ = gpu_ctx(run.shape, w, max_seq)
     greedy = ctx.generate_ar(pr, n_gen)["tokens"]
     accepted = {}
-    for T, seed in ((f32(0.3), 1), (1.0, 2), (1.0, 3)):
+    for T, seed, top_p in ((f32(0.3), 1, 1.0), (1.0, 2, 1.0), (1.0, 3, 1.0), (1.0, 3, f32(0.9)), (f32(1.5), 4, 0.5)):
         o = oracle.Oracle(run.shape, w, max_seq)
-        o.set_sampling(T, seed)
+        o.set_sampling(T, seed, top_p)
         ref, slack = o.ar_generate(pr, n_gen, want_margins=True)
-        ctx.set_sampling(T, seed)
+        ctx.set_sampling(T, seed, top_p)
         ar = ctx.generate_ar(pr, n_gen)["tokens"]
         # fp32 model: logits agree to ~1e-6, so a token can differ only within that of a CDF edge
         diff = np.nonzero(ar != ref)[0]
@@ -114,7 +148,7 @@ def test_tiny_sampled_generation_matches_oracle_and_ar(which, tiny_weights, tiny
             assert slack[diff[0]] < 1e-5, (T, seed, diff[0], slack[diff[0]])
         else:
             assert np.array_equal(ar, ref)
-        accepted[(T, seed)] = 0
+        accepted[(T, seed)] = accepted.get((T, seed), 0)
         for d_max, w_max, thr in ((1, 8, 0.0), (2, 4, 0.25), (3, 3, 0.2), (3, 8, 2.0)):
             tau = inputs.tau_linear(d_max, 1.5, 1.0)
             res = ctx.generate(pr, n_gen, d_max, w_max, tau, thr, trace=True)
@@ -122,11 +156,13 @@ def test_tiny_sampled_generation_matches_oracle_and_ar(which, tiny_weights, tiny
             accepted[(T, seed)] += res["stats"].accepted_drafts
             if not len(diff):
                 o2 = oracle.Oracle(run.shape, w, max_seq)
-                o2.set_sampling(T, seed)
+                o2.set_sampling(T, seed, top_p)
                 _, rounds = o2.specbound_generate(pr, n_gen, d_max, w_max, tau, thr)
                 assert [(r.w, r.emitted, r.accepted_drafts) for r in res["rounds"]] == \
                        [(r.w, r.emitted, r.accepted_drafts) for r in rounds]
     assert not np.array_equal(ar, greedy)
+    ctx.set_sampling(1.0, 3, 1e-6)
+    assert np.array_equal(ctx.generate_ar(pr, n_gen)["tokens"], greedy)                # top_p -> 0: the top-1 alone
     ctx.set_sampling(0.0, 0)
     assert np.array_equal(ctx.generate_ar(pr, n_gen)["tokens"], greedy)                # switching back restores greedy
     ctx.set_sampling(1e-4, 9)
@@ -178,12 +214,12 @@ def test_7b_damped_sampled_run_equals_ar():
     n_gen = 32
     ctx = binding.Context(run.shape, wg, 96, kv_page=64)
     greedy = ctx.generate_ar(pr, n_gen)["tokens"]
-    for T in (0.3, 1.0):
-        ctx.set_sampling(T, 123)
+    for T, top_p in ((0.3, 1.0), (1.0, 1.0), (1.0, 0.9)):
+        ctx.set_sampling(T, 123, top_p)
         ar = ctx.generate_ar(pr, n_gen)["tokens"]
         sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, run.tau, run.threshold)
-        assert np.array_equal(sp["tokens"], ar), T
-        print(f"\n[7b-damped T={T}] accepted drafts {sp['stats'].accepted_drafts}, rounds {sp['stats'].rounds}, "
+        assert np.array_equal(sp["tokens"], ar), (T, top_p)
+        print(f"\n[7b-damped T={T} top_p={top_p}] accepted drafts {sp['stats'].accepted_drafts}, rounds {sp['stats'].rounds}, "
               f"differs from greedy at {int((ar != greedy).sum())} of {n_gen}")
         if T == 0.3:
             assert sp["stats"].accepted_drafts > 0
