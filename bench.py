@@ -435,6 +435,28 @@ def micro_arm(args):
                                 "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
                                 "note": "includes the RMSNorm launch and two small device copies of the stateless entry point"})
             del heads
+    # sampling kernel (decoding strategies of Section 4.3): latency of one launch on m rows of L2-resident logits;
+    # not a bandwidth-bound kernel (one CTA per row, fp64 exponentials), reported in microseconds only
+    for V in (32000, 128256):
+        for m, top_p in ((1, 1.0), (8, 1.0), (1, 0.9), (8, 0.9)):
+            name = f"sample:m={m}:V={V}:top_p={top_p}"
+            if not want(name):
+                continue
+            z = torch.randn((m, V), device="cuda") * 2.5
+            for i in range(3):
+                binding.k_sample(z, 1.0, 1, i, top_p=top_p)
+            torch.cuda.synchronize()
+            times = []
+            for i in range(args.iters):
+                e0, e1 = ev(), ev()
+                e0.record()
+                for k in range(8):   # 8 calls per timing: the queue hides the host's issue time if the kernels are longer
+                    binding.k_sample(z, 1.0, 1, 64 * i + 8 * k, top_p=top_p)
+                e1.record()
+                e1.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e3 / 8)
+            out.setdefault("sample", []).append({"m": m, "V": V, "top_p": top_p, "us": statistics.median(times),
+                                                 "us_min": min(times)})
     print(json.dumps(out), flush=True)
 
 

@@ -185,8 +185,8 @@ int sb_generate_ar(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t
  * layers' top-1 tokens under the annealed threshold; a draft is accepted iff it equals the
  * sampled token of its row, so sb_generate returns exactly what sb_generate_ar returns for the
  * same (temperature, top_p, seed): lossless sample by sample.  The final logits of the
- * <= SB_MAX_W rows go through a [8][vocab] fp32 buffer of the workspace; the exit tests never
- * write logits.  temperature 0 (the default) restores greedy decoding.  Errors: SB_ERR_ARG
+ * <= SB_MAX_W rows go through a [8][vocab] fp32 buffer of the workspace and their exponentials
+ * through a [8][vocab] fp64 one; the exit tests never write logits.  temperature 0 (the default) restores greedy decoding.  Errors: SB_ERR_ARG
  * (negative or NaN temperature, top_p outside (0, 1]), SB_ERR_CAPACITY (vocab > 262144 with
  * temperature > 0). */
 int sb_set_sampling(sb_ctx* ctx, float temperature, float top_p, uint64_t seed);
@@ -200,13 +200,16 @@ double sb_sample_uniform(uint64_t seed, int64_t pos);
 /* Scratch bytes the two calls below need for this shape. */
 size_t sb_k_scratch_bytes(const sb_config* cfg);
 
-/* Sampling kernel alone (the rule of sb_set_sampling): token[j] (device) = inverse-CDF sample of
+/* Sampling kernels alone (the rule of sb_set_sampling): token[j] (device) = inverse-CDF sample of
  * the top_p nucleus of softmax(logits[j][:] / temperature) at sb_sample_uniform(seed, pos0 + j),
- * for m <= SB_MAX_W rows of device fp32 logits [m][vocab].  Asynchronous on `stream`.  Errors:
- * SB_ERR_ARG (null pointer, m outside [1, SB_MAX_W], temperature <= 0, top_p outside (0, 1]),
- * SB_ERR_CAPACITY (vocab > 262144). */
+ * for m <= SB_MAX_W rows of device fp32 logits [m][vocab].  scratch: device memory, 8-byte
+ * aligned, at least sb_k_sample_scratch_bytes(m, vocab) bytes (the rows' fp64 exponentials),
+ * owned by the caller.  Asynchronous on `stream` (two launches).  Errors: SB_ERR_ARG (null
+ * pointer, m outside [1, SB_MAX_W], temperature <= 0, top_p outside (0, 1], scratch misaligned or
+ * too small), SB_ERR_CAPACITY (vocab > 262144). */
+size_t sb_k_sample_scratch_bytes(int32_t m, int32_t vocab);
 int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, float top_p, uint64_t seed,
-                int64_t pos0, int32_t* token, void* stream);
+                int64_t pos0, int32_t* token, void* scratch, size_t scratch_bytes, void* stream);
 
 /* Exit-confidence kernel on m rows of hidden states (Section 3.2, Eq. 2):
  * h device fp32 [m, d]; final_norm / lm_head device in cfg->dtype; tau_l > 0.

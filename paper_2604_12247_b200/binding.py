@@ -66,7 +66,7 @@ class SBError(RuntimeError):
 EXPORTS = ("sb_workspace_bytes", "sb_create", "sb_destroy", "sb_load_weights", "sb_reset", "sb_get_state",
            "sb_selftest_wait_timeout",
            "sb_read_hidden", "sb_prefill", "sb_draft_push", "sb_draft_advance", "sb_exit_confidence", "sb_verify",
-           "sb_generate", "sb_generate_ar", "sb_set_sampling", "sb_sample_uniform", "sb_k_sample", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
+           "sb_generate", "sb_generate_ar", "sb_set_sampling", "sb_sample_uniform", "sb_k_sample", "sb_k_sample_scratch_bytes", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
            "sb_k_layer",
            "sb_tau_schedule", "sb_model_speedup", "sb_set_option", "sb_set_default_option", "sb_strerror")
 
@@ -104,7 +104,9 @@ def lib():
         L.sb_set_sampling.argtypes = [vp, f32, f32, C.c_uint64]
         L.sb_sample_uniform.argtypes = [C.c_uint64, C.c_int64]
         L.sb_sample_uniform.restype = C.c_double
-        L.sb_k_sample.argtypes = [vp, i32, i32, f32, f32, C.c_uint64, C.c_int64, vp, vp]
+        L.sb_k_sample.argtypes = [vp, i32, i32, f32, f32, C.c_uint64, C.c_int64, vp, vp, C.c_size_t, vp]
+        L.sb_k_sample_scratch_bytes.argtypes = [i32, i32]
+        L.sb_k_sample_scratch_bytes.restype = C.c_size_t
         L.sb_k_exit_confidence.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp, vp, C.c_size_t, vp]
         L.sb_k_exit_confidence_static.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp]
         L.sb_k_layer.argtypes = [C.POINTER(Config), C.POINTER(LayerWeights), vp, i32, vp, vp, vp, i32, vp, C.c_size_t, vp]
@@ -304,8 +306,10 @@ def k_sample(logits: torch.Tensor, temperature: float, seed: int, pos0: int, top
     """sb_k_sample on a [m, vocab] fp32 device tensor -> int32 tokens [m] (device)."""
     assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
     tok = torch.empty(logits.shape[0], dtype=torch.int32, device=logits.device)
+    nbytes = lib().sb_k_sample_scratch_bytes(logits.shape[0], logits.shape[1])
+    scratch = torch.empty(nbytes // 8, dtype=torch.float64, device=logits.device)
     _check(lib().sb_k_sample(logits.data_ptr(), logits.shape[0], logits.shape[1], float(temperature), float(top_p), int(seed), int(pos0),
-                             tok.data_ptr(), _stream_handle(stream)), "sb_k_sample")
+                             tok.data_ptr(), scratch.data_ptr(), nbytes, _stream_handle(stream)), "sb_k_sample")
     return tok
 
 

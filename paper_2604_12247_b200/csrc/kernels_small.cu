@@ -659,21 +659,60 @@ void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int
 // together).  z* is found by a radix select over the order-preserving 32-bit keys of the logits, 11 + 11 + 10
 // bits from the top: each pass histograms the MASS of the tokens whose key matches the digits chosen so far and
 // walks the buckets downwards until the mass wanted is reached.  Masses are 2^40 fixed-point integers, so the
-// histogram's atomic additions are exact and order-free, and the result is a pure function of the logits; lanes of
-// a warp that hit the same bucket are merged first (match + three 14-bit integer reductions), so equal logits cost
-// one atomic per warp, not 32.
+// histogram's atomic additions are exact and order-free, and the result is a pure function of the logits (the
+// histogram is kept in three 14-bit parts so that the atomics are 32-bit ones); a warp whose lanes all hit the same
+// bucket (flat or tied logits) merges them first, so equal logits cost one atomic per warp, not 32.
 //
 // CDF walk: the vocabulary is cut into cells of 128 consecutive tokens; a warp sums a cell (coalesced loads, fixed
 // shuffle tree, fp64), the CTA scans the cell sums in order, and the one thread whose cells straddle u * total
 // walks its cell token by token.  The exponentials and sums are fp64 (a few thousand per thread at most), so that
 // for equal logits the token can differ from an fp64 reference only by summation order.
 // Everything is a pure function of (logits, u): deterministic.
+//
+// Two launches.  fp64 exponentials are slow on this GPU (one CTA needs ~35 us for 32000 of them), so they are
+// computed once, by a cluster of 8 CTAs per row (k_sample_exp: slice maxima exchanged through distributed shared
+// memory, then e_v = exp((z_v - max) / T) to an L2-resident scratch row); k_sample, one CTA per row, only reads them.
 // ------------------------------------------------------------------------------------------------
 constexpr int kSampleThreads = 1024;
+constexpr int kExpSlices = 8;
+
+__global__ void __launch_bounds__(kSampleThreads) k_sample_exp(SampleArgs a) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float s_maxw[32];
+    __shared__ float s_slice_max[kExpSlices];      // slot r is written by the CTA of cluster rank r
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int V = a.V, row = blockIdx.x, rank = blockIdx.y;
+    const float* __restrict__ z = a.logits + (size_t)row * V;
+    const int per = (V + kExpSlices - 1) / kExpSlices;
+    const int v0 = min(rank * per, V), v1 = min(v0 + per, V);
+    float mx = -INFINITY;
+    for (int v = v0 + tid; v < v1; v += kSampleThreads) mx = fmaxf(mx, __ldcg(z + v));
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) s_maxw[warp] = mx;
+    __syncthreads();
+    if (tid < kExpSlices) {                        // thread t hands this slice's maximum to the CTA of rank t
+        float sm = s_maxw[0];
+        for (int i = 1; i < 32; ++i) sm = fmaxf(sm, s_maxw[i]);
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&s_slice_max[rank])), "r"(tid));
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(sm) : "memory");
+    }
+    cluster_sync_all();
+    mx = s_slice_max[0];
+    for (int i = 1; i < kExpSlices; ++i) mx = fmaxf(mx, s_slice_max[i]);
+    double* __restrict__ e = a.e + (size_t)row * V;
+    for (int v = v0 + tid; v < v1; v += kSampleThreads) e[v] = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+}
+
 constexpr int kSampleCell = 128;
 constexpr int kSampleMaxCells = kSampleMaxVocab / kSampleCell;
 
 constexpr int kSelectBuckets = 2048;
+
+__device__ __forceinline__ unsigned long long hist_mass(const unsigned int (*h)[kSelectBuckets], int b) {
+    return (unsigned long long)h[0][b] + ((unsigned long long)h[1][b] << 14) + ((unsigned long long)h[2][b] << 28);
+}
 
 // larger logit <-> larger key; -0 and +0 share a key
 __device__ __forceinline__ unsigned int order_key(float z) {
@@ -684,24 +723,20 @@ __device__ __forceinline__ unsigned int order_key(float z) {
 __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     pdl_trigger();
     pdl_wait();
-    __shared__ unsigned long long s_hist[kSelectBuckets];
+    // mass histogram in three 14-bit parts (32-bit shared-memory atomics are native; a part's bucket sum stays below
+    // 2^32 for up to 262144 tokens): mass of bucket b = s_hist[0][b] + (s_hist[1][b] << 14) + (s_hist[2][b] << 28)
+    __shared__ unsigned int s_hist[3][kSelectBuckets];
     __shared__ unsigned long long s_above;
     __shared__ unsigned int s_digit;
     __shared__ double s_cell[kSampleMaxCells];
     __shared__ double s_warp[32];
-    __shared__ float s_maxw[32];
-    __shared__ int s_last;
+    __shared__ int s_last, s_walk_cell;
+    __shared__ double s_walk_run, s_walk_target;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = a.V, row = blockIdx.x;
     const float* __restrict__ z = a.logits + (size_t)row * V;
 
-    float mx = -INFINITY;
-    for (int v = tid; v < V; v += kSampleThreads) mx = fmaxf(mx, __ldcg(z + v));
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) s_maxw[warp] = mx;
-    __syncthreads();
-    mx = s_maxw[0];
-    for (int i = 1; i < 32; ++i) mx = fmaxf(mx, s_maxw[i]);
+    const double* __restrict__ e_row = a.e + (size_t)row * V;
 
     // ---- top-p: key of the smallest logit inside the nucleus (0: every token) ----
     unsigned int kstar = 0;
@@ -713,32 +748,50 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
             const int bits = pass < 2 ? 11 : 10;
             shift -= bits;
             const unsigned int nb = 1u << bits;
-            for (int i = tid; i < kSelectBuckets; i += kSampleThreads) s_hist[i] = 0ull;
+            for (int i = tid; i < 3 * kSelectBuckets; i += kSampleThreads) s_hist[0][i] = 0u;
             __syncthreads();
-            for (int v0 = 0; v0 < V; v0 += kSampleThreads) {
-                const int v = v0 + tid;
-                unsigned int digit = 0xffffffffu;
-                unsigned long long q = 0ull;
-                if (v < V) {
-                    const float zv = __ldcg(z + v);
-                    const unsigned int k = order_key(zv);
-                    if (pass == 0 || (k >> (shift + bits)) == prefix) {
-                        digit = (k >> shift) & (nb - 1);
-                        q = __double2ull_rn(exp(((double)zv - (double)mx) / a.temperature) * 1099511627776.0);   // 2^40
+            constexpr int kBatch = 4;   // tokens per thread per step: their loads are in flight together
+            for (int v0 = 0; v0 < V; v0 += kBatch * kSampleThreads) {
+                unsigned int digit[kBatch];
+                double ev[kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int v = v0 + j * kSampleThreads + tid;
+                    digit[j] = 0xffffffffu;
+                    ev[j] = 0.0;
+                    if (v < V) {
+                        const unsigned int k = order_key(__ldcg(z + v));
+                        if (pass == 0 || (k >> (shift + bits)) == prefix) {
+                            digit[j] = (k >> shift) & (nb - 1);
+                            ev[j] = __ldcg(e_row + v);
+                        }
                     }
                 }
-                const unsigned int peers = __match_any_sync(0xffffffffu, digit);
-                const unsigned int p0 = __reduce_add_sync(peers, (unsigned int)(q & 0x3fffull));
-                const unsigned int p1 = __reduce_add_sync(peers, (unsigned int)((q >> 14) & 0x3fffull));
-                const unsigned int p2 = __reduce_add_sync(peers, (unsigned int)(q >> 28));
-                if (digit != 0xffffffffu && lane == __ffs(peers) - 1)
-                    atomicAdd(&s_hist[digit], (unsigned long long)p0 + ((unsigned long long)p1 << 14) + ((unsigned long long)p2 << 28));
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const unsigned long long q = __double2ull_rn(ev[j] * 1099511627776.0);   // 2^40 fixed point
+                    unsigned int p0 = (unsigned int)(q & 0x3fffull), p1 = (unsigned int)((q >> 14) & 0x3fffull),
+                                 p2 = (unsigned int)(q >> 28);
+                    // equal digits across the whole warp (flat or heavily tied logits) would serialise 32 atomics on
+                    // one word: merge them first (exact integer reductions); otherwise one atomic per lane and part
+                    const bool uniform = __all_sync(0xffffffffu, digit[j] == __shfl_sync(0xffffffffu, digit[j], 0));
+                    if (uniform) {
+                        p0 = __reduce_add_sync(0xffffffffu, p0);
+                        p1 = __reduce_add_sync(0xffffffffu, p1);
+                        p2 = __reduce_add_sync(0xffffffffu, p2);
+                    }
+                    if (digit[j] != 0xffffffffu && (!uniform || lane == 0)) {
+                        if (p0) atomicAdd(&s_hist[0][digit[j]], p0);
+                        if (p1) atomicAdd(&s_hist[1][digit[j]], p1);
+                        if (p2) atomicAdd(&s_hist[2][digit[j]], p2);
+                    }
+                }
             }
             __syncthreads();
             if (warp == 0) {   // walk the buckets from the top: lane l owns the l-th run of nb/32 buckets below the top
                 const int per = nb >> 5;
                 unsigned long long mine = 0ull;
-                for (int j = 0; j < per; ++j) mine += s_hist[nb - 1 - (lane * per + j)];
+                for (int j = 0; j < per; ++j) mine += hist_mass(s_hist, nb - 1 - (lane * per + j));
                 unsigned long long incl = mine;
                 for (int o = 1; o < 32; o <<= 1) {
                     const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
@@ -754,8 +807,9 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
                     unsigned long long run = excl;
                     for (int j = 0; j < per; ++j) {
                         const int b = nb - 1 - (lane * per + j);
-                        if (run + s_hist[b] >= need) { s_digit = b; s_above = above + run; break; }
-                        run += s_hist[b];
+                        const unsigned long long hb = hist_mass(s_hist, b);
+                        if (run + hb >= need) { s_digit = b; s_above = above + run; break; }
+                        run += hb;
                     }
                 }
             }
@@ -773,8 +827,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
         for (int j = 0; j < kSampleCell / 32; ++j) {
             int v = c * kSampleCell + j * 32 + lane;
             if (v < V) {
-                const float zv = __ldcg(z + v);
-                if (order_key(zv) >= kstar) s += exp(((double)zv - (double)mx) / a.temperature);
+                if (kstar == 0u || order_key(__ldcg(z + v)) >= kstar) s += __ldcg(e_row + v);
             }
         }
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -809,19 +862,50 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
         double run = lower;
         int c = c0;
         while (c < c1 - 1 && run + s_cell[c] < target) run += s_cell[c++];
-        const int v0 = c * kSampleCell, v1 = min(v0 + kSampleCell, V);
-        int pick = -1;
-        for (int v = v0; v < v1; ++v) {
-            const float zv = __ldcg(z + v);
-            if (order_key(zv) < kstar) continue;       // outside the nucleus
-            double e = exp(((double)zv - (double)mx) / a.temperature);
-            if (e > 0.0) pick = v;                     // last token with mass, if the walk falls an ulp short
-            run += e;
-            if (run >= target) break;
+        s_walk_cell = c;
+        s_walk_run = run;
+        s_walk_target = target;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // the cell that holds u * total, walked by one warp: lane l sums tokens 4l .. 4l+3 of the cell in order, the lane
+        // sums are scanned in lane order, and the first token whose cumulative mass reaches the target is the sample
+        constexpr int kPerLane = kSampleCell / 32;
+        const int v0 = s_walk_cell * kSampleCell + lane * kPerLane;
+        const double run0 = s_walk_run, tgt = s_walk_target;
+        double ev[kPerLane];
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            const int v = v0 + j;
+            ev[j] = 0.0;
+            if (v < V && (kstar == 0u || order_key(__ldcg(z + v)) >= kstar)) ev[j] = __ldcg(e_row + v);
         }
-        if (pick < 0) pick = v0;
-        a.token[a.r0 + row] = pick;
-        __threadfence();
+        double mine4 = 0.0;
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) mine4 += ev[j];
+        double incl4 = mine4;
+        for (int o = 1; o < 32; o <<= 1) {
+            const double t = __shfl_up_sync(0xffffffffu, incl4, o);
+            if (lane >= o) incl4 += t;
+        }
+        double acc = run0 + (incl4 - mine4);
+        int hit = -1, last_mass = -1;
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            if (ev[j] > 0.0) last_mass = v0 + j;
+            acc += ev[j];
+            if (hit < 0 && ev[j] > 0.0 && acc >= tgt) hit = v0 + j;
+        }
+        const unsigned int hits = __ballot_sync(0xffffffffu, hit >= 0);
+        const unsigned int masses = __ballot_sync(0xffffffffu, last_mass >= 0);
+        int pick;
+        if (hits) pick = __shfl_sync(0xffffffffu, hit, __ffs(hits) - 1);
+        else if (masses) pick = __shfl_sync(0xffffffffu, last_mass, 31 - __clz(masses));   // the walk fell an ulp short
+        else pick = s_walk_cell * kSampleCell;
+        if (lane == 0) {
+            a.token[a.r0 + row] = pick;
+            __threadfence();
+        }
     }
     __syncthreads();
     if (tid == 0) {
@@ -833,6 +917,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     if (s_last) publish_results(a.mirror);
 }
 void launch_sample(cudaStream_t st, const SampleArgs& a) {
+    (void)launch_kc(k_sample_exp, dim3(a.m, kExpSlices), dim3(kSampleThreads), 0, st, kExpSlices, a);
     launch_k(k_sample, dim3(a.m), dim3(kSampleThreads), 0, st, a);
 }
 
