@@ -117,6 +117,7 @@ struct Work {
     float2* rope_tab;      // contexts only: cos/sin of the RoPE angles [n_pages * page][hd/2]
     float* logits;         // contexts only: [8][V] final logits of the rows being sampled (sampling decoding)
     double* sample_e;      // contexts only: [8][V] their exponentials
+    unsigned long long* sample_q;   // contexts only: [8][V] the same as fixed-point integers (top-p)
     void* k_cache;         // [L][n_pages][page][kvd]
     void* v_cache;
 };
@@ -158,10 +159,12 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     W.rope_tab = nullptr;
     W.logits = nullptr;
     W.sample_e = nullptr;
+    W.sample_q = nullptr;
     if (with_state) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
         c.take(W.logits, sizeof(float) * (size_t)kMaxW * D.V);
         c.take(W.sample_e, sizeof(double) * (size_t)kMaxW * D.V);
+        c.take(W.sample_q, sizeof(unsigned long long) * ((size_t)kMaxW * D.V + 64));   // + the slice sums
         c.take(W.rope_tab, sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2));
         size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
         c.take(W.k_cache, kv);
@@ -407,7 +410,7 @@ static void final_tokens(sb_ctx* c, int r0, int m, long long pos0, int* token, c
         return;
     }
     head(e, c->w.lm_head, r0, m, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), e.W.logits);
-    SampleArgs a{e.W.logits, e.W.sample_e, e.D.V, r0, m, (double)c->sample_temperature, (double)c->sample_top_p, c->sample_seed, pos0, token,
+    SampleArgs a{e.W.logits, e.W.sample_e, e.W.sample_q, e.D.V, r0, m, (double)c->sample_temperature, (double)c->sample_top_p, c->sample_seed, pos0, token,
                  reinterpret_cast<unsigned int*>(e.W.res + 57), mir};
     launch_sample(e.st, a);
     e.launches++;
@@ -961,7 +964,7 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
 // Sampling kernel alone: tokens of m rows of device logits.  Its completion counter is the word behind the static
 // scratch (zero at load, left at zero by every launch).
 size_t sb_k_sample_scratch_bytes(int32_t m, int32_t vocab) {
-    return m < 1 || vocab < 1 ? 0 : sizeof(double) * (size_t)m * (size_t)vocab;
+    return m < 1 || vocab < 1 ? 0 : 2 * sizeof(double) * (size_t)m * (size_t)vocab + 512;   // exponentials as fp64 and as fixed point, slice sums
 }
 
 int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, float top_p, uint64_t seed, int64_t pos0,
@@ -973,7 +976,7 @@ int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature
     char* base = nullptr;
     int rc = static_scratch_ptr(&base);
     if (rc) return rc;
-    SampleArgs a{logits, static_cast<double*>(scratch), vocab, 0, m, (double)temperature, (double)top_p, seed, pos0, token,
+    SampleArgs a{logits, static_cast<double*>(scratch), static_cast<unsigned long long*>(scratch) + (size_t)m * vocab, vocab, 0, m, (double)temperature, (double)top_p, seed, pos0, token,
                  reinterpret_cast<unsigned int*>(base + kStaticScratchBytes), Mirror{nullptr, nullptr, 0u}};
     launch_sample((cudaStream_t)stream, a);
     return cuda_ok(cudaGetLastError());

@@ -702,7 +702,29 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_exp(SampleArgs a) {
     mx = s_slice_max[0];
     for (int i = 1; i < kExpSlices; ++i) mx = fmaxf(mx, s_slice_max[i]);
     double* __restrict__ e = a.e + (size_t)row * V;
-    for (int v = v0 + tid; v < v1; v += kSampleThreads) e[v] = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+    unsigned long long* __restrict__ q = a.q + (size_t)row * V;
+    const bool want_q = a.top_p < 1.0;
+    unsigned long long qsum = 0ull;
+    for (int v = v0 + tid; v < v1; v += kSampleThreads) {
+        const double ev = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+        e[v] = ev;
+        if (want_q) {
+            const unsigned long long qv = __double2ull_rn(ev * 1099511627776.0);   // 2^40 fixed point: integer sums are exact in any order
+            q[v] = qv;
+            qsum += qv;
+        }
+    }
+    if (want_q) {   // this slice's integer mass, for the row total that k_sample needs up front
+        __shared__ unsigned long long s_qw[32];
+        for (int o = 16; o > 0; o >>= 1) qsum += __shfl_xor_sync(0xffffffffu, qsum, o);
+        if (lane == 0) s_qw[warp] = qsum;
+        __syncthreads();
+        if (tid == 0) {
+            unsigned long long t = 0ull;
+            for (int i = 0; i < 32; ++i) t += s_qw[i];
+            a.q[(size_t)gridDim.x * V + row * kExpSlices + rank] = t;   // slice sums live behind the [m][V] masses
+        }
+    }
 }
 
 constexpr int kSampleCell = 128;
@@ -726,7 +748,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     // mass histogram in three 14-bit parts (32-bit shared-memory atomics are native; a part's bucket sum stays below
     // 2^32 for up to 262144 tokens): mass of bucket b = s_hist[0][b] + (s_hist[1][b] << 14) + (s_hist[2][b] << 28)
     __shared__ unsigned int s_hist[3][kSelectBuckets];
-    __shared__ unsigned long long s_above;
+    __shared__ unsigned long long s_above, s_wsum[32];
     __shared__ unsigned int s_digit;
     __shared__ double s_cell[kSampleMaxCells];
     __shared__ double s_warp[32];
@@ -737,12 +759,21 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     const float* __restrict__ z = a.logits + (size_t)row * V;
 
     const double* __restrict__ e_row = a.e + (size_t)row * V;
+    const unsigned long long* __restrict__ q_row = a.q + (size_t)row * V;
 
     // ---- top-p: key of the smallest logit inside the nucleus (0: every token) ----
     unsigned int kstar = 0;
     if (a.top_p < 1.0) {
         unsigned int prefix = 0;
-        unsigned long long above = 0, target = 0;   // mass of the keys above the current range; mass wanted
+        unsigned long long total_q = 0ull;
+        for (int i = 0; i < kExpSlices; ++i) total_q += __ldcg(a.q + (size_t)gridDim.x * V + row * kExpSlices + i);
+        unsigned long long above = 0;               // mass of the keys above the current range
+        unsigned long long target = (unsigned long long)ceil(a.top_p * (double)total_q);   // mass wanted
+        target = target < 1ull ? 1ull : (target > total_q ? total_q : target);
+        // Tokens lighter than (1 - top_p) * total / V weigh less than (1 - top_p) * total together, so the tokens at
+        // or above that weight already hold the mass wanted: the lighter ones lie below the threshold logit and never
+        // decide a digit (buckets above the one that mixes both kinds hold none of them).  They skip the histogram.
+        const unsigned long long light = (unsigned long long)((1.0 - a.top_p) * (double)total_q / (double)V * 0.999999);
         int shift = 32;
         for (int pass = 0; pass < 3; ++pass) {
             const int bits = pass < 2 ? 11 : 10;
@@ -750,26 +781,28 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
             const unsigned int nb = 1u << bits;
             for (int i = tid; i < 3 * kSelectBuckets; i += kSampleThreads) s_hist[0][i] = 0u;
             __syncthreads();
-            constexpr int kBatch = 4;   // tokens per thread per step: their loads are in flight together
+            constexpr int kBatch = 8;   // tokens per thread per step: their loads are in flight together
             for (int v0 = 0; v0 < V; v0 += kBatch * kSampleThreads) {
+                // unconditional, clamped loads first: all 2 * kBatch of them are in flight together (a load that waits
+                // for the key test of its own token costs an L2 round trip per token)
+                float zz[kBatch];
+                unsigned long long qv[kBatch];
                 unsigned int digit[kBatch];
-                double ev[kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) zz[j] = __ldcg(z + min(v0 + j * kSampleThreads + tid, V - 1));
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) qv[j] = __ldcg(q_row + min(v0 + j * kSampleThreads + tid, V - 1));
 #pragma unroll
                 for (int j = 0; j < kBatch; ++j) {
                     const int v = v0 + j * kSampleThreads + tid;
-                    digit[j] = 0xffffffffu;
-                    ev[j] = 0.0;
-                    if (v < V) {
-                        const unsigned int k = order_key(__ldcg(z + v));
-                        if (pass == 0 || (k >> (shift + bits)) == prefix) {
-                            digit[j] = (k >> shift) & (nb - 1);
-                            ev[j] = __ldcg(e_row + v);
-                        }
-                    }
+                    const unsigned int k = order_key(zz[j]);
+                    const bool in = v < V && (pass == 0 || (k >> (shift + bits)) == prefix) && qv[j] >= light;
+                    digit[j] = in ? (k >> shift) & (nb - 1) : 0xffffffffu;
+                    if (!in) qv[j] = 0ull;
                 }
 #pragma unroll
                 for (int j = 0; j < kBatch; ++j) {
-                    const unsigned long long q = __double2ull_rn(ev[j] * 1099511627776.0);   // 2^40 fixed point
+                    const unsigned long long q = qv[j];
                     unsigned int p0 = (unsigned int)(q & 0x3fffull), p1 = (unsigned int)((q >> 14) & 0x3fffull),
                                  p2 = (unsigned int)(q >> 28);
                     // equal digits across the whole warp (flat or heavily tied logits) would serialise 32 atomics on
@@ -788,29 +821,25 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
                 }
             }
             __syncthreads();
-            if (warp == 0) {   // walk the buckets from the top: lane l owns the l-th run of nb/32 buckets below the top
-                const int per = nb >> 5;
-                unsigned long long mine = 0ull;
-                for (int j = 0; j < per; ++j) mine += hist_mass(s_hist, nb - 1 - (lane * per + j));
+            {   // walk the buckets from the top: a CTA-wide scan of the bucket masses in descending bucket order; thread t
+                // owns positions 2t and 2t+1 (position p <-> bucket nb-1-p).  Integer sums: exact, exactly one owner.
+                const int pa = 2 * tid;
+                const unsigned long long m0 = pa < (int)nb ? hist_mass(s_hist, nb - 1 - pa) : 0ull;
+                const unsigned long long m1 = pa + 1 < (int)nb ? hist_mass(s_hist, nb - 2 - pa) : 0ull;
+                const unsigned long long mine = m0 + m1;
                 unsigned long long incl = mine;
                 for (int o = 1; o < 32; o <<= 1) {
                     const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
                     if (lane >= o) incl += t;
                 }
-                if (pass == 0) {
-                    const unsigned long long total_q = __shfl_sync(0xffffffffu, incl, 31);
-                    target = (unsigned long long)ceil(a.top_p * (double)total_q);
-                    target = target < 1ull ? 1ull : (target > total_q ? total_q : target);
-                }
-                const unsigned long long need = target - above, excl = incl - mine;
-                if (excl < need && need <= incl) {   // exactly one lane: the range holds at least `need`, and need >= 1
-                    unsigned long long run = excl;
-                    for (int j = 0; j < per; ++j) {
-                        const int b = nb - 1 - (lane * per + j);
-                        const unsigned long long hb = hist_mass(s_hist, b);
-                        if (run + hb >= need) { s_digit = b; s_above = above + run; break; }
-                        run += hb;
-                    }
+                if (lane == 31) s_wsum[warp] = incl;
+                __syncthreads();
+                unsigned long long before = 0ull;
+                for (int i = 0; i < warp; ++i) before += s_wsum[i];
+                const unsigned long long need = target - above, excl = before + incl - mine;
+                if (excl < need && need <= excl + mine) {   // the range holds at least `need`, and need >= 1
+                    if (excl + m0 >= need) { s_digit = nb - 1 - pa; s_above = above + excl; }
+                    else { s_digit = nb - 2 - pa; s_above = above + excl + m0; }
                 }
             }
             __syncthreads();
@@ -826,9 +855,10 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
 #pragma unroll
         for (int j = 0; j < kSampleCell / 32; ++j) {
             int v = c * kSampleCell + j * 32 + lane;
-            if (v < V) {
-                if (kstar == 0u || order_key(__ldcg(z + v)) >= kstar) s += __ldcg(e_row + v);
-            }
+            const int vc = min(v, V - 1);
+            const double ev = __ldcg(e_row + vc);                       // unconditional loads: in flight together
+            const unsigned int kv = kstar ? order_key(__ldcg(z + vc)) : 0xffffffffu;
+            if (v < V && kv >= kstar) s += ev;
         }
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (lane == 0) s_cell[c] = s;
@@ -876,9 +906,10 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
         double ev[kPerLane];
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
-            const int v = v0 + j;
-            ev[j] = 0.0;
-            if (v < V && (kstar == 0u || order_key(__ldcg(z + v)) >= kstar)) ev[j] = __ldcg(e_row + v);
+            const int v = v0 + j, vc = min(v, V - 1);
+            const double e1 = __ldcg(e_row + vc);
+            const unsigned int kv = kstar ? order_key(__ldcg(z + vc)) : 0xffffffffu;
+            ev[j] = v < V && kv >= kstar ? e1 : 0.0;
         }
         double mine4 = 0.0;
 #pragma unroll

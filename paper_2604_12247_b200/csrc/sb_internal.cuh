@@ -270,6 +270,7 @@ constexpr int kSampleMaxVocab = 262144;
 struct SampleArgs {
     const float* logits;       // [m][V] final logits, row r0 first
     double* e;                 // [m][V] scratch: exp((z - row max) / temperature), written by the first kernel
+    unsigned long long* q;     // [m][V] scratch: the same as 2^40 fixed-point integers (top-p select)
     int V, r0, m;
     double temperature;        // sampling temperature T_s > 0
     double top_p;              // nucleus mass; >= 1: the whole vocabulary
