@@ -200,11 +200,11 @@ double sb_sample_uniform(uint64_t seed, int64_t pos);
 /* Scratch bytes the two calls below need for this shape. */
 size_t sb_k_scratch_bytes(const sb_config* cfg);
 
-/* Sampling kernels alone (the rule of sb_set_sampling): token[j] (device) = inverse-CDF sample of
+/* Sampling kernel alone (the rule of sb_set_sampling): token[j] (device) = inverse-CDF sample of
  * the top_p nucleus of softmax(logits[j][:] / temperature) at sb_sample_uniform(seed, pos0 + j),
  * for m <= SB_MAX_W rows of device fp32 logits [m][vocab].  scratch: device memory, 8-byte
  * aligned, at least sb_k_sample_scratch_bytes(m, vocab) bytes (the rows' exponentials, fp64 and fixed point),
- * owned by the caller.  Asynchronous on `stream` (two launches).  Errors: SB_ERR_ARG (null
+ * owned by the caller.  Asynchronous on `stream` (one launch).  Errors: SB_ERR_ARG (null
  * pointer, m outside [1, SB_MAX_W], temperature <= 0, top_p outside (0, 1], scratch misaligned or
  * too small), SB_ERR_CAPACITY (vocab > 262144). */
 size_t sb_k_sample_scratch_bytes(int32_t m, int32_t vocab);

@@ -653,120 +653,117 @@ void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int
 // ------------------------------------------------------------------------------------------------
 // Sampling decoding (Section 4.3, decoding strategies): token = inverse CDF, in vocabulary order, of
 // softmax(z / temperature), restricted to its top-p nucleus when top_p < 1, at the uniform number of the
-// token's sequence position.  One CTA per row.
+// token's sequence position.  One cluster of 8 CTAs per row; every CTA owns a slice of whole 128-token cells.
 //
-// Nucleus: {v : z_v >= z*}, z* the largest logit whose upper set holds top_p of the mass (equal logits enter
-// together).  z* is found by a radix select over the order-preserving 32-bit keys of the logits, 11 + 11 + 10
-// bits from the top: each pass histograms the MASS of the tokens whose key matches the digits chosen so far and
-// walks the buckets downwards until the mass wanted is reached.  Masses are 2^40 fixed-point integers, so the
-// histogram's atomic additions are exact and order-free, and the result is a pure function of the logits (the
-// histogram is kept in three 14-bit parts so that the atomics are 32-bit ones); a warp whose lanes all hit the same
-// bucket (flat or tied logits) merges them first, so equal logits cost one atomic per warp, not 32.
+//  1. slice maxima are exchanged through distributed shared memory; e_v = exp((z_v - max) / T) in fp64 goes to an
+//     L2-resident scratch row (fp64 exponentials are slow on this GPU: ~35 us for 32000 of them on one SM), and,
+//     for top-p, the same as a 2^40 fixed-point integer q_v.
+//  2. Nucleus (top_p < 1): {v : z_v >= z*}, z* the largest logit whose upper set holds top_p of the mass (equal
+//     logits enter together).  z* is found by a radix select over the order-preserving 32-bit keys of the logits,
+//     11 + 11 + 10 bits from the top: each pass, every CTA histograms the integer MASS of its tokens whose key
+//     matches the digits chosen so far (three 14-bit parts: 32-bit shared-memory atomics, exact and order-free),
+//     then sums its share of the buckets over the 8 histograms out of its peers' shared memory and hands the sums
+//     to every CTA, and every CTA scans the buckets from the top until the mass wanted is reached: the same
+//     integers everywhere, so all CTAs choose the same digit.  Tokens
+//     lighter than (1 - top_p) * total / V cannot decide a digit and skip the histogram.
+//  3. CDF walk: every CTA sums its cells' nucleus members (a warp per cell, coalesced loads, fixed shuffle tree,
+//     fp64) into the first CTA's shared memory; that CTA scans the cell sums in order, exactly one thread owns the
+//     interval holding u * total (neighbouring intervals are built from the same additions), and one warp walks
+//     that cell token by token.
 //
-// CDF walk: the vocabulary is cut into cells of 128 consecutive tokens; a warp sums a cell (coalesced loads, fixed
-// shuffle tree, fp64), the CTA scans the cell sums in order, and the one thread whose cells straddle u * total
-// walks its cell token by token.  The exponentials and sums are fp64 (a few thousand per thread at most), so that
-// for equal logits the token can differ from an fp64 reference only by summation order.
-// Everything is a pure function of (logits, u): deterministic.
-//
-// Two launches.  fp64 exponentials are slow on this GPU (one CTA needs ~35 us for 32000 of them), so they are
-// computed once, by a cluster of 8 CTAs per row (k_sample_exp: slice maxima exchanged through distributed shared
-// memory, then e_v = exp((z_v - max) / T) to an L2-resident scratch row); k_sample, one CTA per row, only reads them.
+// fp64 sums and exponentials: for equal logits the token can differ from an fp64 reference only by summation
+// order.  Everything is a pure function of (logits, u): deterministic.  All waits are hardware barriers.
 // ------------------------------------------------------------------------------------------------
 constexpr int kSampleThreads = 1024;
-constexpr int kExpSlices = 8;
-
-__global__ void __launch_bounds__(kSampleThreads) k_sample_exp(SampleArgs a) {
-    pdl_trigger();
-    pdl_wait();
-    __shared__ float s_maxw[32];
-    __shared__ float s_slice_max[kExpSlices];      // slot r is written by the CTA of cluster rank r
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int V = a.V, row = blockIdx.x, rank = blockIdx.y;
-    const float* __restrict__ z = a.logits + (size_t)row * V;
-    const int per = (V + kExpSlices - 1) / kExpSlices;
-    const int v0 = min(rank * per, V), v1 = min(v0 + per, V);
-    float mx = -INFINITY;
-    for (int v = v0 + tid; v < v1; v += kSampleThreads) mx = fmaxf(mx, __ldcg(z + v));
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) s_maxw[warp] = mx;
-    __syncthreads();
-    if (tid < kExpSlices) {                        // thread t hands this slice's maximum to the CTA of rank t
-        float sm = s_maxw[0];
-        for (int i = 1; i < 32; ++i) sm = fmaxf(sm, s_maxw[i]);
-        uint32_t remote;
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&s_slice_max[rank])), "r"(tid));
-        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(sm) : "memory");
-    }
-    cluster_sync_all();
-    mx = s_slice_max[0];
-    for (int i = 1; i < kExpSlices; ++i) mx = fmaxf(mx, s_slice_max[i]);
-    double* __restrict__ e = a.e + (size_t)row * V;
-    unsigned long long* __restrict__ q = a.q + (size_t)row * V;
-    const bool want_q = a.top_p < 1.0;
-    unsigned long long qsum = 0ull;
-    for (int v = v0 + tid; v < v1; v += kSampleThreads) {
-        const double ev = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
-        e[v] = ev;
-        if (want_q) {
-            const unsigned long long qv = __double2ull_rn(ev * 1099511627776.0);   // 2^40 fixed point: integer sums are exact in any order
-            q[v] = qv;
-            qsum += qv;
-        }
-    }
-    if (want_q) {   // this slice's integer mass, for the row total that k_sample needs up front
-        __shared__ unsigned long long s_qw[32];
-        for (int o = 16; o > 0; o >>= 1) qsum += __shfl_xor_sync(0xffffffffu, qsum, o);
-        if (lane == 0) s_qw[warp] = qsum;
-        __syncthreads();
-        if (tid == 0) {
-            unsigned long long t = 0ull;
-            for (int i = 0; i < 32; ++i) t += s_qw[i];
-            a.q[(size_t)gridDim.x * V + row * kExpSlices + rank] = t;   // slice sums live behind the [m][V] masses
-        }
-    }
-}
-
 constexpr int kSampleCell = 128;
 constexpr int kSampleMaxCells = kSampleMaxVocab / kSampleCell;
-
+constexpr int kSampleCtas = 8;
 constexpr int kSelectBuckets = 2048;
 
-__device__ __forceinline__ unsigned long long hist_mass(const unsigned int (*h)[kSelectBuckets], int b) {
-    return (unsigned long long)h[0][b] + ((unsigned long long)h[1][b] << 14) + ((unsigned long long)h[2][b] << 28);
+__device__ __forceinline__ unsigned long long hist_mass(unsigned int h0, unsigned int h1, unsigned int h2) {
+    return (unsigned long long)h0 + ((unsigned long long)h1 << 14) + ((unsigned long long)h2 << 28);
 }
-
 // larger logit <-> larger key; -0 and +0 share a key
 __device__ __forceinline__ unsigned int order_key(float z) {
     const unsigned int b = __float_as_uint(z + 0.0f);
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
+// address of `local` (a shared-memory object of this kernel) in the CTA of cluster rank `rank`
+__device__ __forceinline__ uint32_t peer_smem(const void* local, int rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(local)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ unsigned int peer_ld_u32(uint32_t addr) {
+    unsigned int v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
 
 __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     pdl_trigger();
     pdl_wait();
-    // mass histogram in three 14-bit parts (32-bit shared-memory atomics are native; a part's bucket sum stays below
-    // 2^32 for up to 262144 tokens): mass of bucket b = s_hist[0][b] + (s_hist[1][b] << 14) + (s_hist[2][b] << 28)
+    // mass histogram in three 14-bit parts (a part's bucket sum stays below 2^32 for up to 262144 tokens):
+    // mass of bucket b = s_hist[0][b] + (s_hist[1][b] << 14) + (s_hist[2][b] << 28)
     __shared__ unsigned int s_hist[3][kSelectBuckets];
-    __shared__ unsigned long long s_above, s_wsum[32];
+    __shared__ double s_cell[kSampleMaxCells];          // used in the first CTA of the cluster: every cell's sum
+    // during the select the same words hold the row's merged bucket masses (kSelectBuckets <= kSampleMaxCells)
+    unsigned long long* s_merged = reinterpret_cast<unsigned long long*>(s_cell);
+    __shared__ unsigned long long s_slice_q[kSampleCtas], s_wsum[32], s_above;
+    __shared__ double s_warp[32], s_walk_run, s_walk_target;
+    __shared__ float s_slice_max[kSampleCtas], s_maxw[32];
     __shared__ unsigned int s_digit;
-    __shared__ double s_cell[kSampleMaxCells];
-    __shared__ double s_warp[32];
     __shared__ int s_last, s_walk_cell;
-    __shared__ double s_walk_run, s_walk_target;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int V = a.V, row = blockIdx.x;
+    const int V = a.V, row = blockIdx.x, rank = blockIdx.y;   // cluster = (1, 8, 1): rank in the cluster = blockIdx.y
     const float* __restrict__ z = a.logits + (size_t)row * V;
+    double* __restrict__ e_row = a.e + (size_t)row * V;
+    unsigned long long* __restrict__ q_row = a.q + (size_t)row * V;
+    const bool nucleus = a.top_p < 1.0;
+    const int n_cells = (V + kSampleCell - 1) / kSampleCell;
+    const int cells_per = (n_cells + kSampleCtas - 1) / kSampleCtas;
+    const int c_lo = min(rank * cells_per, n_cells), c_hi = min(c_lo + cells_per, n_cells);
+    const int v_lo = c_lo * kSampleCell, v_hi = min(c_hi * kSampleCell, V);
 
-    const double* __restrict__ e_row = a.e + (size_t)row * V;
-    const unsigned long long* __restrict__ q_row = a.q + (size_t)row * V;
+    // ---- 1. row maximum, exponentials ----
+    float mx = -INFINITY;
+    for (int v = v_lo + tid; v < v_hi; v += kSampleThreads) mx = fmaxf(mx, __ldcg(z + v));
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) s_maxw[warp] = mx;
+    __syncthreads();
+    if (tid < kSampleCtas) {                        // thread t hands this slice's maximum to the CTA of rank t
+        float sm = s_maxw[0];
+        for (int i = 1; i < 32; ++i) sm = fmaxf(sm, s_maxw[i]);
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_smem(&s_slice_max[rank], tid)), "f"(sm) : "memory");
+    }
+    cluster_sync_all();
+    mx = s_slice_max[0];
+    for (int i = 1; i < kSampleCtas; ++i) mx = fmaxf(mx, s_slice_max[i]);
+    unsigned long long qsum = 0ull;
+    for (int v = v_lo + tid; v < v_hi; v += kSampleThreads) {
+        const double ev = exp(((double)__ldcg(z + v) - (double)mx) / a.temperature);
+        e_row[v] = ev;
+        if (nucleus) {
+            const unsigned long long qv = __double2ull_rn(ev * 1099511627776.0);   // 2^40 fixed point: integer sums are exact in any order
+            q_row[v] = qv;
+            qsum += qv;
+        }
+    }
 
-    // ---- top-p: key of the smallest logit inside the nucleus (0: every token) ----
+    // ---- 2. top-p: key of the smallest logit inside the nucleus (0: every token) ----
     unsigned int kstar = 0;
-    if (a.top_p < 1.0) {
-        unsigned int prefix = 0;
+    if (nucleus) {
+        for (int o = 16; o > 0; o >>= 1) qsum += __shfl_xor_sync(0xffffffffu, qsum, o);
+        if (lane == 0) s_wsum[warp] = qsum;
+        __syncthreads();                            // also orders this CTA's e / q stores before its own loads below
+        if (tid < kSampleCtas) {
+            unsigned long long t = 0ull;
+            for (int i = 0; i < 32; ++i) t += s_wsum[i];
+            asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(peer_smem(&s_slice_q[rank], tid)), "l"(t) : "memory");
+        }
+        cluster_sync_all();
         unsigned long long total_q = 0ull;
-        for (int i = 0; i < kExpSlices; ++i) total_q += __ldcg(a.q + (size_t)gridDim.x * V + row * kExpSlices + i);
+        for (int i = 0; i < kSampleCtas; ++i) total_q += s_slice_q[i];
         unsigned long long above = 0;               // mass of the keys above the current range
         unsigned long long target = (unsigned long long)ceil(a.top_p * (double)total_q);   // mass wanted
         target = target < 1ull ? 1ull : (target > total_q ? total_q : target);
@@ -774,6 +771,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
         // or above that weight already hold the mass wanted: the lighter ones lie below the threshold logit and never
         // decide a digit (buckets above the one that mixes both kinds hold none of them).  They skip the histogram.
         const unsigned long long light = (unsigned long long)((1.0 - a.top_p) * (double)total_q / (double)V * 0.999999);
+        unsigned int prefix = 0;
         int shift = 32;
         for (int pass = 0; pass < 3; ++pass) {
             const int bits = pass < 2 ? 11 : 10;
@@ -781,8 +779,8 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
             const unsigned int nb = 1u << bits;
             for (int i = tid; i < 3 * kSelectBuckets; i += kSampleThreads) s_hist[0][i] = 0u;
             __syncthreads();
-            constexpr int kBatch = 8;   // tokens per thread per step: their loads are in flight together
-            for (int v0 = 0; v0 < V; v0 += kBatch * kSampleThreads) {
+            constexpr int kBatch = 4;   // tokens per thread per step
+            for (int v0 = v_lo; v0 < v_hi; v0 += kBatch * kSampleThreads) {
                 // unconditional, clamped loads first: all 2 * kBatch of them are in flight together (a load that waits
                 // for the key test of its own token costs an L2 round trip per token)
                 float zz[kBatch];
@@ -796,7 +794,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
                 for (int j = 0; j < kBatch; ++j) {
                     const int v = v0 + j * kSampleThreads + tid;
                     const unsigned int k = order_key(zz[j]);
-                    const bool in = v < V && (pass == 0 || (k >> (shift + bits)) == prefix) && qv[j] >= light;
+                    const bool in = v < v_hi && (pass == 0 || (k >> (shift + bits)) == prefix) && qv[j] >= light;
                     digit[j] = in ? (k >> shift) & (nb - 1) : 0xffffffffu;
                     if (!in) qv[j] = 0ull;
                 }
@@ -820,12 +818,33 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
                     }
                 }
             }
-            __syncthreads();
-            {   // walk the buckets from the top: a CTA-wide scan of the bucket masses in descending bucket order; thread t
-                // owns positions 2t and 2t+1 (position p <-> bucket nb-1-p).  Integer sums: exact, exactly one owner.
+            cluster_sync_all();                     // every CTA's histogram of this pass is complete
+            {   // Bucket masses of the whole row: this CTA sums its share of the buckets (nb / 8 of them) over the 8
+                // histograms and hands each sum to every CTA's table; integer sums, the same numbers everywhere.
+                const int share = (int)nb / kSampleCtas;
+                if (tid < share) {
+                    const int b = rank * share + tid;
+                    unsigned int h[kSampleCtas][3];
+#pragma unroll
+                    for (int r = 0; r < kSampleCtas; ++r) {
+                        const uint32_t base = peer_smem(&s_hist[0][0], r);
+#pragma unroll
+                        for (int part = 0; part < 3; ++part) h[r][part] = peer_ld_u32(base + 4u * (uint32_t)(part * kSelectBuckets + b));
+                    }
+                    unsigned long long mass = 0ull;
+#pragma unroll
+                    for (int r = 0; r < kSampleCtas; ++r) mass += hist_mass(h[r][0], h[r][1], h[r][2]);
+#pragma unroll
+                    for (int r = 0; r < kSampleCtas; ++r)
+                        asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(peer_smem(&s_merged[b], r)), "l"(mass) : "memory");
+                }
+            }
+            cluster_sync_all();                     // every CTA's table of merged bucket masses is complete
+            {   // Walk the buckets from the top: a CTA-wide scan of the merged masses in descending bucket order; thread t
+                // owns positions 2t and 2t+1 (position p <-> bucket nb-1-p).  Every CTA finds the same bucket.
                 const int pa = 2 * tid;
-                const unsigned long long m0 = pa < (int)nb ? hist_mass(s_hist, nb - 1 - pa) : 0ull;
-                const unsigned long long m1 = pa + 1 < (int)nb ? hist_mass(s_hist, nb - 2 - pa) : 0ull;
+                const unsigned long long m0 = pa < (int)nb ? s_merged[nb - 1 - pa] : 0ull;
+                const unsigned long long m1 = pa + 1 < (int)nb ? s_merged[nb - 2 - pa] : 0ull;
                 const unsigned long long mine = m0 + m1;
                 unsigned long long incl = mine;
                 for (int o = 1; o < 32; o <<= 1) {
@@ -842,32 +861,38 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
                     else { s_digit = nb - 2 - pa; s_above = above + excl + m0; }
                 }
             }
-            __syncthreads();
+            __syncthreads();                        // s_digit, s_above; the next pass may clear this CTA's histogram:
+                                                    // its peers read it before the barrier above
             above = s_above;
             prefix = (prefix << bits) | s_digit;
         }
         kstar = prefix;
+        cluster_sync_all();                         // every CTA is done with its table of merged masses: the cell sums reuse it
+    } else {
+        __syncthreads();                            // this CTA's e stores before its own loads below
     }
 
-    const int n_cells = (V + kSampleCell - 1) / kSampleCell;
-    for (int c = warp; c < n_cells; c += 32) {
+    // ---- 3. cell sums of this CTA's slice, into the first CTA's table ----
+    const uint32_t cell0 = peer_smem(&s_cell[0], 0);
+    for (int c = c_lo + warp; c < c_hi; c += 32) {
         double s = 0.0;
 #pragma unroll
         for (int j = 0; j < kSampleCell / 32; ++j) {
-            int v = c * kSampleCell + j * 32 + lane;
-            const int vc = min(v, V - 1);
+            const int v = c * kSampleCell + j * 32 + lane, vc = min(v, V - 1);
             const double ev = __ldcg(e_row + vc);                       // unconditional loads: in flight together
             const unsigned int kv = kstar ? order_key(__ldcg(z + vc)) : 0xffffffffu;
             if (v < V && kv >= kstar) s += ev;
         }
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) s_cell[c] = s;
+        if (lane == 0)
+            asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(cell0 + 8u * (uint32_t)c), "l"(__double_as_longlong(s)) : "memory");
     }
-    __syncthreads();
+    cluster_sync_all();                             // all cell sums are in place; every CTA's e row is visible
+    if (rank != 0) return;
 
     // exclusive scan of the cell sums in vocabulary order: thread t owns cells [t*per, (t+1)*per)
     const int per = (n_cells + kSampleThreads - 1) / kSampleThreads;
-    const int c0 = tid * per, c1 = min(c0 + per, n_cells);
+    const int c0 = min(tid * per, n_cells), c1 = min(c0 + per, n_cells);
     double mine = 0.0;
     for (int c = c0; c < c1; ++c) mine += s_cell[c];
     double incl = mine;
@@ -941,15 +966,14 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        s_last = atomicInc(a.counter, gridDim.x - 1) == gridDim.x - 1;   // wraps back to zero
+        s_last = atomicInc(a.counter, gridDim.x - 1) == gridDim.x - 1;   // one first-CTA per row; wraps back to zero
         __threadfence();
     }
     __syncthreads();
     if (s_last) publish_results(a.mirror);
 }
 void launch_sample(cudaStream_t st, const SampleArgs& a) {
-    (void)launch_kc(k_sample_exp, dim3(a.m, kExpSlices), dim3(kSampleThreads), 0, st, kExpSlices, a);
-    launch_k(k_sample, dim3(a.m), dim3(kSampleThreads), 0, st, a);
+    (void)launch_kc(k_sample, dim3(a.m, kSampleCtas), dim3(kSampleThreads), 0, st, kSampleCtas, a);
 }
 
 __global__ void k_init_pages(int* pt, int n) {
