@@ -164,7 +164,7 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
         c.take(W.logits, sizeof(float) * (size_t)kMaxW * D.V);
         c.take(W.sample_e, sizeof(double) * (size_t)kMaxW * D.V);
-        c.take(W.sample_q, sizeof(unsigned long long) * ((size_t)kMaxW * D.V + 64));   // + the slice sums
+        c.take(W.sample_q, sizeof(unsigned long long) * (size_t)kMaxW * D.V);
         c.take(W.rope_tab, sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2));
         size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
         c.take(W.k_cache, kv);
@@ -964,7 +964,7 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
 // Sampling kernel alone: tokens of m rows of device logits.  Its completion counter is the word behind the static
 // scratch (zero at load, left at zero by every launch).
 size_t sb_k_sample_scratch_bytes(int32_t m, int32_t vocab) {
-    return m < 1 || vocab < 1 ? 0 : 2 * sizeof(double) * (size_t)m * (size_t)vocab + 512;   // exponentials as fp64 and as fixed point, slice sums
+    return m < 1 || vocab < 1 ? 0 : 2 * sizeof(double) * (size_t)m * (size_t)vocab;   // exponentials as fp64 and as fixed point
 }
 
 int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, float top_p, uint64_t seed, int64_t pos0,

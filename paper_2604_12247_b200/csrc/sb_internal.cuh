@@ -269,7 +269,7 @@ __host__ __device__ inline double sample_uniform(unsigned long long seed, long l
 constexpr int kSampleMaxVocab = 262144;
 struct SampleArgs {
     const float* logits;       // [m][V] final logits, row r0 first
-    double* e;                 // [m][V] scratch: exp((z - row max) / temperature), written by the first kernel
+    double* e;                 // [m][V] scratch: exp((z - row max) / temperature), written in the kernel's first phase
     unsigned long long* q;     // [m][V] scratch: the same as 2^40 fixed-point integers (top-p select)
     int V, r0, m;
     double temperature;        // sampling temperature T_s > 0
