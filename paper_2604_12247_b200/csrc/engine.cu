@@ -15,6 +15,7 @@ namespace sb {
 
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
 static int g_fuse = 3;            // bit 0: SwiGLU in the epilogue of the tcgen05 gate/up GEMM; bit 1: RoPE + append + attention + chunk merge in one launch
+static int g_wide_prefill = 1;    // prefill: 64 prompt rows per pass of the weight-streaming GEMMs (bf16, tcgen05 path)
 static int g_qkv_ahead = 1;       // draft loop: issue the next layer step's norm + QKV GEMM while waiting for the exit decision
 static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
 
@@ -101,6 +102,8 @@ static bool make_dims(const sb_config* c, Dims* o) {
     return true;
 }
 
+constexpr int kWideBlocks = 8, kWideRows = kWideBlocks * kMaxW;   // rows of one wide prefill pass
+
 // Scratch shared by the context and the stateless entry points.
 struct Work {
     int* page_table;
@@ -117,6 +120,10 @@ struct Work {
     float2* rope_tab;      // contexts only: cos/sin of the RoPE angles [n_pages * page][hd/2]
     float* logits;         // contexts only: [8][V] final logits of the rows being sampled (sampling decoding)
     double* sample_e;      // contexts only: [8][V] their exponentials
+    // contexts of bf16 models only: the wide prefill pass (8 blocks of 8 rows per launch of the weight-streaming GEMMs)
+    float* pf_h;           // [64][d]
+    void *pf_act_a, *pf_act_o, *pf_act_f;      // [8][16][d | qd | F]
+    float *pf_p_qkv, *pf_p_o, *pf_p_down;      // [8][kMaxSplit][8][N]
     unsigned long long* sample_q;   // contexts only: [8][V] the same as fixed-point integers (top-p)
     void* k_cache;         // [L][n_pages][page][kvd]
     void* v_cache;
@@ -160,11 +167,22 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     W.logits = nullptr;
     W.sample_e = nullptr;
     W.sample_q = nullptr;
+    W.pf_h = nullptr;
     if (with_state) {
         c.take(W.toks, sizeof(int) * (D.max_seq + 16));
         c.take(W.logits, sizeof(float) * (size_t)kMaxW * D.V);
         c.take(W.sample_e, sizeof(double) * (size_t)kMaxW * D.V);
         c.take(W.sample_q, sizeof(unsigned long long) * (size_t)kMaxW * D.V);
+        if (!D.f32) {
+            c.take(W.pf_h, sizeof(float) * kWideRows * D.d);
+            c.take(W.pf_act_a, es * 2 * kWideRows * D.d);
+            c.take(W.pf_act_o, es * 2 * kWideRows * D.qd);
+            c.take(W.pf_act_f, es * 2 * kWideRows * D.F);
+            const size_t pw = sizeof(float) * kMaxSplit * kWideRows;
+            c.take(W.pf_p_qkv, pw * (D.qd + 2 * D.kvd));
+            c.take(W.pf_p_o, pw * D.d);
+            c.take(W.pf_p_down, pw * D.d);
+        }
         c.take(W.rope_tab, sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2));
         size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
         c.take(W.k_cache, kv);
@@ -205,8 +223,9 @@ static void ensure_act(Exec& e, const void* gain, int r0, int m) {
 static bool tc_path(const Exec& e) { return e.gemm == 1 && !e.D.f32; }
 struct NextGemm { const void* W[2] = {nullptr, nullptr}; int rows = 0, K = 0; const void* act = nullptr; };
 static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, const void* act, float* out, int r0, int m,
-                void* swiglu_out = nullptr, const NextGemm& next = NextGemm()) {
+                void* swiglu_out = nullptr, const NextGemm& next = NextGemm(), int nb = 1) {
     GemmArgs a{};
+    a.nb = nb;
     a.swiglu_out = swiglu_out;
     a.next_W[0] = next.W[0]; a.next_W[1] = next.W[1]; a.next_rows = next.rows; a.next_K = next.K; a.next_act = next.act;
     int tot = 0;
@@ -293,6 +312,70 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     SB_MARK("resid");
     e.launches += 2;
     e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
+}
+
+// Wide prefill pass: one decoder layer for M <= 64 prompt rows at positions pos0 .. pos0+M-1 (bf16 models, tcgen05
+// GEMMs with the SwiGLU epilogue).  The four weight-streaming GEMMs take all rows in ONE launch each (8 blocks of 8
+// rows: the weights are read once for 64 rows instead of once for 8); the small kernels between them run per block of
+// 8 rows on that block's slice of the wide buffers, in block order, so that a block's attention sees the K/V rows
+// the blocks before it appended.  have_act: pf_act_a already holds the rows' RMSNorm with this layer's attention
+// gain (left there by the previous layer).  Ends by adding the MLP output to pf_h and, if next_gain is given,
+// leaving the rows' RMSNorm with that gain in pf_act_a.
+static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int M, int pos0,
+                            bool have_act, const void* next_gain) {
+    using T = __nv_bfloat16;
+    const Dims& D = e.D;
+    Work& W = e.W;
+    const int nblk = (M + kMaxW - 1) / kMaxW;
+    auto rows_of = [&](int b) { return M - b * kMaxW < kMaxW ? M - b * kMaxW : kMaxW; };
+    auto h_of = [&](int b) { return W.pf_h + (size_t)b * kMaxW * D.d; };
+    auto act_of = [&](void* base, int b, int K) { return (void*)((char*)base + (size_t)b * 16 * K * sizeof(T)); };
+    if (!have_act)
+        for (int b = 0; b < nblk; ++b) {
+            launch_resid_norm<T>(e.st, h_of(b), nullptr, 0, D.d, (const T*)lw.attn_norm, D.eps, act_of(W.pf_act_a, b, D.d), 0, rows_of(b));
+            e.launches++;
+        }
+    const void* wqkv[3] = {lw.wq, lw.wk, lw.wv};
+    int nqkv[3] = {D.qd, D.kvd, D.kvd};
+    const int n_qkv = D.qd + 2 * D.kvd;
+    const int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.pf_act_a, W.pf_p_qkv, 0, M, nullptr, NextGemm(), kWideBlocks);
+    for (int b = 0; b < nblk; ++b) {
+        float* p_qkv = W.pf_p_qkv + (size_t)b * s_qkv * kMaxW * n_qkv;
+        AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, act_of(W.pf_act_o, b, D.qd), D.H, D.Hkv, D.hd, D.page,
+                    D.page_shift, pos0 + b * kMaxW, 0, rows_of(b), D.chunk, p_qkv, s_qkv, W.rope_tab, W.status, {}};
+        for (int i = 0; i < D.hd / 2; ++i) aa.inv_freq[i] = D.inv_freq[i];
+        bool fused = false;
+        if (g_fuse & 2) fused = launch_attention_fused<T>(e.st, aa);
+        if (fused) {
+            e.launches += 1;
+        } else {
+            RopeArgs ra{p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
+                        pos0 + b * kMaxW, 0, rows_of(b), D.rope_base, W.rope_tab, {}};
+            for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
+            launch_rope_append<T>(e.st, ra);
+            launch_attention<T>(e.st, aa);
+            e.launches += 3;
+        }
+    }
+    const void* wo[1] = {lw.wo};
+    int no[1] = {D.d};
+    const int s_o = gemm(e, wo, no, 1, D.qd, W.pf_act_o, W.pf_p_o, 0, M, nullptr, NextGemm(), kWideBlocks);
+    for (int b = 0; b < nblk; ++b) {
+        launch_resid_norm<T>(e.st, h_of(b), W.pf_p_o + (size_t)b * s_o * kMaxW * D.d, s_o, D.d, (const T*)lw.mlp_norm, D.eps,
+                             act_of(W.pf_act_a, b, D.d), 0, rows_of(b));
+        e.launches++;
+    }
+    const void* wgu[2] = {lw.w_gate, lw.w_up};
+    int ngu[2] = {D.F, D.F};
+    gemm(e, wgu, ngu, 2, D.d, W.pf_act_a, nullptr, 0, M, W.pf_act_f, NextGemm(), kWideBlocks);   // SwiGLU in the epilogue
+    const void* wd[1] = {lw.w_down};
+    int nd[1] = {D.d};
+    const int s_d = gemm(e, wd, nd, 1, D.F, W.pf_act_f, W.pf_p_down, 0, M, nullptr, NextGemm(), kWideBlocks);
+    for (int b = 0; b < nblk; ++b) {
+        launch_resid_norm<T>(e.st, h_of(b), W.pf_p_down + (size_t)b * s_d * kMaxW * D.d, s_d, D.d, (const T*)next_gain, D.eps,
+                             act_of(W.pf_act_a, b, D.d), 0, rows_of(b));
+        e.launches++;
+    }
 }
 
 // exit-confidence / final-head kernel on rows r0 .. r0+m-1; act_a must hold their final RMSNorm
@@ -610,6 +693,7 @@ int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_L2_PREFETCH) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_QKV_AHEAD) { g_qkv_ahead = value != 0; return SB_OK; }
+    if (key == SB_OPT_WIDE_PREFILL) { g_wide_prefill = value != 0; return SB_OK; }
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
     if (key == SB_OPT_FUSE) { if (value < 0 || value > 3) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;
@@ -649,7 +733,29 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
         return SB_ERR_CUDA;
     c->h2d += sizeof(int) * n_prompt;
     int m = 0;
-    for (int p0 = 0; p0 < n_prompt; p0 += m) {
+    int done = 0;
+    // Wide passes (bf16 models on the tcgen05 path with the SwiGLU epilogue): 64 prompt rows per pass, so the weights
+    // are streamed once per 64 rows; what is left over (fewer than 16 rows) goes through 8-row passes below.
+    if (tc_path(e) && (g_fuse & 1) && g_wide_prefill && e.W.pf_h) {
+        while (n_prompt - done >= 2 * kMaxW) {
+            const int M = n_prompt - done < kWideRows ? n_prompt - done : kWideRows;
+            launch_embed<__nv_bfloat16>(e.st, (const __nv_bfloat16*)c->w.embed, e.D.d, e.W.toks + done, 0, 0, M, e.W.pf_h);
+            e.launches++;
+            for (int l = 1; l <= e.D.L; ++l)
+                layer_step_wide(e, c->layers[l - 1], c->kc(l), c->vc(l), M, done, l > 1,
+                                l < e.D.L ? c->layers[l].attn_norm : nullptr);
+            done += M;
+            if (done == n_prompt) {   // the last 8-row block's hidden rows are what the first generated token comes from
+                const int nblk = (M + kMaxW - 1) / kMaxW;
+                m = M - (nblk - 1) * kMaxW;
+                if (cudaMemcpyAsync(e.W.h, e.W.pf_h + (size_t)(nblk - 1) * kMaxW * e.D.d, sizeof(float) * m * e.D.d,
+                                    cudaMemcpyDeviceToDevice, e.st) != cudaSuccess)
+                    return SB_ERR_CUDA;
+                e.act_gain = nullptr;
+            }
+        }
+    }
+    for (int p0 = done; p0 < n_prompt; p0 += m) {
         m = n_prompt - p0 < kMaxW ? n_prompt - p0 : kMaxW;
         bool last = p0 + m == n_prompt;
         SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, e.W.toks + p0, 0, 0, m, e.W.h));

@@ -31,7 +31,10 @@ constexpr int kStageA = kTileRows * kBK * 2;  // 16 KB
 constexpr int kStageB = 16 * kBK * 2;         // 2 KB
 constexpr int kProducers = 4;                 // producer warps
 constexpr int kTcThreads = (kProducers + 5) * 32;
-static int smem_bytes(int stages) { return stages * (kStageA + kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+static int smem_bytes(int stages, int nb = 1) { return stages * (kStageA + nb * kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+// Wide mode (prefill): nb = 8 blocks of 8 activation rows ride through one launch (MMA N = 128); the stages are
+// twice as large, so one CTA per SM with the usual depth.
+constexpr int kWideBlocks = 8, kWideStages = 6;
 // Two CTAs per SM (each with its own producers, MMA issuer and TMEM accumulators) stream measurably
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;
@@ -165,8 +168,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;              // SWIZZLE_128B
     return d;
 }
-// instruction descriptor: D = f32, A = B = bf16, both K-major, N = 16, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+// instruction descriptor: D = f32, A = B = bf16, both K-major, N columns (16 per block of 8 activation rows), M = 128
+__host__ __device__ constexpr uint32_t idesc_n(uint32_t n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24); }
 
 // The four epilogue warps agree on whether to go on: each has waited (bounded) for the accumulator on its
 // own, and a named barrier that one of them skipped would hang the others.  ok_s is [2][4], alternating per call.
@@ -212,8 +215,12 @@ struct WorkIter {
     }
 };
 
-template <bool kHead, bool kPair>
+template <bool kHead, bool kPair, int NB = 1>
 __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ TcParams p) {
+    static_assert(!kHead || NB == 1, "the LM-head mode handles one block of rows");
+    constexpr int kStageBn = NB * kStageB;          // activation tile of a stage: 16 operand rows per block
+    constexpr uint32_t kCols = 16u * NB;            // TMEM columns of one accumulator
+    constexpr uint32_t kIdesc = idesc_n(kCols);
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_s;
@@ -226,7 +233,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
     const uint32_t tiles = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
     const int kStages = p.stages;
     const uint32_t smA = tiles, smB = tiles + kStages * kStageA;
-    const uint32_t bars = smB + kStages * kStageB;             // 8-byte mbarriers
+    const uint32_t bars = smB + kStages * kStageBn;            // 8-byte mbarriers
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
     auto tfull_bar = [&](int b) { return bars + 8u * (2 * kStages + b); };
@@ -246,15 +253,15 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kProducers) {   // TMEM: 32 columns = two 16-column accumulators
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(32));
+    if (warp == kProducers) {   // TMEM: two accumulators of 16 columns per block of rows
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2u * kCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
-    const uint32_t stage_bytes = (uint32_t)p.R * (kBK * 2) + kStageB;
+    const uint32_t stage_bytes = (uint32_t)p.R * (kBK * 2) + kStageBn;
 
     if (warp < kProducers) {
         // ------------------------------ TMA producers ------------------------------
@@ -301,7 +308,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             }
             pdl_wait();
             for (int f0 = warp; f0 < fill; f0 += kProducers) {
-                tma_load_2d(smB + f0 * kStageB, &p.tmB, w0.kb * kBK, 0, full_bar(f0));
+                tma_load_2d(smB + f0 * kStageBn, &p.tmB, w0.kb * kBK, 0, full_bar(f0));
                 for (int j = 0; j < kProducers; ++j) w0.next(p);
             }
             for (; w.valid(); fill += kProducers) {
@@ -310,7 +317,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_s, p.status, 1u)) break;
                 mbar_expect_tx(full_bar(stage), stage_bytes);
                 load_a(stage, w);
-                tma_load_2d(smB + stage * kStageB, &p.tmB, w.kb * kBK, 0, full_bar(stage));
+                tma_load_2d(smB + stage * kStageBn, &p.tmB, w.kb * kBK, 0, full_bar(stage));
                 for (int j = 0; j < kProducers; ++j) w.next(p);
             }
         } else {
@@ -328,11 +335,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 uint32_t use = (uint32_t)(n_local >> 1);   // how often this accumulator was used before
                 if (!(ok = mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, &abort_s, p.status, 2u))) break;
                 tc_fence_after();
-                uint32_t d_tmem = tmem_base + (uint32_t)buf * 16u;
+                uint32_t d_tmem = tmem_base + (uint32_t)buf * kCols;
                 for (int kb = it.kb0; kb < it.kb1; ++kb) {
                     if (!(ok = mbar_wait(full_bar(stage), phase, &abort_s, p.status, 3u))) break;
                     tc_fence_after();
-                    uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageB);
+                    uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageBn);
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k)   // +32 bytes per 16-element k step inside the swizzle row
                         tc_mma(d_tmem, da + 2u * k, db + 2u * k, kIdesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
@@ -363,51 +370,56 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             if (kPair) ok = epi_vote(ok, ok_s, n_local, q, lane);   // the pair epilogue synchronises the four warps
             if (!ok) break;
             tc_fence_after();
-            uint32_t v[16];
-            tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 16u, v);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator may be overwritten
-            if (kPair) {
-                // warps 2-3 hold the up projections (tile rows 64 ..): hand them to the thread that holds the
-                // gate projection of the same column, which writes silu(gate) * up as the next GEMM's operand
-                float z[kMaxW];
-#pragma unroll
-                for (int i = 0; i < kMaxW; ++i) z[i] = __uint_as_float(v[i]) + __uint_as_float(v[i + 8]);
-                if (q >= 2) {
-#pragma unroll
-                    for (int i = 0; i < kMaxW; ++i) up_s[i * 64 + (row_in_tile - 64)] = z[i];
+            const int n = it.row0 + row_in_tile;
+            const int s = item / p.n_chunks;
+#pragma unroll 1
+            for (int blk = 0; blk < NB; ++blk) {           // one block of 8 activation rows = 16 accumulator columns
+                uint32_t v[16];
+                tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * kCols + (uint32_t)blk * 16u, v);
+                if (blk == NB - 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator may be overwritten
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int col = it.row0 + row_in_tile;
-                if (q < 2 && row_in_tile < p.pair_half && col < p.n_rows[0]) {
-                    const size_t F = (size_t)p.n_rows[0];
+                const int row_base = blk * kMaxW;          // first activation row of this block
+                if (kPair) {
+                    // warps 2-3 hold the up projections (tile rows 64 ..): hand them to the thread that holds the
+                    // gate projection of the same column, which writes silu(gate) * up as the next GEMM's operand
+                    float z[kMaxW];
 #pragma unroll
-                    for (int i = 0; i < kMaxW; ++i) {
-                        if (i >= p.r0 && i < p.r0 + p.m) {
-                            const float g = z[i], u = up_s[i * 64 + row_in_tile];
-                            const float val = g / (1.f + expf(-g)) * u;
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
-                            p.swiglu_out[(size_t)i * F + col] = hi;
-                            p.swiglu_out[(size_t)(i + 8) * F + col] = __float2bfloat16_rn(val - __bfloat162float(hi));
+                    for (int i = 0; i < kMaxW; ++i) z[i] = __uint_as_float(v[i]) + __uint_as_float(v[i + 8]);
+                    if (q >= 2) {
+#pragma unroll
+                        for (int i = 0; i < kMaxW; ++i) up_s[i * 64 + (row_in_tile - 64)] = z[i];
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int col = it.row0 + row_in_tile;
+                    if (q < 2 && row_in_tile < p.pair_half && col < p.n_rows[0]) {
+                        const size_t F = (size_t)p.n_rows[0];
+                        __nv_bfloat16* dst = p.swiglu_out + (size_t)blk * 16 * F;   // [16][F] per block: high halves, low halves
+#pragma unroll
+                        for (int i = 0; i < kMaxW; ++i) {
+                            if (row_base + i >= p.r0 && row_base + i < p.r0 + p.m) {
+                                const float g = z[i], u = up_s[i * 64 + row_in_tile];
+                                const float val = g / (1.f + expf(-g)) * u;
+                                const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+                                dst[(size_t)i * F + col] = hi;
+                                dst[(size_t)(i + 8) * F + col] = __float2bfloat16_rn(val - __bfloat162float(hi));
+                            }
                         }
                     }
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");   // up_s may be overwritten by the next item
-                continue;
-            }
-            int n = it.row0 + row_in_tile;
-            if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
-                int s = item / p.n_chunks;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");   // up_s may be overwritten by the next block / item
+                } else if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
 #pragma unroll
-                for (int i = 0; i < kMaxW; ++i) {
-                    if (i >= p.r0 && i < p.r0 + p.m) {
-                        float z = __uint_as_float(v[i]) + __uint_as_float(v[i + 8]);
-                        if (kHead) {
-                            soft_push(tr[i], z, n, p.inv_tau);
-                            if (p.logits_dbg) p.logits_dbg[(size_t)(i - p.r0) * p.n_total + n] = z;
-                        } else {
-                            p.out[((size_t)s * kMaxW + i) * p.n_total + p.n_off[it.mat] + n] = z;
+                    for (int i = 0; i < kMaxW; ++i) {
+                        if (row_base + i >= p.r0 && row_base + i < p.r0 + p.m) {
+                            float z = __uint_as_float(v[i]) + __uint_as_float(v[i + 8]);
+                            if (kHead) {
+                                soft_push(tr[i], z, n, p.inv_tau);
+                                if (p.logits_dbg) p.logits_dbg[(size_t)(i - p.r0) * p.n_total + n] = z;
+                            } else {   // split-K partials [block][split][8][n_total]
+                                p.out[(((size_t)blk * p.S + s) * kMaxW + i) * p.n_total + p.n_off[it.mat] + n] = z;
+                            }
                         }
                     }
                 }
@@ -438,7 +450,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
     __syncthreads();
     if (warp == kProducers) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kCols));
     }
     if (!kHead) return;
 
@@ -541,20 +553,20 @@ static int choose_pair_half(int n_rows, int G) {
 }
 
 static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_end, int n_mats, int K, const void* act,
-                        bool head, bool pair = false) {
+                        bool head, bool pair = false, int nb = 1) {
     std::vector<uint64_t> key;
     for (int j = 0; j < n_mats; ++j) { key.push_back((uint64_t)(uintptr_t)W[j]); key.push_back((uint64_t)n_end[j]); }
     key.push_back((uint64_t)K);
     key.push_back((uint64_t)(uintptr_t)act);
-    key.push_back((head ? 1 : 0) + (pair ? 2 : 0));
+    key.push_back((head ? 1 : 0) + (pair ? 2 : 0) + 4 * nb);
     key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_split_penalty_pm << 40));
     auto it = cache->plans.find(key);
     if (it != cache->plans.end()) return it->second;
     TcPlan* pl = new TcPlan();
     memset(&pl->p, 0, sizeof(pl->p));
     TcParams& p = pl->p;
-    int G = sm_count() * g_ctas_per_sm;
-    p.stages = g_stages;
+    int G = sm_count() * (nb > 1 ? 1 : g_ctas_per_sm);
+    p.stages = nb > 1 ? kWideStages : g_stages;
     p.n_mats = n_mats;
     p.KB = (K + kBK - 1) / kBK;
     int prev = 0;
@@ -576,20 +588,21 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     p.n_chunks = chunks;
     p.n_items = chunks * p.S;
     pl->grid = p.n_items < G ? p.n_items : G;
-    bool ok = make_map(&p.tmB, act, 16, K, 16);
+    bool ok = make_map(&p.tmB, act, 16 * nb, K, 16 * nb);
     for (int j = 0; j < n_mats && ok; ++j) ok = make_map(&p.tmA[j], W[j], p.n_rows[j], K, pair ? p.pair_half : p.R);
     if (!ok) { delete pl; return nullptr; }
     cache->plans[key] = pl;
     return pl;
 }
 
-template <bool kHead, bool kPair> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
+template <bool kHead, bool kPair, int NB = 1> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaFuncSetAttribute(k_tc<kHead, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(kMaxStages));
+        cudaFuncSetAttribute(k_tc<kHead, kPair, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             NB > 1 ? smem_bytes(kWideStages, NB) : smem_bytes(kMaxStages));
         attr_set = true;
     }
-    launch_k(k_tc<kHead, kPair>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages), st, p);
+    launch_k(k_tc<kHead, kPair, NB>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages, NB), st, p);
 }
 
 bool tc_set_split_penalty(int per_mille) {
@@ -637,11 +650,13 @@ bool tc_set_tuning(int stages, int ctas_per_sm) {
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status) {
     const bool pair = a.swiglu_out != nullptr;
     if (pair && (a.n_mats != 2 || a.n_end[1] != 2 * a.n_end[0])) return -1;
-    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false, pair);
+    const int nb = a.nb > 1 ? kWideBlocks : 1;
+    if (a.nb > 1 && a.nb != kWideBlocks) return -1;
+    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false, pair, nb);
     if (!pl) return -1;
     TcParams p = pl->p;
     p.out = a.out; p.n_total = a.n_total; p.r0 = a.r0; p.m = a.m; p.status = status;
-    if (a.next_W[0] && g_l2_next_every > 0) {   // announce a later pair-mode GEMM: same plan that GEMM will use
+    if (a.next_W[0] && g_l2_next_every > 0 && nb == 1) {   // announce a later pair-mode GEMM: same plan that GEMM will use
         const void* nW[2] = {a.next_W[0], a.next_W[1]};
         int n_end[2] = {a.next_rows, 2 * a.next_rows};
         TcPlan* nx = get_plan(cache, nW, n_end, 2, a.next_K, a.next_act, false, true);
@@ -653,9 +668,11 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsig
     }
     if (pair) {
         p.swiglu_out = reinterpret_cast<__nv_bfloat16*>(a.swiglu_out);
-        launch<false, true>(st, pl, p);
+        if (nb > 1) launch<false, true, kWideBlocks>(st, pl, p);
+        else launch<false, true>(st, pl, p);
     } else {
-        launch<false, false>(st, pl, p);
+        if (nb > 1) launch<false, false, kWideBlocks>(st, pl, p);
+        else launch<false, false>(st, pl, p);
     }
     return p.S;
 }

@@ -302,6 +302,10 @@ struct GemmArgs {          // out[s][row][n] = sum_k act[row][k] * W[n][k]   for
     const void* next_W[2];
     int next_rows, next_K;
     const void* next_act;
+    // tcgen05 kernel only, wide mode (prefill): nb = 8 blocks of 8 activation rows in one launch.  act is then
+    // [nb][16][K] (block b = rows 8b .. 8b+7: high halves, low halves), out is [nb][n_split][8][n_total],
+    // swiglu_out [nb][16][n_end[0]], and r0 / m count rows over all blocks (0 .. 63).  0 or 1: one block.
+    int nb;
 };
 
 struct HeadArgs {          // exit-confidence / final-head kernel
