@@ -124,6 +124,8 @@ struct Work {
     float* pf_h;           // [64][d]
     void *pf_act_a, *pf_act_o, *pf_act_f;      // [8][16][d | qd | F]
     float *pf_p_qkv, *pf_p_o, *pf_p_down;      // [8][kMaxSplit][8][N]
+    float *pf_q, *pf_attn_part;                // [64][qd]; [8][max_chunks][8][H][hd+2]
+    size_t pf_attn_stride;                     // floats per block of pf_attn_part
     unsigned long long* sample_q;   // contexts only: [8][V] the same as fixed-point integers (top-p)
     void* k_cache;         // [L][n_pages][page][kvd]
     void* v_cache;
@@ -182,6 +184,9 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
             c.take(W.pf_p_qkv, pw * (D.qd + 2 * D.kvd));
             c.take(W.pf_p_o, pw * D.d);
             c.take(W.pf_p_down, pw * D.d);
+            c.take(W.pf_q, sizeof(float) * kWideRows * D.qd);
+            W.pf_attn_stride = (size_t)max_chunks * kMaxW * D.H * (D.hd + 2);
+            c.take(W.pf_attn_part, sizeof(float) * kWideBlocks * W.pf_attn_stride);
         }
         c.take(W.rope_tab, sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2));
         size_t kv = es * (size_t)D.L * D.n_pages * D.page * D.kvd;
@@ -316,9 +321,9 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
 
 // Wide prefill pass: one decoder layer for M <= 64 prompt rows at positions pos0 .. pos0+M-1 (bf16 models, tcgen05
 // GEMMs with the SwiGLU epilogue).  The four weight-streaming GEMMs take all rows in ONE launch each (8 blocks of 8
-// rows: the weights are read once for 64 rows instead of once for 8); the small kernels between them run per block of
-// 8 rows on that block's slice of the wide buffers, in block order, so that a block's attention sees the K/V rows
-// the blocks before it appended.  have_act: pf_act_a already holds the rows' RMSNorm with this layer's attention
+// rows: the weights are read once for 64 rows instead of once for 8); so do the residual/RMSNorm kernel and the
+// RoPE/append kernel; the attention kernels run all full blocks in one launch (a block per grid.z), after the append,
+// so that a block's attention sees the K/V rows of the blocks before it.  have_act: pf_act_a already holds the rows' RMSNorm with this layer's attention
 // gain (left there by the previous layer).  Ends by adding the MLP output to pf_h and, if next_gain is given,
 // leaving the rows' RMSNorm with that gain in pf_act_a.
 static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int M, int pos0,
@@ -326,56 +331,53 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
     using T = __nv_bfloat16;
     const Dims& D = e.D;
     Work& W = e.W;
-    const int nblk = (M + kMaxW - 1) / kMaxW;
-    auto rows_of = [&](int b) { return M - b * kMaxW < kMaxW ? M - b * kMaxW : kMaxW; };
-    auto h_of = [&](int b) { return W.pf_h + (size_t)b * kMaxW * D.d; };
     auto act_of = [&](void* base, int b, int K) { return (void*)((char*)base + (size_t)b * 16 * K * sizeof(T)); };
-    if (!have_act)
-        for (int b = 0; b < nblk; ++b) {
-            launch_resid_norm<T>(e.st, h_of(b), nullptr, 0, D.d, (const T*)lw.attn_norm, D.eps, act_of(W.pf_act_a, b, D.d), 0, rows_of(b));
-            e.launches++;
-        }
+    if (!have_act) {
+        launch_resid_norm<T>(e.st, W.pf_h, nullptr, 0, D.d, (const T*)lw.attn_norm, D.eps, W.pf_act_a, 0, M);
+        e.launches++;
+    }
     const void* wqkv[3] = {lw.wq, lw.wk, lw.wv};
     int nqkv[3] = {D.qd, D.kvd, D.kvd};
-    const int n_qkv = D.qd + 2 * D.kvd;
     const int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, W.pf_act_a, W.pf_p_qkv, 0, M, nullptr, NextGemm(), kWideBlocks);
-    for (int b = 0; b < nblk; ++b) {
-        float* p_qkv = W.pf_p_qkv + (size_t)b * s_qkv * kMaxW * n_qkv;
-        AttnArgs aa{W.q, k_cache_l, v_cache_l, W.page_table, W.attn_part, act_of(W.pf_act_o, b, D.qd), D.H, D.Hkv, D.hd, D.page,
-                    D.page_shift, pos0 + b * kMaxW, 0, rows_of(b), D.chunk, p_qkv, s_qkv, W.rope_tab, W.status, {}};
-        for (int i = 0; i < D.hd / 2; ++i) aa.inv_freq[i] = D.inv_freq[i];
-        bool fused = false;
-        if (g_fuse & 2) fused = launch_attention_fused<T>(e.st, aa);
-        if (fused) {
-            e.launches += 1;
-        } else {
-            RopeArgs ra{p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                        pos0 + b * kMaxW, 0, rows_of(b), D.rope_base, W.rope_tab, {}};
-            for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
-            launch_rope_append<T>(e.st, ra);
+    // RoPE + K/V append for all rows in one launch, then the separate attention kernels over all full blocks of 8
+    // rows at once (grid.z = block; every block sees the K/V rows of the blocks before it, already appended), then
+    // the ragged last block, if any, by itself
+    {
+        RopeArgs ra{W.pf_p_qkv, s_qkv, W.pf_q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
+                    pos0, 0, M, D.rope_base, W.rope_tab, {}};
+        for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
+        launch_rope_append<T>(e.st, ra);
+        e.launches++;
+        const int n_full = M / kMaxW, rem = M - n_full * kMaxW;
+        if (n_full > 0) {
+            AttnArgs aa{W.pf_q, k_cache_l, v_cache_l, W.page_table, W.pf_attn_part, W.pf_act_o, D.H, D.Hkv, D.hd, D.page,
+                        D.page_shift, pos0, 0, kMaxW, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
+            aa.n_blocks = n_full;
+            aa.part_block_stride = W.pf_attn_stride;
             launch_attention<T>(e.st, aa);
-            e.launches += 3;
+            e.launches += 2;
+        }
+        if (rem > 0) {
+            AttnArgs aa{W.pf_q + (size_t)n_full * kMaxW * D.qd, k_cache_l, v_cache_l, W.page_table,
+                        W.pf_attn_part + (size_t)n_full * W.pf_attn_stride, act_of(W.pf_act_o, n_full, D.qd), D.H, D.Hkv, D.hd,
+                        D.page, D.page_shift, pos0 + n_full * kMaxW, 0, rem, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
+            launch_attention<T>(e.st, aa);
+            e.launches += 2;
         }
     }
     const void* wo[1] = {lw.wo};
     int no[1] = {D.d};
     const int s_o = gemm(e, wo, no, 1, D.qd, W.pf_act_o, W.pf_p_o, 0, M, nullptr, NextGemm(), kWideBlocks);
-    for (int b = 0; b < nblk; ++b) {
-        launch_resid_norm<T>(e.st, h_of(b), W.pf_p_o + (size_t)b * s_o * kMaxW * D.d, s_o, D.d, (const T*)lw.mlp_norm, D.eps,
-                             act_of(W.pf_act_a, b, D.d), 0, rows_of(b));
-        e.launches++;
-    }
+    launch_resid_norm<T>(e.st, W.pf_h, W.pf_p_o, s_o, D.d, (const T*)lw.mlp_norm, D.eps, W.pf_act_a, 0, M);   // all rows
+    e.launches++;
     const void* wgu[2] = {lw.w_gate, lw.w_up};
     int ngu[2] = {D.F, D.F};
     gemm(e, wgu, ngu, 2, D.d, W.pf_act_a, nullptr, 0, M, W.pf_act_f, NextGemm(), kWideBlocks);   // SwiGLU in the epilogue
     const void* wd[1] = {lw.w_down};
     int nd[1] = {D.d};
     const int s_d = gemm(e, wd, nd, 1, D.F, W.pf_act_f, W.pf_p_down, 0, M, nullptr, NextGemm(), kWideBlocks);
-    for (int b = 0; b < nblk; ++b) {
-        launch_resid_norm<T>(e.st, h_of(b), W.pf_p_down + (size_t)b * s_d * kMaxW * D.d, s_d, D.d, (const T*)next_gain, D.eps,
-                             act_of(W.pf_act_a, b, D.d), 0, rows_of(b));
-        e.launches++;
-    }
+    launch_resid_norm<T>(e.st, W.pf_h, W.pf_p_down, s_d, D.d, (const T*)next_gain, D.eps, W.pf_act_a, 0, M);
+    e.launches++;
 }
 
 // exit-confidence / final-head kernel on rows r0 .. r0+m-1; act_a must hold their final RMSNorm

@@ -370,9 +370,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             if (kPair) ok = epi_vote(ok, ok_s, n_local, q, lane);   // the pair epilogue synchronises the four warps
             if (!ok) break;
             tc_fence_after();
-            const int n = it.row0 + row_in_tile;
-            const int s = item / p.n_chunks;
-#pragma unroll 1
             for (int blk = 0; blk < NB; ++blk) {           // one block of 8 activation rows = 16 accumulator columns
                 uint32_t v[16];
                 tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * kCols + (uint32_t)blk * 16u, v);
@@ -409,7 +406,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                         }
                     }
                     asm volatile("bar.sync 1, 128;" ::: "memory");   // up_s may be overwritten by the next block / item
-                } else if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
+                    continue;
+                }
+                const int n = it.row0 + row_in_tile;
+                if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
+                    const int s = item / p.n_chunks;
 #pragma unroll
                     for (int i = 0; i < kMaxW; ++i) {
                         if (row_base + i >= p.r0 && row_base + i < p.r0 + p.m) {

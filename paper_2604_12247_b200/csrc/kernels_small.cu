@@ -34,7 +34,7 @@ void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, i
 // ------------------------------------------------------------------------------------------------
 constexpr int kNormThreads = 1024;
 constexpr int kNormVec = 2;   // float4 per thread: rows up to 1024 * 2 * 4 = 8192 wide
-template <typename T>
+template <typename T, bool kWide>
 __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__ h, const float* __restrict__ part,
                                                             int n_split, int d, const T* __restrict__ gain, float eps,
                                                             void* __restrict__ act, int r0, unsigned int* __restrict__ clear16) {
@@ -43,8 +43,11 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
     pdl_wait();
     // optional: zero 16 words for the kernels that follow (the stateless calls' status word and ticket)
     if (clear16 && blockIdx.x == 0 && threadIdx.x < 16) clear16[threadIdx.x] = 0u;
-    int row = r0 + blockIdx.x;
-    float4* hr = reinterpret_cast<float4*>(h + (size_t)row * d);
+    // kWide: rows beyond the first 8 (wide prefill passes) live in further blocks of 8: their split-K partials are
+    // [block][split][8][d] and their operand rows [block][Act rows][d]; the hidden rows are contiguous
+    const int row_all = r0 + blockIdx.x, blk = kWide ? row_all / kMaxW : 0, row = row_all - blk * kMaxW;
+    float4* hr = reinterpret_cast<float4*>(h + (size_t)row_all * d);
+    const float* __restrict__ part_b = part + ((size_t)blk * n_split * kMaxW + row) * d;   // this row's first partial
     const int nv = d >> 2;
     float4 v[kNormVec], g4[kNormVec];
     float ss = 0.f;
@@ -56,7 +59,7 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
             v[j] = hr[k4];
             if (gain) g4[j] = load_gain4(gain, k4 << 2);
             if (part) {
-                float4 p = sum_splits4(reinterpret_cast<const float4*>(part + (size_t)row * d) + k4, (size_t)kMaxW * d / 4, n_split);
+                float4 p = sum_splits4(reinterpret_cast<const float4*>(part_b) + k4, (size_t)kMaxW * d / 4, n_split);
                 v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
                 hr[k4] = v[j];
             }
@@ -72,7 +75,7 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
     for (int w = 0; w < kNormThreads / 32; ++w) tot += red[w];
     float inv = rsqrtf(tot / (float)d + eps);
     using A = Act<T>;
-    typename A::type* a = reinterpret_cast<typename A::type*>(act);
+    typename A::type* a = reinterpret_cast<typename A::type*>(act) + (size_t)blk * A::rows * d;
 #pragma unroll
     for (int j = 0; j < kNormVec; ++j) {
         int k4 = threadIdx.x + j * kNormThreads;
@@ -84,7 +87,8 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
 template <typename T>
 void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d, const T* gain, float eps,
                        void* act, int r0, int m, unsigned int* clear16) {
-    launch_k(k_resid_norm<T>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16);
+    if (r0 + m > kMaxW) launch_k(k_resid_norm<T, true>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16);
+    else launch_k(k_resid_norm<T, false>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -137,7 +141,8 @@ __global__ void k_rope_append(RopeArgs a) {
     int i = threadIdx.x;
     int qd = a.H * a.hd, kvd = a.Hkv * a.hd, ntot = qd + 2 * kvd;
     int col = head * a.hd;   // q heads, then k heads, then v heads are contiguous in the GEMM output
-    const float* p0 = a.qkv + (size_t)row * ntot + col + i;
+    const int blk = row / kMaxW;   // partials of rows beyond the first 8 (wide prefill passes): [block][split][8][ntot]
+    const float* p0 = a.qkv + ((size_t)blk * a.n_split * kMaxW + (row - blk * kMaxW)) * ntot + col + i;
     float x0 = sum_splits(p0, (size_t)kMaxW * ntot, a.n_split);
     float x1 = sum_splits(p0 + half, (size_t)kMaxW * ntot, a.n_split);
     bool is_v = head >= a.H + a.Hkv;
@@ -216,6 +221,13 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
     const int kvh = blockIdx.x, c = blockIdx.y;
+    if (!kFused && a.n_blocks > 1) {                 // several blocks of 8 rows in one launch: this CTA's block
+        const int blk = blockIdx.z;
+        a.q += (size_t)blk * kMaxW * a.H * HD;
+        a.part += (size_t)blk * a.part_block_stride;
+        a.pos0 += blk * kMaxW;
+        if (c * kAttnChunk > a.pos0 + a.r0 + a.m - 1) return;   // a chunk beyond this block's last position
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
     const int kvd = a.Hkv * HD, qd = a.H * HD;
@@ -509,6 +521,14 @@ __global__ void k_attn_combine(AttnArgs a) {
     pdl_wait();
     int hq = blockIdx.x, row = a.r0 + blockIdx.y, e = threadIdx.x;
     int hd = a.hd;
+    using A = Act<T>;
+    typename A::type* act_out = reinterpret_cast<typename A::type*>(a.act_out);
+    if (a.n_blocks > 1) {                            // several blocks of 8 rows in one launch: this CTA's block
+        const int blk = blockIdx.z;
+        a.part += (size_t)blk * a.part_block_stride;
+        a.pos0 += blk * kMaxW;
+        act_out += (size_t)blk * A::rows * a.H * hd;
+    }
     int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own
     float M = -INFINITY, L = 0.f, O = 0.f;
     constexpr int kBatch = 8;   // chunks whose partials are loaded together (one L2 round trip per batch)
@@ -533,8 +553,7 @@ __global__ void k_attn_combine(AttnArgs a) {
             }
         }
     }
-    using A = Act<T>;
-    A::store(reinterpret_cast<typename A::type*>(a.act_out), row, hq * hd + e, a.H * hd, O / L);
+    A::store(act_out, row, hq * hd + e, a.H * hd, O / L);
 }
 
 static size_t attn_smem(int P, int HD, size_t elt, bool fused) {
@@ -583,14 +602,15 @@ static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid, i
 }
 
 template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) {
-    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
-    dim3 grid(a.Hkv, n_chunks);
+    const int nz = a.n_blocks > 1 ? a.n_blocks : 1;
+    int n_chunks = (a.pos0 + a.r0 + (nz - 1) * kMaxW + a.m - 1) / kAttnChunk + 1;   // up to the last block's last position
+    dim3 grid(a.Hkv, n_chunks, nz);
     switch (a.hd) {
         case 32: launch_attn_partial<T, 32, false>(st, a, grid, 0); break;
         case 64: launch_attn_partial<T, 64, false>(st, a, grid, 0); break;
         default: launch_attn_partial<T, 128, false>(st, a, grid, 0); break;
     }
-    launch_k(k_attn_combine<T>, dim3(a.H, a.m), dim3(a.hd), 0, st, a);
+    launch_k(k_attn_combine<T>, dim3(a.H, a.m, nz), dim3(a.hd), 0, st, a);
 }
 
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a) {

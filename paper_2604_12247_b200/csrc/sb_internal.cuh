@@ -341,12 +341,17 @@ struct AttnArgs {
     const float2* rope_tab;   // nullable: cos/sin [position][hd/2] (launch_rope_table)
     unsigned int* status;     // device status word: a staging copy that never completes raises code 5 here
     double inv_freq[64];   // as in RopeArgs
+    // separate kernels only: n_blocks > 1 runs that many blocks of 8 rows in one launch (grid.z = block); block b
+    // takes rows 8b .. 8b+7 of q ([8 n_blocks][H*hd]), its own partials (part + b * part_block_stride), its own 16
+    // operand rows of act_out, and sits at positions pos0 + 8b ..; r0 must be 0 and m = 8
+    int n_blocks = 0;
+    size_t part_block_stride = 0;
 };
 
 struct RopeArgs {
-    const float* qkv;      // partials [n_split][8][qd + 2 kvd]
+    const float* qkv;      // partials [block][n_split][8][qd + 2 kvd]; block = row / 8 (one block unless m > 8)
     int n_split;
-    float* q;              // [8][qd]
+    float* q;              // [m][qd]
     void* k_cache;
     void* v_cache;
     const int* page_table;
