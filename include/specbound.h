@@ -281,8 +281,8 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                    issues the RMSNorm and QKV GEMM of the layer step that follows if the row does not exit
  *                    (they write scratch only; on an exit they are discarded).  Results do not depend on it.
  *   SB_OPT_WIDE_PREFILL (default option only) 1 (default) = sb_prefill of a bf16 model on the tcgen05 path (with the
- *                    SwiGLU epilogue on) sends 64 prompt rows per pass through the weight-streaming GEMMs (the
- *                    weights are read once per 64 rows) and the fewer than 16 rows left over through 8-row passes;
+ *                    SwiGLU epilogue on) sends up to 128 prompt rows per pass through the weight-streaming GEMMs (the
+ *                    weights are read once per 128 rows) and the fewer than 16 rows left over through 8-row passes;
  *                    0 = 8-row passes only.  Both are deterministic; they may differ in the split-K summation order,
  *                    i.e. in the last bits of the K/V cache and of the first token's logits. */
 enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,

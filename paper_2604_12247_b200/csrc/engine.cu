@@ -15,7 +15,7 @@ namespace sb {
 
 static int g_default_gemm = -1;   // -1: pick tcgen05 for bf16 when available
 static int g_fuse = 3;            // bit 0: SwiGLU in the epilogue of the tcgen05 gate/up GEMM; bit 1: RoPE + append + attention + chunk merge in one launch
-static int g_wide_prefill = 1;    // prefill: 64 prompt rows per pass of the weight-streaming GEMMs (bf16, tcgen05 path)
+static int g_wide_prefill = 1;    // prefill: up to 128 prompt rows per pass of the weight-streaming GEMMs (bf16, tcgen05 path)
 static int g_qkv_ahead = 1;       // draft loop: issue the next layer step's norm + QKV GEMM while waiting for the exit decision
 static int g_trace = 0;           // 1: the stateless layer call times every launch with CUDA events and prints them
 
@@ -102,7 +102,7 @@ static bool make_dims(const sb_config* c, Dims* o) {
     return true;
 }
 
-constexpr int kWideBlocks = 8, kWideRows = kWideBlocks * kMaxW;   // rows of one wide prefill pass
+constexpr int kWideRows = kWideBlocks * kMaxW;   // rows of one wide prefill pass
 
 // Scratch shared by the context and the stateless entry points.
 struct Work {
@@ -120,11 +120,11 @@ struct Work {
     float2* rope_tab;      // contexts only: cos/sin of the RoPE angles [n_pages * page][hd/2]
     float* logits;         // contexts only: [8][V] final logits of the rows being sampled (sampling decoding)
     double* sample_e;      // contexts only: [8][V] their exponentials
-    // contexts of bf16 models only: the wide prefill pass (8 blocks of 8 rows per launch of the weight-streaming GEMMs)
-    float* pf_h;           // [64][d]
-    void *pf_act_a, *pf_act_o, *pf_act_f;      // [8][16][d | qd | F]
-    float *pf_p_qkv, *pf_p_o, *pf_p_down;      // [8][kMaxSplit][8][N]
-    float *pf_q, *pf_attn_part;                // [64][qd]; [8][max_chunks][8][H][hd+2]
+    // contexts of bf16 models only: the wide prefill pass (kWideBlocks = B blocks of 8 rows per launch of the GEMMs)
+    float* pf_h;           // [8 B][d]
+    void *pf_act_a, *pf_act_o, *pf_act_f;      // [B][16][d | qd | F]
+    float *pf_p_qkv, *pf_p_o, *pf_p_down;      // [B][kMaxSplit][8][N]
+    float *pf_q, *pf_attn_part;                // [8 B][qd]; [B][max_chunks][8][H][hd+2]
     size_t pf_attn_stride;                     // floats per block of pf_attn_part
     unsigned long long* sample_q;   // contexts only: [8][V] the same as fixed-point integers (top-p)
     void* k_cache;         // [L][n_pages][page][kvd]
@@ -319,9 +319,9 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
 }
 
-// Wide prefill pass: one decoder layer for M <= 64 prompt rows at positions pos0 .. pos0+M-1 (bf16 models, tcgen05
-// GEMMs with the SwiGLU epilogue).  The four weight-streaming GEMMs take all rows in ONE launch each (8 blocks of 8
-// rows: the weights are read once for 64 rows instead of once for 8); so do the residual/RMSNorm kernel and the
+// Wide prefill pass: one decoder layer for M <= 8 * kWideBlocks prompt rows at positions pos0 .. pos0+M-1 (bf16 models, tcgen05
+// GEMMs with the SwiGLU epilogue).  The four weight-streaming GEMMs take all rows in ONE launch each (blocks of 8
+// rows: the weights are read once for 128 rows instead of once for 8); so do the residual/RMSNorm kernel and the
 // RoPE/append kernel; the attention kernels run all full blocks in one launch (a block per grid.z), after the append,
 // so that a block's attention sees the K/V rows of the blocks before it.  have_act: pf_act_a already holds the rows' RMSNorm with this layer's attention
 // gain (left there by the previous layer).  Ends by adding the MLP output to pf_h and, if next_gain is given,
@@ -736,8 +736,8 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
     c->h2d += sizeof(int) * n_prompt;
     int m = 0;
     int done = 0;
-    // Wide passes (bf16 models on the tcgen05 path with the SwiGLU epilogue): 64 prompt rows per pass, so the weights
-    // are streamed once per 64 rows; what is left over (fewer than 16 rows) goes through 8-row passes below.
+    // Wide passes (bf16 models on the tcgen05 path with the SwiGLU epilogue): up to 128 prompt rows per pass, so the
+    // weights are streamed once per 128 rows; what is left over (fewer than 16 rows) goes through 8-row passes below.
     if (tc_path(e) && (g_fuse & 1) && g_wide_prefill && e.W.pf_h) {
         while (n_prompt - done >= 2 * kMaxW) {
             const int M = n_prompt - done < kWideRows ? n_prompt - done : kWideRows;

@@ -32,9 +32,11 @@ constexpr int kStageB = 16 * kBK * 2;         // 2 KB
 constexpr int kProducers = 4;                 // producer warps
 constexpr int kTcThreads = (kProducers + 5) * 32;
 static int smem_bytes(int stages, int nb = 1) { return stages * (kStageA + nb * kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
-// Wide mode (prefill): nb = 8 blocks of 8 activation rows ride through one launch (MMA N = 128); the stages are
-// twice as large, so one CTA per SM with the usual depth.
-constexpr int kWideBlocks = 8, kWideStages = 6;
+// Wide mode (prefill): kWideBlocks blocks of 8 activation rows ride through one launch (MMA N = 16 per block); a stage
+// is 16 KB of weights + 2 KB per block of activations, so one CTA per SM with 4 stages (>= the number of producers).
+constexpr int kWideStages = 4;
+static_assert(kWideStages * (kStageA + kWideBlocks * kStageB) + 1280 <= 227 * 1024, "wide stages exceed shared memory");
+static_assert(2 * 16 * kWideBlocks <= 512, "two wide accumulators exceed tensor memory");
 // Two CTAs per SM (each with its own producers, MMA issuer and TMEM accumulators) stream measurably
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;

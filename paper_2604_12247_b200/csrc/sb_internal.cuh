@@ -284,6 +284,10 @@ struct SampleArgs {
 // ---------------------------------------------------------------------------------------------
 // Launch arguments
 // ---------------------------------------------------------------------------------------------
+// Wide mode of the tcgen05 GEMM (prefill): blocks of 8 activation rows that ride through one launch.  16 blocks =
+// 128 rows: MMA N = 256, two 256-column accumulators = all of an SM's tensor memory, one CTA per SM.
+constexpr int kWideBlocks = 16;
+
 struct GemmArgs {          // out[s][row][n] = sum_k act[row][k] * W[n][k]   for rows r0 .. r0+m-1
     const void* W[3];      // up to three matrices sharing K and the activation operand
     int n_end[3];          // cumulative row counts: matrix j owns output columns [n_end[j-1], n_end[j])
@@ -302,9 +306,9 @@ struct GemmArgs {          // out[s][row][n] = sum_k act[row][k] * W[n][k]   for
     const void* next_W[2];
     int next_rows, next_K;
     const void* next_act;
-    // tcgen05 kernel only, wide mode (prefill): nb = 8 blocks of 8 activation rows in one launch.  act is then
+    // tcgen05 kernel only, wide mode (prefill): nb = kWideBlocks blocks of 8 activation rows in one launch.  act is then
     // [nb][16][K] (block b = rows 8b .. 8b+7: high halves, low halves), out is [nb][n_split][8][n_total],
-    // swiglu_out [nb][16][n_end[0]], and r0 / m count rows over all blocks (0 .. 63).  0 or 1: one block.
+    // swiglu_out [nb][16][n_end[0]], and r0 / m count rows over all blocks.  0 or 1: one block.
     int nb;
 };
 

@@ -1,4 +1,4 @@
-"""Wide prefill passes (64 prompt rows per launch of the weight-streaming GEMMs) against the 8-row passes and the
+"""Wide prefill passes (up to 128 prompt rows per launch of the weight-streaming GEMMs) against the 8-row passes and the
 oracle.  What prefill leaves behind is the K/V cache of every layer and the first generated token; both are checked
 through what is computed from them: the first token, the hidden state of that token after every layer (it attends
 over all cached prompt positions of each layer), and the tokens decoded afterwards."""
@@ -27,8 +27,8 @@ def _hidden_after_prefill(ctx, prompt, n_layers):
     return first, hid
 
 
-# 16: the smallest wide pass; 64 / 128: whole passes; 70: a wide pass + 6 rows through an 8-row pass; 100: a second,
-# ragged wide pass (36 rows = 4 blocks and a half); 130 + a page size of 16: passes that straddle pages
+# 16: the smallest wide pass; 64, 70, 100: one ragged wide pass (70 and 100 end in a partial block of 8 rows); 128: a
+# whole pass; 130: a whole pass + 2 rows through an 8-row pass.  Page size 16: passes straddle pages
 @pytest.mark.parametrize("n_prompt", [16, 64, 70, 100, 128, 130])
 def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt):
     shape = SMALL_BF16
@@ -74,7 +74,7 @@ def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt):
 
 
 def test_wide_prefill_at_the_bench_shape_matches_narrow_first_token_and_tokens():
-    """7B shape, 200-token prompt (three wide passes + one 8-row pass): same first token and decoded tokens as the
+    """7B shape, 200-token prompt (a whole wide pass + a ragged one of 72 rows): same first token and decoded tokens as the
     8-row passes, and the oracle's teacher-forced check on the first tokens."""
     run = inputs.RUNS["7b-damped"]
     wg = inputs.make_weights(run.shape, run.seed, device="cuda", damp_rho=run.damp_rho)
