@@ -28,8 +28,8 @@ def _hidden_after_prefill(ctx, prompt, n_layers):
 
 
 # 16: the smallest wide pass; 64, 70, 100: one ragged wide pass (70 and 100 end in a partial block of 8 rows); 128: a
-# whole pass; 130: a whole pass + 2 rows through an 8-row pass.  Page size 16: passes straddle pages
-@pytest.mark.parametrize("n_prompt", [16, 64, 70, 100, 128, 130])
+# whole pass; 130: a whole pass + 2 rows through an 8-row pass; 300: two whole passes and a ragged one.  Page size 16
+@pytest.mark.parametrize("n_prompt", [16, 64, 70, 100, 128, 130, 300])
 def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt):
     shape = SMALL_BF16
     w = inputs.make_weights(shape, 5, damp_rho=0.3)
