@@ -497,7 +497,7 @@ static void final_tokens(sb_ctx* c, int r0, int m, long long pos0, int* token, c
     head(e, c->w.lm_head, r0, m, 1.f, 2.f, c->conf_d(), c->token_d(), c->flag_d(), e.W.logits);
     SampleArgs a{e.W.logits, e.W.sample_e, e.W.sample_q, e.D.V, r0, m, (double)c->sample_temperature, (double)c->sample_top_p, c->sample_seed, pos0, token,
                  reinterpret_cast<unsigned int*>(e.W.res + 57), mir};
-    launch_sample(e.st, a);
+    if (!launch_sample(e.st, a)) e.err = SB_ERR_CUDA;
     e.launches++;
 }
 
@@ -1086,7 +1086,7 @@ int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature
     if (rc) return rc;
     SampleArgs a{logits, static_cast<double*>(scratch), static_cast<unsigned long long*>(scratch) + (size_t)m * vocab, vocab, 0, m, (double)temperature, (double)top_p, seed, pos0, token,
                  reinterpret_cast<unsigned int*>(base + kStaticScratchBytes), Mirror{nullptr, nullptr, 0u}};
-    launch_sample((cudaStream_t)stream, a);
+    if (!launch_sample((cudaStream_t)stream, a)) { (void)cudaGetLastError(); return SB_ERR_CUDA; }
     return cuda_ok(cudaGetLastError());
 }
 

@@ -992,8 +992,8 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     __syncthreads();
     if (s_last) publish_results(a.mirror);
 }
-void launch_sample(cudaStream_t st, const SampleArgs& a) {
-    (void)launch_kc(k_sample, dim3(a.m, kSampleCtas), dim3(kSampleThreads), 0, st, kSampleCtas, a);
+bool launch_sample(cudaStream_t st, const SampleArgs& a) {
+    return launch_kc(k_sample, dim3(a.m, kSampleCtas), dim3(kSampleThreads), 0, st, kSampleCtas, a) == cudaSuccess;
 }
 
 __global__ void k_init_pages(int* pt, int n) {

@@ -382,7 +382,7 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror);
-void launch_sample(cudaStream_t st, const SampleArgs& a);
+bool launch_sample(cudaStream_t st, const SampleArgs& a);   // false: the cluster launch was refused
 void launch_init_pages(cudaStream_t st, int* page_table, int n_pages);
 
 // ---- launchers (gemm_simt.cu) ----
