@@ -40,6 +40,17 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
                                                             void* __restrict__ act, int r0, unsigned int* __restrict__ clear16) {
     __shared__ float red[kNormThreads / 32];
     pdl_trigger();
+    // the gains are weights: no kernel writes them, so they are requested before the grid-dependency wait (a layer's
+    // gains were last touched a whole token ago and come from HBM)
+    const int nv = d >> 2;
+    float4 g4[kNormVec];
+    if (gain) {
+#pragma unroll
+        for (int j = 0; j < kNormVec; ++j) {
+            int k4 = threadIdx.x + j * kNormThreads;
+            if (k4 < nv) g4[j] = load_gain4(gain, k4 << 2);
+        }
+    }
     pdl_wait();
     // optional: zero 16 words for the kernels that follow (the stateless calls' status word and ticket)
     if (clear16 && blockIdx.x == 0 && threadIdx.x < 16) clear16[threadIdx.x] = 0u;
@@ -48,8 +59,7 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
     const int row_all = r0 + blockIdx.x, blk = kWide ? row_all / kMaxW : 0, row = row_all - blk * kMaxW;
     float4* hr = reinterpret_cast<float4*>(h + (size_t)row_all * d);
     const float* __restrict__ part_b = part + ((size_t)blk * n_split * kMaxW + row) * d;   // this row's first partial
-    const int nv = d >> 2;
-    float4 v[kNormVec], g4[kNormVec];
+    float4 v[kNormVec];
     float ss = 0.f;
     // every load of a thread is independent: the hidden row, all partials and the gains are in flight at once
 #pragma unroll
@@ -57,7 +67,6 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
         int k4 = threadIdx.x + j * kNormThreads;
         if (k4 < nv) {
             v[j] = hr[k4];
-            if (gain) g4[j] = load_gain4(gain, k4 << 2);
             if (part) {
                 float4 p = sum_splits4(reinterpret_cast<const float4*>(part_b) + k4, (size_t)kMaxW * d / 4, n_split);
                 v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
