@@ -354,6 +354,7 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
                         D.page_shift, pos0, 0, kMaxW, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
             aa.n_blocks = n_full;
             aa.part_block_stride = W.pf_attn_stride;
+            aa.pos_pred0 = pos0;
             launch_attention<T>(e.st, aa);
             e.launches += 2;
         }
@@ -361,6 +362,7 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
             AttnArgs aa{W.pf_q + (size_t)n_full * kMaxW * D.qd, k_cache_l, v_cache_l, W.page_table,
                         W.pf_attn_part + (size_t)n_full * W.pf_attn_stride, act_of(W.pf_act_o, n_full, D.qd), D.H, D.Hkv, D.hd,
                         D.page, D.page_shift, pos0 + n_full * kMaxW, 0, rem, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
+            aa.pos_pred0 = pos0;   // the pass's RoPE/append launch wrote the rows of the full blocks too
             launch_attention<T>(e.st, aa);
             e.launches += 2;
         }

@@ -24,7 +24,14 @@ __global__ void k_embed(const T* __restrict__ embed, int d, const int* __restric
 }
 template <typename T>
 void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, int tok_scalar, int row0, int m, float* h) {
+    // Every step of a row (a prompt block, a drafted token, an autoregressive token) starts with this kernel, and it is
+    // launched WITHOUT programmatic dependent launch: it starts only after everything before it in the stream has
+    // completed.  The kernels behind it may therefore rely on what earlier steps wrote (the K/V rows of earlier
+    // positions) being complete even before their own grid-dependency wait returns.
+    const bool saved = g_use_pdl;
+    g_use_pdl = false;
     launch_k(k_embed<T>, dim3(m), dim3(256), 0, st, embed, d, toks_dev, tok_scalar, row0, h);
+    g_use_pdl = saved;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -230,6 +237,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
     const int kvh = blockIdx.x, c = blockIdx.y;
+    const int pos_pred0 = a.pos_pred0 >= 0 ? a.pos_pred0 : a.pos0 + a.r0;   // separate kernels: first position the preceding RoPE/append launch wrote
     if (!kFused && a.n_blocks > 1) {                 // several blocks of 8 rows in one launch: this CTA's block
         const int blk = blockIdx.z;
         a.q += (size_t)blk * kMaxW * a.H * HD;
@@ -260,26 +268,48 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     // and no kernel of a launch sequence writes it: like the weights it may be read before the wait.
     int my_page = 0;
     if (my_t < pos_new0) my_page = a.page_table[my_t >> a.page_shift];
-    pdl_wait();
+    // Rows of EARLIER steps of this layer (positions below pos_done) are complete when this kernel starts: between such
+    // steps the stream holds a launch without programmatic overlap (the embedding kernel that starts every step, or
+    // the clear of a stateless call).  Their copies -- the long, cold loads of this kernel -- start before the
+    // grid-dependency wait.  Separate kernels: the RoPE/append kernel right before this one wrote the rows from
+    // pos_done on; they are staged after the wait, on the same barrier (the warp arrives with the second batch).
+    const int pos_done = kFused ? pos_new0 : pos_pred0;
     __syncthreads();   // barriers initialised
     // 1. stage the block's K rows (first warp of the block) or V rows (second warp): one TMA copy per row of an
     //    earlier launch; rows beyond the last position are zeroed (their probabilities are 0, but 0 * garbage
     //    must stay 0); rows this launch creates are written in step 2
+    constexpr uint32_t kRowBytes = HD * (uint32_t)sizeof(T);
     {
-        constexpr uint32_t kRowBytes = HD * (uint32_t)sizeof(T);
-        const bool old_row = my_t < pos_new0;
+        const bool early = my_t < pos_done;
         const uint32_t bar = smem_u32(&stage_bar[v]);
-        const unsigned n_old = __popc(__ballot_sync(0xffffffffu, old_row));
-        if (lane == 0) mbar_expect_tx(bar, n_old * kRowBytes);
+        const unsigned n_early = __popc(__ballot_sync(0xffffffffu, early));
+        if (lane == 0) {
+            if (kFused) mbar_expect_tx(bar, n_early * kRowBytes);
+            else mbar_expect_tx_only(bar, n_early * kRowBytes);
+        }
         __syncwarp();
         unsigned char* row = (hsel ? V_w : K_w) + lane * ROWB;
-        if (old_row) {
+        if (early) {
             const T* src = reinterpret_cast<const T*>(hsel ? a.v_cache : a.k_cache) +
                            ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
             bulk_load(smem_u32(row), src, kRowBytes, bar);
         } else if (my_t > pos_last) {
 #pragma unroll
             for (int j = 0; j < (int)kRowBytes / 16; ++j) reinterpret_cast<uint4*>(row)[j] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    pdl_wait();
+    if (!kFused) {   // the rows the RoPE/append kernel just wrote
+        const bool late = my_t >= pos_done && my_t < pos_new0;
+        const uint32_t bar = smem_u32(&stage_bar[v]);
+        const unsigned n_late = __popc(__ballot_sync(0xffffffffu, late));
+        if (lane == 0) mbar_expect_tx(bar, n_late * kRowBytes);
+        __syncwarp();
+        if (late) {
+            unsigned char* row = (hsel ? V_w : K_w) + lane * ROWB;
+            const T* src = reinterpret_cast<const T*>(hsel ? a.v_cache : a.k_cache) +
+                           ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+            bulk_load(smem_u32(row), src, kRowBytes, bar);
         }
     }
     // 2. while those copies fly: q, and (fused) the new positions' K and V

@@ -81,6 +81,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// adds to the bytes the current phase waits for, without arriving
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -350,6 +354,9 @@ struct AttnArgs {
     // operand rows of act_out, and sits at positions pos0 + 8b ..; r0 must be 0 and m = 8
     int n_blocks = 0;
     size_t part_block_stride = 0;
+    // separate kernels only: first position that the RoPE/append launch preceding this one wrote (-1: pos0 + r0).
+    // K/V rows below it belong to earlier steps and may be fetched before the grid-dependency wait.
+    int pos_pred0 = -1;
 };
 
 struct RopeArgs {
