@@ -319,13 +319,13 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
 }
 
-// Wide prefill pass: one decoder layer for M <= 8 * kWideBlocks prompt rows at positions pos0 .. pos0+M-1 (bf16 models, tcgen05
-// GEMMs with the SwiGLU epilogue).  The four weight-streaming GEMMs take all rows in ONE launch each (blocks of 8
-// rows: the weights are read once for 128 rows instead of once for 8); so do the residual/RMSNorm kernel and the
-// RoPE/append kernel; the attention kernels run all full blocks in one launch (a block per grid.z), after the append,
-// so that a block's attention sees the K/V rows of the blocks before it.  have_act: pf_act_a already holds the rows' RMSNorm with this layer's attention
-// gain (left there by the previous layer).  Ends by adding the MLP output to pf_h and, if next_gain is given,
-// leaving the rows' RMSNorm with that gain in pf_act_a.
+// Wide prefill pass: one decoder layer for M <= 8 * kWideBlocks prompt rows at positions pos0 .. pos0+M-1 (bf16
+// models, tcgen05 GEMMs with the SwiGLU epilogue).  The four weight-streaming GEMMs take all rows in ONE launch each
+// (blocks of 8 rows: the weights are read once for 128 rows instead of once for 8); so do the residual/RMSNorm
+// kernel and the RoPE/append kernel; the attention kernels run all full blocks in one launch (a block per grid.z),
+// after the append, so that a block's attention sees the K/V rows of the blocks before it.  have_act: pf_act_a
+// already holds the rows' RMSNorm with this layer's attention gain (left there by the previous layer).  Ends by
+// adding the MLP output to pf_h and, if next_gain is given, leaving the rows' RMSNorm with that gain in pf_act_a.
 static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int M, int pos0,
                             bool have_act, const void* next_gain) {
     using T = __nv_bfloat16;
