@@ -186,9 +186,9 @@ int sb_generate_ar(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t
  * sampled token of its row, so sb_generate returns exactly what sb_generate_ar returns for the
  * same (temperature, top_p, seed): lossless sample by sample.  The final logits of the
  * <= SB_MAX_W rows go through a [8][vocab] fp32 buffer of the workspace and their exponentials
- * through two [8][vocab] 8-byte ones; the exit tests never write logits.  temperature 0 (the default) restores greedy decoding.  Errors: SB_ERR_ARG
- * (negative or NaN temperature, top_p outside (0, 1]), SB_ERR_CAPACITY (vocab > 262144 with
- * temperature > 0). */
+ * through two [8][vocab] 8-byte ones; the exit tests never write logits.  temperature 0 (the
+ * default) restores greedy decoding.  Errors: SB_ERR_ARG (negative or NaN temperature, top_p
+ * outside (0, 1]), SB_ERR_CAPACITY (vocab > 262144 with temperature > 0). */
 int sb_set_sampling(sb_ctx* ctx, float temperature, float top_p, uint64_t seed);
 
 /* The counter-based uniform number in (0, 1) behind sb_set_sampling: the splitmix64 output function
@@ -197,19 +197,20 @@ double sb_sample_uniform(uint64_t seed, int64_t pos);
 
 /* ---- stateless kernel entry points (micro-benchmarks, unit parity) ---------------------------- */
 
-/* Scratch bytes the two calls below need for this shape. */
-size_t sb_k_scratch_bytes(const sb_config* cfg);
-
 /* Sampling kernel alone (the rule of sb_set_sampling): token[j] (device) = inverse-CDF sample of
  * the top_p nucleus of softmax(logits[j][:] / temperature) at sb_sample_uniform(seed, pos0 + j),
  * for m <= SB_MAX_W rows of device fp32 logits [m][vocab].  scratch: device memory, 8-byte
- * aligned, at least sb_k_sample_scratch_bytes(m, vocab) bytes (the rows' exponentials, fp64 and fixed point),
- * owned by the caller.  Asynchronous on `stream` (one launch).  Errors: SB_ERR_ARG (null
+ * aligned, at least sb_k_sample_scratch_bytes(m, vocab) bytes (the rows' exponentials, fp64 and
+ * fixed point), owned by the caller.  Asynchronous on `stream` (one launch).  Errors: SB_ERR_ARG (null
  * pointer, m outside [1, SB_MAX_W], temperature <= 0, top_p outside (0, 1], scratch misaligned or
  * too small), SB_ERR_CAPACITY (vocab > 262144). */
 size_t sb_k_sample_scratch_bytes(int32_t m, int32_t vocab);
 int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature, float top_p, uint64_t seed,
                 int64_t pos0, int32_t* token, void* scratch, size_t scratch_bytes, void* stream);
+
+/* Scratch bytes the two calls below need for this shape. */
+size_t sb_k_scratch_bytes(const sb_config* cfg);
+
 
 /* Exit-confidence kernel on m rows of hidden states (Section 3.2, Eq. 2):
  * h device fp32 [m, d]; final_norm / lm_head device in cfg->dtype; tau_l > 0.
