@@ -583,6 +583,7 @@ int orc_teacher_forced(orc_ctx* o, const int32_t* tokens, int n_total, int from,
  *   p >= threshold for the first script_len drafted rows (in drafting order):
  *   script[k] = e >= 1 -> row k exits at layer e with that layer's greedy token;
  *   script[k] = 0      -> row k does not exit (difficult token).
+ * tau[l-1] <= 0: layer l is not tested for an exit (probe-layer mask); scripted or not, no row exits there.
  * rounds / max_rounds: optional trace. Returns the number of rounds, or -1. */
 int orc_specbound_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int n_gen,
                            int d_max, int w_max, const double* tau, double threshold,
@@ -620,6 +621,10 @@ int orc_specbound_generate(orc_ctx* o, const int32_t* prompt, int n_prompt, int 
                 orc_layer_forward(o, l, h + (size_t)r0 * d, r + 1 - r0, n + r0);
                 for (int i = r0; i <= r; ++i) { depth[i] = l; R.layers_done[i]++; }
                 R.layer_steps++;
+                /* probe-layer mask (a reading of Section 3.2's "first layer where p >= threshold" for callers that
+                 * do not want every layer tested): a layer whose temperature is <= 0 is walked but not tested,
+                 * so no exit can happen there */
+                if (!(tau[l - 1] > 0.0)) continue;
                 double p; int t;
                 exit_logits(o, l, h + (size_t)r * d, z);
                 confidence_from_logits(z, V, tau[l - 1], &p, &t);

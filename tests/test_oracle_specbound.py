@@ -69,8 +69,8 @@ def test_speculative_equals_autoregressive_over_grid(which, tiny_weights, tiny_d
         assert {0, 1, 2, 3}.issubset(seen_acc) and {1, 2, 4, 8}.issubset(seen_w)
 
 
-def test_contract_runs_as_specified(tiny_weights, tiny_damped_weights):
-    """Config 'tiny' as written, and its damped variant: tokens equal AR, trace is sane."""
+def test_tiny_workloads_run_as_defined(tiny_weights, tiny_damped_weights):
+    """Workload 'tiny' as defined, and its damped variant: tokens equal AR, trace is sane."""
     for which, w in (("tiny", tiny_weights), ("tiny-damped", tiny_damped_weights)):
         run = inputs.RUNS[which]
         pr = inputs.make_prompt(run.shape, run.n_prompt, run.seed).numpy()
@@ -127,6 +127,51 @@ def test_scenario_long_shallow_chain():
     assert r.layer_steps == 14 + 4 + 2
     assert r.probes == 14
     assert all(r.layers_done[i] == EIGHT.n_layers for i in range(r.w))
+
+
+MASKS = [(0, 1, 1), (1, 0, 1), (1, 1, 0), (0, 0, 1), (0, 1, 0), (1, 0, 0), (0, 0, 0)]
+
+
+def test_probe_layer_mask(tiny_damped_weights):
+    """Probe-layer mask (tau_l <= 0: layer l is walked but not tested).  Pins:
+    * the output is still plain greedy decoding, for every mask (the exactness claim of Section 3.3 does not depend
+      on where exits are looked for);
+    * a masked layer never appears as an exit layer, and a row is charged one probe per UNMASKED layer it walked;
+    * a masked run is the unmasked algorithm with a test that cannot pass at that layer: temperature 1e30 there makes
+      the confidence 1/V < threshold, and that run must agree round for round (width, depth, exit layers, drafts,
+      accepted, emitted) -- only the probe count differs, by exactly the probes spent on hopeless layers;
+    * masking every layer turns each round into one autoregressive step that went d_max deep (w = 1, no draft)."""
+    run = inputs.RUNS["tiny-damped"]
+    shape, w = run.shape, tiny_damped_weights
+    pr = inputs.make_prompt(shape, run.n_prompt, run.seed).numpy()
+    n_gen, d_max, w_max, thr = 24, 3, 4, 0.3
+    base = (1.6, 1.3, 1.0)
+    ar = oracle.Oracle(shape, w, 64).ar_generate(pr, n_gen)
+    seen_exit_layers = set()
+    for mask in MASKS:
+        tau_masked = tuple(t if on else 0.0 for t, on in zip(base, mask))
+        tau_hopeless = tuple(t if on else 1e30 for t, on in zip(base, mask))
+        out, rounds = _run(shape, w, pr, n_gen, d_max, w_max, tau_masked, thr)
+        out_h, rounds_h = _run(shape, w, pr, n_gen, d_max, w_max, tau_hopeless, thr)
+        assert np.array_equal(out, ar) and np.array_equal(out_h, ar), mask
+        check_round_invariants(rounds, shape.n_layers, d_max, w_max)
+        assert len(rounds) == len(rounds_h)
+        for r, q in zip(rounds, rounds_h):
+            assert (r.w, r.D, r.emitted, r.accepted_drafts, r.layer_steps) == (q.w, q.D, q.emitted, q.accepted_drafts, q.layer_steps)
+            assert list(r.exit_layer[:r.w]) == list(q.exit_layer[:q.w]) and list(r.draft[:r.w]) == list(q.draft[:q.w])
+            walked = [e if e else d_max for e in r.exit_layer[:r.w]]          # layers each row's own draft step walked
+            assert r.probes == sum(sum(mask[:n]) for n in walked)
+            assert q.probes == sum(walked)
+            for e in r.exit_layer[:r.w]:
+                assert e == 0 or mask[e - 1] == 1
+                seen_exit_layers.add(e)
+        if not any(mask):
+            assert all(r.w == 1 and r.D == d_max and r.draft[0] == -1 and r.probes == 0 for r in rounds)
+    assert {1, 2, 3}.issubset(seen_exit_layers)      # the masks really moved exits between layers
+    # negative temperatures mask as well, and the unmasked schedule is untouched by the feature
+    out_a, rounds_a = _run(shape, w, pr, n_gen, d_max, w_max, (-1.0, 1.3, 1.0), thr)
+    out_b, rounds_b = _run(shape, w, pr, n_gen, d_max, w_max, (0.0, 1.3, 1.0), thr)
+    assert np.array_equal(out_a, out_b) and [r.probes for r in rounds_a] == [r.probes for r in rounds_b]
 
 
 def test_bad_arguments_are_refused(tiny_weights):
