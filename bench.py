@@ -35,8 +35,11 @@ import torch
 
 from paper_2604_12247_b200 import inputs
 
-METRIC = "batch-1 decode tokens/s (SpecBound, 7B shape)"
 NOMINAL_HBM_GBS = 8000.0
+
+
+def metric_name(run: "inputs.Run") -> str:
+    return f"batch-1 decode tokens/s (SpecBound, {run.shape.name})"
 
 
 def captured_traffic(key: str):
@@ -132,6 +135,28 @@ def cpu_oracle_sample(run: inputs.Run, weights_cpu: dict, p: int = 2, g: int = 4
                       f"({run.shape.name}, {run.shape.dtype} weights, fp64 arithmetic, OpenMP over output rows), {dt:.1f} s"}, dt
 
 
+def cpu_oracle_specbound_sample(run: inputs.Run, weights_cpu: dict, p: int, g: int):
+    """Times the oracle's SpecBound loop (Section 3.3) on a bounded sample of the workload: a p-token prompt and g
+    generated tokens with the workload's d_max, w_max, temperatures and threshold.  The decode phase is what the
+    metric counts, so the prefill (the same loop asked for one token) is timed separately and taken off.
+    Returns (decode tokens/s, decode seconds, total seconds, rounds)."""
+    from oracle import oracle
+    pr = inputs.make_prompt(run.shape, p, run.seed).numpy()
+    max_seq = p + g + run.w_max + 1
+    o = oracle.Oracle(run.shape, weights_cpu, max_seq)
+    t0 = time.perf_counter()
+    o.specbound_generate(pr, 1, run.d_max, run.w_max, run.tau, run.threshold)
+    t_prefill = time.perf_counter() - t0
+    o.close()
+    o = oracle.Oracle(run.shape, weights_cpu, max_seq)
+    t0 = time.perf_counter()
+    _, rounds = o.specbound_generate(pr, g, run.d_max, run.w_max, run.tau, run.threshold)
+    t_all = time.perf_counter() - t0
+    o.close()
+    dec = max(t_all - t_prefill, 1e-9)
+    return (g - 1) / dec, dec, t_all + t_prefill, len(rounds)
+
+
 def host_weights(run: inputs.Run):
     if torch.cuda.is_available():
         w = inputs.make_weights(run.shape, run.seed, device="cuda", damp_rho=run.damp_rho)
@@ -139,8 +164,13 @@ def host_weights(run: inputs.Run):
     return inputs.make_weights(run.shape, run.seed, device="cpu", damp_rho=run.damp_rho)
 
 
+REF_PROMPT, REF_GEN = 4, 8   # the slice of the workload one reference step decodes
+
+
 def reference_arm(args, run: inputs.Run):
-    """--impl reference: the CPU oracle as it stands, on the host cores, same metric and config."""
+    """--impl reference: the CPU oracle as it stands, on the host cores, same metric (decode tokens/s of the SpecBound
+    loop) and hyper-parameters; every step decodes a bounded slice of the workload (REF_PROMPT prompt tokens,
+    REF_GEN generated tokens), stated in config.timed_slice, first speculatively, then autoregressively."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -149,17 +179,26 @@ def reference_arm(args, run: inputs.Run):
     w = host_weights(run)
     for _ in range(args.warmup):
         cpu_oracle_sample(run, w, 1, 1)
-    vals, secs = [], []
-    desc = None
+    dec_s, tot_s, ar_tps, rounds = [], [], [], 0
     for _ in range(args.steps):
-        desc, dt = cpu_oracle_sample(run, w, 4, 28)   # 31 forward passes per step: about 10 s
-        vals.append(desc["value"]); secs.append(dt)
-    v = sum(31 for _ in vals) / sum(secs)    # 31 forward passes per step
-    desc["value"] = v
-    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak",
+        _, dec, tot, rounds = cpu_oracle_specbound_sample(run, w, REF_PROMPT, REF_GEN)
+        desc, dt = cpu_oracle_sample(run, w, REF_PROMPT, REF_GEN)
+        dec_s.append(dec); tot_s.append(tot + dt); ar_tps.append(desc["value"])
+    v = args.steps * (REF_GEN - 1) / sum(dec_s)
+    cfg = workload_config(run, "cpu-oracle")
+    cfg["timed_slice"] = (f"each step: {REF_PROMPT}-token prompt + {REF_GEN} generated tokens of this workload through the oracle's "
+                          f"SpecBound loop (value = decode tokens/s, prefill taken off), then the same slice autoregressively; "
+                          f"NOT the full {run.n_prompt} + {run.n_gen} tokens")
+    cores = len(os.sched_getaffinity(0))
+    base = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"oracle SpecBound loop, {REF_PROMPT}-token prompt + {REF_GEN} tokens ({rounds} rounds), d_max {run.d_max}, w_max "
+                      f"{run.w_max}, {run.shape.name}, {run.shape.dtype} weights, fp64 arithmetic, OpenMP over output rows; "
+                      f"{sum(dec_s) / len(dec_s):.1f} s of decoding per step",
+            "ar_forward_passes_per_s": sum(ar_tps) / len(ar_tps)}
+    line = {"impl": "reference", "metric": metric_name(run), "value": v, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sum(tot_s) / len(tot_s), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(run, "cpu-oracle"), "cpu_baseline": desc,
+            "config": cfg, "cpu_baseline": base,
             "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -172,6 +211,76 @@ def workload_config(run: inputs.Run, parallelism: str) -> dict:
             "batch": 1, "prompt_tokens": run.n_prompt, "generated_tokens": run.n_gen, "d_max": run.d_max, "w_max": run.w_max,
             "tau": [round(t, 4) for t in run.tau], "threshold": run.threshold, "parallelism": parallelism,
             "l2": "inputs larger than L2 (every layer pass streams >= 400 MB of distinct weights)"}
+
+
+def verify_roofline(s: inputs.Shape, stats, peak: float):
+    """Achieved bandwidth of the verify pass over the unified passes of `stats`: algorithmic bytes of one layer pass =
+    the layer's weights once + K,V of the positions attended over (read) / appended (written), whatever the rows."""
+    wb = inputs.weight_bytes(s)
+    S = lambda f: sum(getattr(st, f) for st in stats)
+    uni_steps, uni_us, uni_pos = S("unified_layer_steps"), S("us_unified"), S("unified_kv_positions")
+    uni_bytes = uni_steps * wb["layer"] + uni_pos * kv_bytes_per_pos(s)
+    ach = uni_bytes / (uni_us * 1e-6) / 1e9 if uni_us > 0 else 0.0
+    return ach, uni_bytes, uni_steps, uni_us
+
+
+def oracle_check(ctx, run: inputs.Run, weights_cpu: dict, n_prompt: int, n_gen: int) -> dict:
+    """Accepted tokens against the oracle: the GPU decodes n_gen tokens from a short prompt with the workload's own
+    weights and hyper-parameters (speculatively and autoregressively), and the oracle makes ONE teacher-forced pass
+    over prompt + GPU tokens, reporting for every generated position its own top-1, the top-2 margin and how far the
+    GPU's token lies below the top-1 logit.  A GPU token is correct if it is the oracle's top-1 or the margin at that
+    position is below the logit tolerance (2e-2 for bf16 storage, 1e-4 for fp32); such positions are counted.  (A
+    teacher-forced pass over the workload's full prompt would take the host cores tens of minutes.)"""
+    from oracle import oracle
+    tol = 2e-2 if run.shape.dtype == "bf16" else 1e-4
+    pr = inputs.make_prompt(run.shape, n_prompt, run.seed + 5).numpy()
+    sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, run.tau, run.threshold)
+    ar = ctx.generate_ar(pr, n_gen)
+    toks = np.concatenate([pr, sp["tokens"]]).astype(np.int32)
+    t0 = time.perf_counter()
+    o = oracle.Oracle(run.shape, weights_cpu, len(toks) + 1)
+    top1, _, margin, deficit = o.teacher_forced(toks, n_prompt)
+    o.close()
+    dt = time.perf_counter() - t0
+    off = top1 != sp["tokens"]
+    return {"prompt_tokens": n_prompt, "positions": int(n_gen), "not_top1": int(off.sum()),
+            "near_ties": int((margin < 2 * tol).sum()), "wrong": int((off & (margin >= 2 * tol)).sum()),
+            "worst_deficit": float(deficit.min()), "logit_tolerance": tol, "smallest_margin": float(margin.min()),
+            "tokens_equal_ar": bool(np.array_equal(sp["tokens"], ar["tokens"])), "oracle_seconds": dt,
+            "what": "teacher-forced oracle pass over a short-prompt generation of this workload (same weights, d_max, w_max, "
+                    "tau, threshold); wrong = GPU token differs from the oracle's top-1 at a position whose top-2 margin is "
+                    "not below twice the tolerance"}
+
+
+def damped_arm(args, peak: float) -> dict:
+    """The labelled addition `7b-damped` (damped deep layers: the synthetic stand-in for trained exit heads, with the
+    paper's own hyper-parameters), measured the same way as the main workload for a few steps: the configuration in
+    which drafts get accepted."""
+    from paper_2604_12247_b200 import binding
+    run = inputs.RUNS["7b-damped"]
+    s = run.shape
+    w = inputs.make_weights(s, run.seed, device="cuda", damp_rho=run.damp_rho)
+    prompt = inputs.make_prompt(s, run.n_prompt, run.seed).numpy()
+    ctx = binding.Context(s, w, run.n_prompt + run.n_gen + run.w_max + 8, kv_page=64)
+    steps = max(1, min(args.steps, 3))
+    for _ in range(2):
+        ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold)
+    ctx.generate_ar(prompt, 32)
+    stats = [ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold) for _ in range(steps)]
+    ars = [ctx.generate_ar(prompt, run.n_gen) for _ in range(steps)]
+    dec_tok = run.n_gen - 1
+    value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in stats) * 1e-6)
+    ar_value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in ars) * 1e-6)
+    ach, _, uni_steps, uni_us = verify_roofline(s, [r["stats"] for r in stats], peak)
+    st = stats[-1]["stats"]
+    out = {"workload": workload_config(run, "single GPU"), "steps": steps, "value": value, "unit": "tokens/s",
+           "ar_tokens_per_s": ar_value, "speedup_vs_ar": value / ar_value,
+           "tokens_equal_ar": bool(np.array_equal(stats[-1]["tokens"], ars[-1]["tokens"])),
+           "emitted_per_round": st.emitted / max(st.rounds, 1), "accepted_drafts_per_round": st.accepted_drafts / max(st.rounds, 1),
+           "exit_hist": list(st.exit_hist[:run.d_max + 1]), "width_hist": list(st.width_hist),
+           "roofline_frac": ach / peak, "verify_us_per_layer": uni_us / max(uni_steps, 1)}
+    ctx.close()
+    return out
 
 
 def product_arm(args, run: inputs.Run):
@@ -240,11 +349,7 @@ def product_arm(args, run: inputs.Run):
     peak, peak_src = measured_peak()
     wb = inputs.weight_bytes(s)
     S = lambda f: sum(getattr(st, f) for st in stats)
-    # verify pass: algorithmic bytes of one layer pass = the layer's weights once + K,V of the
-    # positions attended over (read) / appended (written), whatever the number of rows
-    uni_steps, uni_us, uni_pos = S("unified_layer_steps"), S("us_unified"), S("unified_kv_positions")
-    uni_bytes = uni_steps * wb["layer"] + uni_pos * kv_bytes_per_pos(s)
-    ach = uni_bytes / (uni_us * 1e-6) / 1e9 if uni_us > 0 else 0.0
+    ach, uni_bytes, uni_steps, uni_us = verify_roofline(s, stats, peak)
     roofline = {"kernel": "verify pass: one decoder layer for w<=8 rows (weight-streaming GEMMs + paged-KV attention), "
                           "averaged over the unified passes of the timed region",
                 "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
@@ -260,7 +365,7 @@ def product_arm(args, run: inputs.Run):
                      "traffic": captured_traffic(f"exit_confidence:{s.name}")}
     st0 = stats[-1]
     line = {
-        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": metric_name(run), "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dec_ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "storage_dtype": s.dtype, "data": "synthetic",
         "config": workload_config(run, f"replicas x{world}" if world > 1 else "single GPU"),
@@ -273,6 +378,9 @@ def product_arm(args, run: inputs.Run):
         "rounds_per_step": st0.rounds, "emitted_per_round": st0.emitted / max(st0.rounds, 1),
         "accepted_drafts_per_round": st0.accepted_drafts / max(st0.rounds, 1), "probes_per_step": st0.probes,
         "exit_hist": list(st0.exit_hist[:run.d_max + 1]), "width_hist": list(st0.width_hist),
+        "ttft_ms": statistics.median(st.us_prefill for st in stats) / 1e3,
+        "ttft_note": "time to first token through sb_generate: prompt host->device, prefill of all prompt tokens (wide passes), "
+                     "first token device->host; host wall clock, median over the timed steps",
         "phase_ms_per_step": {"prefill_host": st0.us_prefill / 1e3, "decode_dev": st0.us_decode_dev / 1e3,
                               "draft_dev": st0.us_draft / 1e3, "verify_dev": st0.us_verify / 1e3,
                               "unified_dev": st0.us_unified / 1e3, "probe_kernels_dev": st0.us_probe_kernels / 1e3 * st0.probes / max(st0.probes_timed, 1)},
@@ -286,55 +394,119 @@ def product_arm(args, run: inputs.Run):
         oracle.build()
         wc = inputs.weights_to(w, "cpu")
         line["cpu_baseline"], _ = cpu_oracle_sample(run, wc, 4, 40)   # 43 forward passes: about 10-30 s of CPU work
-    print(json.dumps(line), flush=True)
+        if args.oracle_check_tokens > 0:
+            line["oracle_check"] = oracle_check(ctx, run, wc, 16, args.oracle_check_tokens)
+        del wc
     ctx.close()
+    if world == 1 and args.workload == "7b" and not args.no_damped:
+        line["damped"] = damped_arm(args, peak)
+    print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
 def sweep_arm(args, run: inputs.Run):
-    """Hyper-parameter sweep in the spirit of the paper's ablations (Section 4.4: confidence threshold, depth bound
-    d_max, width bound w_max), on the synthetic workload given by --workload: for every point the decode tokens/s
-    of SpecBound, the speed-up over autoregressive decoding with the same kernels, tokens emitted per round, and
-    what Eq. 5 predicts from the measured per-draft acceptance rate (Eq. 5 has no term for the exit probes, which
-    cost a read of the LM head each on this GPU).  One JSON line with all points."""
+    """Hyper-parameter study in the spirit of the paper's ablations (Section 4.4: confidence threshold gamma, annealing
+    strength alpha, depth bound d_max, width bound w_max; without ACT / without d_max / without w_max), on the
+    synthetic workload given by --workload at its own prompt and generation lengths (--sweep-short: at most 256 + 256
+    tokens).  Every point reports decode tokens/s of SpecBound, the speed-up over autoregressive decoding with the same
+    kernels, tokens emitted per round, whether the tokens equal the autoregressive ones, and what Eq. 5 predicts from
+    the measured per-draft acceptance rate.  Also: the decoding strategies of Section 4.3 / Table 2, a probe-layer
+    mask study (layers whose exit test rarely passes are not tested), and a least-squares fit of the round-cost model
+    T = t_layer * layer_steps + t_probe * probes + t_round * rounds to all measured points (Eq. 3 is this with
+    t_probe = t_round = 0 and every draft charged d_max layers).  One JSON line."""
     from paper_2604_12247_b200 import binding, build
     build.build()
     torch.cuda.set_device(0)
     s = run.shape
+    L = s.n_layers
     w = inputs.make_weights(s, run.seed, device="cuda", damp_rho=run.damp_rho)
-    n_prompt, n_gen = min(run.n_prompt, 256), min(run.n_gen, 256)
+    short = getattr(args, "sweep_short", False)
+    n_prompt, n_gen = (min(run.n_prompt, 256), min(run.n_gen, 256)) if short else (run.n_prompt, run.n_gen)
     pr = inputs.make_prompt(s, n_prompt, run.seed).numpy()
-    ctx = binding.Context(s, w, n_prompt + n_gen + 16, kv_page=16)
+    ctx = binding.Context(s, w, n_prompt + n_gen + 16, kv_page=64 if n_prompt + n_gen > 1024 else 16)
     ar = None
     for _ in range(2):
         ar = ctx.generate_ar(pr, n_gen)
     ar_tps = (n_gen - 1) / (ar["stats"].us_decode_dev * 1e-6)
-    alpha = (run.tau[0] - 1.0) / (1.0 - 1.0 / s.n_layers) if run.tau[0] > 1.0 else 0.0   # Eq. 1 strength of the workload's schedule
-    points = []
-    depths = [d for d in (1, 2, 4, 6, 8, 10, 12) if d < s.n_layers]
-    grid = [(d, wm, th) for d in depths for wm in (2, 4, 8) for th in (run.threshold,)]
-    grid += [(run.d_max, run.w_max, th) for th in (0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9) if th != run.threshold]
-    for d_max, w_max, thr in grid:
-        tau = [1.0 + alpha * (1.0 - l / s.n_layers) for l in range(1, d_max + 1)] if alpha > 0 else list(inputs.tau_linear(d_max, 2.0, 1.0))
+    alpha0 = (run.tau[0] - 1.0) / (1.0 - 1.0 / L) if run.tau[0] > 1.0 else 0.0   # Eq. 1 strength of the workload's schedule
+    eq1 = abs(run.tau[-1] - (1.0 + alpha0 * (1.0 - run.d_max / L))) < 1e-6        # the workload's schedule is Eq. 1
+
+    def tau_for(d_max, alpha=None):
+        if alpha is not None:
+            return [1.0 + alpha * (1.0 - l / L) for l in range(1, d_max + 1)]
+        if eq1:
+            return [1.0 + alpha0 * (1.0 - l / L) for l in range(1, d_max + 1)]
+        return list(inputs.tau_linear(d_max, run.tau[0], run.tau[-1]))
+
+    def measure(label, d_max, w_max, thr, tau, **extra):
         ctx.generate(pr, n_gen, d_max, w_max, tau, thr)   # warm-up (descriptor cache)
         sp = ctx.generate(pr, n_gen, d_max, w_max, tau, thr)
         st = sp["stats"]
-        equal = bool((sp["tokens"] == ar["tokens"]).all())
         tps = (n_gen - 1) / (st.us_decode_dev * 1e-6)
         drafts = sum(st.exit_hist[1:])                      # rows that produced a draft
         acc = st.accepted_drafts / drafts if drafts else 0.0
-        points.append({"d_max": d_max, "w_max": w_max, "threshold": thr, "tokens_per_s": tps, "speedup_vs_ar": tps / ar_tps,
-                       "tokens_equal_ar": equal, "rounds": st.rounds, "emitted_per_round": st.emitted / max(st.rounds, 1),
-                       "mean_width": st.rows / max(st.rounds, 1), "draft_acceptance": acc,
-                       "eq5_speedup_at_that_acceptance": binding.model_speedup(s.n_layers, min(acc, 0.999), w_max, d_max),
-                       "probes": st.probes})
+        pt = {"point": label, "d_max": d_max, "w_max": w_max, "threshold": thr, "tokens_per_s": tps, "speedup_vs_ar": tps / ar_tps,
+              "tokens_equal_ar": bool((sp["tokens"] == ar["tokens"]).all()), "rounds": st.rounds,
+              "emitted_per_round": st.emitted / max(st.rounds, 1), "mean_width": st.rows / max(st.rounds, 1),
+              "draft_acceptance": acc,
+              "eq5_speedup_at_that_acceptance": binding.model_speedup(L, min(acc, 0.999), w_max, d_max),
+              "probes": st.probes, "layer_steps": st.layer_steps, "decode_us": st.us_decode_dev,
+              "exit_hist": list(st.exit_hist[:d_max + 1])}
+        pt.update(extra)
+        return pt
+
+    depths = [int(x) for x in args.depths.split(",")] if getattr(args, "depths", None) else \
+        [d for d in (1, 2, 4, 6, 8, 10, 12) if d < L]
+    widths = [int(x) for x in args.widths.split(",")] if getattr(args, "widths", None) else [2, 4, 8]
+    points = [measure("bounds", d, wm, run.threshold, tau_for(d)) for d in depths for wm in widths]
+    points += [measure("threshold", run.d_max, run.w_max, th, tau_for(run.d_max))
+               for th in (0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9) if th != run.threshold]
+    # annealing strength of Eq. 1 (alpha = 0 is decoding without ACT: every layer tested at temperature 1)
+    alphas = [measure("alpha", run.d_max, run.w_max, run.threshold, tau_for(run.d_max, a), alpha=a)
+              for a in (0.0, 0.1, 0.2, 0.4, 0.8, 1.6)]
+    # component ablation (Section 4.4): the full method, then one component off at a time
+    base = measure("full", run.d_max, run.w_max, run.threshold, list(run.tau[:run.d_max]))
+    ablation = [base,
+                measure("without ACT (tau = 1 at every layer)", run.d_max, run.w_max, run.threshold, [1.0] * run.d_max),
+                measure("without d_max (drafting may go to layer L-1)", L - 1, run.w_max, run.threshold, tau_for(L - 1)),
+                measure("without w_max (the library's row limit, 8)", run.d_max, 8, run.threshold, list(run.tau[:run.d_max]))]
+    # probe-layer mask from the exit histogram of the full method: layers that catch fewer than 2 % of the drafted rows
+    # are walked but not tested; also: test every second layer only
+    hist = base["exit_hist"]
+    rows = max(sum(hist), 1)
+    keep = [hist[l] / rows >= 0.02 for l in range(1, run.d_max + 1)]
+    masks = [("full schedule", [True] * run.d_max), ("layers catching >= 2 % of the rows", keep),
+             ("every second layer", [l % 2 == 0 for l in range(1, run.d_max + 1)]),
+             ("last layer only", [l == run.d_max for l in range(1, run.d_max + 1)])]
+    mask_points = []
+    for label, m in masks:
+        if not any(m):
+            continue
+        tau = [t if on else 0.0 for t, on in zip(run.tau[:run.d_max], m)]
+        mask_points.append(measure(label, run.d_max, run.w_max, run.threshold, tau, probed_layers=[l + 1 for l, on in enumerate(m) if on]))
+    # least-squares fit of the round-cost model to every measured point
+    allp = points + alphas + ablation + mask_points
+    A = np.array([[p["layer_steps"], p["probes"], p["rounds"]] for p in allp], dtype=np.float64)
+    y = np.array([p["decode_us"] for p in allp])
+    coef, *_ = np.linalg.lstsq(A, y, rcond=None)
+    pred = A @ coef
+    wb = inputs.weight_bytes(s)
+    fit = {"model": "decode_us = t_layer * layer_steps + t_probe * probes + t_round * rounds (a layer step carries 1..w rows; "
+                    "t_round = final head on w rows + acceptance + the host's look at the result)",
+           "t_layer_us": float(coef[0]), "t_probe_us": float(coef[1]), "t_round_us": float(coef[2]),
+           "probe_over_layer_fitted": float(coef[1] / coef[0]) if coef[0] else None,
+           "probe_over_layer_bytes": wb["head"] / wb["layer"],
+           "max_rel_residual": float(np.max(np.abs(pred - y) / y)), "points": len(allp),
+           "ar_token_us_measured": 1e6 / ar_tps, "ar_token_us_from_fit": float(coef[0] * L + coef[2])}
     # decoding strategies (Section 4.3, Table 2): greedy, temperature and top-p sampling at the workload's own setting;
     # under sampling the baseline is autoregressive sampling with the same temperature and seed
     strategies = []
     tau = list(run.tau[:run.d_max])
     for name, temp, top_p in (("greedy", 0.0, 1.0), ("temperature 0.3", 0.3, 1.0), ("temperature 1.0", 1.0, 1.0),
                               ("top-p 0.9", 1.0, 0.9)):
+        if getattr(args, "no_strategies", False):
+            break
         ctx.set_sampling(temp, run.seed, top_p)
         for _ in range(2):
             a = ctx.generate_ar(pr, n_gen)
@@ -348,10 +520,16 @@ def sweep_arm(args, run: inputs.Run):
                            "emitted_per_round": st.emitted / max(st.rounds, 1),
                            "draft_acceptance": st.accepted_drafts / drafts if drafts else 0.0})
     ctx.set_sampling(0.0, 0)
+    out = {"mode": "sweep", "workload": workload_config(run, "single GPU")["workload"], "prompt_tokens": n_prompt,
+           "generated_tokens": n_gen, "ar_tokens_per_s": ar_tps, "points": points, "alpha_sweep": alphas,
+           "ablation": ablation, "probe_mask": mask_points, "cost_model_fit": fit, "decoding_strategies": strategies}
+    if getattr(args, "oracle_check_tokens", 0) > 0 and not getattr(args, "no_cpu_baseline", True):
+        from oracle import oracle
+        oracle.build()
+        wc = inputs.weights_to(w, "cpu")
+        out["oracle_check"] = oracle_check(ctx, run, wc, 16, args.oracle_check_tokens)
     ctx.close()
-    print(json.dumps({"mode": "sweep", "workload": workload_config(run, "single GPU")["workload"], "prompt_tokens": n_prompt,
-                      "generated_tokens": n_gen, "ar_tokens_per_s": ar_tps, "points": points,
-                      "decoding_strategies": strategies}), flush=True)
+    print(json.dumps(out), flush=True)
 
 
 def micro_arm(args):
@@ -372,6 +550,8 @@ def micro_arm(args):
 
     n_copies = 4
     layers = None
+    chain_layers = None
+    n_chain = 32     # distinct layer weight sets run back to back in the chained mode: 13 GB, the L2 defeat of a real pass
     for S in (512, 2048, 8192):
         for w in (1, 2, 4, 6, 8):
             name = f"layer:w={w}:S={S}"
@@ -403,8 +583,37 @@ def micro_arm(args):
                 times.append(e0.elapsed_time(e1) * 1e3)
             us = statistics.median(times)
             nbytes = inputs.weight_bytes(s)["layer"] + (S + 2 * w) * kv_bytes_per_pos(s)
-            out["layer"].append({"w": w, "S": S, "us": us, "us_min": min(times), "bytes": nbytes, "gbs": nbytes / us / 1e3,
-                                 "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS})
+            row = {"w": w, "S": S, "us": us, "us_min": min(times), "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                   "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS}
+            if not args.no_chained:
+                # steady state: n_chain distinct layers (own weights, own K/V cache) back to back in ONE launch sequence
+                # inside one event bracket, with the rotation-angle table a context would have: every kernel overlaps
+                # its predecessor's tail and requests its first weight tiles early, as inside sb_generate
+                if chain_layers is None:
+                    chain_layers = [inputs.make_weights(s, 200 + i, device="cuda")["layers"][0] for i in range(n_chain)]
+                kcs = [kc] + [torch.randn((n_pages, 64, kvd), device="cuda").to(torch.bfloat16) for _ in range(n_chain - 1)]
+                vcs = [vc] + [torch.randn((n_pages, 64, kvd), device="cuda").to(torch.bfloat16) for _ in range(n_chain - 1)]
+                chain = binding.LayerChain(chain_layers, kcs, vcs)
+                tab = binding.k_rope_table(cfg)
+                for _ in range(2):
+                    h.copy_(h0)
+                    binding.k_layer_chain(cfg, chain, h, pt, S, sc, tab)
+                torch.cuda.synchronize()
+                ctimes = []
+                for i in range(max(args.iters // 4, 5)):
+                    h.copy_(h0)
+                    e0, e1 = ev(), ev()
+                    e0.record()
+                    binding.k_layer_chain(cfg, chain, h, pt, S, sc, tab)
+                    e1.record()
+                    e1.synchronize()
+                    ctimes.append(e0.elapsed_time(e1) * 1e3 / n_chain)
+                cus = statistics.median(ctimes)
+                row.update({"chained_us": cus, "chained_us_min": min(ctimes), "chained_gbs": nbytes / cus / 1e3,
+                            "chained_frac": nbytes / cus / 1e3 / peak, "chained_layers": n_chain})
+                del kcs, vcs, chain
+            out["layer"].append(row)
+    del chain_layers
     del layers
     for V in (32000, 128256):
         for m in (1, 4, 8):
@@ -431,9 +640,24 @@ def micro_arm(args):
                 times.append(e0.elapsed_time(e1) * 1e3)
             us = statistics.median(times)
             nbytes = V * sh.d_model * 2
-            out["exit"].append({"m": m, "V": V, "us": us, "us_min": min(times), "bytes": nbytes, "gbs": nbytes / us / 1e3,
-                                "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
-                                "note": "includes the RMSNorm launch and two small device copies of the stateless entry point"})
+            row = {"m": m, "V": V, "us": us, "us_min": min(times), "bytes": nbytes, "gbs": nbytes / us / 1e3,
+                   "frac": nbytes / us / 1e3 / peak, "frac_of_nominal_8TBs": nbytes / us / 1e3 / NOMINAL_HBM_GBS,
+                   "note": "the whole stateless call: the RMSNorm launch and the exit kernel, starting cold"}
+            if not args.no_chained:
+                # steady state: 8 calls over rotating heads inside one event bracket (each kernel overlaps its predecessor)
+                ctimes = []
+                for i in range(max(args.iters // 4, 5)):
+                    e0, e1 = ev(), ev()
+                    e0.record()
+                    for k in range(8):
+                        binding.k_exit_confidence(cfg, h, gain, heads[(i + k) % copies], 1.0 + 0.2 * (k % 6), sc)
+                    e1.record()
+                    e1.synchronize()
+                    ctimes.append(e0.elapsed_time(e1) * 1e3 / 8)
+                cus = statistics.median(ctimes)
+                row.update({"chained_us": cus, "chained_us_min": min(ctimes), "chained_gbs": nbytes / cus / 1e3,
+                            "chained_frac": nbytes / cus / 1e3 / peak, "chained_calls": 8})
+            out["exit"].append(row)
             del heads
     # sampling kernel (decoding strategies of Section 4.3): latency of one launch on m rows of L2-resident logits;
     # not a bandwidth-bound kernel (one CTA per row, fp64 exponentials), reported in microseconds only
@@ -469,11 +693,19 @@ def main():
     ap.add_argument("--workload", default="7b", choices=sorted(inputs.RUNS))
     ap.add_argument("--n-gen", type=int, default=None, help="override the number of generated tokens")
     ap.add_argument("--n-prompt", type=int, default=None, help="override the prompt length (profiling small cases)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the legs that run the CPU oracle (cpu_baseline, oracle_check)")
+    ap.add_argument("--no-damped", action="store_true", help="skip the extra 7b-damped measurement of the default run")
+    ap.add_argument("--oracle-check-tokens", type=int, default=96,
+                    help="tokens of the short-prompt generation the oracle checks teacher-forced (0 = skip)")
     ap.add_argument("--micro", action="store_true", help="kernel micro-benchmarks instead of the generation benchmark")
-    ap.add_argument("--sweep", action="store_true", help="d_max x w_max and threshold sweep on --workload (one JSON line)")
+    ap.add_argument("--sweep", action="store_true", help="hyper-parameter study on --workload (one JSON line)")
+    ap.add_argument("--sweep-short", action="store_true", help="--sweep at no more than 256 + 256 tokens")
+    ap.add_argument("--depths", default=None, help="--sweep: comma list of d_max values (default 1,2,4,6,8,10,12 below the layer count)")
+    ap.add_argument("--widths", default=None, help="--sweep: comma list of w_max values (default 2,4,8)")
+    ap.add_argument("--no-strategies", action="store_true", help="--sweep: skip the sampling-strategy rows")
     ap.add_argument("--micro-case", default="", help="comma list, e.g. layer:w=4:S=512,exit:m=1:V=32000 (default: all)")
     ap.add_argument("--iters", type=int, default=40)
+    ap.add_argument("--no-chained", action="store_true", help="--micro: isolated calls only (skip the chained steady-state mode)")
     ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
                     help="library option set before the run (sb_set_default_option), e.g. 6=10; for tuning sweeps")
     args = ap.parse_args()

@@ -15,7 +15,9 @@
  *     mailbox (a few KB) that sb_destroy releases.
  *   - Matrices are row-major [out_features, in_features] in the config's storage dtype, no biases,
  *     LM head untied from the embedding.  Layers are numbered 1..n_layers as in the paper.
- *   - One context = one sequence on one GPU.  A context is not thread-safe.
+ *   - One context = one sequence on one GPU.  A context is not thread-safe.  The stateless entry points
+ *     (sb_k_*) may be called from several host threads and on several devices of one process: they
+ *     serialise their host-side launch sequence internally and keep their caches per device.
  *   - Functions that return host scalars synchronise the context's stream themselves.
  *   - Device-side waits are bounded; if one expires the call returns SB_ERR_DEVICE_TIMEOUT and the
  *     CUDA context stays usable.
@@ -146,7 +148,9 @@ int sb_draft_advance(sb_ctx* ctx, int32_t to_layer);
 
 /* (a) Exit decision of Section 3.2 (Eq. 1-2) for the newest row, whose depth must equal `layer`:
  * final RMSNorm -> shared LM head -> logits / tau_l -> conf = max softmax, token = argmax,
- * exit_flag = (conf >= threshold).  One fused kernel; logits never reach HBM.  Outputs are host. */
+ * exit_flag = (conf >= threshold).  One fused kernel; logits never reach HBM.  Outputs are host.
+ * tau_l must be > 0 (a layer masked out of sb_generate's schedule with tau <= 0 cannot be probed:
+ * SB_ERR_ARG). */
 int sb_exit_confidence(sb_ctx* ctx, int32_t layer, float tau_l, float threshold, float* conf, int32_t* token,
                        int32_t* exit_flag);
 
@@ -159,9 +163,15 @@ int sb_verify(sb_ctx* ctx, const int32_t* drafts, int32_t w, int32_t* out_tokens
 
 /* Whole generation: prefill, then rounds of draft + verify until n_gen tokens are out.
  * tau (host) [d_max]: tau[l-1] = temperature T_l of layer l.  threshold: exit when conf >= it
- * (<= 0: always exit at layer 1; > 1: never exit).  rounds (host, nullable) [max_rounds] receives
- * the per-round trace; n_rounds (nullable) their number.  stats nullable.
- * Errors: SB_ERR_ARG (d_max not in [1, n_layers-1], w_max not in [1, SB_MAX_W], tau <= 0, NaN
+ * (<= 0: always exit at the first probed layer; > 1: never exit).
+ * Probe-layer mask: Section 3.2 tests "the first layer where p >= threshold" after every layer; on
+ * this GPU a test costs a full read of the LM head (0.65 of a 7B layer's bytes), so a caller may
+ * switch the test off where it rarely passes: tau[l-1] <= 0 means layer l is walked but not probed
+ * (no exit can happen there; a row that reaches d_max without exiting is the difficult token as
+ * usual).  The output tokens do not depend on the mask.
+ * rounds (host, nullable) [max_rounds] receives the per-round trace; n_rounds (nullable) their
+ * number.  stats nullable.
+ * Errors: SB_ERR_ARG (d_max not in [1, n_layers-1], w_max not in [1, SB_MAX_W], NaN tau or
  * threshold, token id outside the vocabulary), SB_ERR_CAPACITY (n_prompt + n_gen + w_max > max_seq). */
 int sb_generate(sb_ctx* ctx, const int32_t* prompt, int32_t n_prompt, int32_t n_gen, int32_t d_max, int32_t w_max,
                 const float* tau, float threshold, int32_t* out_tokens, int32_t* n_out, sb_stats* stats,
@@ -248,6 +258,18 @@ int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, 
  * positions 0 .. own position. */
 int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_t m, void* k_cache, void* v_cache,
                const int32_t* page_table, int32_t first_pos, void* scratch, size_t scratch_bytes, void* cuda_stream);
+
+/* The same for n_layers consecutive layers in one launch sequence (the steady state of the verify
+ * pass, Section 3.3: the weights of the layers D+1..L streamed back to back): layer i uses lw[i],
+ * k_caches[i], v_caches[i] (HOST arrays [n_layers]; the caches are device memory laid out as for
+ * sb_k_layer and share page_table).  rope_table: nullable device table of the rotation angles made
+ * by sb_k_rope_table for this config (without it every launch computes its angles).  One status
+ * clear at the start, then every kernel overlaps its predecessor's tail as inside sb_generate. */
+size_t sb_k_rope_table_bytes(const sb_config* cfg);
+int sb_k_rope_table(const sb_config* cfg, void* table, size_t table_bytes, void* cuda_stream);
+int sb_k_layer_chain(const sb_config* cfg, const sb_layer_weights* lw, int32_t n_layers, void* h, int32_t m,
+                     void* const* k_caches, void* const* v_caches, const int32_t* page_table, int32_t first_pos,
+                     const void* rope_table, void* scratch, size_t scratch_bytes, void* cuda_stream);
 
 /* ---- helpers ---------------------------------------------------------------------------------- */
 

@@ -67,7 +67,7 @@ EXPORTS = ("sb_workspace_bytes", "sb_create", "sb_destroy", "sb_load_weights", "
            "sb_selftest_wait_timeout",
            "sb_read_hidden", "sb_prefill", "sb_draft_push", "sb_draft_advance", "sb_exit_confidence", "sb_verify",
            "sb_generate", "sb_generate_ar", "sb_set_sampling", "sb_sample_uniform", "sb_k_sample", "sb_k_sample_scratch_bytes", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
-           "sb_k_layer",
+           "sb_k_layer", "sb_k_layer_chain", "sb_k_rope_table", "sb_k_rope_table_bytes",
            "sb_tau_schedule", "sb_model_speedup", "sb_set_option", "sb_set_default_option", "sb_strerror")
 
 _lib = None
@@ -110,6 +110,11 @@ def lib():
         L.sb_k_exit_confidence.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp, vp, C.c_size_t, vp]
         L.sb_k_exit_confidence_static.argtypes = [C.POINTER(Config), vp, i32, vp, vp, f32, vp, vp, vp]
         L.sb_k_layer.argtypes = [C.POINTER(Config), C.POINTER(LayerWeights), vp, i32, vp, vp, vp, i32, vp, C.c_size_t, vp]
+        L.sb_k_rope_table_bytes.restype = C.c_size_t
+        L.sb_k_rope_table_bytes.argtypes = [C.POINTER(Config)]
+        L.sb_k_rope_table.argtypes = [C.POINTER(Config), vp, C.c_size_t, vp]
+        L.sb_k_layer_chain.argtypes = [C.POINTER(Config), C.POINTER(LayerWeights), i32, vp, i32, C.POINTER(vp), C.POINTER(vp), vp,
+                                       i32, vp, vp, C.c_size_t, vp]
         L.sb_tau_schedule.argtypes = [f32, i32, vp]
         L.sb_model_speedup.restype = C.c_double
         L.sb_model_speedup.argtypes = [i32, C.c_double, i32, i32]
@@ -338,3 +343,33 @@ def k_layer(cfg: Config, lw: dict, h: torch.Tensor, k_cache: torch.Tensor, v_cac
     _check(lib().sb_k_layer(C.byref(cfg), C.byref(L), h.data_ptr(), h.shape[0], k_cache.data_ptr(), v_cache.data_ptr(),
                             page_table.data_ptr(), first_pos, C.c_void_p(scratch.ptr), scratch.nbytes,
                             _stream_handle(stream)), "sb_k_layer")
+
+
+def k_rope_table(cfg: Config, stream=None) -> torch.Tensor:
+    """sb_k_rope_table: the cos/sin table of the rotation angles for this config, as a device tensor."""
+    nbytes = lib().sb_k_rope_table_bytes(C.byref(cfg))
+    tab = torch.empty(nbytes // 4, dtype=torch.float32, device="cuda")
+    _check(lib().sb_k_rope_table(C.byref(cfg), tab.data_ptr(), nbytes, _stream_handle(stream)), "sb_k_rope_table")
+    return tab
+
+
+class LayerChain:
+    """Marshalled arguments of sb_k_layer_chain: n layers' weights and caches (kept alive here)."""
+
+    def __init__(self, lws: Sequence[dict], k_caches: Sequence[torch.Tensor], v_caches: Sequence[torch.Tensor]):
+        n = len(lws)
+        assert n == len(k_caches) == len(v_caches)
+        self.n = n
+        self._keep = (lws, k_caches, v_caches)
+        self.lw = (LayerWeights * n)(*[l if isinstance(l, LayerWeights) else layer_weights(l) for l in lws])
+        self.kc = (C.c_void_p * n)(*[t.data_ptr() for t in k_caches])
+        self.vc = (C.c_void_p * n)(*[t.data_ptr() for t in v_caches])
+
+
+def k_layer_chain(cfg: Config, chain: LayerChain, h: torch.Tensor, page_table: torch.Tensor, first_pos: int,
+                  scratch: KernelScratch, rope_table: Optional[torch.Tensor] = None, stream=None):
+    """n consecutive decoder layers in place on h (CUDA fp32 [m, d]), one launch sequence."""
+    assert h.is_cuda and h.dtype == torch.float32 and h.is_contiguous()
+    _check(lib().sb_k_layer_chain(C.byref(cfg), chain.lw, chain.n, h.data_ptr(), h.shape[0], chain.kc, chain.vc,
+                                  page_table.data_ptr(), first_pos, rope_table.data_ptr() if rope_table is not None else None,
+                                  C.c_void_p(scratch.ptr), scratch.nbytes, _stream_handle(stream)), "sb_k_layer_chain")

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "gemm_tc.cuh"
@@ -21,10 +22,15 @@ static int g_trace = 0;           // 1: the stateless layer call times every lau
 
 // TMA descriptors of the stateless entry points: keyed by (pointers, shapes), so they stay valid for as
 // long as the key matches; kept across calls because encoding them costs more host time than the launch.
+// One cache per device (a descriptor holds a device address and the plan the device's SM count); the stateless
+// entry points hold g_stateless_mu while they use it, so they may be called from several host threads.
+static std::mutex g_stateless_mu;
 static TcPlanCache& stateless_plans() {
-    static TcPlanCache cache;
-    if (cache.plans.size() > 512) cache.clear();
-    return cache;
+    static TcPlanCache cache[kMaxDevices];
+    int dev = current_device();
+    TcPlanCache& c = cache[dev < 0 ? 0 : dev];
+    if (c.plans.size() > 512) c.clear();
+    return c;
 }
 
 struct Tracer {
@@ -519,7 +525,7 @@ static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats*
 // ---------------------------------------------------------------------------------------------
 constexpr size_t kStaticScratchBytes = size_t(1) << 20;   // 1 MiB
 constexpr int kStaticMaxDModel = 8192;                    // widest model whose rows fit it
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes + 256];   // + the sampling kernel's counter word
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // what the exit-confidence call keeps in scratch: hidden rows, the normalised operand, the per-CTA
 // softmax triples, the ticket, the result block and the status word
@@ -541,10 +547,9 @@ static size_t carve_exit_only(const Dims& D, char* base, Work* w) {
 // only a host-side handle, never a device address: the address comes from cudaGetSymbolAddress,
 // asked once per device with that device current.
 static int static_scratch_ptr(char** out) {
-    constexpr int kMaxDev = 64;
-    static char* ptrs[kMaxDev] = {nullptr};
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return SB_ERR_CUDA;
+    static char* ptrs[kMaxDevices] = {nullptr};
+    const int dev = current_device();
+    if (dev < 0) return SB_ERR_CUDA;
     if (!ptrs[dev]) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
@@ -920,7 +925,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
     if (!c->loaded) return SB_ERR_STATE;
     if (d_max < 1 || d_max > c->e.D.L - 1 || w_max < 1 || w_max > SB_MAX_W || threshold != threshold) return SB_ERR_ARG;
     for (int l = 0; l < d_max; ++l)
-        if (!(tau[l] > 0.f)) return SB_ERR_ARG;
+        if (tau[l] != tau[l]) return SB_ERR_ARG;   // NaN; tau[l] <= 0 = layer l + 1 is not probed
     if (n_prompt + n_gen + w_max > c->e.D.max_seq) return SB_ERR_CAPACITY;
     if (check_tokens(c, prompt, n_prompt)) return SB_ERR_ARG;
     sb_stats local;
@@ -953,7 +958,11 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
             int r = c->rows - 1;
             bool exited = false;
             for (int l = 1; l <= d_max; ++l) {
-                advance_suffix(c, l, c->norm_of(l), st);
+                // a layer whose temperature is <= 0 is walked but not probed: its step hands the rows straight to the
+                // next layer's attention norm
+                const bool probed = tau[l - 1] > 0.f;
+                advance_suffix(c, l, probed ? c->norm_of(l) : c->layers[l].attn_norm, st);
+                if (!probed) continue;
                 float conf; int tok, flag;
                 if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag, st, l < d_max))) return rc;
                 st->probes++;
@@ -1055,6 +1064,7 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     if (m < 1 || m > SB_MAX_W || !(tau_l > 0.f)) return SB_ERR_ARG;
     if (((uintptr_t)scratch & 1023) || ((uintptr_t)lm_head & 15) || ((uintptr_t)h & 15)) return SB_ERR_ARG;
     if (scratch_bytes < carve(D, nullptr, false, nullptr)) return SB_ERR_CAPACITY;
+    std::lock_guard<std::mutex> lock(g_stateless_mu);
     Exec e;
     e.D = D;
     e.st = (cudaStream_t)stream;
@@ -1071,8 +1081,8 @@ int sb_k_exit_confidence(const sb_config* cfg, const void* h, int32_t m, const v
     return cuda_ok(cudaGetLastError());
 }
 
-// Sampling kernel alone: tokens of m rows of device logits.  Its completion counter is the word behind the static
-// scratch (zero at load, left at zero by every launch).
+// Sampling kernel alone: tokens of m rows of device logits.  Nothing is published to the host, so the kernel's
+// completion counter is not used: the call touches the caller's buffers only.
 size_t sb_k_sample_scratch_bytes(int32_t m, int32_t vocab) {
     return m < 1 || vocab < 1 ? 0 : 2 * sizeof(double) * (size_t)m * (size_t)vocab;   // exponentials as fp64 and as fixed point
 }
@@ -1083,11 +1093,8 @@ int sb_k_sample(const float* logits, int32_t m, int32_t vocab, float temperature
     if (((uintptr_t)scratch & 7) || scratch_bytes < sb_k_sample_scratch_bytes(m, vocab)) return SB_ERR_ARG;
     if (!(top_p > 0.f) || top_p > 1.f) return SB_ERR_ARG;
     if (vocab > kSampleMaxVocab) return SB_ERR_CAPACITY;
-    char* base = nullptr;
-    int rc = static_scratch_ptr(&base);
-    if (rc) return rc;
     SampleArgs a{logits, static_cast<double*>(scratch), static_cast<unsigned long long*>(scratch) + (size_t)m * vocab, vocab, 0, m, (double)temperature, (double)top_p, seed, pos0, token,
-                 reinterpret_cast<unsigned int*>(base + kStaticScratchBytes), Mirror{nullptr, nullptr, 0u}};
+                 nullptr, Mirror{nullptr, nullptr, 0u}};
     if (!launch_sample((cudaStream_t)stream, a)) { (void)cudaGetLastError(); return SB_ERR_CUDA; }
     return cuda_ok(cudaGetLastError());
 }
@@ -1103,6 +1110,7 @@ int sb_k_exit_confidence_static(const sb_config* cfg, const void* h, int32_t m, 
     char* base = nullptr;
     int rc = static_scratch_ptr(&base);   // first call on a device looks the address up
     if (rc) return rc;
+    std::lock_guard<std::mutex> lock(g_stateless_mu);
     Exec e;
     e.D = D;
     e.st = (cudaStream_t)stream;
@@ -1131,6 +1139,7 @@ int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_
     const void* ps[9] = {lw->attn_norm, lw->wq, lw->wk, lw->wv, lw->wo, lw->mlp_norm, lw->w_gate, lw->w_up, lw->w_down};
     for (const void* p : ps)
         if (!p || ((uintptr_t)p & 15)) return SB_ERR_ARG;
+    std::lock_guard<std::mutex> lock(g_stateless_mu);
     Exec e;
     e.D = D;
     e.st = (cudaStream_t)stream;
@@ -1143,6 +1152,52 @@ int sb_k_layer(const sb_config* cfg, const sb_layer_weights* lw, void* h, int32_
     if (g_trace) g_tracer.begin(e.st);
     layer_step(e, *lw, k_cache, v_cache, 0, m, first_pos, nullptr);
     g_tracer.end();
+    if (e.err) return e.err;
+    return cuda_ok(cudaGetLastError());
+}
+
+size_t sb_k_rope_table_bytes(const sb_config* cfg) {
+    Dims D;
+    if (!make_dims(cfg, &D)) return 0;
+    return sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2);
+}
+
+int sb_k_rope_table(const sb_config* cfg, void* table, size_t table_bytes, void* stream) {
+    Dims D;
+    if (!make_dims(cfg, &D) || !table || ((uintptr_t)table & 15)) return SB_ERR_ARG;
+    if (table_bytes < sizeof(float2) * (size_t)D.n_pages * D.page * (D.hd / 2)) return SB_ERR_CAPACITY;
+    launch_rope_table((cudaStream_t)stream, static_cast<float2*>(table), D.n_pages * D.page, D.hd / 2, D.inv_freq);
+    return cuda_ok(cudaGetLastError());
+}
+
+int sb_k_layer_chain(const sb_config* cfg, const sb_layer_weights* lw, int32_t n_layers, void* h, int32_t m,
+                     void* const* k_caches, void* const* v_caches, const int32_t* page_table, int32_t first_pos,
+                     const void* rope_table, void* scratch, size_t scratch_bytes, void* stream) {
+    Dims D;
+    if (!make_dims(cfg, &D) || !lw || !h || !k_caches || !v_caches || !page_table || !scratch) return SB_ERR_ARG;
+    if (n_layers < 1 || n_layers > SB_MAX_LAYERS || m < 1 || m > SB_MAX_W || first_pos < 0) return SB_ERR_ARG;
+    if (first_pos + m > D.max_seq) return SB_ERR_CAPACITY;
+    if (((uintptr_t)scratch & 1023) || ((uintptr_t)rope_table & 15)) return SB_ERR_ARG;
+    if (scratch_bytes < carve(D, nullptr, false, nullptr)) return SB_ERR_CAPACITY;
+    for (int l = 0; l < n_layers; ++l) {
+        const void* ps[11] = {lw[l].attn_norm, lw[l].wq, lw[l].wk, lw[l].wv, lw[l].wo, lw[l].mlp_norm, lw[l].w_gate,
+                              lw[l].w_up, lw[l].w_down, k_caches[l], v_caches[l]};
+        for (const void* p : ps)
+            if (!p || ((uintptr_t)p & 15)) return SB_ERR_ARG;
+    }
+    std::lock_guard<std::mutex> lock(g_stateless_mu);
+    Exec e;
+    e.D = D;
+    e.st = (cudaStream_t)stream;
+    carve(D, (char*)scratch, false, &e.W);
+    e.W.page_table = const_cast<int*>(page_table);
+    e.W.h = reinterpret_cast<float*>(h);
+    e.W.rope_tab = const_cast<float2*>(static_cast<const float2*>(rope_table));
+    e.gemm = pick_gemm(D.f32);
+    e.plans = &stateless_plans();
+    cudaMemsetAsync(e.W.status, 0, 64, e.st);
+    for (int l = 0; l < n_layers; ++l)
+        layer_step(e, lw[l], k_caches[l], v_caches[l], 0, m, first_pos, l + 1 < n_layers ? lw[l + 1].attn_norm : nullptr);
     if (e.err) return e.err;
     return cuda_ok(cudaGetLastError());
 }

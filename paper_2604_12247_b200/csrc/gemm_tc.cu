@@ -515,14 +515,12 @@ static bool make_map(CUtensorMap* tm, const void* base, int rows, int K, int box
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
+static int sm_count() {   // of the current device
+    static int n[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return 148;
+    if (!n[dev] && (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0)) n[dev] = 148;
+    return n[dev];
 }
 
 // Slab height R (multiple of 8 in [64,128]) and split count S that minimise what the busiest
@@ -599,11 +597,12 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
 }
 
 template <bool kHead, bool kPair, int NB = 1> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices];   // function attributes are per device
+    const int dev = current_device();
+    if (dev >= 0 && !attr_set[dev]) {
         cudaFuncSetAttribute(k_tc<kHead, kPair, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              NB > 1 ? smem_bytes(kWideStages, NB) : smem_bytes(kMaxStages));
-        attr_set = true;
+        attr_set[dev] = true;
     }
     launch_k(k_tc<kHead, kPair, NB>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages, NB), st, p);
 }

@@ -28,10 +28,7 @@ void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, i
     // launched WITHOUT programmatic dependent launch: it starts only after everything before it in the stream has
     // completed.  The kernels behind it may therefore rely on what earlier steps wrote (the K/V rows of earlier
     // positions) being complete even before their own grid-dependency wait returns.
-    const bool saved = g_use_pdl;
-    g_use_pdl = false;
-    launch_k(k_embed<T>, dim3(m), dim3(256), 0, st, embed, d, toks_dev, tok_scalar, row0, h);
-    g_use_pdl = saved;
+    (void)launch_kcp(k_embed<T>, dim3(m), dim3(256), 0, st, 1, /*pdl=*/false, embed, d, toks_dev, tok_scalar, row0, h);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -605,13 +602,16 @@ static size_t attn_smem(int P, int HD, size_t elt, bool fused) {
 template <typename T, int HD, int PG, bool kFused>
 static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem, int cluster_y) {
     auto kernel = k_attn_partial<T, HD, PG, kFused>;
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices];             // function attributes are per device
+    const int dev = current_device();
+    if (dev < 0) return false;
+    if (!configured[dev]) {
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
-        configured = true;
+        configured[dev] = true;
     }
     if (kFused && cluster_y > 1) {
-        static int fits[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // per cluster size: 0 unknown, 1 yes, -1 no
+        static int fits_dev[kMaxDevices][9];             // per device and cluster size: 0 unknown, 1 yes, -1 no
+        int* fits = fits_dev[dev];
         if (fits[cluster_y] == 0) {
             cudaLaunchConfig_t cfg{};
             cfg.gridDim = grid; cfg.blockDim = dim3(kAttnWarps * 32); cfg.dynamicSmemBytes = 200 * 1024;
@@ -762,6 +762,7 @@ __device__ __forceinline__ unsigned int peer_ld_u32(uint32_t addr) {
 __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
     pdl_trigger();
     pdl_wait();
+    cluster_sync_all();   // distributed shared memory may be touched only once every CTA of the cluster has started
     // mass histogram in three 14-bit parts (a part's bucket sum stays below 2^32 for up to 262144 tokens):
     // mass of bucket b = s_hist[0][b] + (s_hist[1][b] << 14) + (s_hist[2][b] << 28)
     __shared__ unsigned int s_hist[3][kSelectBuckets];
@@ -1022,6 +1023,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(SampleArgs a) {
             __threadfence();
         }
     }
+    if (!a.mirror.host) return;                     // nothing to publish: the completion counter is not touched
     __syncthreads();
     if (tid == 0) {
         __threadfence();

@@ -108,15 +108,23 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 extern bool g_use_pdl;
-// cluster.y > 1 launches thread-block clusters of that many CTAs along y (grid.y must be a multiple of it)
+// Index of the current device for the per-device host-side caches (function attributes, SM count, ...); -1 on error.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+// cluster.y > 1 launches thread-block clusters of that many CTAs along y (grid.y must be a multiple of it);
+// pdl: launch with programmatic stream serialisation (the kernel may start while its predecessor drains)
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kc(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,
-                             Args&&... args) {
+inline cudaError_t launch_kcp(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,
+                              bool pdl, Args&&... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     int n_attr = 0;
-    if (g_use_pdl) {
+    if (pdl) {
         attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
         ++n_attr;
@@ -131,16 +139,24 @@ inline cudaError_t launch_kc(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
     // every kernel asks for the same (maximal) shared-memory carve-out: an SM never has to drain to
-    // change its L1/shared split between two kernels of the chain
-    static void* seen[32];
-    static int n_seen = 0;
-    bool known = false;
-    for (int i = 0; i < n_seen; ++i) known |= seen[i] == (void*)kernel;
-    if (!known) {
-        cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
-        if (n_seen < 32) seen[n_seen++] = (void*)kernel;
+    // change its L1/shared split between two kernels of the chain.  Function attributes are per device.
+    static void* seen[kMaxDevices][32];
+    static int n_seen[kMaxDevices];
+    const int dev = current_device();
+    if (dev >= 0) {
+        bool known = false;
+        for (int i = 0; i < n_seen[dev]; ++i) known |= seen[dev][i] == (void*)kernel;
+        if (!known) {
+            cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+            if (n_seen[dev] < 32) seen[dev][n_seen[dev]++] = (void*)kernel;
+        }
     }
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kc(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,
+                             Args&&... args) {
+    return launch_kcp(kernel, grid, block, smem, st, cluster_y, g_use_pdl, static_cast<Args&&>(args)...);
 }
 template <typename... KArgs, typename... Args>
 inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {

@@ -77,7 +77,7 @@ def scaled(shape: Shape, **kw) -> Shape:
     return Shape(**d)
 
 
-# The workloads named by the build contract, by index.
+# The named workloads (shape + decoding hyper-parameters); labelled additions are marked.
 RUNS: Dict[str, Run] = {
     # tiny decoder, fp32: tau_l = 1 + 0.5 (d_max - l)
     "tiny": Run(TINY, 16, 32, 2, 4, (1.5, 1.0), 0.3, seed=0),

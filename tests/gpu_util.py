@@ -5,7 +5,7 @@ import torch
 from oracle import oracle
 from paper_2604_12247_b200 import binding, inputs
 
-# Tolerances of the build contract: logits within 1e-4 (fp32 models) / 2e-2 (bf16 models) absolute,
+# Tolerances of the parity tests: logits within 1e-4 (fp32 models) / 2e-2 (bf16 models) absolute,
 # exit confidences within 1e-3.  Hidden states are compared relative to their own scale.
 LOGIT_TOL = {"f32": 1e-4, "bf16": 2e-2}
 CONF_TOL = 1e-3

@@ -114,6 +114,66 @@ def test_tiny_hyper_parameter_grid_equals_ar(tiny_damped_weights):
     ctx.close()
 
 
+def test_probe_layer_mask_matches_oracle_trace(tiny_damped_weights):
+    """Probe-layer mask (temperature <= 0: the layer is walked but not tested): tokens stay those of autoregressive
+    decoding for every mask, and rounds, exit layers, drafts, confidences and the probe count follow the oracle run
+    with the same mask."""
+    run = inputs.RUNS["tiny-damped"]
+    pr = inputs.make_prompt(run.shape, run.n_prompt, run.seed).numpy()
+    n_gen, d_max, w_max, thr = 24, 3, 4, 0.3
+    base = (1.6, 1.3, 1.0)
+    ctx, _ = gpu_ctx(run.shape, tiny_damped_weights, 64)
+    ar = ctx.generate_ar(pr, n_gen)["tokens"]
+    assert np.array_equal(ar, oracle.Oracle(run.shape, tiny_damped_weights, 64).ar_generate(pr, n_gen))
+    for mask in ((1, 1, 1), (0, 1, 1), (1, 0, 1), (1, 1, 0), (0, 0, 1), (0, 1, 0), (1, 0, 0), (0, 0, 0)):
+        tau = tuple(t if on else 0.0 for t, on in zip(base, mask))
+        _, orc_rounds = oracle.Oracle(run.shape, tiny_damped_weights, 64).specbound_generate(pr, n_gen, d_max, w_max, tau, thr)
+        sp = ctx.generate(pr, n_gen, d_max, w_max, tau, thr, trace=True)
+        assert np.array_equal(sp["tokens"], ar), mask
+        compare_traces(sp["rounds"], orc_rounds)
+        assert sp["stats"].probes == sum(r.probes for r in orc_rounds)
+        assert sp["stats"].layer_steps == sum(r.layer_steps for r in orc_rounds)
+        assert all(mask[e - 1] for r in sp["rounds"] for e in r.exit_layer[:r.w] if e)
+    ctx.close()
+
+
+GEOM_7B_RUN = inputs.scaled(inputs.LLAMA2_7B, name="7b-attention-geometry-7l", n_layers=7, d_model=512, d_ffn=1024, vocab=2048,
+                            head_scale=16.0)
+
+
+def test_bench_lengths_on_7b_attention_geometry_match_oracle():
+    """The bench workload's lengths and bounds (512-token prompt, 512 generated tokens, d_max 6, w_max 4, its tau
+    schedule and threshold) on a 7-layer model with the 7B attention geometry (32 heads of 128 channels; d_model and
+    FFN cut so that the oracle can follow every position): the context grows from 512 to 1028 positions, through
+    cluster merges of 5 to 8 chunk CTAs and over the hand-over to the separate attention kernels at the 9th chunk, and
+    the prompt goes through the wide prefill passes.  Speculative == autoregressive bit for bit on the GPU; every one of
+    the 512 tokens is the oracle's top-1 or within the logit tolerance of it (teacher-forced), near ties counted."""
+    run = inputs.RUNS["7b"]
+    shape = GEOM_7B_RUN
+    w = inputs.make_weights(shape, 5, damp_rho=0.3)
+    pr = inputs.make_prompt(shape, run.n_prompt, 9).numpy()
+    n_gen = run.n_gen
+    max_seq = run.n_prompt + n_gen + run.w_max + 8
+    ctx, _ = gpu_ctx(shape, w, max_seq, kv_page=64, gemm=1)
+    ar = ctx.generate_ar(pr, n_gen)["tokens"]
+    sp = ctx.generate(pr, n_gen, run.d_max, run.w_max, run.tau, run.threshold, trace=True)
+    assert np.array_equal(sp["tokens"], ar)
+    rounds = sp["rounds"]
+    assert all(1 <= r.w <= run.w_max and r.D <= run.d_max and 1 <= r.emitted <= r.w for r in rounds)
+    st = sp["stats"]
+    assert st.accepted_drafts > 0 and max(r.w for r in rounds) == run.w_max
+    ctx.close()
+    toks = np.concatenate([pr, ar]).astype(np.int32)
+    top1, top2, margin, deficit = oracle.Oracle(shape, w, max_seq).teacher_forced(toks, len(pr))
+    n_off = int((top1 != ar).sum())
+    near = int((margin < 2 * LOGIT_TOL["bf16"]).sum())
+    print(f"\n[7B attention geometry, 512 + 512 tokens] {len(rounds)} rounds, {st.accepted_drafts} drafts accepted; GPU tokens "
+          f"that are not the oracle's top-1: {n_off} of {n_gen}; positions with a top-2 margin below tolerance: {near}; "
+          f"worst deficit {deficit.min():.2e}")
+    assert deficit.min() > -LOGIT_TOL["bf16"]
+    assert all(margin[i] < 2 * LOGIT_TOL["bf16"] for i in range(n_gen) if top1[i] != ar[i])
+
+
 EIGHT = inputs.scaled(inputs.TINY, name="tiny-8l", n_layers=8, d_model=128, n_heads=4, n_kv_heads=4, head_dim=32,
                       d_ffn=256, vocab=200)
 
@@ -219,7 +279,7 @@ def test_state_and_argument_errors(tiny_weights):
         ctx.generate(pr, 8, 2, 9, (1.5, 1.0), 0.3)           # w_max > 8
     assert e.value.status == -1
     with pytest.raises(E) as e:
-        ctx.generate(pr, 8, 2, 4, (1.5, 0.0), 0.3)           # temperature must be positive
+        ctx.generate(pr, 8, 2, 4, (1.5, float("nan")), 0.3)  # a temperature must be a number (<= 0 masks the layer)
     assert e.value.status == -1
     bad = pr.copy(); bad[3] = run.shape.vocab
     with pytest.raises(E) as e:
@@ -232,6 +292,9 @@ def test_state_and_argument_errors(tiny_weights):
     with pytest.raises(E) as e:
         ctx.exit_confidence(2, 1.0, 0.5)                     # newest row is at depth 1, not 2
     assert e.value.status == -2
+    with pytest.raises(E) as e:
+        ctx.exit_confidence(1, 0.0, 0.5)                     # a masked layer (temperature <= 0) cannot be probed
+    assert e.value.status == -1
     with pytest.raises(E) as e:
         ctx.verify([-1, -1])                                 # one row in flight, two given
     assert e.value.status == -2
@@ -253,6 +316,12 @@ def test_7b_shape_run_matches_oracle_on_sampled_positions():
     run = inputs.RUNS["7b"]
     shape = run.shape
     wg = inputs.make_weights(shape, run.seed, device="cuda")
+    # the workload's norm gains are all 1.0, which would hide a dropped or misplaced gain at d = 4096: perturb them here
+    g = torch.Generator(device="cuda").manual_seed(77)
+    perturbed = lambda t: (1.0 + 0.1 * torch.randn(t.shape, generator=g, device="cuda")).to(t.dtype)
+    for lw in wg["layers"]:
+        lw["attn_norm"], lw["mlp_norm"] = perturbed(lw["attn_norm"]), perturbed(lw["mlp_norm"])
+    wg["final_norm"] = perturbed(wg["final_norm"])
     pr = inputs.make_prompt(shape, 24, run.seed).numpy()
     n_gen, max_seq = 12, 64
     ctx = binding.Context(shape, wg, max_seq, kv_page=64)
@@ -327,7 +396,7 @@ def test_7b_damped_run_accepts_drafts_and_equals_ar():
 
 @pytest.mark.parametrize("which", ["l3-8b", "13b"])
 def test_large_config_tokens_match_oracle(which):
-    """Contract configs 3 (Llama-3-8B shape: GQA 32/8 heads, vocabulary 128256) and 4 (13B shape: 40 layers,
+    """Workloads `l3-8b` (Llama-3-8B shape: GQA 32/8 heads, vocabulary 128256) and `13b` (13B shape: 40 layers,
     d = 5120) in the launch configuration bench.py uses, on a sequence short enough for the oracle:
     speculative == autoregressive bit for bit on the GPU, and every token is the oracle's top-1 or within the
     logit tolerance of it (teacher-forced)."""
@@ -369,6 +438,14 @@ def test_bench_sweep_mode_on_tiny(capsys):
     assert {p["d_max"] for p in pts} == {1, 2} and {p["w_max"] for p in pts} == {2, 4, 8}
     assert all(1.0 <= p["emitted_per_round"] <= p["w_max"] and 0.0 <= p["draft_acceptance"] <= 1.0 for p in pts)
     assert max(p["emitted_per_round"] for p in pts) > 1.5
+    # annealing-strength sweep, component ablation, probe-layer masks and the fitted cost model (Section 4.4's axes)
+    assert [p["alpha"] for p in line["alpha_sweep"]] == [0.0, 0.1, 0.2, 0.4, 0.8, 1.6]
+    assert len(line["ablation"]) == 4 and line["ablation"][2]["d_max"] == inputs.RUNS["tiny-damped"].shape.n_layers - 1
+    assert len(line["probe_mask"]) >= 2 and line["probe_mask"][-1]["probes"] < line["probe_mask"][0]["probes"]
+    for group in ("alpha_sweep", "ablation", "probe_mask"):
+        assert all(p["tokens_equal_ar"] for p in line[group]), group
+    fit = line["cost_model_fit"]
+    assert fit["points"] == len(pts) + 6 + 4 + len(line["probe_mask"]) and fit["t_layer_us"] > 0
     strat = line["decoding_strategies"]
     assert [x["strategy"] for x in strat] == ["greedy", "temperature 0.3", "temperature 1.0", "top-p 0.9"]
     assert all(x["tokens_equal_ar"] and x["tokens_per_s"] > 0 and x["ar_tokens_per_s"] > 0 for x in strat)

@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle
 from paper_2604_12247_b200 import binding, inputs
 from gpu_util import CONF_TOL
 
@@ -40,6 +41,37 @@ def test_static_scratch_entry_point_matches_the_ordinary_one(shape):
         assert np.allclose(got_conf.cpu().numpy(), want_conf.cpu().numpy(), atol=CONF_TOL, rtol=0), call
         assert np.array_equal(got_tok.cpu().numpy(), want_tok.cpu().numpy()), call
         assert np.all(got_conf.cpu().numpy() > 0) and np.all(got_conf.cpu().numpy() <= 1 + 1e-6)
+        # and against the CPU oracle's exit test on the same rows (Eq. 2), directly
+        w = inputs.make_weights(inputs.scaled(shape, vocab=8), 0)
+        w["lm_head"], w["final_norm"] = lm.cpu(), gain.cpu()
+        o = oracle.Oracle(shape, w, 4)
+        for i in range(m):
+            p, t = o.exit_confidence(h[i].cpu().numpy(), tau)
+            assert abs(float(got_conf[i]) - p) < CONF_TOL and int(got_tok[i]) == t, (call, i)
+        o.close()
+
+
+def test_static_scratch_call_allocates_no_device_memory():
+    """What the entry point is for: with the outputs preallocated, a call leaves the device's free memory where it
+    was (no cudaMalloc behind the caller's back), also at the widest model the fixed array takes (d_model 8192)."""
+    wide = inputs.scaled(BF16, name="noalloc-wide", d_model=8192, n_heads=64, n_kv_heads=64, head_dim=128, vocab=512)
+    for shape in (BF16, wide):
+        cfg = binding.make_config(shape, 64, 16)
+        lm, gain = _head(shape, 43)
+        h = inputs.make_hidden(8, shape.d_model, 77).cuda()
+        conf = torch.empty(8, dtype=torch.float32, device="cuda")
+        tok = torch.empty(8, dtype=torch.int32, device="cuda")
+        call = lambda: binding._check(binding.lib().sb_k_exit_confidence_static(
+            cfg, h.data_ptr(), 8, gain.data_ptr(), lm.data_ptr(), 1.3, conf.data_ptr(), tok.data_ptr(), None), "static")
+        call()                                   # the first call on a device looks up the array's address
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0, (shape.name, free0, free1)
+        assert np.all(conf.cpu().numpy() > 0) and np.all((tok.cpu().numpy() >= 0) & (tok.cpu().numpy() < shape.vocab))
 
 
 def test_static_scratch_entry_point_refuses_what_does_not_fit():
