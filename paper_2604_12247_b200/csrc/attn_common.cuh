@@ -1,0 +1,94 @@
+// Arithmetic shared by the attention kernels (one-launch cluster kernel, separate chunk kernel, streaming kernel
+// for long contexts, chunk merge).  Every kernel computes a (row, query head) pair's attention the same way:
+//
+//   32-position block : scores by one fmaf chain per position over the channels in order; block maximum and sum of
+//                       exp(score - maximum) by warp butterflies; out = sum_t p_t V_t by one fmaf chain per channel
+//   128-position chunk: its four blocks merged at once: M = max m_j, L = sum_j l_j f_j, O = sum_j o_j f_j with
+//                       f_j = exp(m_j - M), in block order
+//   8-chunk group     : the chunks folded one after the other, in chunk order
+//   whole context     : the groups folded one after the other, in group order;  out = O / L
+//
+// The roundings below are explicit (no contraction left to the compiler) so that the kernels agree bit for bit and a
+// row's result depends on its own position only, never on the rows that ride along or on the launch that computes it.
+#pragma once
+#include "sb_internal.cuh"
+
+namespace sb {
+
+constexpr int kPosWarps = 4;                  // 32-position blocks per chunk
+constexpr int kAttnChunk = 128;               // positions per chunk
+constexpr int kChunkGroup = 8;                // chunks per group of the two-level fold
+constexpr unsigned long long kStageWaitCycles = 2000000000ull;   // bound of the wait for staging copies (~1 s)
+
+template <typename T> __device__ __forceinline__ void unpack16(const uint4& u, float (&f)[16 / sizeof(T)]);
+template <> __device__ __forceinline__ void unpack16<float>(const uint4& u, float (&f)[4]) {
+    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+}
+template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& u, float (&f)[8]) {
+    const uint32_t r[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = __uint_as_float(r[j] << 16);
+        f[2 * j + 1] = __uint_as_float(r[j] & 0xffff0000u);
+    }
+}
+// E consecutive channels (E = 1, 2 or 4) of a staged V row as floats; p is E * sizeof(T)-byte aligned
+template <typename T, int E> __device__ __forceinline__ void load_channels(const unsigned char* p, float (&f)[E]);
+template <> __device__ __forceinline__ void load_channels<float, 1>(const unsigned char* p, float (&f)[1]) { f[0] = *reinterpret_cast<const float*>(p); }
+template <> __device__ __forceinline__ void load_channels<float, 2>(const unsigned char* p, float (&f)[2]) {
+    const float2 v = *reinterpret_cast<const float2*>(p); f[0] = v.x; f[1] = v.y;
+}
+template <> __device__ __forceinline__ void load_channels<float, 4>(const unsigned char* p, float (&f)[4]) {
+    const float4 v = *reinterpret_cast<const float4*>(p); f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+template <> __device__ __forceinline__ void load_channels<__nv_bfloat16, 1>(const unsigned char* p, float (&f)[1]) {
+    f[0] = __uint_as_float((uint32_t)*reinterpret_cast<const unsigned short*>(p) << 16);
+}
+template <> __device__ __forceinline__ void load_channels<__nv_bfloat16, 2>(const unsigned char* p, float (&f)[2]) {
+    const uint32_t r = *reinterpret_cast<const uint32_t*>(p);
+    f[0] = __uint_as_float(r << 16); f[1] = __uint_as_float(r & 0xffff0000u);
+}
+template <> __device__ __forceinline__ void load_channels<__nv_bfloat16, 4>(const unsigned char* p, float (&f)[4]) {
+    const uint2 r = *reinterpret_cast<const uint2*>(p);
+    f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+    f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+}
+
+// 1 / sqrt(head_dim) as every kernel forms it
+__device__ __forceinline__ float attn_score_scale(int hd) { return rsqrtf((float)hd); }
+
+// Softmax pieces of one 32-position block for one pair: lane = position.  `on`: the position is visible to the
+// pair's row (causal mask).  Returns this lane's probability relative to the block maximum; m = block maximum
+// (-inf if no position is visible), l = sum of the probabilities.
+__device__ __forceinline__ float attn_block_softmax(float score, float scale, bool on, float& m_out, float& l_out) {
+    const float s = on ? __fmul_rn(score, scale) : -INFINITY;
+    float m = s;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float pt = 0.f;
+    m_out = -INFINITY;
+    l_out = 0.f;
+    if (m > -INFINITY) {
+        pt = on ? expf(__fsub_rn(s, m)) : 0.f;
+        m_out = m;
+        l_out = warp_sum(pt);
+    }
+    return pt;
+}
+// weight of a block partial with maximum m inside a chunk whose maximum is M
+__device__ __forceinline__ float attn_block_weight(float m, float M) { return expf(__fsub_rn(m, M)); }
+// acc + x * f in one rounding (the chunk's L and O sums)
+__device__ __forceinline__ float attn_weighted_add(float acc, float x, float f) { return __fmaf_rn(x, f, acc); }
+// One step of the in-order fold: the running (M, L) takes in a partial (mc, lc); f0 and f1 are the factors by which the
+// running and the incoming out vectors are scaled (attn_fold_out).  Call only for mc > -inf.
+__device__ __forceinline__ void attn_fold(float& M, float& L, float mc, float lc, float& f0, float& f1) {
+    const float nm = fmaxf(M, mc);
+    f0 = expf(__fsub_rn(M, nm));
+    f1 = expf(__fsub_rn(mc, nm));
+    L = __fmaf_rn(L, f0, __fmul_rn(lc, f1));
+    M = nm;
+}
+__device__ __forceinline__ float attn_fold_out(float O, float oc, float f0, float f1) { return __fmaf_rn(O, f0, __fmul_rn(oc, f1)); }
+__device__ __forceinline__ float attn_finish(float O, float L) { return __fdiv_rn(O, L); }
+
+}  // namespace sb

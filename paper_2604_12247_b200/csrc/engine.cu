@@ -289,7 +289,11 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
         for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
         SB_T(e, launch_rope_append<T>(e.st, ra));
         SB_MARK("rope");
-        SB_T(e, launch_attention<T>(e.st, aa));
+        // long contexts: warps streaming whole chunks (bit-identical to the separate chunk kernel, which the option
+        // that switches the one-launch attention off also restores here)
+        bool streamed = false;
+        if ((g_fuse & 2) && (pos0 + r0 + m - 1) / D.chunk + 1 > 8) SB_T(e, streamed = launch_attention_stream<T>(e.st, aa));
+        if (!streamed) SB_T(e, launch_attention<T>(e.st, aa));
         SB_MARK("attn");
         e.launches += 3;
     }

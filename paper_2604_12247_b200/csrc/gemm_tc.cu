@@ -515,13 +515,7 @@ static bool make_map(CUtensorMap* tm, const void* base, int rows, int K, int box
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int sm_count() {   // of the current device
-    static int n[kMaxDevices];
-    const int dev = current_device();
-    if (dev < 0) return 148;
-    if (!n[dev] && (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0)) n[dev] = 148;
-    return n[dev];
-}
+static int sm_count() { return device_sm_count(); }
 
 // Slab height R (multiple of 8 in [64,128]) and split count S that minimise what the busiest
 // CTA streams.  Depends on the shape only, never on the number of rows.

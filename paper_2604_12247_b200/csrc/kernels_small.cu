@@ -2,6 +2,7 @@
 // decode attention over the paged KV cache (split-KV, warp-shuffle reductions), SwiGLU,
 // greedy acceptance.  All of them are deterministic and row-invariant: what they compute for one
 // row never depends on which other rows ride along in the same launch.
+#include "attn_common.cuh"
 #include "sb_internal.cuh"
 
 namespace sb {
@@ -192,24 +193,8 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 // A warp sweeps its pairs PG at a time.  Per-block partials (max, sum, out) are merged in block order into one
 // partial per (chunk, row, head); the chunks are merged by k_attn_combine or, in the fused kernel, by the cluster.
 // ------------------------------------------------------------------------------------------------
-constexpr int kPosWarps = 4;                  // 32-position blocks per chunk
 constexpr int kAttnWarps = 2 * kPosWarps;     // two warps per block: each takes half of the (row, query head) pairs
-constexpr int kAttnChunk = 128;
-constexpr unsigned long long kStageWaitCycles = 2000000000ull;   // bound of the wait for the staging copies (~1 s)
 constexpr int kMaxPairGroup = 8;
-
-template <typename T> __device__ __forceinline__ void unpack16(const uint4& u, float (&f)[16 / sizeof(T)]);
-template <> __device__ __forceinline__ void unpack16<float>(const uint4& u, float (&f)[4]) {
-    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
-}
-template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& u, float (&f)[8]) {
-    const uint32_t r[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        f[2 * j] = __uint_as_float(r[j] << 16);
-        f[2 * j + 1] = __uint_as_float(r[j] & 0xffff0000u);
-    }
-}
 
 // PG = (row, query head) pairs handled per sweep over the staged tile: the largest of 8, 4, 2, 1 that
 // divides the pair count, so that the inner loops carry no run-time predicates.
@@ -394,7 +379,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     }
     __syncthreads();   // q_s, the rows of step 2 and both warps' tiles are complete
 
-    const float scale = rsqrtf((float)HD);
+    const float scale = attn_score_scale(HD);
     const int P0 = (P + 1) / 2;   // pairs [0, P0) go to the first warp of a block, [P0, P) to the second
     for (int pg = hsel ? P0 : 0; pg < (hsel ? P : P0); pg += kPairGroup) {
         // ---- scores: lane = position ----
@@ -422,21 +407,9 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         float mx[kPairGroup], ls[kPairGroup];
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
-            mx[pp] = -INFINITY;
-            ls[pp] = 0.f;
-            float pt = 0.f;
             int i = (pg + pp) / G;
             bool on = my_t <= a.pos0 + a.r0 + i;         // causal: a row sees positions <= its own
-            float s = on ? sc[pp] * scale : -INFINITY;
-            float m = s;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            if (m > -INFINITY) {
-                pt = on ? expf(s - m) : 0.f;
-                mx[pp] = m;
-                ls[pp] = warp_sum(pt);
-            }
-            P_w[pp * 32 + lane] = pt;
+            P_w[pp * 32 + lane] = attn_block_softmax(sc[pp], scale, on, mx[pp], ls[pp]);
         }
         __syncwarp();
         // ---- out = sum_t p_t V_t: lane = channels lane*E .. lane*E+E-1 ----
@@ -450,9 +423,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
             float vf[4][E];
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {
-                const T* vp = reinterpret_cast<const T*>(V_w + (t4 * 4 + tt) * ROWB) + lane * E;
-#pragma unroll
-                for (int e = 0; e < E; ++e) vf[tt][e] = to_f32(vp[e]);
+                load_channels<T, E>(V_w + (t4 * 4 + tt) * ROWB + lane * E * (int)sizeof(T), vf[tt]);
             }
 #pragma unroll
             for (int pp = 0; pp < kPairGroup; ++pp) {
@@ -493,9 +464,9 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
                 const float* src = mrg + ((size_t)w * P + p) * (HD + 2);
                 float mw = src[HD];
                 if (mw > -INFINITY) {
-                    float f = expf(mw - M);
-                    L += src[HD + 1] * f;
-                    O += src[e] * f;
+                    const float f = attn_block_weight(mw, M);
+                    L = attn_weighted_add(L, src[HD + 1], f);
+                    O = attn_weighted_add(O, src[e], f);
                 }
             }
         }
@@ -535,28 +506,30 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 if (mc[u] > -INFINITY) {
-                    float nm = fmaxf(M, mc[u]);
-                    float f0 = expf(M - nm), f1 = expf(mc[u] - nm);
-                    L = L * f0 + lc[u] * f1;
-                    O = O * f0 + oc[u] * f1;
-                    M = nm;
+                    float f0, f1;
+                    attn_fold(M, L, mc[u], lc[u], f0, f1);
+                    O = attn_fold_out(O, oc[u], f0, f1);
                 }
             }
             using A = Act<T>;
-            A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (kvh * G + g) * HD + e, a.H * HD, O / L);
+            A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (kvh * G + g) * HD + e, a.H * HD, attn_finish(O, L));
         }
     }
     __syncthreads();
     cluster_sync_all();   // a CTA's shared memory stays alive until its peers have read it
 }
 
-// grid = (H, m), block = hd: merge the chunk partials of one (row, head) in chunk order.
+// Merge of the chunk partials of one (row, query head): grid = (H, m), 8 warps, lane = hd / 32 channels.
+// Two levels, both in order: warp g folds the chunks 8g .. 8g+7 of its group one after the other (all their loads are
+// issued before the first use: one L2 round trip), then the first warp folds the group partials one after the other.
+// A context of up to 8 chunks is one group, which is the fold the one-launch kernel does through its cluster.
 template <typename T>
-__global__ void k_attn_combine(AttnArgs a) {
+__global__ void __launch_bounds__(kChunkGroup * 32) k_attn_combine(AttnArgs a) {
+    __shared__ float grp[kChunkGroup][128 + 2];
     pdl_trigger();
     pdl_wait();
-    int hq = blockIdx.x, row = a.r0 + blockIdx.y, e = threadIdx.x;
-    int hd = a.hd;
+    const int hq = blockIdx.x, row = a.r0 + blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hd = a.hd, E = hd >> 5;                // channels per lane: 1, 2 or 4
     using A = Act<T>;
     typename A::type* act_out = reinterpret_cast<typename A::type*>(a.act_out);
     if (a.n_blocks > 1) {                            // several blocks of 8 rows in one launch: this CTA's block
@@ -565,31 +538,62 @@ __global__ void k_attn_combine(AttnArgs a) {
         a.pos0 += blk * kMaxW;
         act_out += (size_t)blk * A::rows * a.H * hd;
     }
-    int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own
-    float M = -INFINITY, L = 0.f, O = 0.f;
-    constexpr int kBatch = 8;   // chunks whose partials are loaded together (one L2 round trip per batch)
-    for (int c0 = 0; c0 < n_chunks; c0 += kBatch) {
-        float mc[kBatch], lc[kBatch], oc[kBatch];
+    const int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own
+    const int n_groups = (n_chunks + kChunkGroup - 1) / kChunkGroup;
+    float Mf = -INFINITY, Lf = 0.f, Of[4] = {0.f, 0.f, 0.f, 0.f};   // the first warp's running result
+    for (int g0 = 0; g0 < n_groups; g0 += kChunkGroup) {
+        const int g = g0 + warp;
+        if (g < n_groups) {
+            float mc[kChunkGroup], lc[kChunkGroup], oc[kChunkGroup][4];
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const bool ok = c0 + u < n_chunks;
-            const float* src = a.part + (((size_t)(ok ? c0 + u : 0) * kMaxW + row) * a.H + hq) * (hd + 2);
-            mc[u] = ok ? __ldcg(src + hd) : -INFINITY;
-            lc[u] = ok ? __ldcg(src + hd + 1) : 0.f;
-            oc[u] = ok ? __ldcg(src + e) : 0.f;
-        }
+            for (int u = 0; u < kChunkGroup; ++u) {
+                const int c = g * kChunkGroup + u;
+                const bool ok = c < n_chunks;
+                const float* src = a.part + (((size_t)(ok ? c : 0) * kMaxW + row) * a.H + hq) * (hd + 2);
+                mc[u] = ok ? __ldcg(src + hd) : -INFINITY;
+                lc[u] = ok ? __ldcg(src + hd + 1) : 0.f;
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            if (mc[u] > -INFINITY) {
-                float nm = fmaxf(M, mc[u]);
-                float f0 = expf(M - nm), f1 = expf(mc[u] - nm);
-                L = L * f0 + lc[u] * f1;
-                O = O * f0 + oc[u] * f1;
-                M = nm;
+                for (int e = 0; e < 4; ++e) oc[u][e] = (ok && e < E) ? __ldcg(src + lane * E + e) : 0.f;
+            }
+            float M = -INFINITY, L = 0.f, O[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int u = 0; u < kChunkGroup; ++u) {
+                if (mc[u] > -INFINITY) {
+                    float f0, f1;
+                    attn_fold(M, L, mc[u], lc[u], f0, f1);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) O[e] = attn_fold_out(O[e], oc[u][e], f0, f1);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (e < E) grp[warp][lane * E + e] = O[e];
+            if (lane == 0) {
+                grp[warp][hd] = M;
+                grp[warp][hd + 1] = L;
             }
         }
+        __syncthreads();
+        if (warp == 0) {
+            const int n_here = min(kChunkGroup, n_groups - g0);
+            for (int w = 0; w < n_here; ++w) {
+                const float mg = grp[w][hd];
+                if (mg > -INFINITY) {
+                    float f0, f1;
+                    attn_fold(Mf, Lf, mg, grp[w][hd + 1], f0, f1);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (e < E) Of[e] = attn_fold_out(Of[e], grp[w][lane * E + e], f0, f1);
+                }
+            }
+        }
+        __syncthreads();
     }
-    A::store(act_out, row, hq * hd + e, a.H * hd, O / L);
+    if (warp == 0) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (e < E) A::store(act_out, row, hq * hd + lane * E + e, a.H * hd, attn_finish(Of[e], Lf));
+    }
 }
 
 static size_t attn_smem(int P, int HD, size_t elt, bool fused) {
@@ -649,7 +653,12 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) 
         case 64: launch_attn_partial<T, 64, false>(st, a, grid, 0); break;
         default: launch_attn_partial<T, 128, false>(st, a, grid, 0); break;
     }
-    launch_k(k_attn_combine<T>, dim3(a.H, a.m, nz), dim3(a.hd), 0, st, a);
+    launch_k(k_attn_combine<T>, dim3(a.H, a.m, nz), dim3(kChunkGroup * 32), 0, st, a);
+}
+
+template <typename T> void launch_attention_combine(cudaStream_t st, const AttnArgs& a) {
+    const int nz = a.n_blocks > 1 ? a.n_blocks : 1;
+    launch_k(k_attn_combine<T>, dim3(a.H, a.m, nz), dim3(kChunkGroup * 32), 0, st, a);
 }
 
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a) {
@@ -1052,6 +1061,7 @@ void launch_init_pages(cudaStream_t st, int* page_table, int n_pages) {
     template void launch_rope_append<T>(cudaStream_t, const RopeArgs&);                                             \
     template void launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
     template bool launch_attention_fused<T>(cudaStream_t, const AttnArgs&);                                         \
+    template void launch_attention_combine<T>(cudaStream_t, const AttnArgs&);                                       \
     template void launch_swiglu<T>(cudaStream_t, const float*, int, int, void*, int, int);
 SB_INST(float)
 SB_INST(__nv_bfloat16)

@@ -115,6 +115,13 @@ inline int current_device() {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
     return dev;
 }
+inline int device_sm_count() {   // SMs of the current device (148 if the query fails)
+    static int n[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return 148;
+    if (!n[dev] && (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0)) n[dev] = 148;
+    return n[dev];
+}
 // cluster.y > 1 launches thread-block clusters of that many CTAs along y (grid.y must be a multiple of it);
 // pdl: launch with programmatic stream serialisation (the kernel may start while its predecessor drains)
 template <typename... KArgs, typename... Args>
@@ -403,6 +410,11 @@ template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
 // Returns false without launching when the shape is not covered (more than 8 chunks of 128 positions, or the
 // device cannot co-schedule the cluster): the caller then runs launch_rope_append + launch_attention.
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a);
+// Long contexts (attn_stream.cu): the chunk partials by warps that each stream whole chunks through a private ring of
+// staging tiles, then the chunk merge; a.q must hold the rotated queries and the cache the new rows (launch_rope_append
+// first).  Same results, bit for bit, as launch_attention.  Returns false without launching if the shape is not covered.
+template <typename T> bool launch_attention_stream(cudaStream_t st, const AttnArgs& a);
+template <typename T> void launch_attention_combine(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror);
 bool launch_sample(cudaStream_t st, const SampleArgs& a);   // false: the cluster launch was refused

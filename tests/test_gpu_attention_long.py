@@ -33,7 +33,7 @@ K_SCALE = 3.0
 # 1024, 1025: hand-over to the separate kernels (9 chunks); 2048: 17 chunks; 8184: 64 chunks, the longest context of
 # the micro-benchmarks
 CASES = [(1, 511), (8, 511), (4, 512), (8, 896), (8, 1016), (1, 1023), (8, 1017), (4, 1023), (1, 1024), (8, 1024),
-         (4, 1025), (1, 2048), (8, 2048), (4, 8184), (8, 8184), (1, 8191)]
+         (4, 1025), (2, 1500), (3, 1790), (1, 2048), (8, 2048), (6, 2500), (5, 4000), (4, 8184), (8, 8184), (1, 8191)]
 
 
 class Geometry:
@@ -71,13 +71,19 @@ class Geometry:
         self.scratch = binding.KernelScratch(self.cfg)
         self.lw = {k: v.cuda() for k, v in self.w["layers"][0].items()}
 
-    def gpu(self, h, first_pos):
+    def gpu(self, h, first_pos, pre=None):
+        """The layer on rows h at first_pos ..; pre = (K rows, V rows) cached at the positions right before first_pos
+        in place of the history (rows an earlier pass appended)."""
         m = h.shape[0]
         kc, vc = self.kc0.clone(), self.vc0.clone()
         # positions from first_pos on are what the pass appends: whatever they held must not matter
         idx = self.phys[first_pos:].cuda()
         kc[idx] = 7.0
         vc[idx] = -7.0
+        if pre is not None and len(pre[0]):
+            at = self.phys[first_pos - len(pre[0]):first_pos].cuda()
+            kc[at] = torch.from_numpy(pre[0]).to(kc.dtype).cuda()
+            vc[at] = torch.from_numpy(pre[1]).to(vc.dtype).cuda()
         hg = h.clone().cuda()
         binding.k_layer(self.cfg, self.lw, hg, kc, vc, self.pt, first_pos, self.scratch)
         torch.cuda.synchronize()
@@ -142,3 +148,23 @@ def test_dropping_one_chunk_would_be_seen(geometry):
     moved = np.abs(blind_h - ref_h).max() / np.abs(ref_h).max()
     print(f"\n[{g.shape.name}] hiding one chunk of 128 positions moves the hidden state by {moved:.2e}")
     assert moved > 5 * HIDDEN_TOL["bf16"]
+
+
+@pytest.mark.parametrize("first_pos", [1021, 2050])
+def test_long_context_rows_do_not_depend_on_companions(geometry, first_pos):
+    """Row i of a 6-row pass is bit-identical to the same row run alone once the earlier rows' K,V are cached, also
+    where the pass straddles the 1024-position hand-over between the attention kernels (rows at 1021 .. 1023 alone go
+    through the one-launch kernel, in company through the long-context kernels) and deep inside a long context: what
+    makes speculative decoding return exactly the autoregressive tokens at any length."""
+    g = geometry
+    m = 6
+    h = inputs.make_hidden(m, g.shape.d_model, 5 + first_pos)
+    binding.set_default_gemm(1)
+    try:
+        all_h, all_k, all_v = g.gpu(h, first_pos)
+        for i in range(m):
+            one_h, one_k, one_v = g.gpu(h[i:i + 1], first_pos + i, pre=(all_k[:i], all_v[:i]))
+            assert np.array_equal(one_h[0], all_h[i]), (g.shape.name, first_pos, i)
+            assert np.array_equal(one_k[0], all_k[i]) and np.array_equal(one_v[0], all_v[i])
+    finally:
+        binding.set_default_gemm(-1)
