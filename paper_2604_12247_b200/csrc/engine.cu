@@ -284,18 +284,24 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
         e.launches += 1;
         SB_MARK("attn");
     } else {
-        RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
-                    pos0, r0, m, D.rope_base, W.rope_tab, {}};
-        for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
-        SB_T(e, launch_rope_append<T>(e.st, ra));
-        SB_MARK("rope");
-        // long contexts: warps streaming whole chunks (bit-identical to the separate chunk kernel, which the option
-        // that switches the one-launch attention off also restores here)
-        bool streamed = false;
-        if ((g_fuse & 2) && (pos0 + r0 + m - 1) / D.chunk + 1 > 8) SB_T(e, streamed = launch_attention_stream<T>(e.st, aa));
-        if (!streamed) SB_T(e, launch_attention<T>(e.st, aa));
-        SB_MARK("attn");
-        e.launches += 3;
+        // more than 8 chunks: the chunk kernel with the same front end, then the chunk merge (two launches)
+        bool front = false;
+        if (g_fuse & 2) SB_T(e, front = launch_attention_front<T>(e.st, aa));
+        if (front) {
+            e.launches += 2;
+            SB_MARK("attn");
+        } else {
+            RopeArgs ra{W.p_qkv, s_qkv, W.q, k_cache_l, v_cache_l, W.page_table, D.H, D.Hkv, D.hd, D.page, D.page_shift,
+                        pos0, r0, m, D.rope_base, W.rope_tab, {}};
+            for (int i = 0; i < D.hd / 2; ++i) ra.inv_freq[i] = D.inv_freq[i];
+            SB_T(e, launch_rope_append<T>(e.st, ra));
+            SB_MARK("rope");
+            bool ok = false;
+            SB_T(e, ok = launch_attention<T>(e.st, aa));
+            if (!ok) e.err = SB_ERR_UNSUPPORTED;
+            SB_MARK("attn");
+            e.launches += 3;
+        }
     }
     const void* wo[1] = {lw.wo};
     int no[1] = {D.d};
@@ -365,7 +371,7 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
             aa.n_blocks = n_full;
             aa.part_block_stride = W.pf_attn_stride;
             aa.pos_pred0 = pos0;
-            launch_attention<T>(e.st, aa);
+            if (!launch_attention<T>(e.st, aa)) e.err = SB_ERR_UNSUPPORTED;
             e.launches += 2;
         }
         if (rem > 0) {
@@ -373,7 +379,7 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
                         W.pf_attn_part + (size_t)n_full * W.pf_attn_stride, act_of(W.pf_act_o, n_full, D.qd), D.H, D.Hkv, D.hd,
                         D.page, D.page_shift, pos0 + n_full * kMaxW, 0, rem, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
             aa.pos_pred0 = pos0;   // the pass's RoPE/append launch wrote the rows of the full blocks too
-            launch_attention<T>(e.st, aa);
+            if (!launch_attention<T>(e.st, aa)) e.err = SB_ERR_UNSUPPORTED;
             e.launches += 2;
         }
     }

@@ -193,34 +193,72 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 // A warp sweeps its pairs PG at a time.  Per-block partials (max, sum, out) are merged in block order into one
 // partial per (chunk, row, head); the chunks are merged by k_attn_combine or, in the fused kernel, by the cluster.
 // ------------------------------------------------------------------------------------------------
-constexpr int kAttnWarps = 2 * kPosWarps;     // two warps per block: each takes half of the (row, query head) pairs
 constexpr int kMaxPairGroup = 8;
 
-// PG = (row, query head) pairs handled per sweep over the staged tile: the largest of 8, 4, 2, 1 that
-// divides the pair count, so that the inner loops carry no run-time predicates.
-//
-// kFused: the kernel also does what precedes and follows it.  q is summed from the QKV split-K
-// partials and rotated here (every chunk CTA redoes it: a few hundred values); the CTA whose chunk
-// holds the new positions sums, rotates and rounds their K and V, appends them to the cache and puts
-// them straight into its staged tile; the chunk CTAs of a KV head form one thread-block cluster
-// (grid.y = cluster size = number of chunks <= 8) and merge the chunk partials, read from one another's
-// shared memory, in chunk order (each CTA takes a share of the outputs).  Same arithmetic in the same order as
-// k_rope_append + k_attn_partial<.., false> + k_attn_combine: bit-identical results.
+// Shared-memory layout of k_attn_partial: rotated queries [Ppad][HD] fp32 | K tiles [4][32][padded row] | V tiles
+// [4][32][row] | probabilities per warp [PG][32] | block partials [4][Ppad][HD+2] | (mode 1) chunk partial [Ppad][HD+2].
+// With one warp per block and few pairs, a block's partial is written over its own K tile, which is dead by then.
+struct AttnLayout {
+    int Ppad, rowb_k, rowb_v;
+    size_t off_k, off_v, off_p, off_mrg, off_out, total;
+    bool alias;
+    __host__ __device__ AttnLayout(int P, int HD, int elt, int PG, int WPB, bool want_out) {
+        Ppad = (P + PG - 1) / PG * PG;
+        rowb_k = HD * elt + 16;      // padded pitch: lane-per-row 16-byte reads of K are conflict-free
+        rowb_v = HD * elt;           // V is read a whole row per warp
+        off_k = (size_t)Ppad * HD * 4;
+        off_v = off_k + (size_t)kPosWarps * 32 * rowb_k;
+        off_p = off_v + (size_t)kPosWarps * 32 * rowb_v;
+        off_mrg = off_p + (size_t)kPosWarps * WPB * PG * 32 * 4;
+        alias = WPB == 1 && (size_t)Ppad * (HD + 2) * 4 <= (size_t)32 * rowb_k;
+        off_out = off_mrg + (alias ? 0 : (size_t)kPosWarps * Ppad * (HD + 2) * 4);
+        total = off_out + (want_out ? (size_t)Ppad * (HD + 2) * 4 : 0);
+    }
+};
+
+// mbarrier wait that lets the hardware park the thread for up to `ns` nanoseconds instead of spinning
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
+// PG = (row, query head) pairs handled per sweep over a staged block: 1, 2, 4 or 8; the pair count is padded to a
+// multiple of it (padding pairs compute on zero queries and are never written), so the inner loops carry no
+// run-time predicates and each K element is unpacked once for up to 8 pairs.
+// WPB = warps per 32-position block: 1 (the warp takes every pair; up to 8 pairs) or 2 (the groups of 8 pairs are
+// split between two warps; grouped-query models with several rows).
+// kMode 0: the rotated queries and every cached row come from memory (launch_rope_append ran before); chunk
+//          partials go to global memory for k_attn_combine.
+// kMode 1: the kernel also does what precedes and follows it.  q is summed from the QKV split-K partials and rotated
+//          here (every chunk CTA redoes it: a few hundred values); the CTA whose chunk holds the new positions sums,
+//          rotates and rounds their K and V, appends them to the cache and puts them straight into its staged tile;
+//          the chunk CTAs of a KV head form one thread-block cluster (grid.y = cluster size = number of chunks <= 8)
+//          and merge the chunk partials, read from one another's shared memory, in chunk order.
+// kMode 2: the front end of mode 1, the partials to global memory (contexts of more than 8 chunks).
+// Same arithmetic in the same order in every mode: bit-identical results.
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-template <typename T, int HD, int PG, bool kFused>
-__global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
+template <typename T, int HD, int PG, int kMode, int WPB>
+__global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs a) {
+    constexpr bool kFront = kMode != 0, kCluster = kMode == 1;
     constexpr int kPairGroup = PG;
     constexpr int E = HD / 32;                       // channels per lane in P.V
     constexpr int EPP = 16 / (int)sizeof(T);         // elements per 16-byte piece
     constexpr int PPR = HD / EPP;                    // pieces per K/V row
-    constexpr int ROWB = HD * (int)sizeof(T) + 16;   // padded row pitch: lane-per-row 16-byte reads are conflict-free
+    constexpr int ROWB_K = HD * (int)sizeof(T) + 16, ROWB_V = HD * (int)sizeof(T);
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
     const int kvh = blockIdx.x, c = blockIdx.y;
-    const int pos_pred0 = a.pos_pred0 >= 0 ? a.pos_pred0 : a.pos0 + a.r0;   // separate kernels: first position the preceding RoPE/append launch wrote
-    if (!kFused && a.n_blocks > 1) {                 // several blocks of 8 rows in one launch: this CTA's block
+    const int pos_pred0 = a.pos_pred0 >= 0 ? a.pos_pred0 : a.pos0 + a.r0;   // mode 0: first position the preceding RoPE/append launch wrote
+    if (!kFront && a.n_blocks > 1) {                 // several blocks of 8 rows in one launch: this CTA's block
         const int blk = blockIdx.z;
         a.q += (size_t)blk * kMaxW * a.H * HD;
         a.part += (size_t)blk * a.part_block_stride;
@@ -230,20 +268,27 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
     const int kvd = a.Hkv * HD, qd = a.H * HD;
-    float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD]
-    unsigned char* kv_s = smem + (size_t)P * HD * 4;                                // per warp: K[32], V[32]
-    const int v = warp & (kPosWarps - 1), hsel = warp / kPosWarps;   // position block; which half of the pairs
-    unsigned char* K_w = kv_s + (size_t)v * 64 * ROWB;
-    unsigned char* V_w = K_w + 32 * ROWB;
-    float* P_w = reinterpret_cast<float*>(kv_s + (size_t)kPosWarps * 64 * ROWB) + warp * kMaxPairGroup * 32;   // [PG][32]
-    float* mrg = reinterpret_cast<float*>(kv_s + (size_t)kPosWarps * 64 * ROWB) + kAttnWarps * kMaxPairGroup * 32;   // [4][P][HD+2]
-    float* out_s = mrg + (size_t)kPosWarps * P * (HD + 2);   // kFused: this chunk's merged partial [P][HD+2]
+    const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB, kCluster);
+    const int Ppad = lay.Ppad;
+    float* q_s = reinterpret_cast<float*>(smem);                                   // [Ppad][HD]
+    unsigned char* k_tiles = smem + lay.off_k;
+    unsigned char* v_tiles = smem + lay.off_v;
+    const int v = warp & (kPosWarps - 1), hsel = warp / kPosWarps;   // position block; which share of the pair groups
+    unsigned char* K_w = k_tiles + (size_t)v * 32 * ROWB_K;
+    unsigned char* V_w = v_tiles + (size_t)v * 32 * ROWB_V;
+    float* P_w = reinterpret_cast<float*>(smem + lay.off_p) + warp * PG * 32;       // [PG][32]
+    // block partial of block w: [Ppad][HD+2]
+    auto mrg_blk = [&](int w) -> float* {
+        return lay.alias ? reinterpret_cast<float*>(k_tiles + (size_t)w * 32 * ROWB_K)
+                         : reinterpret_cast<float*>(smem + lay.off_mrg) + (size_t)w * Ppad * (HD + 2);
+    };
+    float* out_s = reinterpret_cast<float*>(smem + lay.off_out);   // mode 1: this chunk's merged partial [Ppad][HD+2]
     __shared__ __align__(8) unsigned long long stage_bar[kPosWarps];
-    if (threadIdx.x < kPosWarps) mbar_init(smem_u32(&stage_bar[threadIdx.x]), 2);   // one arrival per warp of the block
+    if (threadIdx.x < kPosWarps) mbar_init(smem_u32(&stage_bar[threadIdx.x]), WPB);   // one arrival per warp of the block
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 
     const int pos_last = a.pos0 + a.r0 + a.m - 1;
-    const int pos_new0 = kFused ? a.pos0 + a.r0 : pos_last + 1;   // first position whose K,V this launch creates
+    const int pos_new0 = kFront ? a.pos0 + a.r0 : pos_last + 1;   // first position whose K,V this launch creates
     const int tbase = c * kAttnChunk + v * 32;
     const int my_t = tbase + lane;
     // The page table is set up when the context is created (or, for the stateless call, before the call)
@@ -253,56 +298,62 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
     // Rows of EARLIER steps of this layer (positions below pos_done) are complete when this kernel starts: between such
     // steps the stream holds a launch without programmatic overlap (the embedding kernel that starts every step, or
     // the clear of a stateless call).  Their copies -- the long, cold loads of this kernel -- start before the
-    // grid-dependency wait.  Separate kernels: the RoPE/append kernel right before this one wrote the rows from
+    // grid-dependency wait.  Mode 0: the RoPE/append kernel right before this one wrote the rows from
     // pos_done on; they are staged after the wait, on the same barrier (the warp arrives with the second batch).
-    const int pos_done = kFused ? pos_new0 : pos_pred0;
+    const int pos_done = kFront ? pos_new0 : pos_pred0;
     __syncthreads();   // barriers initialised
-    // 1. stage the block's K rows (first warp of the block) or V rows (second warp): one TMA copy per row of an
-    //    earlier launch; rows beyond the last position are zeroed (their probabilities are 0, but 0 * garbage
-    //    must stay 0); rows this launch creates are written in step 2
+    // 1. stage the block's K and V rows: one TMA copy per row of an earlier launch (two warps per block: the first
+    //    takes K, the second V); rows beyond the last position are zeroed (their probabilities are 0, but
+    //    0 * garbage must stay 0); rows this launch creates are written in step 2
     constexpr uint32_t kRowBytes = HD * (uint32_t)sizeof(T);
+    const int which0 = WPB == 2 ? hsel : 0, which1 = WPB == 2 ? hsel + 1 : 2;   // 0 = K, 1 = V
     {
         const bool early = my_t < pos_done;
         const uint32_t bar = smem_u32(&stage_bar[v]);
         const unsigned n_early = __popc(__ballot_sync(0xffffffffu, early));
         if (lane == 0) {
-            if (kFused) mbar_expect_tx(bar, n_early * kRowBytes);
-            else mbar_expect_tx_only(bar, n_early * kRowBytes);
+            if (kFront) mbar_expect_tx(bar, (uint32_t)(which1 - which0) * n_early * kRowBytes);
+            else mbar_expect_tx_only(bar, (uint32_t)(which1 - which0) * n_early * kRowBytes);
         }
         __syncwarp();
-        unsigned char* row = (hsel ? V_w : K_w) + lane * ROWB;
-        if (early) {
-            const T* src = reinterpret_cast<const T*>(hsel ? a.v_cache : a.k_cache) +
-                           ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
-            bulk_load(smem_u32(row), src, kRowBytes, bar);
-        } else if (my_t > pos_last) {
+        for (int which = which0; which < which1; ++which) {
+            unsigned char* row = which ? V_w + lane * ROWB_V : K_w + lane * ROWB_K;
+            if (early) {
+                const T* src = reinterpret_cast<const T*>(which ? a.v_cache : a.k_cache) +
+                               ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                bulk_load(smem_u32(row), src, kRowBytes, bar);
+            } else if (my_t > pos_last) {
 #pragma unroll
-            for (int j = 0; j < (int)kRowBytes / 16; ++j) reinterpret_cast<uint4*>(row)[j] = make_uint4(0u, 0u, 0u, 0u);
+                for (int j = 0; j < (int)kRowBytes / 16; ++j) reinterpret_cast<uint4*>(row)[j] = make_uint4(0u, 0u, 0u, 0u);
+            }
         }
     }
     pdl_wait();
-    if (!kFused) {   // the rows the RoPE/append kernel just wrote
+    if (!kFront) {   // the rows the RoPE/append kernel just wrote
         const bool late = my_t >= pos_done && my_t < pos_new0;
         const uint32_t bar = smem_u32(&stage_bar[v]);
         const unsigned n_late = __popc(__ballot_sync(0xffffffffu, late));
-        if (lane == 0) mbar_expect_tx(bar, n_late * kRowBytes);
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(which1 - which0) * n_late * kRowBytes);
         __syncwarp();
         if (late) {
-            unsigned char* row = (hsel ? V_w : K_w) + lane * ROWB;
-            const T* src = reinterpret_cast<const T*>(hsel ? a.v_cache : a.k_cache) +
-                           ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
-            bulk_load(smem_u32(row), src, kRowBytes, bar);
+            for (int which = which0; which < which1; ++which) {
+                unsigned char* row = which ? V_w + lane * ROWB_V : K_w + lane * ROWB_K;
+                const T* src = reinterpret_cast<const T*>(which ? a.v_cache : a.k_cache) +
+                               ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                bulk_load(smem_u32(row), src, kRowBytes, bar);
+            }
         }
     }
-    // 2. while those copies fly: q, and (fused) the new positions' K and V
-    if (kFused) {
+    // 2. while those copies fly: q, and (front end) the new positions' K and V
+    for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[idx] = 0.f;   // padding pairs
+    if (kFront) {
         constexpr int half = HD / 2;
         constexpr int kBatch = 4;   // work items whose partial sums are requested together
         const int ntot = qd + 2 * kvd;
         const size_t sstride = (size_t)kMaxW * ntot;
         // work items: P * half rotation pairs of q, then, for each new position of this chunk, half rotation pairs
         // of K and half element pairs of V (rounded to the storage type, written to the cache and into the staged
-        // tile of the warp that owns the position)
+        // tile of the block that owns the position)
         const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
         const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
         struct Item { int kind, pos, e2, p; };   // kind 0: q pair of (row, head) pair p; 1: K pair; 2: V pair of position pos
@@ -352,7 +403,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
                     dst[it.e2] = y0;
                     dst[it.e2 + half] = y1;
                     int tl = it.pos - c * kAttnChunk;
-                    T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
+                    T* srow = reinterpret_cast<T*>(is_v ? v_tiles + (size_t)tl * ROWB_V : k_tiles + (size_t)tl * ROWB_K);
                     srow[it.e2] = y0;
                     srow[it.e2 + half] = y1;
                 }
@@ -369,7 +420,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         const uint32_t bar = smem_u32(&stage_bar[v]);
         if (!mbar_try_wait(bar, 0)) {
             const unsigned long long t0 = clock64();
-            while (!mbar_try_wait(bar, 0)) {
+            while (!mbar_try_wait_parked(bar, 0, 2000u)) {
                 if (clock64() - t0 > kStageWaitCycles) {
                     if (a.status) atomicExch(a.status, 5u);
                     break;
@@ -377,11 +428,13 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
             }
         }
     }
-    __syncthreads();   // q_s, the rows of step 2 and both warps' tiles are complete
+    __syncthreads();   // q_s, the rows of step 2 and every block's tiles are complete
 
     const float scale = attn_score_scale(HD);
-    const int P0 = (P + 1) / 2;   // pairs [0, P0) go to the first warp of a block, [P0, P) to the second
-    for (int pg = hsel ? P0 : 0; pg < (hsel ? P : P0); pg += kPairGroup) {
+    // this warp's share of the pair groups
+    const int n_grp = Ppad / PG, grp_split = WPB == 2 ? (n_grp + 1) / 2 : n_grp;
+    const int pg_begin = hsel ? grp_split * PG : 0, pg_end = hsel ? Ppad : grp_split * PG;
+    for (int pg = pg_begin; pg < pg_end; pg += kPairGroup) {
         // ---- scores: lane = position ----
         float sc[kPairGroup];
 #pragma unroll
@@ -389,7 +442,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
 #pragma unroll 2
         for (int piece = 0; piece < PPR; ++piece) {
             float kf[EPP];
-            unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB + piece * 16), kf);
+            unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB_K + piece * 16), kf);
 #pragma unroll
             for (int pp = 0; pp < kPairGroup; ++pp) {
                 const float4* qv = reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP);
@@ -422,9 +475,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         for (int t4 = 0; t4 < 8; ++t4) {
             float vf[4][E];
 #pragma unroll
-            for (int tt = 0; tt < 4; ++tt) {
-                load_channels<T, E>(V_w + (t4 * 4 + tt) * ROWB + lane * E * (int)sizeof(T), vf[tt]);
-            }
+            for (int tt = 0; tt < 4; ++tt) load_channels<T, E>(V_w + (t4 * 4 + tt) * ROWB_V + lane * E * (int)sizeof(T), vf[tt]);
 #pragma unroll
             for (int pp = 0; pp < kPairGroup; ++pp) {
                 float4 p4 = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
@@ -437,10 +488,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
                 }
             }
         }
-        __syncwarp();
+        __syncwarp();   // every lane is done with its K row and with P_w: the block partial may go over the K tile
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
-            float* dst = mrg + ((size_t)v * P + pg + pp) * (HD + 2);
+            float* dst = mrg_blk(v) + (size_t)(pg + pp) * (HD + 2);
 #pragma unroll
             for (int e = 0; e < E; ++e) dst[lane * E + e] = o[pp][e];
             if (lane == 0) {
@@ -450,35 +501,37 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_partial(AttnArgs a) {
         }
     }
     __syncthreads();
-    // merge the four warps in warp order; thread -> (pair, channel)
-    for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
-        int p = idx / HD, e = idx - p * HD;
-        int i = p / G, g = p - i * G;
+    // merge the four blocks in block order; thread -> (pair, two channels)
+    for (int idx = threadIdx.x; idx < P * (HD / 2); idx += blockDim.x) {
+        const int p = idx / (HD / 2), e = (idx - p * (HD / 2)) * 2;
+        const int i = p / G, g = p - i * G;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kPosWarps; ++w) M = fmaxf(M, mrg[((size_t)w * P + p) * (HD + 2) + HD]);
-        float L = 0.f, O = 0.f;
+        for (int w = 0; w < kPosWarps; ++w) M = fmaxf(M, mrg_blk(w)[(size_t)p * (HD + 2) + HD]);
+        float L = 0.f, O0 = 0.f, O1 = 0.f;
         if (M > -INFINITY) {
 #pragma unroll
             for (int w = 0; w < kPosWarps; ++w) {
-                const float* src = mrg + ((size_t)w * P + p) * (HD + 2);
-                float mw = src[HD];
+                const float* src = mrg_blk(w) + (size_t)p * (HD + 2);
+                const float mw = src[HD];
                 if (mw > -INFINITY) {
                     const float f = attn_block_weight(mw, M);
+                    const float2 o2 = *reinterpret_cast<const float2*>(src + e);
                     L = attn_weighted_add(L, src[HD + 1], f);
-                    O = attn_weighted_add(O, src[e], f);
+                    O0 = attn_weighted_add(O0, o2.x, f);
+                    O1 = attn_weighted_add(O1, o2.y, f);
                 }
             }
         }
-        float* dst = kFused ? out_s + (size_t)p * (HD + 2)
-                            : a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
-        dst[e] = O;
+        float* dst = kCluster ? out_s + (size_t)p * (HD + 2)
+                              : a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
+        *reinterpret_cast<float2*>(dst + e) = make_float2(O0, O1);
         if (e == 0) {
             dst[HD] = M;
             dst[HD + 1] = L;
         }
     }
-    if (!kFused) return;
+    if (!kCluster) return;
     // ---- chunk merge across the cluster (one CTA per chunk of this KV head) ----
     __syncthreads();
     cluster_sync_all();   // every chunk's partial is in its CTA's out_s
@@ -596,16 +649,14 @@ __global__ void __launch_bounds__(kChunkGroup * 32) k_attn_combine(AttnArgs a) {
     }
 }
 
-static size_t attn_smem(int P, int HD, size_t elt, bool fused) {
-    const int rowb = HD * (int)elt + 16;
-    return (size_t)P * HD * 4 + (size_t)kPosWarps * 64 * rowb + (size_t)kAttnWarps * kMaxPairGroup * 32 * 4 +
-           (size_t)kPosWarps * P * (HD + 2) * 4 + (fused ? (size_t)P * (HD + 2) * 4 : 0);
-}
-// cluster_y = 0: plain launch; > 0: the fused kernel as clusters of that many chunk CTAs.  Returns false if the
+// cluster_y = 0: plain launch; > 0: mode 1 as clusters of that many chunk CTAs.  Returns false if the
 // device cannot co-schedule such a cluster (nothing is launched then).
-template <typename T, int HD, int PG, bool kFused>
-static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem, int cluster_y) {
-    auto kernel = k_attn_partial<T, HD, PG, kFused>;
+template <typename T, int HD, int PG, int kMode, int WPB>
+static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
+    auto kernel = k_attn_partial<T, HD, PG, kMode, WPB>;
+    const int P = a.m * (a.H / a.Hkv);
+    const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB, kMode == 1);
+    const dim3 block(kPosWarps * WPB * 32);
     static bool configured[kMaxDevices];             // function attributes are per device
     const int dev = current_device();
     if (dev < 0) return false;
@@ -613,12 +664,13 @@ static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
         configured[dev] = true;
     }
-    if (kFused && cluster_y > 1) {
+    if (lay.total > 200 * 1024) return false;
+    if (kMode == 1 && cluster_y > 1) {
         static int fits_dev[kMaxDevices][9];             // per device and cluster size: 0 unknown, 1 yes, -1 no
         int* fits = fits_dev[dev];
         if (fits[cluster_y] == 0) {
             cudaLaunchConfig_t cfg{};
-            cfg.gridDim = grid; cfg.blockDim = dim3(kAttnWarps * 32); cfg.dynamicSmemBytes = 200 * 1024;
+            cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 200 * 1024;
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = (unsigned)cluster_y; at[0].val.clusterDim.z = 1;
@@ -629,31 +681,33 @@ static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t
         }
         if (fits[cluster_y] < 0) return false;
     }
-    return launch_kc(kernel, grid, dim3(kAttnWarps * 32), smem, st, kFused ? cluster_y : 1, a) == cudaSuccess;
+    return launch_kc(kernel, grid, block, lay.total, st, kMode == 1 ? cluster_y : 1, a) == cudaSuccess;
 }
-template <typename T, int HD, bool kFused>
+template <typename T, int HD, int kMode>
 static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
     const int P = a.m * (a.H / a.Hkv);
-    size_t smem = attn_smem(P, HD, sizeof(T), kFused);
-    // pairs per sweep: the largest of 8, 4, 2, 1 that divides what each of a block's two warps gets
-    const int P0 = (P + 1) / 2, P1 = P - P0;
-    auto divides = [&](int g) { return P0 % g == 0 && P1 % g == 0; };
-    if (divides(8)) return launch_attn_pg<T, HD, 8, kFused>(st, a, grid, smem, cluster_y);
-    if (divides(4)) return launch_attn_pg<T, HD, 4, kFused>(st, a, grid, smem, cluster_y);
-    if (divides(2)) return launch_attn_pg<T, HD, 2, kFused>(st, a, grid, smem, cluster_y);
-    return launch_attn_pg<T, HD, 1, kFused>(st, a, grid, smem, cluster_y);
+    // up to 8 pairs: one warp per block sweeps them all at once (pair count padded to 1, 2, 4 or 8); more (grouped-query
+    // models with several rows): groups of 8, split between two warps per block
+    if (P > 8) return launch_attn_pg<T, HD, 8, kMode, 2>(st, a, grid, cluster_y);
+    if (P > 4) return launch_attn_pg<T, HD, 8, kMode, 1>(st, a, grid, cluster_y);
+    if (P > 2) return launch_attn_pg<T, HD, 4, kMode, 1>(st, a, grid, cluster_y);
+    if (P > 1) return launch_attn_pg<T, HD, 2, kMode, 1>(st, a, grid, cluster_y);
+    return launch_attn_pg<T, HD, 1, kMode, 1>(st, a, grid, cluster_y);
 }
 
-template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a) {
+template <typename T> bool launch_attention(cudaStream_t st, const AttnArgs& a) {
     const int nz = a.n_blocks > 1 ? a.n_blocks : 1;
     int n_chunks = (a.pos0 + a.r0 + (nz - 1) * kMaxW + a.m - 1) / kAttnChunk + 1;   // up to the last block's last position
     dim3 grid(a.Hkv, n_chunks, nz);
+    bool ok;
     switch (a.hd) {
-        case 32: launch_attn_partial<T, 32, false>(st, a, grid, 0); break;
-        case 64: launch_attn_partial<T, 64, false>(st, a, grid, 0); break;
-        default: launch_attn_partial<T, 128, false>(st, a, grid, 0); break;
+        case 32: ok = launch_attn_partial<T, 32, 0>(st, a, grid, 0); break;
+        case 64: ok = launch_attn_partial<T, 64, 0>(st, a, grid, 0); break;
+        default: ok = launch_attn_partial<T, 128, 0>(st, a, grid, 0); break;
     }
-    launch_k(k_attn_combine<T>, dim3(a.H, a.m, nz), dim3(kChunkGroup * 32), 0, st, a);
+    if (!ok) return false;
+    launch_attention_combine<T>(st, a);
+    return true;
 }
 
 template <typename T> void launch_attention_combine(cudaStream_t st, const AttnArgs& a) {
@@ -666,10 +720,26 @@ template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArg
     if (n_chunks > 8) return false;   // portable cluster size
     dim3 grid(a.Hkv, n_chunks);
     switch (a.hd) {
-        case 32: return launch_attn_partial<T, 32, true>(st, a, grid, n_chunks);
-        case 64: return launch_attn_partial<T, 64, true>(st, a, grid, n_chunks);
-        default: return launch_attn_partial<T, 128, true>(st, a, grid, n_chunks);
+        case 32: return launch_attn_partial<T, 32, 1>(st, a, grid, n_chunks);
+        case 64: return launch_attn_partial<T, 64, 1>(st, a, grid, n_chunks);
+        default: return launch_attn_partial<T, 128, 1>(st, a, grid, n_chunks);
     }
+}
+
+// Contexts of any length in two launches: the chunk kernel with its front end (RoPE, cache append) and the chunk merge.
+template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a) {
+    if (a.n_blocks > 1) return false;
+    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
+    dim3 grid(a.Hkv, n_chunks);
+    bool ok;
+    switch (a.hd) {
+        case 32: ok = launch_attn_partial<T, 32, 2>(st, a, grid, 0); break;
+        case 64: ok = launch_attn_partial<T, 64, 2>(st, a, grid, 0); break;
+        default: ok = launch_attn_partial<T, 128, 2>(st, a, grid, 0); break;
+    }
+    if (!ok) return false;
+    launch_attention_combine<T>(st, a);
+    return true;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1059,9 +1129,10 @@ void launch_init_pages(cudaStream_t st, int* page_table, int n_pages) {
     template void launch_embed<T>(cudaStream_t, const T*, int, const int*, int, int, int, float*);                  \
     template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int, unsigned int*); \
     template void launch_rope_append<T>(cudaStream_t, const RopeArgs&);                                             \
-    template void launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
+    template bool launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
     template bool launch_attention_fused<T>(cudaStream_t, const AttnArgs&);                                         \
     template void launch_attention_combine<T>(cudaStream_t, const AttnArgs&);                                       \
+    template bool launch_attention_front<T>(cudaStream_t, const AttnArgs&);                                         \
     template void launch_swiglu<T>(cudaStream_t, const float*, int, int, void*, int, int);
 SB_INST(float)
 SB_INST(__nv_bfloat16)

@@ -405,15 +405,16 @@ template <typename T> void launch_resid_norm(cudaStream_t st, float* h, const fl
 template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a);
 // cos/sin of pos * inv_freq[i] for pos < n_pos, i < half, as [pos][half]
 void launch_rope_table(cudaStream_t st, float2* tab, int n_pos, int half, const double* inv_freq);
-template <typename T> void launch_attention(cudaStream_t st, const AttnArgs& a);
+// false: the shape is not covered (too many (row, query head) pairs per KV head for the shared memory of an SM); nothing launched
+template <typename T> bool launch_attention(cudaStream_t st, const AttnArgs& a);
 // RoPE + cache append + attention + chunk merge in one launch (a.qkv, a.n_split, a.inv_freq set; a.q unused).
 // Returns false without launching when the shape is not covered (more than 8 chunks of 128 positions, or the
 // device cannot co-schedule the cluster): the caller then runs launch_rope_append + launch_attention.
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a);
-// Long contexts (attn_stream.cu): the chunk partials by warps that each stream whole chunks through a private ring of
-// staging tiles, then the chunk merge; a.q must hold the rotated queries and the cache the new rows (launch_rope_append
-// first).  Same results, bit for bit, as launch_attention.  Returns false without launching if the shape is not covered.
-template <typename T> bool launch_attention_stream(cudaStream_t st, const AttnArgs& a);
+// Contexts of any length (a.qkv, a.n_split, a.inv_freq set; a.q unused): the chunk kernel with RoPE and cache append
+// in its front end, then the chunk merge: two launches.  Same results, bit for bit, as launch_rope_append +
+// launch_attention.  Returns false without launching if the shape is not covered.
+template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_attention_combine(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror);
