@@ -197,7 +197,7 @@ constexpr int kMaxPairGroup = 8;
 
 // Shared-memory layout of k_attn_partial: rotated queries [Ppad][HD] fp32 | K tiles [4][32][padded row] | V tiles
 // [4][32][row] | probabilities per warp [PG][32] | block partials [4][Ppad][HD+2] | (mode 1) chunk partial [Ppad][HD+2].
-// With one warp per block and few pairs, a block's partial is written over its own K tile, which is dead by then.
+// Where it fits, a block's partial is written over the block's own K tile once its warps are done with the scores.
 struct AttnLayout {
     int Ppad, rowb_k, rowb_v;
     size_t off_k, off_v, off_p, off_mrg, off_out, total;
@@ -210,7 +210,8 @@ struct AttnLayout {
         off_v = off_k + (size_t)kPosWarps * 32 * rowb_k;
         off_p = off_v + (size_t)kPosWarps * 32 * rowb_v;
         off_mrg = off_p + (size_t)kPosWarps * WPB * PG * 32 * 4;
-        alias = WPB == 1 && (size_t)Ppad * (HD + 2) * 4 <= (size_t)32 * rowb_k;
+        // only where every warp makes at most one sweep: a second sweep would read the K tile again
+        alias = (size_t)Ppad * (HD + 2) * 4 <= (size_t)32 * rowb_k && Ppad / PG <= WPB;
         off_out = off_mrg + (alias ? 0 : (size_t)kPosWarps * Ppad * (HD + 2) * 4);
         total = off_out + (want_out ? (size_t)Ppad * (HD + 2) * 4 : 0);
     }
@@ -434,6 +435,11 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     // this warp's share of the pair groups
     const int n_grp = Ppad / PG, grp_split = WPB == 2 ? (n_grp + 1) / 2 : n_grp;
     const int pg_begin = hsel ? grp_split * PG : 0, pg_end = hsel ? Ppad : grp_split * PG;
+    // Where the block partial goes over the K tile and two warps share the block, both must be done with the scores
+    // first: a named barrier of the block's two warps, which EVERY warp executes exactly once (the layout allows that
+    // overlay only if no warp makes more than one sweep; a warp without pairs arrives after the loop).
+    const bool pair_barrier = WPB == 2 && lay.alias;
+    bool arrived = false;
     for (int pg = pg_begin; pg < pg_end; pg += kPairGroup) {
         // ---- scores: lane = position ----
         float sc[kPairGroup];
@@ -443,17 +449,21 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         for (int piece = 0; piece < PPR; ++piece) {
             float kf[EPP];
             unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB_K + piece * 16), kf);
+            // per pair one fmaf chain over the channels in order; the pairs' chains are independent and interleaved
 #pragma unroll
-            for (int pp = 0; pp < kPairGroup; ++pp) {
-                const float4* qv = reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP);
+            for (int v4 = 0; v4 < EPP / 4; ++v4) {
+                float4 qq[kPairGroup];
 #pragma unroll
-                for (int v4 = 0; v4 < EPP / 4; ++v4) {
-                    float4 qq = qv[v4];
-                    sc[pp] = fmaf(qq.x, kf[4 * v4], sc[pp]);
-                    sc[pp] = fmaf(qq.y, kf[4 * v4 + 1], sc[pp]);
-                    sc[pp] = fmaf(qq.z, kf[4 * v4 + 2], sc[pp]);
-                    sc[pp] = fmaf(qq.w, kf[4 * v4 + 3], sc[pp]);
-                }
+                for (int pp = 0; pp < kPairGroup; ++pp)
+                    qq[pp] = *reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP + 4 * v4);
+#pragma unroll
+                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].x, kf[4 * v4], sc[pp]);
+#pragma unroll
+                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].y, kf[4 * v4 + 1], sc[pp]);
+#pragma unroll
+                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].z, kf[4 * v4 + 2], sc[pp]);
+#pragma unroll
+                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].w, kf[4 * v4 + 3], sc[pp]);
             }
         }
         // ---- softmax pieces of this warp's 32 positions (warp-shuffle max and sum) ----
@@ -476,19 +486,32 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
             float vf[4][E];
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) load_channels<T, E>(V_w + (t4 * 4 + tt) * ROWB_V + lane * E * (int)sizeof(T), vf[tt]);
+            // per (pair, channel) one fmaf chain over the positions in order; the chains are independent and interleaved
+            float4 p4[kPairGroup];
 #pragma unroll
-            for (int pp = 0; pp < kPairGroup; ++pp) {
-                float4 p4 = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
+            for (int pp = 0; pp < kPairGroup; ++pp) p4[pp] = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    o[pp][e] = fmaf(p4.x, vf[0][e], o[pp][e]);
-                    o[pp][e] = fmaf(p4.y, vf[1][e], o[pp][e]);
-                    o[pp][e] = fmaf(p4.z, vf[2][e], o[pp][e]);
-                    o[pp][e] = fmaf(p4.w, vf[3][e], o[pp][e]);
-                }
-            }
+            for (int pp = 0; pp < kPairGroup; ++pp)
+#pragma unroll
+                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].x, vf[0][e], o[pp][e]);
+#pragma unroll
+            for (int pp = 0; pp < kPairGroup; ++pp)
+#pragma unroll
+                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].y, vf[1][e], o[pp][e]);
+#pragma unroll
+            for (int pp = 0; pp < kPairGroup; ++pp)
+#pragma unroll
+                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].z, vf[2][e], o[pp][e]);
+#pragma unroll
+            for (int pp = 0; pp < kPairGroup; ++pp)
+#pragma unroll
+                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].w, vf[3][e], o[pp][e]);
         }
-        __syncwarp();   // every lane is done with its K row and with P_w: the block partial may go over the K tile
+        __syncwarp();   // every lane is done with its K row and with P_w
+        if (pair_barrier && !arrived) {   // ... and so is the block's other warp, before the block partial goes over the K tile
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + v) : "memory");
+            arrived = true;
+        }
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
             float* dst = mrg_blk(v) + (size_t)(pg + pp) * (HD + 2);
@@ -500,6 +523,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
             }
         }
     }
+    if (pair_barrier && !arrived) asm volatile("bar.sync %0, 64;" ::"r"(1 + v) : "memory");
     __syncthreads();
     // merge the four blocks in block order; thread -> (pair, two channels)
     for (int idx = threadIdx.x; idx < P * (HD / 2); idx += blockDim.x) {
@@ -686,13 +710,13 @@ static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, int cl
 template <typename T, int HD, int kMode>
 static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
     const int P = a.m * (a.H / a.Hkv);
-    // up to 8 pairs: one warp per block sweeps them all at once (pair count padded to 1, 2, 4 or 8); more (grouped-query
-    // models with several rows): groups of 8, split between two warps per block
+    // Two warps per 32-position block share the pairs (latency hides behind warps, not behind instruction-level
+    // parallelism: one warp per block with twice the pairs measured slower at every context length); pairs per sweep =
+    // what one of the two warps gets, padded to 1, 2, 4 or 8.
     if (P > 8) return launch_attn_pg<T, HD, 8, kMode, 2>(st, a, grid, cluster_y);
-    if (P > 4) return launch_attn_pg<T, HD, 8, kMode, 1>(st, a, grid, cluster_y);
-    if (P > 2) return launch_attn_pg<T, HD, 4, kMode, 1>(st, a, grid, cluster_y);
-    if (P > 1) return launch_attn_pg<T, HD, 2, kMode, 1>(st, a, grid, cluster_y);
-    return launch_attn_pg<T, HD, 1, kMode, 1>(st, a, grid, cluster_y);
+    if (P > 4) return launch_attn_pg<T, HD, 4, kMode, 2>(st, a, grid, cluster_y);
+    if (P > 2) return launch_attn_pg<T, HD, 2, kMode, 2>(st, a, grid, cluster_y);
+    return launch_attn_pg<T, HD, 1, kMode, 2>(st, a, grid, cluster_y);   // one pair: the second warp still stages the V rows
 }
 
 template <typename T> bool launch_attention(cudaStream_t st, const AttnArgs& a) {
