@@ -50,6 +50,8 @@ typedef enum { SB_F32 = 0, SB_BF16 = 1 } sb_dtype;
 #define SB_MAX_LAYERS 64
 
 typedef struct {
+    /* supported: n_layers <= 64, d_model <= 8192 (multiple of 8), head_dim 32 / 64 / 128, n_heads a multiple of
+     * n_kv_heads with at most 4 query heads per KV head, d_ffn a multiple of 8 */
     int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
     float rope_base, rms_eps;
     int32_t dtype;   /* sb_dtype: storage of weights and of the KV cache; arithmetic is fp32 */

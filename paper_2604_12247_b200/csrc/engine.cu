@@ -90,6 +90,8 @@ static bool make_dims(const sb_config* c, Dims* o) {
         c->d_ffn < 8 || c->vocab < 2 || c->max_seq < 1)
         return false;
     if (c->n_heads % c->n_kv_heads) return false;
+    // the attention kernels keep all (row, query head) pairs of a KV head in one CTA's shared memory: 8 rows x 4 heads
+    if (c->n_heads / c->n_kv_heads > 4) return false;
     if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
     if (c->d_model % 8 || c->d_ffn % 8 || c->d_model > 8192) return false;
     if (c->dtype != SB_F32 && c->dtype != SB_BF16) return false;

@@ -31,22 +31,12 @@ constexpr int kStageA = kTileRows * kBK * 2;  // 16 KB
 constexpr int kStageB = 16 * kBK * 2;         // 2 KB
 constexpr int kProducers = 4;                 // producer warps
 constexpr int kTcThreads = (kProducers + 5) * 32;
-// Wide mode (prefill): kWideBlocks blocks of 8 activation rows ride through one launch.  A work item is TWO weight
-// tiles (2 x 128 rows) against one activation tile, so the [256][64] activation tile -- which every CTA has to pull
-// out of L2 -- is read once per 256 weight rows instead of once per 128.  The high and the low halves of an
-// activation row are accumulated into the SAME tensor-memory column (two MMAs per weight tile and k step: the
-// operand descriptor's 8-row-group stride of 2048 bytes walks the high rows, the same + 1024 bytes the low rows), so
-// an accumulator is 128 columns = the 128 prompt rows in order, and two tiles x two buffers fill the 512 columns.
-// A stage is 2 x 16 KB of weights + 32 KB of activations: one CTA per SM with 3 stages and 3 producer warps.
-constexpr int kWideStages = 3;
-constexpr int kWideProducers = 3;
-constexpr int kWideSlabs = 2;
-static int smem_bytes(int stages, int nb = 1) {
-    return stages * ((nb > 1 ? kWideSlabs : 1) * kStageA + nb * kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/;
-}
-static_assert(kWideStages * (kWideSlabs * kStageA + kWideBlocks * kStageB) + 1280 <= 227 * 1024, "wide stages exceed shared memory");
-static_assert(2 * kWideSlabs * 8 * kWideBlocks <= 512, "the wide accumulators exceed tensor memory");
-static_assert(kWideStages >= kWideProducers, "a producer must never lag two barrier phases behind");
+static int smem_bytes(int stages, int nb = 1) { return stages * (kStageA + nb * kStageB) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+// Wide mode (prefill): kWideBlocks blocks of 8 activation rows ride through one launch (MMA N = 16 per block); a stage
+// is 16 KB of weights + 2 KB per block of activations, so one CTA per SM with 4 stages (>= the number of producers).
+constexpr int kWideStages = 4;
+static_assert(kWideStages * (kStageA + kWideBlocks * kStageB) + 1280 <= 227 * 1024, "wide stages exceed shared memory");
+static_assert(2 * 16 * kWideBlocks <= 512, "two wide accumulators exceed tensor memory");
 // Two CTAs per SM (each with its own producers, MMA issuer and TMEM accumulators) stream measurably
 // faster than one CTA with twice the pipeline depth.
 static int g_stages = 6, g_ctas_per_sm = 2;
@@ -63,7 +53,6 @@ struct alignas(64) TcParams {
     int n_off[3];       // first output column of each matrix
     int n_chunks, R, S, KB, n_items;
     int stages;
-    int slabs_per_item;   // weight tiles per work item: 1; wide mode: 2 (chunk counts then count pairs of tiles)
     // L2 prefetch on behalf of a later (pair mode) GEMM whose weights this kernel's idle wait can hide
     CUtensorMap tmN[2];
     int next_half, next_chunks, next_KB, next_every;   // next_every = 0: none
@@ -173,10 +162,10 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 // shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t group_stride = 1024) {
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);
     d |= (uint64_t)1 << 16;              // leading byte offset (unused for swizzled K-major): 16 bytes
-    d |= (uint64_t)(group_stride >> 4) << 32;   // stride byte offset between 8-row groups
+    d |= (uint64_t)(1024 >> 4) << 32;    // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;              // descriptor version of sm_100
     d |= (uint64_t)2 << 61;              // SWIZZLE_128B
     return d;
@@ -195,21 +184,15 @@ __device__ __forceinline__ bool epi_vote(bool ok, volatile int* ok_s, int n_call
 
 struct ItemInfo {
     int mat, row0, kb0, kb1;
-    int n_slabs;   // weight tiles of the item: 1; wide mode: 2, or 1 at the ragged end of a matrix
 };
 __device__ __forceinline__ ItemInfo decode_item(const TcParams& p, int item) {
     int chunk = item % p.n_chunks, s = item / p.n_chunks;
-    const int per = p.slabs_per_item;   // 1, wide mode 2
-    if (p.pair_half) {                  // never split along k
-        const int row0 = chunk * per * p.pair_half;
-        return ItemInfo{0, row0, 0, p.KB, (per == 2 && row0 + p.pair_half < p.n_rows[0]) ? 2 : 1};
-    }
+    if (p.pair_half) return ItemInfo{0, chunk * p.pair_half, 0, p.KB};   // never split along k
     int j = 0, base = 0;
     while (j < p.n_mats - 1 && chunk >= p.chunk_end[j]) base = p.chunk_end[j++];
     ItemInfo it;
     it.mat = j;
-    it.row0 = (chunk - base) * per * p.R;
-    it.n_slabs = (per == 2 && it.row0 + p.R < p.n_rows[j]) ? 2 : 1;
+    it.row0 = (chunk - base) * p.R;
     it.kb0 = (int)((long long)s * p.KB / p.S);
     it.kb1 = (int)((long long)(s + 1) * p.KB / p.S);
     return it;
@@ -237,14 +220,8 @@ struct WorkIter {
 template <bool kHead, bool kPair, int NB = 1>
 __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ TcParams p) {
     static_assert(!kHead || NB == 1, "the LM-head mode handles one block of rows");
-    constexpr bool kWide = NB > 1;
     constexpr int kStageBn = NB * kStageB;          // activation tile of a stage: 16 operand rows per block
-    constexpr int kStageAn = (kWide ? kWideSlabs : 1) * kStageA;   // weight tile(s) of a stage
-    constexpr int kProd = kWide ? kWideProducers : kProducers;     // producer warps at work
-    // TMEM columns of one weight tile's accumulator: narrow 16 (8 high + 8 low columns); wide 8 per block (the high and
-    // low halves are accumulated into one column)
-    constexpr uint32_t kCols = kWide ? 8u * NB : 16u;
-    constexpr uint32_t kBufCols = (kWide ? kWideSlabs : 1) * kCols;   // columns of one accumulator buffer
+    constexpr uint32_t kCols = 16u * NB;            // TMEM columns of one accumulator
     constexpr uint32_t kIdesc = idesc_n(kCols);
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_s;
@@ -257,7 +234,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
     const int kStages = p.stages;
-    const uint32_t smA = tiles, smB = tiles + kStages * kStageAn;
+    const uint32_t smA = tiles, smB = tiles + kStages * kStageA;
     const uint32_t bars = smB + kStages * kStageBn;            // 8-byte mbarriers
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
@@ -279,19 +256,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kProducers) {   // TMEM: two accumulators of 16 columns per block of rows
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2u * kBufCols));
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2u * kCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
-    // bytes one pipeline fill brings: the item's weight tile(s) + the activation tile
-    auto stage_bytes = [&](const ItemInfo& it) { return (uint32_t)(it.n_slabs * p.R) * (kBK * 2) + kStageBn; };
+    const uint32_t stage_bytes = (uint32_t)p.R * (kBK * 2) + kStageBn;
 
-    if (warp < kProd) {
+    if (warp < kProducers) {
         // ------------------------------ TMA producers ------------------------------
-        // Producer j owns pipeline fills j, j + kProd, ...  The weight tiles of the first
+        // Producer j owns pipeline fills j, j + kProducers, ...  The weight tiles of the first
         // pipeline fill do not depend on the preceding kernel, so they are requested BEFORE the
         // grid-dependency wait; the activation tiles (written by that kernel) follow after it.
         if (lane == 0) {
@@ -300,27 +276,22 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
             }
             const uint64_t pol = policy_evict_first();
-            // weight tile(s) of one pipeline fill; pair mode: gate rows to tile rows 0 .., up rows to tile rows 64 ..;
-            // wide mode: the item's second tile 16 KB further on
+            // weight tile(s) of one pipeline fill; pair mode: gate rows to tile rows 0 .., up rows to tile rows 64 ..
             auto load_a = [&](int st, const WorkIter& wi) {
-                for (int sl = 0; sl < wi.it.n_slabs; ++sl) {
-                    const uint32_t dst = smA + st * kStageAn + sl * kStageA;
-                    if (kPair) {
-                        const int row = wi.it.row0 + sl * p.pair_half;
-                        tma_load_2d_hint(dst, &p.tmA[0], wi.kb * kBK, row, full_bar(st), pol);
-                        tma_load_2d_hint(dst + 64 * kBK * 2, &p.tmA[1], wi.kb * kBK, row, full_bar(st), pol);
-                    } else {
-                        tma_load_2d_hint(dst, &p.tmA[wi.it.mat], wi.kb * kBK, wi.it.row0 + sl * p.R, full_bar(st), pol);
-                    }
+                if (kPair) {
+                    tma_load_2d_hint(smA + st * kStageA, &p.tmA[0], wi.kb * kBK, wi.it.row0, full_bar(st), pol);
+                    tma_load_2d_hint(smA + st * kStageA + 64 * kBK * 2, &p.tmA[1], wi.kb * kBK, wi.it.row0, full_bar(st), pol);
+                } else {
+                    tma_load_2d_hint(smA + st * kStageA, &p.tmA[wi.it.mat], wi.kb * kBK, wi.it.row0, full_bar(st), pol);
                 }
             };
             WorkIter w(p), w0(p);
             for (int j = 0; j < warp; ++j) { w.next(p); w0.next(p); }
             int fill = warp;
-            for (; w.valid() && fill < kStages; fill += kProd) {
-                mbar_expect_tx(full_bar(fill), stage_bytes(w.it));
+            for (; w.valid() && fill < kStages; fill += kProducers) {
+                mbar_expect_tx(full_bar(fill), stage_bytes);
                 load_a(fill, w);
-                for (int j = 0; j < kProd; ++j) w.next(p);
+                for (int j = 0; j < kProducers; ++j) w.next(p);
             }
             // Still waiting for the predecessor kernel, and so will the kernels after this one: HBM would
             // sit idle.  Ask TMA to bring every next_every-th k block of the weights of a GEMM that runs
@@ -328,7 +299,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             // HBM side by side.
             if (p.next_every > 0) {
                 for (int c = blockIdx.x; c < p.next_chunks; c += gridDim.x)
-                    for (int kb = warp * p.next_every; kb < p.next_KB; kb += kProd * p.next_every) {
+                    for (int kb = warp * p.next_every; kb < p.next_KB; kb += kProducers * p.next_every) {
                         asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(&p.tmN[0]), "r"(kb * kBK),
                                      "r"(c * p.next_half)
                                      : "memory");
@@ -338,24 +309,22 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                     }
             }
             pdl_wait();
-            for (int f0 = warp; f0 < fill; f0 += kProd) {
+            for (int f0 = warp; f0 < fill; f0 += kProducers) {
                 tma_load_2d(smB + f0 * kStageBn, &p.tmB, w0.kb * kBK, 0, full_bar(f0));
-                for (int j = 0; j < kProd; ++j) w0.next(p);
+                for (int j = 0; j < kProducers; ++j) w0.next(p);
             }
-            for (; w.valid(); fill += kProd) {
+            for (; w.valid(); fill += kProducers) {
                 int stage = fill % kStages;
                 uint32_t phase = (uint32_t)(fill / kStages) & 1u;
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_s, p.status, 1u)) break;
-                mbar_expect_tx(full_bar(stage), stage_bytes(w.it));
+                mbar_expect_tx(full_bar(stage), stage_bytes);
                 load_a(stage, w);
                 tma_load_2d(smB + stage * kStageBn, &p.tmB, w.kb * kBK, 0, full_bar(stage));
-                for (int j = 0; j < kProd; ++j) w.next(p);
+                for (int j = 0; j < kProducers; ++j) w.next(p);
             }
         } else {
             pdl_wait();
         }
-    } else if (warp < kProducers) {
-        pdl_wait();   // wide mode: a producer warp without work
     } else if (warp == kProducers) {
         // ------------------------------ MMA issuer ------------------------------
         pdl_wait();
@@ -368,28 +337,14 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
                 uint32_t use = (uint32_t)(n_local >> 1);   // how often this accumulator was used before
                 if (!(ok = mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, &abort_s, p.status, 2u))) break;
                 tc_fence_after();
-                uint32_t d_tmem = tmem_base + (uint32_t)buf * kBufCols;
+                uint32_t d_tmem = tmem_base + (uint32_t)buf * kCols;
                 for (int kb = it.kb0; kb < it.kb1; ++kb) {
                     if (!(ok = mbar_wait(full_bar(stage), phase, &abort_s, p.status, 3u))) break;
                     tc_fence_after();
-                    if constexpr (kWide) {
-                        // operand rows 16b .. 16b+7 = high halves of block b, 16b+8 .. = low halves: a group stride of
-                        // 2048 bytes walks one kind; both kinds go into the same accumulator column
-                        const uint64_t db_hi = smem_desc(smB + stage * kStageBn, 2048), db_lo = smem_desc(smB + stage * kStageBn + 1024, 2048);
+                    uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageBn);
 #pragma unroll
-                        for (int k = 0; k < kBK / 16; ++k) {
-                            for (int sl = 0; sl < it.n_slabs; ++sl) {
-                                const uint64_t da = smem_desc(smA + stage * kStageAn + sl * kStageA);
-                                tc_mma(d_tmem + (uint32_t)sl * kCols, da + 2u * k, db_hi + 2u * k, kIdesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
-                                tc_mma(d_tmem + (uint32_t)sl * kCols, da + 2u * k, db_lo + 2u * k, kIdesc, 1u);
-                            }
-                        }
-                    } else {
-                        uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageBn);
-#pragma unroll
-                        for (int k = 0; k < kBK / 16; ++k)   // +32 bytes per 16-element k step inside the swizzle row
-                            tc_mma(d_tmem, da + 2u * k, db + 2u * k, kIdesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
-                    }
+                    for (int k = 0; k < kBK / 16; ++k)   // +32 bytes per 16-element k step inside the swizzle row
+                        tc_mma(d_tmem, da + 2u * k, db + 2u * k, kIdesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
                     tc_commit(empty_bar(stage));          // frees the stage once these MMAs have read it
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
@@ -417,61 +372,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
             if (kPair) ok = epi_vote(ok, ok_s, n_local, q, lane);   // the pair epilogue synchronises the four warps
             if (!ok) break;
             tc_fence_after();
-            if constexpr (kWide) {
-                // wide mode: column c of a tile's accumulator = prompt row c (block c / 8, row c % 8), high + low already
-                // summed by the tensor core; 16 columns per load = two blocks of 8 rows
-                const int s_split = item / p.n_chunks;
-                for (int sl = 0; sl < it.n_slabs; ++sl) {
-                    for (int g = 0; g < (int)kCols / 16; ++g) {
-                        uint32_t v[16];
-                        tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * kBufCols + (uint32_t)sl * kCols + (uint32_t)g * 16u, v);
-                        if (sl == it.n_slabs - 1 && g == (int)kCols / 16 - 1) {
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(tempty_bar(buf));   // accumulator may be overwritten
-                        }
-#pragma unroll
-                        for (int hb = 0; hb < 2; ++hb) {
-                            const int blk = 2 * g + hb, row_base = blk * kMaxW;   // this block of 8 rows
-                            if (kPair) {
-                                // warps 2-3 hold the up projections (tile rows 64 ..): hand them to the thread that holds the
-                                // gate projection of the same column, which writes silu(gate) * up as the next GEMM's operand
-                                if (q >= 2) {
-#pragma unroll
-                                    for (int i = 0; i < kMaxW; ++i) up_s[i * 64 + (row_in_tile - 64)] = __uint_as_float(v[8 * hb + i]);
-                                }
-                                asm volatile("bar.sync 1, 128;" ::: "memory");
-                                const int col = it.row0 + sl * p.pair_half + row_in_tile;
-                                if (q < 2 && row_in_tile < p.pair_half && col < p.n_rows[0]) {
-                                    const size_t F = (size_t)p.n_rows[0];
-                                    __nv_bfloat16* dst = p.swiglu_out + (size_t)blk * 16 * F;   // [16][F] per block: high halves, low halves
-#pragma unroll
-                                    for (int i = 0; i < kMaxW; ++i) {
-                                        if (row_base + i >= p.r0 && row_base + i < p.r0 + p.m) {
-                                            const float gt = __uint_as_float(v[8 * hb + i]), u = up_s[i * 64 + row_in_tile];
-                                            const float val = gt / (1.f + expf(-gt)) * u;
-                                            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
-                                            dst[(size_t)i * F + col] = hi;
-                                            dst[(size_t)(i + 8) * F + col] = __float2bfloat16_rn(val - __bfloat162float(hi));
-                                        }
-                                    }
-                                }
-                                asm volatile("bar.sync 1, 128;" ::: "memory");   // up_s may be overwritten by the next block / item
-                            } else {
-                                const int n = it.row0 + sl * p.R + row_in_tile;
-                                if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
-#pragma unroll
-                                    for (int i = 0; i < kMaxW; ++i) {
-                                        if (row_base + i >= p.r0 && row_base + i < p.r0 + p.m)   // split-K partials [block][split][8][n_total]
-                                            p.out[(((size_t)blk * p.S + s_split) * kMaxW + i) * p.n_total + p.n_off[it.mat] + n] = __uint_as_float(v[8 * hb + i]);
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
-                continue;
-            }
             for (int blk = 0; blk < NB; ++blk) {           // one block of 8 activation rows = 16 accumulator columns
                 uint32_t v[16];
                 tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * kCols + (uint32_t)blk * 16u, v);
@@ -553,7 +453,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
     __syncthreads();
     if (warp == kProducers) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kBufCols));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kCols));
     }
     if (!kHead) return;
 
@@ -619,17 +519,16 @@ static int sm_count() { return device_sm_count(); }
 
 // Slab height R (multiple of 8 in [64,128]) and split count S that minimise what the busiest
 // CTA streams.  Depends on the shape only, never on the number of rows.
-// `per` = weight tiles per work item (wide mode: 2; an item then streams up to 2 R rows).
-static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int per, int* R_out, int* S_out) {
+static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out) {
     double best = 1e300;
     int bR = 128, bS = 1;
     for (int S = 1; S <= max_split && S <= KB; ++S)
         for (int R = 128; R >= 64; R -= 8) {
             long long chunks = 0;
-            for (int j = 0; j < n_mats; ++j) chunks += ((n_rows[j] + R - 1) / R + per - 1) / per;
+            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + R - 1) / R;
             long long items = chunks * S;
-            long long rounds = (items + G - 1) / G;
-            double cost = (double)rounds * per * R * ((KB + S - 1) / S) * (1.0 + 0.001 * g_split_penalty_pm * S);   // each split adds partial traffic and consumer loads
+            long long per = (items + G - 1) / G;
+            double cost = (double)per * R * ((KB + S - 1) / S) * (1.0 + 0.001 * g_split_penalty_pm * S);   // each split adds partial traffic and consumer loads
             if (cost < best - 1e-9) { best = cost; bR = R; bS = S; }
         }
     *R_out = bR;
@@ -637,12 +536,12 @@ static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, i
 }
 
 // Pair mode: rows of each kind per item (multiple of 8 in [32,64]) that minimise what the busiest CTA streams.
-static int choose_pair_half(int n_rows, int G, int per) {
+static int choose_pair_half(int n_rows, int G) {
     double best = 1e300;
     int bh = 64;
     for (int h = 64; h >= 32; h -= 8) {
-        long long items = ((n_rows + h - 1) / h + per - 1) / per;
-        double cost = (double)((items + G - 1) / G) * h * per;
+        long long items = (n_rows + h - 1) / h;
+        double cost = (double)((items + G - 1) / G) * h;
         if (cost < best - 1e-9) { best = cost; bh = h; }
     }
     return bh;
@@ -663,23 +562,21 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     TcParams& p = pl->p;
     int G = sm_count() * (nb > 1 ? 1 : g_ctas_per_sm);
     p.stages = nb > 1 ? kWideStages : g_stages;
-    const int per = nb > 1 ? kWideSlabs : 1;   // weight tiles per work item
-    p.slabs_per_item = per;
     p.n_mats = n_mats;
     p.KB = (K + kBK - 1) / kBK;
     int prev = 0;
     for (int j = 0; j < n_mats; ++j) { p.n_rows[j] = n_end[j] - prev; p.n_off[j] = prev; prev = n_end[j]; }
     int chunks = 0;
     if (pair) {
-        p.pair_half = choose_pair_half(p.n_rows[0], G, per);
+        p.pair_half = choose_pair_half(p.n_rows[0], G);
         p.R = 2 * p.pair_half;
         p.S = 1;
-        chunks = ((p.n_rows[0] + p.pair_half - 1) / p.pair_half + per - 1) / per;
+        chunks = (p.n_rows[0] + p.pair_half - 1) / p.pair_half;
         for (int j = 0; j < 3; ++j) p.chunk_end[j] = chunks;
     } else {
-        choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, per, &p.R, &p.S);
+        choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
         for (int j = 0; j < 3; ++j) {
-            if (j < n_mats) chunks += ((p.n_rows[j] + p.R - 1) / p.R + per - 1) / per;
+            if (j < n_mats) chunks += (p.n_rows[j] + p.R - 1) / p.R;
             p.chunk_end[j] = chunks;
         }
     }

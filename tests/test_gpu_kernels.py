@@ -242,6 +242,50 @@ def test_layer_under_fusion_and_prefetch_options(shape):
         assert np.abs(a[0] - b[0]).max() <= 1e-5 * np.abs(b[0]).max()
 
 
+@pytest.mark.parametrize("first_pos,m", [(40, 5), (1100, 3)])
+def test_layer_chain_equals_single_layer_calls(first_pos, m):
+    """sb_k_layer_chain (n layers in one launch sequence, optionally with the rotation-angle table of sb_k_rope_table) gives
+    bit for bit what n successive sb_k_layer calls give: hidden rows and the K/V rows appended to every layer's cache."""
+    shape = inputs.scaled(LAYER_HD128, name="chain-hd128", n_layers=3)
+    w = inputs.make_weights(shape, 25, std=0.05)
+    page, max_seq = 16, 1200
+    kvd = shape.n_kv_heads * shape.head_dim
+    cfg = binding.make_config(shape, max_seq, page)
+    n_pages = (max_seq + page - 1) // page
+    pt = torch.arange(n_pages, dtype=torch.int32, device="cuda")
+    hist = [inputs.make_kv(max_seq, kvd, 40 + l, shape.dtype) for l in range(shape.n_layers)]
+    assert n_pages * page == max_seq
+
+    def caches():   # fresh per-layer caches holding the history
+        return ([k.reshape(n_pages, page, kvd).clone().cuda() for k, _ in hist],
+                [v.reshape(n_pages, page, kvd).clone().cuda() for _, v in hist])
+
+    lws = [{k: v.cuda() for k, v in lw.items()} for lw in w["layers"]]
+    h0 = inputs.make_hidden(m, shape.d_model, 91).cuda()
+    binding.set_default_gemm(1)
+    try:
+        sc = binding.KernelScratch(cfg)
+        kc1, vc1 = caches()
+        h1 = h0.clone()
+        for l in range(shape.n_layers):
+            binding.k_layer(cfg, lws[l], h1, kc1[l], vc1[l], pt, first_pos, sc)
+        torch.cuda.synchronize()
+        tab = binding.k_rope_table(cfg)
+        for table in (None, tab):
+            kc2, vc2 = caches()
+            h2 = h0.clone()
+            binding.k_layer_chain(cfg, binding.LayerChain(lws, kc2, vc2), h2, pt, first_pos, sc, table)
+            torch.cuda.synchronize()
+            assert torch.equal(h1, h2)
+            for l in range(shape.n_layers):
+                assert torch.equal(kc1[l], kc2[l]) and torch.equal(vc1[l], vc2[l])
+    finally:
+        binding.set_default_gemm(-1)
+    with pytest.raises(binding.SBError) as e:
+        binding.k_layer_chain(cfg, binding.LayerChain(lws, kc2, vc2), h2, pt, max_seq - 1, sc, None)   # rows past max_seq
+    assert e.value.status == -3
+
+
 def test_layer_rejects_bad_arguments():
     shape = LAYER_BF16
     w = inputs.make_weights(shape, 23)
