@@ -273,7 +273,18 @@ def damped_arm(args, peak: float) -> dict:
     ar_value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in ars) * 1e-6)
     ach, _, uni_steps, uni_us = verify_roofline(s, [r["stats"] for r in stats], peak)
     st = stats[-1]["stats"]
+    # the same with the probe-layer mask that did best in the hyper-parameter study: only every second layer is tested
+    tau_m = [t if l % 2 == 0 else 0.0 for l, t in enumerate(run.tau, start=1)]
+    ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, tau_m, run.threshold)
+    masked = [ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, tau_m, run.threshold) for _ in range(steps)]
+    m_value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in masked) * 1e-6)
+    mst = masked[-1]["stats"]
     out = {"workload": workload_config(run, "single GPU"), "steps": steps, "value": value, "unit": "tokens/s",
+           "every_second_layer_probed": {"value": m_value, "speedup_vs_ar": m_value / ar_value,
+                                         "tokens_equal_ar": bool(np.array_equal(masked[-1]["tokens"], ars[-1]["tokens"])),
+                                         "emitted_per_round": mst.emitted / max(mst.rounds, 1), "probes_per_step": mst.probes,
+                                         "tau": [round(t, 4) for t in tau_m]},
+           "probes_per_step": st.probes,
            "ar_tokens_per_s": ar_value, "speedup_vs_ar": value / ar_value,
            "tokens_equal_ar": bool(np.array_equal(stats[-1]["tokens"], ars[-1]["tokens"])),
            "emitted_per_round": st.emitted / max(st.rounds, 1), "accepted_drafts_per_round": st.accepted_drafts / max(st.rounds, 1),
