@@ -252,19 +252,19 @@ def oracle_check(ctx, run: inputs.Run, weights_cpu: dict, n_prompt: int, n_gen: 
                     "not below twice the tolerance"}
 
 
-def damped_arm(args, peak: float) -> dict:
-    """The labelled addition `7b-damped` (damped deep layers: the synthetic stand-in for trained exit heads, with the
-    paper's own hyper-parameters), measured the same way as the main workload for a few steps: the configuration in
-    which drafts get accepted."""
+def side_arm(args, workload: str, peak: float, masked: bool = False, steps: int = 3) -> dict:
+    """Another workload measured the same way as the main one, for a few steps, as extra keys of the default run's
+    line: `7b-damped` (damped deep layers: the synthetic stand-in for trained exit heads, with the paper's own
+    hyper-parameters -- the configuration in which drafts get accepted; also with the probe-layer mask that did best in
+    the hyper-parameter study) and the other full-size shapes (`l3-8b`, `13b`) at their own lengths."""
     from paper_2604_12247_b200 import binding
-    run = inputs.RUNS["7b-damped"]
+    run = inputs.RUNS[workload]
     s = run.shape
     w = inputs.make_weights(s, run.seed, device="cuda", damp_rho=run.damp_rho)
     prompt = inputs.make_prompt(s, run.n_prompt, run.seed).numpy()
     ctx = binding.Context(s, w, run.n_prompt + run.n_gen + run.w_max + 8, kv_page=64)
-    steps = max(1, min(args.steps, 3))
-    for _ in range(2):
-        ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold)
+    steps = max(1, min(args.steps, steps))
+    ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold)
     ctx.generate_ar(prompt, 32)
     stats = [ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold) for _ in range(steps)]
     ars = [ctx.generate_ar(prompt, run.n_gen) for _ in range(steps)]
@@ -273,23 +273,26 @@ def damped_arm(args, peak: float) -> dict:
     ar_value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in ars) * 1e-6)
     ach, _, uni_steps, uni_us = verify_roofline(s, [r["stats"] for r in stats], peak)
     st = stats[-1]["stats"]
-    # the same with the probe-layer mask that did best in the hyper-parameter study: only every second layer is tested
-    tau_m = [t if l % 2 == 0 else 0.0 for l, t in enumerate(run.tau, start=1)]
-    ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, tau_m, run.threshold)
-    masked = [ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, tau_m, run.threshold) for _ in range(steps)]
-    m_value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in masked) * 1e-6)
-    mst = masked[-1]["stats"]
+    wb = inputs.weight_bytes(s)
+    probe_us = sum(r["stats"].us_probe_kernels for r in stats) / max(sum(r["stats"].probes_timed for r in stats), 1)
     out = {"workload": workload_config(run, "single GPU"), "steps": steps, "value": value, "unit": "tokens/s",
-           "every_second_layer_probed": {"value": m_value, "speedup_vs_ar": m_value / ar_value,
-                                         "tokens_equal_ar": bool(np.array_equal(masked[-1]["tokens"], ars[-1]["tokens"])),
-                                         "emitted_per_round": mst.emitted / max(mst.rounds, 1), "probes_per_step": mst.probes,
-                                         "tau": [round(t, 4) for t in tau_m]},
-           "probes_per_step": st.probes,
            "ar_tokens_per_s": ar_value, "speedup_vs_ar": value / ar_value,
            "tokens_equal_ar": bool(np.array_equal(stats[-1]["tokens"], ars[-1]["tokens"])),
            "emitted_per_round": st.emitted / max(st.rounds, 1), "accepted_drafts_per_round": st.accepted_drafts / max(st.rounds, 1),
-           "exit_hist": list(st.exit_hist[:run.d_max + 1]), "width_hist": list(st.width_hist),
-           "roofline_frac": ach / peak, "verify_us_per_layer": uni_us / max(uni_steps, 1)}
+           "probes_per_step": st.probes, "exit_hist": list(st.exit_hist[:run.d_max + 1]), "width_hist": list(st.width_hist),
+           "ttft_ms": st.us_prefill / 1e3,
+           "roofline_frac": ach / peak, "verify_us_per_layer": uni_us / max(uni_steps, 1),
+           "roofline_exit_frac": wb["head"] / (probe_us * 1e-6) / 1e9 / peak if probe_us > 0 else None}
+    if masked:   # only every second layer is tested for an exit
+        tau_m = [t if l % 2 == 0 else 0.0 for l, t in enumerate(run.tau, start=1)]
+        ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, tau_m, run.threshold)
+        runs = [ctx.generate(prompt, run.n_gen, run.d_max, run.w_max, tau_m, run.threshold) for _ in range(steps)]
+        m_value = steps * dec_tok / (sum(r["stats"].us_decode_dev for r in runs) * 1e-6)
+        mst = runs[-1]["stats"]
+        out["every_second_layer_probed"] = {"value": m_value, "speedup_vs_ar": m_value / ar_value,
+                                            "tokens_equal_ar": bool(np.array_equal(runs[-1]["tokens"], ars[-1]["tokens"])),
+                                            "emitted_per_round": mst.emitted / max(mst.rounds, 1), "probes_per_step": mst.probes,
+                                            "tau": [round(t, 4) for t in tau_m]}
     ctx.close()
     return out
 
@@ -410,7 +413,9 @@ def product_arm(args, run: inputs.Run):
         del wc
     ctx.close()
     if world == 1 and args.workload == "7b" and not args.no_damped:
-        line["damped"] = damped_arm(args, peak)
+        line["damped"] = side_arm(args, "7b-damped", peak, masked=True)
+        if not args.no_other_shapes:
+            line["other_shapes"] = {name: side_arm(args, name, peak, steps=1) for name in ("l3-8b", "13b")}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -705,7 +710,8 @@ def main():
     ap.add_argument("--n-gen", type=int, default=None, help="override the number of generated tokens")
     ap.add_argument("--n-prompt", type=int, default=None, help="override the prompt length (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the legs that run the CPU oracle (cpu_baseline, oracle_check)")
-    ap.add_argument("--no-damped", action="store_true", help="skip the extra 7b-damped measurement of the default run")
+    ap.add_argument("--no-damped", action="store_true", help="skip the extra workloads of the default run (7b-damped, l3-8b, 13b)")
+    ap.add_argument("--no-other-shapes", action="store_true", help="skip the l3-8b and 13b measurements of the default run")
     ap.add_argument("--oracle-check-tokens", type=int, default=96,
                     help="tokens of the short-prompt generation the oracle checks teacher-forced (0 = skip)")
     ap.add_argument("--micro", action="store_true", help="kernel micro-benchmarks instead of the generation benchmark")
