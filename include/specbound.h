@@ -307,9 +307,10 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                    (they write scratch only; on an exit they are discarded).  Results do not depend on it.
  *   SB_OPT_WIDE_PREFILL (default option only) 1 (default) = sb_prefill of a bf16 model on the tcgen05 path (with the
  *                    SwiGLU epilogue on) sends up to 128 prompt rows per pass through the weight-streaming GEMMs (the
- *                    weights are read once per 128 rows) and the fewer than 16 rows left over through 8-row passes;
- *                    0 = 8-row passes only.  Both are deterministic; they may differ in the split-K summation order,
- *                    i.e. in the last bits of the K/V cache and of the first token's logits. */
+ *                    weights are read once per 128 rows), with a tiled causal attention kernel on the tensor cores, and
+ *                    the fewer than 16 rows left over through 8-row passes; 2 = the same passes with the decode attention
+ *                    kernels (a block of 8 rows at a time); 0 = 8-row passes only.  All are deterministic; they may differ
+ *                    in summation order, i.e. in the last bits of the K/V cache and of the first token's logits. */
 enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,
        SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7, SB_OPT_QKV_AHEAD = 8, SB_OPT_WIDE_PREFILL = 9 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);

@@ -367,7 +367,13 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
         launch_rope_append<T>(e.st, ra);
         e.launches++;
         const int n_full = M / kMaxW, rem = M - n_full * kMaxW;
-        if (n_full > 0) {
+        // tiled causal attention on the tensor cores: one launch for all rows of the pass
+        bool tiled = false;
+        if (g_wide_prefill == 1 && (D.hd == 64 || D.hd == 128))
+            tiled = launch_attention_prefill(e.st, W.pf_q, k_cache_l, v_cache_l, W.page_table, W.pf_act_o, D.H, D.Hkv, D.hd, D.page,
+                                             D.page_shift, pos0, M);
+        if (tiled) e.launches++;
+        if (!tiled && n_full > 0) {
             AttnArgs aa{W.pf_q, k_cache_l, v_cache_l, W.page_table, W.pf_attn_part, W.pf_act_o, D.H, D.Hkv, D.hd, D.page,
                         D.page_shift, pos0, 0, kMaxW, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
             aa.n_blocks = n_full;
@@ -376,7 +382,7 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
             if (!launch_attention<T>(e.st, aa)) e.err = SB_ERR_UNSUPPORTED;
             e.launches += 2;
         }
-        if (rem > 0) {
+        if (!tiled && rem > 0) {
             AttnArgs aa{W.pf_q + (size_t)n_full * kMaxW * D.qd, k_cache_l, v_cache_l, W.page_table,
                         W.pf_attn_part + (size_t)n_full * W.pf_attn_stride, act_of(W.pf_act_o, n_full, D.qd), D.H, D.Hkv, D.hd,
                         D.page, D.page_shift, pos0 + n_full * kMaxW, 0, rem, D.chunk, nullptr, 0, W.rope_tab, W.status, {}};
@@ -714,7 +720,7 @@ int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_L2_PREFETCH) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_QKV_AHEAD) { g_qkv_ahead = value != 0; return SB_OK; }
-    if (key == SB_OPT_WIDE_PREFILL) { g_wide_prefill = value != 0; return SB_OK; }
+    if (key == SB_OPT_WIDE_PREFILL) { if (value < 0 || value > 2) return SB_ERR_ARG; g_wide_prefill = value; return SB_OK; }
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
     if (key == SB_OPT_FUSE) { if (value < 0 || value > 3) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;

@@ -416,6 +416,11 @@ template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArg
 // launch_attention.  Returns false without launching if the shape is not covered.
 template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a);
 template <typename T> void launch_attention_combine(cudaStream_t st, const AttnArgs& a);
+// Tiled causal attention of a wide prefill pass on the tensor cores (attn_prefill.cu; bf16 caches, head_dim 64 or 128):
+// q [M][H * hd] fp32 rotated queries of the rows at positions pos0 .., whose K/V rows are in the cache already;
+// act_out: the output projection's operand in the block-major layout of the wide GEMMs.  false: shape not covered.
+bool launch_attention_prefill(cudaStream_t st, const float* q, const void* k_cache, const void* v_cache, const int* page_table,
+                              void* act_out, int H, int Hkv, int hd, int page, int page_shift, int pos0, int M);
 template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int n_split, int F, void* act, int r0, int m);
 void launch_accept(cudaStream_t st, const int* g, const int* drafts8, int w, int max_emit, int* result, const Mirror& mirror);
 bool launch_sample(cudaStream_t st, const SampleArgs& a);   // false: the cluster launch was refused

@@ -29,8 +29,10 @@ def _hidden_after_prefill(ctx, prompt, n_layers):
 
 # 16: the smallest wide pass; 64, 70, 100: one ragged wide pass (70 and 100 end in a partial block of 8 rows); 128: a
 # whole pass; 130: a whole pass + 2 rows through an 8-row pass; 300: two whole passes and a ragged one.  Page size 16
+# wide_mode 1: the tiled tensor-core attention kernel of the wide passes (the default); 2: the decode attention kernels
+@pytest.mark.parametrize("wide_mode", [1, 2])
 @pytest.mark.parametrize("n_prompt", [16, 64, 70, 100, 128, 130, 300])
-def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt):
+def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt, wide_mode):
     shape = SMALL_BF16
     w = inputs.make_weights(shape, 5, damp_rho=0.3)
     pr = inputs.make_prompt(shape, n_prompt, 17).numpy()
@@ -44,10 +46,14 @@ def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt):
         ar_n = ctx_n.generate_ar(pr, 12)["tokens"]
         ctx_n.close()
     finally:
+        assert binding.lib().sb_set_default_option(OPT_WIDE_PREFILL, wide_mode) == 0
+    try:
+        ctx, _ = gpu_ctx(shape, w, max_seq, gemm=1)
+        first, hid = _hidden_after_prefill(ctx, pr, L)
+        res = ctx.generate_ar(pr, 12)
+        sp = ctx.generate(pr, 12, 2, 4, inputs.tau_linear(2, 1.5, 1.0), 0.3)
+    finally:
         assert binding.lib().sb_set_default_option(OPT_WIDE_PREFILL, 1) == 0
-    ctx, _ = gpu_ctx(shape, w, max_seq, gemm=1)
-    first, hid = _hidden_after_prefill(ctx, pr, L)
-    res = ctx.generate_ar(pr, 12)
     ar = res["tokens"]
     assert res["stats"].kernel_launches < launches_n          # the wide passes really ran
     # against the 8-row passes: the same arithmetic up to the split-K summation order
@@ -68,7 +74,6 @@ def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt):
     if n_off == 0:
         assert np.array_equal(ar, ar_n)
     # speculative decoding from the same cache equals autoregressive decoding, bit for bit
-    sp = ctx.generate(pr, 12, 2, 4, inputs.tau_linear(2, 1.5, 1.0), 0.3)
     assert np.array_equal(sp["tokens"], ar)
     ctx.close()
 
