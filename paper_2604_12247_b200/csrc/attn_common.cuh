@@ -54,6 +54,34 @@ template <> __device__ __forceinline__ void load_channels<__nv_bfloat16, 4>(cons
     f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
 }
 
+// ---- rotary embedding: rotate-half pairing (i, i + hd/2), angle = pos * base^(-2i/hd) ----
+// cos and sin of the angle pos * inv_freq[i]
+__device__ __forceinline__ float2 rope_cos_sin(const double* inv_freq, int pos, int i) {
+    // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
+    // the fp32 sincos sees a small argument
+    double ang = (double)pos * inv_freq[i];
+    ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+    float s, c;
+    sincosf((float)ang, &s, &c);
+    return make_float2(c, s);
+}
+// cos/sin of the angle of rotation pair i at position pos; tab (nullable) = rope_cos_sin tabulated as
+// [position][hd/2] by k_rope_table: the same values, one load instead of the math
+__device__ __forceinline__ float2 rope_fetch(const double* inv_freq, const float2* __restrict__ tab, int half, int pos, int i) {
+    return tab ? __ldg(tab + (size_t)pos * half + i) : rope_cos_sin(inv_freq, pos, i);
+}
+// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head
+__device__ __forceinline__ void rope_apply(float2 cs, float& x0, float& x1) {
+    // explicit roundings: the compiler must not contract these into fused multiply-adds differently at
+    // different call sites (the separate and the fused kernels have to agree bit for bit)
+    float y0 = __fsub_rn(__fmul_rn(x0, cs.x), __fmul_rn(x1, cs.y)), y1 = __fadd_rn(__fmul_rn(x1, cs.x), __fmul_rn(x0, cs.y));
+    x0 = y0;
+    x1 = y1;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // 1 / sqrt(head_dim) as every kernel forms it
 __device__ __forceinline__ float attn_score_scale(int hd) { return rsqrtf((float)hd); }
 

@@ -110,29 +110,6 @@ void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split
 // write q (fp32) and append k, v to the paged cache in the storage dtype.
 // grid = (H + 2 Hkv, m), block = hd/2 threads (one rotation pair each).
 // ------------------------------------------------------------------------------------------------
-// cos and sin of the angle pos * inv_freq[i]
-__device__ __forceinline__ float2 rope_cos_sin(const double* inv_freq, int pos, int i) {
-    // the angle is formed and reduced to [-pi, pi] in fp64 (exact for every position), then
-    // the fp32 sincos sees a small argument
-    double ang = (double)pos * inv_freq[i];
-    ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
-    float s, c;
-    sincosf((float)ang, &s, &c);
-    return make_float2(c, s);
-}
-// cos/sin of the angle of rotation pair i at position pos; tab (nullable) = rope_cos_sin tabulated as
-// [position][hd/2] by k_rope_table: the same values, one load instead of the math
-__device__ __forceinline__ float2 rope_fetch(const double* inv_freq, const float2* __restrict__ tab, int half, int pos, int i) {
-    return tab ? __ldg(tab + (size_t)pos * half + i) : rope_cos_sin(inv_freq, pos, i);
-}
-// rotate the pair (x0, x1) = elements (i, i + hd/2) of a head
-__device__ __forceinline__ void rope_apply(float2 cs, float& x0, float& x1) {
-    // explicit roundings: the compiler must not contract these into fused multiply-adds differently at
-    // different call sites (the separate and the fused kernels have to agree bit for bit)
-    float y0 = __fsub_rn(__fmul_rn(x0, cs.x), __fmul_rn(x1, cs.y)), y1 = __fadd_rn(__fmul_rn(x1, cs.x), __fmul_rn(x0, cs.y));
-    x0 = y0;
-    x1 = y1;
-}
 struct RopeFreq { double inv_freq[64]; };
 __global__ void k_rope_table(float2* tab, int n_pos, int half, RopeFreq f) {
     int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -196,13 +173,13 @@ template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a
 constexpr int kMaxPairGroup = 8;
 
 // Shared-memory layout of k_attn_partial: rotated queries [Ppad][HD] fp32 | K tiles [4][32][padded row] | V tiles
-// [4][32][row] | probabilities per warp [PG][32] | block partials [4][Ppad][HD+2] | (mode 1) chunk partial [Ppad][HD+2].
+// [4][32][row] | probabilities per warp [PG][32] | block partials [4][Ppad][HD+2].
 // Where it fits, a block's partial is written over the block's own K tile once its warps are done with the scores.
 struct AttnLayout {
     int Ppad, rowb_k, rowb_v;
-    size_t off_k, off_v, off_p, off_mrg, off_out, total;
+    size_t off_k, off_v, off_p, off_mrg, total;
     bool alias;
-    __host__ __device__ AttnLayout(int P, int HD, int elt, int PG, int WPB, bool want_out) {
+    __host__ __device__ AttnLayout(int P, int HD, int elt, int PG, int WPB) {
         Ppad = (P + PG - 1) / PG * PG;
         rowb_k = HD * elt + 16;      // padded pitch: lane-per-row 16-byte reads of K are conflict-free
         rowb_v = HD * elt;           // V is read a whole row per warp
@@ -212,8 +189,7 @@ struct AttnLayout {
         off_mrg = off_p + (size_t)kPosWarps * WPB * PG * 32 * 4;
         // only where every warp makes at most one sweep: a second sweep would read the K tile again
         alias = (size_t)Ppad * (HD + 2) * 4 <= (size_t)32 * rowb_k && Ppad / PG <= WPB;
-        off_out = off_mrg + (alias ? 0 : (size_t)kPosWarps * Ppad * (HD + 2) * 4);
-        total = off_out + (want_out ? (size_t)Ppad * (HD + 2) * 4 : 0);
+        total = off_mrg + (alias ? 0 : (size_t)kPosWarps * Ppad * (HD + 2) * 4);
     }
 };
 
@@ -222,21 +198,14 @@ struct AttnLayout {
 // run-time predicates and each K element is unpacked once for up to 8 pairs.
 // WPB = warps per 32-position block: 1 (the warp takes every pair; up to 8 pairs) or 2 (the groups of 8 pairs are
 // split between two warps; grouped-query models with several rows).
-// kMode 0: the rotated queries and every cached row come from memory (launch_rope_append ran before); chunk
-//          partials go to global memory for k_attn_combine.
-// kMode 1: the kernel also does what precedes and follows it.  q is summed from the QKV split-K partials and rotated
-//          here (every chunk CTA redoes it: a few hundred values); the CTA whose chunk holds the new positions sums,
-//          rotates and rounds their K and V, appends them to the cache and puts them straight into its staged tile;
-//          the chunk CTAs of a KV head form one thread-block cluster (grid.y = cluster size = number of chunks <= 8)
-//          and merge the chunk partials, read from one another's shared memory, in chunk order.
-// kMode 2: the front end of mode 1, the partials to global memory (contexts of more than 8 chunks).
-// Same arithmetic in the same order in every mode: bit-identical results.
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-template <typename T, int HD, int PG, int kMode, int WPB>
+// kFront false: the rotated queries and every cached row come from memory (launch_rope_append ran before).
+// kFront true : the kernel also does what precedes it.  q is summed from the QKV split-K partials and rotated here
+//          (every chunk CTA redoes it: a few hundred values); the CTA whose chunk holds the new positions sums,
+//          rotates and rounds their K and V, appends them to the cache and puts them straight into its staged tile.
+// The chunk partials go to global memory for k_attn_combine.  Same arithmetic in the same order in both forms and in
+// the one-launch cluster kernel of the short contexts (attn_cluster.cu): bit-identical results.
+template <typename T, int HD, int PG, bool kFront, int WPB>
 __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs a) {
-    constexpr bool kFront = kMode != 0, kCluster = kMode == 1;
     constexpr int kPairGroup = PG;
     constexpr int E = HD / 32;                       // channels per lane in P.V
     constexpr int EPP = 16 / (int)sizeof(T);         // elements per 16-byte piece
@@ -245,7 +214,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
     const int kvh = blockIdx.x, c = blockIdx.y;
-    const int pos_pred0 = a.pos_pred0 >= 0 ? a.pos_pred0 : a.pos0 + a.r0;   // mode 0: first position the preceding RoPE/append launch wrote
+    const int pos_pred0 = a.pos_pred0 >= 0 ? a.pos_pred0 : a.pos0 + a.r0;   // separate form: first position the preceding RoPE/append launch wrote
     if (!kFront && a.n_blocks > 1) {                 // several blocks of 8 rows in one launch: this CTA's block
         const int blk = blockIdx.z;
         a.q += (size_t)blk * kMaxW * a.H * HD;
@@ -258,7 +227,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     const int g_shift = (G & (G - 1)) == 0 ? __ffs(G) - 1 : -1;   // G is 1, 2 or 4 in practice: a shift instead of a division
     auto row_of = [&](int p) { return g_shift >= 0 ? p >> g_shift : p / G; };
     const int kvd = a.Hkv * HD, qd = a.H * HD;
-    const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB, kCluster);
+    const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const int Ppad = lay.Ppad;
     float* q_s = reinterpret_cast<float*>(smem);                                   // [Ppad][HD]
     unsigned char* k_tiles = smem + lay.off_k;
@@ -272,7 +241,6 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         return lay.alias ? reinterpret_cast<float*>(k_tiles + (size_t)w * 32 * ROWB_K)
                          : reinterpret_cast<float*>(smem + lay.off_mrg) + (size_t)w * Ppad * (HD + 2);
     };
-    float* out_s = reinterpret_cast<float*>(smem + lay.off_out);   // mode 1: this chunk's merged partial [Ppad][HD+2]
     const int pos_last = a.pos0 + a.r0 + a.m - 1;
     const int pos_new0 = kFront ? a.pos0 + a.r0 : pos_last + 1;   // first position whose K,V this launch creates
     const int tbase = c * kAttnChunk + v * 32;
@@ -280,7 +248,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     // Rows of EARLIER steps of this layer (positions below pos_done) are complete when this kernel starts: between such
     // steps the stream holds a launch without programmatic overlap (the embedding kernel that starts every step, or
     // the clear of a stateless call).  Their copies -- the long, cold loads of this kernel -- start before the
-    // grid-dependency wait.  Mode 0: the RoPE/append kernel right before this one wrote the rows from
+    // grid-dependency wait.  Separate form: the RoPE/append kernel right before this one wrote the rows from
     // pos_done on; they are staged after the wait.  (The page table is set up when the context is created -- or, for
     // the stateless call, before the call -- and no kernel of a launch sequence writes it: like the weights it may be
     // read before the wait.)
@@ -502,53 +470,13 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 }
             }
         }
-        float* dst = kCluster ? out_s + (size_t)p * (HD + 2)
-                              : a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
+        float* dst = a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
         *reinterpret_cast<float2*>(dst + e) = make_float2(O0, O1);
         if (e == 0) {
             dst[HD] = M;
             dst[HD + 1] = L;
         }
     }
-    if (!kCluster) return;
-    // ---- chunk merge across the cluster (one CTA per chunk of this KV head) ----
-    __syncthreads();
-    cluster_sync_all();   // every chunk's partial is in its CTA's out_s
-    {   // every CTA of the cluster merges its share of the (pair, channel) outputs
-        const uint32_t out_local = (uint32_t)__cvta_generic_to_shared(out_s);
-        constexpr int kBatch = 8;
-        for (int idx = c * blockDim.x + threadIdx.x; idx < P * HD; idx += gridDim.y * blockDim.x) {
-            int p = idx / HD, e = idx - p * HD;
-            int i = row_of(p), g = p - i * G;
-            int row = a.r0 + i;
-            int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own (<= cluster size)
-            float M = -INFINITY, L = 0.f, O = 0.f;
-            float mc[kBatch], lc[kBatch], oc[kBatch];
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                mc[u] = -INFINITY; lc[u] = 0.f; oc[u] = 0.f;
-                if (u < n_chunks) {
-                    uint32_t base;
-                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(base) : "r"(out_local + (uint32_t)(p * (HD + 2)) * 4u), "r"(u));
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mc[u]) : "r"(base + (uint32_t)HD * 4u) : "memory");
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(lc[u]) : "r"(base + (uint32_t)(HD + 1) * 4u) : "memory");
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(oc[u]) : "r"(base + (uint32_t)e * 4u) : "memory");
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                if (mc[u] > -INFINITY) {
-                    float f0, f1;
-                    attn_fold(M, L, mc[u], lc[u], f0, f1);
-                    O = attn_fold_out(O, oc[u], f0, f1);
-                }
-            }
-            using A = Act<T>;
-            A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (kvh * G + g) * HD + e, a.H * HD, attn_finish(O, L));
-        }
-    }
-    __syncthreads();
-    cluster_sync_all();   // a CTA's shared memory stays alive until its peers have read it
 }
 
 // Merge of the chunk partials of one (row, query head): grid = (H, m), 8 warps, lane = hd / 32 channels.
@@ -628,13 +556,12 @@ __global__ void __launch_bounds__(kChunkGroup * 32) k_attn_combine(AttnArgs a) {
     }
 }
 
-// cluster_y = 0: plain launch; > 0: mode 1 as clusters of that many chunk CTAs.  Returns false if the
-// device cannot co-schedule such a cluster (nothing is launched then).
-template <typename T, int HD, int PG, int kMode, int WPB>
-static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
-    auto kernel = k_attn_partial<T, HD, PG, kMode, WPB>;
+// Returns false if the pairs do not fit in shared memory (nothing is launched then).
+template <typename T, int HD, int PG, bool kFront, int WPB>
+static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid) {
+    auto kernel = k_attn_partial<T, HD, PG, kFront, WPB>;
     const int P = a.m * (a.H / a.Hkv);
-    const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB, kMode == 1);
+    const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const dim3 block(kPosWarps * WPB * 32);
     static bool configured[kMaxDevices];             // function attributes are per device
     const int dev = current_device();
@@ -644,34 +571,18 @@ static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, int cl
         configured[dev] = true;
     }
     if (lay.total > 200 * 1024) return false;
-    if (kMode == 1 && cluster_y > 1) {
-        static int fits_dev[kMaxDevices][9];             // per device and cluster size: 0 unknown, 1 yes, -1 no
-        int* fits = fits_dev[dev];
-        if (fits[cluster_y] == 0) {
-            cudaLaunchConfig_t cfg{};
-            cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 200 * 1024;
-            cudaLaunchAttribute at[1];
-            at[0].id = cudaLaunchAttributeClusterDimension;
-            at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = (unsigned)cluster_y; at[0].val.clusterDim.z = 1;
-            cfg.attrs = at; cfg.numAttrs = 1;
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-            fits[cluster_y] = n > 0 ? 1 : -1;
-        }
-        if (fits[cluster_y] < 0) return false;
-    }
-    return launch_kc(kernel, grid, block, lay.total, st, kMode == 1 ? cluster_y : 1, a) == cudaSuccess;
+    return launch_kc(kernel, grid, block, lay.total, st, 1, a) == cudaSuccess;
 }
-template <typename T, int HD, int kMode>
-static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
+template <typename T, int HD, bool kFront>
+static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid) {
     const int P = a.m * (a.H / a.Hkv);
     // Two warps per 32-position block share the pairs (latency hides behind warps, not behind instruction-level
     // parallelism: one warp per block with twice the pairs measured slower at every context length); pairs per sweep =
     // what one of the two warps gets, padded to 1, 2, 4 or 8.
-    if (P > 8) return launch_attn_pg<T, HD, 8, kMode, 2>(st, a, grid, cluster_y);
-    if (P > 4) return launch_attn_pg<T, HD, 4, kMode, 2>(st, a, grid, cluster_y);
-    if (P > 2) return launch_attn_pg<T, HD, 2, kMode, 2>(st, a, grid, cluster_y);
-    return launch_attn_pg<T, HD, 1, kMode, 2>(st, a, grid, cluster_y);   // one pair: the second warp still stages the V rows
+    if (P > 8) return launch_attn_pg<T, HD, 8, kFront, 2>(st, a, grid);
+    if (P > 4) return launch_attn_pg<T, HD, 4, kFront, 2>(st, a, grid);
+    if (P > 2) return launch_attn_pg<T, HD, 2, kFront, 2>(st, a, grid);
+    return launch_attn_pg<T, HD, 1, kFront, 2>(st, a, grid);   // one pair: the second warp still stages the V rows
 }
 
 template <typename T> bool launch_attention(cudaStream_t st, const AttnArgs& a) {
@@ -680,9 +591,9 @@ template <typename T> bool launch_attention(cudaStream_t st, const AttnArgs& a) 
     dim3 grid(a.Hkv, n_chunks, nz);
     bool ok;
     switch (a.hd) {
-        case 32: ok = launch_attn_partial<T, 32, 0>(st, a, grid, 0); break;
-        case 64: ok = launch_attn_partial<T, 64, 0>(st, a, grid, 0); break;
-        default: ok = launch_attn_partial<T, 128, 0>(st, a, grid, 0); break;
+        case 32: ok = launch_attn_partial<T, 32, false>(st, a, grid); break;
+        case 64: ok = launch_attn_partial<T, 64, false>(st, a, grid); break;
+        default: ok = launch_attn_partial<T, 128, false>(st, a, grid); break;
     }
     if (!ok) return false;
     launch_attention_combine<T>(st, a);
@@ -694,17 +605,6 @@ template <typename T> void launch_attention_combine(cudaStream_t st, const AttnA
     launch_k(k_attn_combine<T>, dim3(a.H, a.m, nz), dim3(kChunkGroup * 32), 0, st, a);
 }
 
-template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a) {
-    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
-    if (n_chunks > 8) return false;   // portable cluster size
-    dim3 grid(a.Hkv, n_chunks);
-    switch (a.hd) {
-        case 32: return launch_attn_partial<T, 32, 1>(st, a, grid, n_chunks);
-        case 64: return launch_attn_partial<T, 64, 1>(st, a, grid, n_chunks);
-        default: return launch_attn_partial<T, 128, 1>(st, a, grid, n_chunks);
-    }
-}
-
 // Contexts of any length in two launches: the chunk kernel with its front end (RoPE, cache append) and the chunk merge.
 template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a) {
     if (a.n_blocks > 1) return false;
@@ -712,9 +612,9 @@ template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArg
     dim3 grid(a.Hkv, n_chunks);
     bool ok;
     switch (a.hd) {
-        case 32: ok = launch_attn_partial<T, 32, 2>(st, a, grid, 0); break;
-        case 64: ok = launch_attn_partial<T, 64, 2>(st, a, grid, 0); break;
-        default: ok = launch_attn_partial<T, 128, 2>(st, a, grid, 0); break;
+        case 32: ok = launch_attn_partial<T, 32, true>(st, a, grid); break;
+        case 64: ok = launch_attn_partial<T, 64, true>(st, a, grid); break;
+        default: ok = launch_attn_partial<T, 128, true>(st, a, grid); break;
     }
     if (!ok) return false;
     launch_attention_combine<T>(st, a);
@@ -1109,7 +1009,6 @@ void launch_init_pages(cudaStream_t st, int* page_table, int n_pages) {
     template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int, unsigned int*); \
     template void launch_rope_append<T>(cudaStream_t, const RopeArgs&);                                             \
     template bool launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
-    template bool launch_attention_fused<T>(cudaStream_t, const AttnArgs&);                                         \
     template void launch_attention_combine<T>(cudaStream_t, const AttnArgs&);                                       \
     template bool launch_attention_front<T>(cudaStream_t, const AttnArgs&);                                         \
     template void launch_swiglu<T>(cudaStream_t, const float*, int, int, void*, int, int);
