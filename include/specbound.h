@@ -309,7 +309,8 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                    SwiGLU epilogue on) sends up to 128 prompt rows per pass through the weight-streaming GEMMs (the
  *                    weights are read once per 128 rows), with a tiled causal attention kernel on the tensor cores, and
  *                    the fewer than 16 rows left over through 8-row passes; 2 = the same passes with the decode attention
- *                    kernels (a block of 8 rows at a time); 0 = 8-row passes only.  All are deterministic; they may differ
+ *                    kernels (a block of 8 rows at a time); 3 = as 1, but every work item of a wide GEMM on one CTA instead of
+ *                    a pair of CTAs sharing one activation tile; 0 = 8-row passes only.  All are deterministic; they may differ
  *                    in summation order, i.e. in the last bits of the K/V cache and of the first token's logits. */
 enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,
        SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7, SB_OPT_QKV_AHEAD = 8, SB_OPT_WIDE_PREFILL = 9 };

@@ -3,7 +3,7 @@
 // A pass carries up to 128 prompt rows per layer.  The decode attention kernel (CUDA cores, one CTA per 128 cached
 // positions and block of 8 rows) re-reads and re-unpacks the cached K/V for every block of 8 rows; here a CTA takes a
 // tile of 16 prompt rows of ONE query head and walks the cached positions 0 .. (last row's position) in blocks of 64,
-// staged once per tile by 16-byte asynchronous copies (double-buffered), with the two contractions on the tensor cores
+// staged once per tile by 16-byte asynchronous copies (three buffers, two blocks in flight), with the two contractions on the tensor cores
 // (mma.sync m16n8k16, bf16 x bf16 -> fp32):
 //
 //   scores   S = Q K^T : Q is fp32; it enters as its high and low bf16 halves (two MMAs), so the product is as
@@ -24,6 +24,7 @@ namespace sb {
 constexpr int kPfRows = 16;          // prompt rows per CTA
 constexpr int kPfBlock = 64;         // cached positions per staged block
 constexpr int kPfWarps = 4;
+constexpr int kPfStages = 3;         // staged blocks in flight per CTA (104 KB at 128 channels: two CTAs per SM)
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
@@ -60,9 +61,9 @@ __global__ void __launch_bounds__(kPfWarps * 32) k_attn_prefill(PrefillAttnArgs 
     constexpr int kTile = kPfBlock * ROWB;               // one staged K or V block
     constexpr int KS = HD / 16;                          // k steps of the score contraction
     constexpr int NT = HD / 8;                           // n tiles of the output
-    extern __shared__ __align__(16) unsigned char smem[];   // [2 buffers][K block | V block]; reused for the final merge
+    extern __shared__ __align__(16) unsigned char smem[];   // [kPfStages buffers][K block | V block]; reused for the final merge
     pdl_trigger();
-    const int h = blockIdx.x, tile = blockIdx.y;
+    const int h = blockIdx.x, tile = (int)gridDim.y - 1 - (int)blockIdx.y;   // the tiles with the most positions start first
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tig = lane & 3;
     const int G = a.H / a.Hkv, kvh = h / G;
     const int kvd = a.Hkv * HD, qd = a.H * HD;
@@ -93,6 +94,7 @@ __global__ void __launch_bounds__(kPfWarps * 32) k_attn_prefill(PrefillAttnArgs 
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
     stage(0, 0);
+    if (n_blocks > 1) stage(1, 1);
 
     // this thread's query fragments: rows g and g + 8 of the tile, high and low halves
     uint32_t qh[KS][4], ql[KS][4];
@@ -120,9 +122,13 @@ __global__ void __launch_bounds__(kPfWarps * 32) k_attn_prefill(PrefillAttnArgs 
     for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
 
     for (int blk = 0; blk < n_blocks; ++blk) {
-        const int buf = blk & 1;
-        if (blk + 1 < n_blocks) {
-            stage(blk + 1, buf ^ 1);
+        const int buf = blk % kPfStages;
+        // two blocks ahead (its buffer was released by the barrier that ended the previous iteration); the copies of
+        // a CTA are latency, not bandwidth: the more of them are in flight the better
+        if (blk + 2 < n_blocks) {
+            stage(blk + 2, (blk + 2) % kPfStages);
+            asm volatile("cp.async.wait_group 2;" ::: "memory");
+        } else if (blk + 1 < n_blocks) {
             asm volatile("cp.async.wait_group 1;" ::: "memory");
         } else {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -246,7 +252,7 @@ bool launch_attention_prefill(cudaStream_t st, const float* q, const void* k_cac
     PrefillAttnArgs a{q, static_cast<const __nv_bfloat16*>(k_cache), static_cast<const __nv_bfloat16*>(v_cache), page_table,
                       static_cast<__nv_bfloat16*>(act_out), H, Hkv, page, page_shift, pos0, M};
     const dim3 grid(H, (M + kPfRows - 1) / kPfRows), block(kPfWarps * 32);
-    const size_t smem = (size_t)4 * kPfBlock * (hd * 2 + 16);
+    const size_t smem = (size_t)kPfStages * 2 * kPfBlock * (hd * 2 + 16);
     static bool configured[kMaxDevices][2];
     const int dev = current_device();
     if (dev < 0) return false;

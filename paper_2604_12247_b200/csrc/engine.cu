@@ -369,7 +369,7 @@ static void layer_step_wide(Exec& e, const sb_layer_weights& lw, void* k_cache_l
         const int n_full = M / kMaxW, rem = M - n_full * kMaxW;
         // tiled causal attention on the tensor cores: one launch for all rows of the pass
         bool tiled = false;
-        if (g_wide_prefill == 1 && (D.hd == 64 || D.hd == 128))
+        if (g_wide_prefill != 2 && (D.hd == 64 || D.hd == 128))
             tiled = launch_attention_prefill(e.st, W.pf_q, k_cache_l, v_cache_l, W.page_table, W.pf_act_o, D.H, D.Hkv, D.hd, D.page,
                                              D.page_shift, pos0, M);
         if (tiled) e.launches++;
@@ -473,8 +473,8 @@ static int cuda_ok(cudaError_t err) { return err == cudaSuccess ? SB_OK : SB_ERR
 static int fetch_results(sb_ctx* c) {
     if (cudaMemcpyAsync(c->mailbox, c->e.W.res, sizeof(int) * 49, cudaMemcpyDeviceToHost, c->e.st) != cudaSuccess)
         return SB_ERR_CUDA;
-    if (cudaStreamSynchronize(c->e.st) != cudaSuccess) return SB_ERR_CUDA;
-    if (cudaGetLastError() != cudaSuccess) return SB_ERR_CUDA;
+    if (report_cuda("stream synchronize", cudaStreamSynchronize(c->e.st)) != cudaSuccess) return SB_ERR_CUDA;
+    if (report_cuda("last error", cudaGetLastError()) != cudaSuccess) return SB_ERR_CUDA;
     if (c->e.err) return c->e.err;
     c->d2h += sizeof(int) * 49;
     if (c->mailbox[48] != 0) return SB_ERR_DEVICE_TIMEOUT;
@@ -720,7 +720,12 @@ int sb_set_default_option(int32_t key, int32_t value) {
     if (key == SB_OPT_L2_PREFETCH) return tc_set_l2_prefetch(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_SPLIT_PENALTY) return tc_set_split_penalty(value) ? SB_OK : SB_ERR_ARG;
     if (key == SB_OPT_QKV_AHEAD) { g_qkv_ahead = value != 0; return SB_OK; }
-    if (key == SB_OPT_WIDE_PREFILL) { if (value < 0 || value > 2) return SB_ERR_ARG; g_wide_prefill = value; return SB_OK; }
+    if (key == SB_OPT_WIDE_PREFILL) {
+        if (value < 0 || value > 3) return SB_ERR_ARG;
+        g_wide_prefill = value;
+        tc_set_wide_cta_pairs(value != 3);
+        return SB_OK;
+    }
     if (key == SB_OPT_PDL) { g_use_pdl = value != 0; return SB_OK; }
     if (key == SB_OPT_FUSE) { if (value < 0 || value > 3) return SB_ERR_ARG; g_fuse = value; return SB_OK; }
     if (key == SB_OPT_TC_TUNING) return tc_set_tuning(value / 16, value % 16) ? SB_OK : SB_ERR_ARG;

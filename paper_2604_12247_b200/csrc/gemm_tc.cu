@@ -479,6 +479,354 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
 }
 
 // ---------------------------------------------------------------------------------------------
+// Wide passes (prefill, 128 activation rows) on CTA PAIRS: tcgen05.mma.cta_group::2, M = 256, N = 256.
+//
+// In the one-CTA wide form every CTA re-reads the whole [256][K] activation operand from L2 for its 128 weight rows:
+// 3 bytes reach the SMs per weight byte, and that L2 -> SM traffic, not HBM, bounds the pass.  Here two CTAs of a
+// cluster (one per SM) share one activation tile: each stages ITS 128 weight rows (the M half it accumulates in its
+// own tensor memory) and ITS HALF of the activation operand (operand rows 128 r .. 128 r + 127 of the [256][64]
+// tile = blocks 8 r .. 8 r + 7); the MMA, issued by one thread of the first CTA, reads both halves out of both CTAs'
+// shared memory.  2 bytes per weight byte, stages of 32 KB, six of them, both accumulators double-buffered.
+//
+// Barriers: "full" lives in the first CTA (the leader) and counts the bytes of BOTH CTAs' copies (each CTA issues its
+// own TMA copies with the pair form of the instruction, which may complete on the peer's barrier -- no cluster
+// multicast anywhere); "stage empty" and "accumulator full" exist in both CTAs and are signalled together by the
+// leader's tcgen05.commit; "accumulator empty" lives in the leader and takes the arrivals of both CTAs' epilogue
+// warps.  Every wait is bounded as in k_tc.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPairStages = 6;
+constexpr int kStageB2 = 128 * kBK * 2;       // this CTA's half of the activation tile: 16 KB
+constexpr uint32_t kPairCols = 256;           // TMEM columns of one accumulator (16 per block of 8 rows)
+static int smem_bytes_pair() { return kPairStages * (kStageA + kStageB2) + 1024 + 256; }
+static_assert(kPairStages * (kStageA + kStageB2) + 1280 + 16384 + 512 <= 227 * 1024, "pair stages exceed shared memory");
+__host__ __device__ constexpr uint32_t idesc_pair() { return (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24); }
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_pair() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// pair form of the TMA tile copy: destination in this CTA, completion on a barrier of either CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar_cluster, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], "
+        "[%4], %5;" ::"r"(dst),
+        "l"(tm), "r"(x), "r"(y), "r"(bar_cluster), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// completion of the MMAs issued so far arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(both)
+                 : "memory");
+}
+
+// 64 consecutive accumulator columns of this warp's 32 lanes (no wait: pair with tc_wait_ld)
+__device__ __forceinline__ void tc_ld64_nowait(uint32_t taddr, uint32_t (&v)[64]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Work items of the pair kernel: (slab of 2 R weight rows, k split); CTA r of the pair takes rows row0 + r R ..
+// (gate/up: columns row0 + r h .. of both matrices).  Clusters stride over the items.
+__device__ __forceinline__ ItemInfo decode_item_pair(const TcParams& p, int item, int rank) {
+    ItemInfo it = decode_item(p, item);
+    if (p.pair_half) it.row0 = (item % p.n_chunks) * 2 * p.pair_half + rank * p.pair_half;
+    else it.row0 = 2 * it.row0 + rank * p.R;       // decode_item counted slabs of R rows; a pair slab is 2 R
+    return it;
+}
+
+template <bool kPair>
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant__ TcParams p) {
+    constexpr int NB = kWideBlocks;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile int abort_s;
+    __shared__ float xch_s[kPair ? 2 : 1][kPair ? 4 : 1][kMaxW][kPair ? 64 : 1];   // gate/up: exchange area of the epilogue warps
+    __shared__ volatile int ok_s[8];
+
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    constexpr int kStages = kPairStages;
+    const uint32_t smA = tiles, smB = tiles + kStages * kStageA;
+    const uint32_t bars = smB + kStages * kStageB2;
+    auto full_bar = [&](int s) { return bars + 8u * s; };                       // used in the leader
+    auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };          // both CTAs
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * kStages + b); };      // both CTAs
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * kStages + 2 + b); }; // used in the leader
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const int cluster_id = (int)(blockIdx.x >> 1), n_clusters = (int)(gridDim.x >> 1);   // clusters of two CTAs along x (the pair of a 2-CTA MMA)
+    pdl_trigger();
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);       // the leader's arrive.expect_tx; the bytes of both CTAs
+            mbar_init(empty_bar(s), 1);      // the leader's commit
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);      // the leader's commit
+            mbar_init(tempty_bar(b), 8);     // four epilogue warps of each CTA
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kProducers) {   // both accumulators of both CTAs: the same warp of each CTA takes part
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2u * kPairCols));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_pair();        // the peer's barriers exist before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t a_bytes = kPair ? 2u * (uint32_t)p.pair_half * (kBK * 2) : (uint32_t)p.R * (kBK * 2);
+    const uint32_t stage_bytes = 2u * (a_bytes + (uint32_t)kStageB2);   // what both CTAs bring per fill
+
+    if (warp < kProducers) {
+        // ------------------------------ TMA producers (both CTAs) ------------------------------
+        if (lane == 0) {
+            if (warp == 0) {
+                for (int j = 0; j < p.n_mats; ++j) asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmA[j]) : "memory");
+                asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tmB) : "memory");
+            }
+            const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+            // position in this cluster's sequence of (item, k block) fills
+            int item = cluster_id, kb = 0;
+            ItemInfo it{};
+            auto start_item = [&]() { if (item < p.n_items) { it = decode_item_pair(p, item, (int)rank); kb = it.kb0; } };
+            auto advance = [&]() {
+                if (item >= p.n_items) return;
+                if (++kb < it.kb1) return;
+                item += n_clusters;
+                start_item();
+            };
+            start_item();
+            for (int j = 0; j < warp; ++j) advance();
+            auto load_a = [&](int st, uint32_t bar) {
+                if (kPair) {
+                    tma_load_2d_pair(smA + st * kStageA, &p.tmA[0], kb * kBK, it.row0, bar, pol_w);
+                    tma_load_2d_pair(smA + st * kStageA + 64 * kBK * 2, &p.tmA[1], kb * kBK, it.row0, bar, pol_w);
+                } else {
+                    tma_load_2d_pair(smA + st * kStageA, &p.tmA[it.mat], kb * kBK, it.row0, bar, pol_w);
+                }
+            };
+            // The weight tiles of the first pipeline fill do not depend on the preceding kernel: requested before the
+            // grid-dependency wait; the activation tiles follow after it.
+            int fill = warp;
+            int kb_first[(kStages + kProducers - 1) / kProducers];
+            int n_first = 0;
+            for (; item < p.n_items && fill < kStages; fill += kProducers) {
+                if (rank == 0) mbar_expect_tx(full_bar(fill), stage_bytes);
+                load_a(fill, map_to_cta(full_bar(fill), 0));
+                kb_first[n_first++] = kb;
+                for (int j = 0; j < kProducers; ++j) advance();
+            }
+            pdl_wait();
+            for (int j = 0; j < n_first; ++j) {
+                const int f0 = warp + j * kProducers;
+                tma_load_2d_pair(smB + f0 * kStageB2, &p.tmB, kb_first[j] * kBK, 128 * (int)rank, map_to_cta(full_bar(f0), 0), pol_a);
+            }
+            for (; item < p.n_items; fill += kProducers) {
+                const int stage = fill % kStages;
+                const uint32_t phase = (uint32_t)(fill / kStages) & 1u;
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_s, p.status, 1u)) break;
+                if (rank == 0) mbar_expect_tx(full_bar(stage), stage_bytes);
+                const uint32_t bar = map_to_cta(full_bar(stage), 0);
+                load_a(stage, bar);
+                tma_load_2d_pair(smB + stage * kStageB2, &p.tmB, kb * kBK, 128 * (int)rank, bar, pol_a);
+                for (int j = 0; j < kProducers; ++j) advance();
+            }
+        } else {
+            pdl_wait();
+        }
+    } else if (warp == kProducers) {
+        // ------------------------------ MMA issuer (one thread of the leader) ------------------------------
+        pdl_wait();
+        if (rank == 0 && lane == 0) {
+            int stage = 0, phase = 0, n_local = 0;
+            bool ok = true;
+            for (int item = cluster_id; item < p.n_items && ok; item += n_clusters, ++n_local) {
+                const ItemInfo it = decode_item(p, item);
+                const int buf = n_local & 1;
+                const uint32_t use = (uint32_t)(n_local >> 1);
+                if (!(ok = mbar_wait(tempty_bar(buf), (use & 1u) ^ 1u, &abort_s, p.status, 2u))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kPairCols;
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!(ok = mbar_wait(full_bar(stage), phase, &abort_s, p.status, 3u))) break;
+                    tc_fence_after();
+                    const uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageB2);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)
+                        tc_mma_pair(d_tmem, da + 2u * k, db + 2u * k, idesc_pair(), (kb > it.kb0 || k > 0) ? 1u : 0u);
+                    tc_commit_pair(empty_bar(stage));     // frees the stage in both CTAs once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+                if (ok) tc_commit_pair(tfull_bar(buf));   // accumulators of both CTAs complete
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (128 threads of each CTA) ------------------------------
+        // An item's mainloop is short at 128 rows (a few microseconds), so the epilogue must not be a chain of small
+        // tensor-memory loads: four loads of 64 columns (4 blocks of 8 rows) per item, the next one in flight while
+        // the current one is stored.
+        pdl_wait();
+        const int q = warp & 3;
+        const int row_in_tile = q * 32 + lane;
+        const int n_groups = (p.r0 + p.m + 4 * kMaxW - 1) / (4 * kMaxW);   // groups of 4 blocks that hold rows of this pass (<= 4)
+        int n_local = 0;
+        bool ok = true;
+        for (int item = cluster_id; item < p.n_items && ok; item += n_clusters, ++n_local) {
+            const ItemInfo it = decode_item_pair(p, item, (int)rank);
+            const int buf = n_local & 1;
+            const uint32_t use = (uint32_t)(n_local >> 1);
+            if (lane == 0) ok = mbar_wait_relaxed(tfull_bar(buf), use & 1u, &abort_s, p.status, 4u);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            if (kPair) ok = epi_vote(ok, ok_s, n_local, q, lane);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * kPairCols;
+            // One group of 4 blocks: finish what sits in v.  The code of a group is kept small and the loop over the
+            // groups is NOT unrolled beyond the two register buffers: an item's epilogue runs once, straight-line code
+            // of thousands of instructions would all be cold instruction-cache misses (measured: 7 us per item).
+            auto finish_group = [&](int g, const uint32_t (&v)[64]) {
+                if constexpr (kPair) {
+                    // tile rows 0-63 (warps 0-1) hold gate projections, rows 64-127 (warps 2-3) the up projections of the
+                    // same columns.  Of the group's four blocks the gate warps finish blocks 0-1 and the up warps blocks
+                    // 2-3: each side hands the other its values for the blocks it does not finish, through a
+                    // double-buffered exchange area (one barrier per group).
+                    float (*xb)[kMaxW][64] = xch_s[g & 1];
+                    const int c = row_in_tile & 63;
+                    const bool up_side = q >= 2;
+                    // (register indices stay compile-time: both candidates are formed, one is selected)
+                    float mine[2][kMaxW];
+#pragma unroll
+                    for (int b = 0; b < 2; ++b) {
+#pragma unroll
+                        for (int i = 0; i < kMaxW; ++i) {
+                            const float lo2 = __uint_as_float(v[b * 16 + i]) + __uint_as_float(v[b * 16 + 8 + i]);
+                            const float hi2 = __uint_as_float(v[(b + 2) * 16 + i]) + __uint_as_float(v[(b + 2) * 16 + 8 + i]);
+                            xb[up_side ? b : b + 2][i][c] = up_side ? lo2 : hi2;    // the block the other side finishes
+                            mine[b][i] = up_side ? hi2 : lo2;
+                        }
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int col = it.row0 + c;
+                    if (c < p.pair_half && col < p.n_rows[0]) {
+                        const size_t F = (size_t)p.n_rows[0];
+#pragma unroll
+                        for (int b = 0; b < 2; ++b) {
+                            const int bk = up_side ? b + 2 : b;    // block (within the group) finished here
+                            const int blk = g * 4 + bk;
+                            __nv_bfloat16* dst = p.swiglu_out + (size_t)blk * 16 * F + col;
+#pragma unroll
+                            for (int i = 0; i < kMaxW; ++i) {
+                                const int row = blk * kMaxW + i;
+                                if (row >= p.r0 && row < p.r0 + p.m) {
+                                    const float other = xb[bk][i][c];
+                                    const float gt = up_side ? other : mine[b][i], u = up_side ? mine[b][i] : other;
+                                    const float val = gt / (1.f + expf(-gt)) * u;
+                                    const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+                                    dst[(size_t)i * F] = hi;
+                                    dst[(size_t)(i + 8) * F] = __float2bfloat16_rn(val - __bfloat162float(hi));
+                                }
+                            }
+                        }
+                    }
+                } else {
+                    const int n = it.row0 + row_in_tile;
+                    if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
+                        const int s = item / p.n_chunks;
+                        // partials [block][split][8][n_total]
+                        float* o = p.out + (((size_t)(g * 4) * p.S + s) * kMaxW) * p.n_total + p.n_off[it.mat] + n;
+                        const size_t blk_stride = (size_t)p.S * kMaxW * p.n_total;
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+#pragma unroll
+                            for (int i = 0; i < kMaxW; ++i) {
+                                const int row = (g * 4 + b) * kMaxW + i;
+                                if (row >= p.r0 && row < p.r0 + p.m)
+                                    o[b * blk_stride + (size_t)i * p.n_total] = __uint_as_float(v[b * 16 + i]) + __uint_as_float(v[b * 16 + 8 + i]);
+                            }
+                        }
+                    }
+                }
+            };
+            if constexpr (kPair) {     // one register buffer: the exchange needs the registers
+                uint32_t va[64];
+#pragma unroll 1
+                for (int g = 0; g < n_groups; ++g) {
+                    tc_ld64_nowait(t0 + (uint32_t)g * 64u, va);
+                    tc_wait_ld();
+                    finish_group(g, va);
+                }
+            } else {
+                uint32_t va[64], vb[64];
+                tc_ld64_nowait(t0, va);
+#pragma unroll 1
+                for (int g = 0; g < n_groups; g += 2) {     // two groups per trip: one register buffer each, the next load in flight
+                    tc_wait_ld();
+                    if (g + 1 < n_groups) tc_ld64_nowait(t0 + (uint32_t)(g + 1) * 64u, vb);
+                    finish_group(g, va);
+                    if (g + 1 < n_groups) {
+                        tc_wait_ld();
+                        if (g + 2 < n_groups) tc_ld64_nowait(t0 + (uint32_t)(g + 2) * 64u, va);
+                        finish_group(g + 1, vb);
+                    }
+                }
+            }
+            // every load of this accumulator has completed (the last group's wait): it may be overwritten
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0));
+            if (kPair) asm volatile("bar.sync 1, 128;" ::: "memory");   // the exchange buffers are free for the next item
+        }
+    }
+
+    if (abort_s) {   // a wait expired: give copies and MMAs still in flight time to land before leaving
+        unsigned long long t0 = clock64();
+        while (clock64() - t0 < 4000000ull) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_pair();   // neither CTA's shared memory, barriers or tensor memory go away while the peer may still use them
+    if (warp == kProducers) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kPairCols));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Host side: tensor maps and work decomposition
 // ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -519,16 +867,22 @@ static int sm_count() { return device_sm_count(); }
 
 // Slab height R (multiple of 8 in [64,128]) and split count S that minimise what the busiest
 // CTA streams.  Depends on the shape only, never on the number of rows.
-static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out) {
+// per_item: CTAs that share a work item (a slab is then per_item * R rows); penalty_pm: cost of one more split.
+static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out, int per_item = 1,
+                         int penalty_pm = -1) {
+    if (penalty_pm < 0) penalty_pm = g_split_penalty_pm;
     double best = 1e300;
     int bR = 128, bS = 1;
     for (int S = 1; S <= max_split && S <= KB; ++S)
         for (int R = 128; R >= 64; R -= 8) {
             long long chunks = 0;
-            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + R - 1) / R;
+            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + per_item * R - 1) / (per_item * R);
             long long items = chunks * S;
             long long per = (items + G - 1) / G;
-            double cost = (double)per * R * ((KB + S - 1) / S) * (1.0 + 0.001 * g_split_penalty_pm * S);   // each split adds partial traffic and consumer loads
+            // what a CTA moves into its shared memory per k block: its R weight rows and, for CTA pairs in a wide pass
+            // (bound by the L2 -> SM traffic), its 128-row half of the activation tile as well
+            const int rows_moved = per_item == 2 ? R + 128 : R;
+            double cost = (double)per * rows_moved * ((KB + S - 1) / S) * (1.0 + 0.001 * penalty_pm * S);   // each split adds partial traffic and consumer loads
             if (cost < best - 1e-9) { best = cost; bR = R; bS = S; }
         }
     *R_out = bR;
@@ -536,54 +890,58 @@ static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, i
 }
 
 // Pair mode: rows of each kind per item (multiple of 8 in [32,64]) that minimise what the busiest CTA streams.
-static int choose_pair_half(int n_rows, int G) {
+static int choose_pair_half(int n_rows, int G, int per_item = 1) {
     double best = 1e300;
     int bh = 64;
     for (int h = 64; h >= 32; h -= 8) {
-        long long items = (n_rows + h - 1) / h;
-        double cost = (double)((items + G - 1) / G) * h;
+        long long items = (n_rows + per_item * h - 1) / (per_item * h);
+        double cost = (double)((items + G - 1) / G) * (per_item == 2 ? 2 * h + 128 : h);   // rows moved per k block, as in choose_split
         if (cost < best - 1e-9) { best = cost; bh = h; }
     }
     return bh;
 }
 
+static int max_pair_clusters();
+// cta_pair: plan for k_tc_pair (a work item is a slab of 2 R rows for a cluster of two CTAs)
 static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_end, int n_mats, int K, const void* act,
-                        bool head, bool pair = false, int nb = 1) {
+                        bool head, bool pair = false, int nb = 1, bool cta_pair = false) {
     std::vector<uint64_t> key;
     for (int j = 0; j < n_mats; ++j) { key.push_back((uint64_t)(uintptr_t)W[j]); key.push_back((uint64_t)n_end[j]); }
     key.push_back((uint64_t)K);
     key.push_back((uint64_t)(uintptr_t)act);
-    key.push_back((head ? 1 : 0) + (pair ? 2 : 0) + 4 * nb);
+    key.push_back((head ? 1 : 0) + (pair ? 2 : 0) + 4 * nb + (cta_pair ? 1024 : 0));
     key.push_back((uint64_t)g_stages * 16 + g_ctas_per_sm + ((uint64_t)g_split_penalty_pm << 40));
     auto it = cache->plans.find(key);
     if (it != cache->plans.end()) return it->second;
     TcPlan* pl = new TcPlan();
     memset(&pl->p, 0, sizeof(pl->p));
     TcParams& p = pl->p;
-    int G = sm_count() * (nb > 1 ? 1 : g_ctas_per_sm);
-    p.stages = nb > 1 ? kWideStages : g_stages;
+    int G = cta_pair ? max_pair_clusters() : sm_count() * (nb > 1 ? 1 : g_ctas_per_sm);   // CTAs, or clusters, that share the items
+    if (G > sm_count() / 2 && cta_pair) G = sm_count() / 2;
+    p.stages = cta_pair ? kPairStages : nb > 1 ? kWideStages : g_stages;
     p.n_mats = n_mats;
     p.KB = (K + kBK - 1) / kBK;
     int prev = 0;
     for (int j = 0; j < n_mats; ++j) { p.n_rows[j] = n_end[j] - prev; p.n_off[j] = prev; prev = n_end[j]; }
     int chunks = 0;
+    const int per_item = cta_pair ? 2 : 1;   // CTAs that share a work item
     if (pair) {
-        p.pair_half = choose_pair_half(p.n_rows[0], G);
+        p.pair_half = choose_pair_half(p.n_rows[0], G, per_item);
         p.R = 2 * p.pair_half;
         p.S = 1;
-        chunks = (p.n_rows[0] + p.pair_half - 1) / p.pair_half;
+        chunks = (p.n_rows[0] + per_item * p.pair_half - 1) / (per_item * p.pair_half);
         for (int j = 0; j < 3; ++j) p.chunk_end[j] = chunks;
     } else {
-        choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
+        choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S, per_item, cta_pair ? 30 : g_split_penalty_pm);
         for (int j = 0; j < 3; ++j) {
-            if (j < n_mats) chunks += (p.n_rows[j] + p.R - 1) / p.R;
+            if (j < n_mats) chunks += (p.n_rows[j] + per_item * p.R - 1) / (per_item * p.R);
             p.chunk_end[j] = chunks;
         }
     }
     p.n_chunks = chunks;
     p.n_items = chunks * p.S;
-    pl->grid = p.n_items < G ? p.n_items : G;
-    bool ok = make_map(&p.tmB, act, 16 * nb, K, 16 * nb);
+    pl->grid = (p.n_items < G ? p.n_items : G) * per_item;
+    bool ok = make_map(&p.tmB, act, 16 * nb, K, cta_pair ? 128 : 16 * nb);
     for (int j = 0; j < n_mats && ok; ++j) ok = make_map(&p.tmA[j], W[j], p.n_rows[j], K, pair ? p.pair_half : p.R);
     if (!ok) { delete pl; return nullptr; }
     cache->plans[key] = pl;
@@ -600,6 +958,44 @@ template <bool kHead, bool kPair, int NB = 1> static void launch(cudaStream_t st
     }
     launch_k(k_tc<kHead, kPair, NB>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes(p.stages, NB), st, p);
 }
+
+template <bool kPair> static void pair_func_attr() {
+    static bool attr_set[kMaxDevices];
+    const int dev = current_device();
+    if (dev >= 0 && !attr_set[dev]) {
+        cudaFuncSetAttribute(k_tc_pair<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_pair());
+        attr_set[dev] = true;
+    }
+}
+template <bool kPair> static bool launch_pair(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
+    pair_func_attr<kPair>();
+    const bool ok = launch_kcp(k_tc_pair<kPair>, dim3(pl->grid), dim3(kTcThreads), (size_t)smem_bytes_pair(), st, dim3(2, 1, 1), g_use_pdl, p) == cudaSuccess;
+    if (!ok && getenv("SB_DEBUG")) fprintf(stderr, "[specbound] k_tc_pair: grid %d, smem %d, items %d, clusters at once %d\n", pl->grid, smem_bytes_pair(), p.n_items, max_pair_clusters());
+    return ok;
+}
+// Clusters of two k_tc_pair CTAs the device can hold at once (a GPC with an odd number of usable SMs leaves one out):
+// the persistent grid must not exceed it, or the last cluster would run as a second wave.  0 = cannot run.
+static int max_pair_clusters() {
+    static int n[kMaxDevices];   // 0 unknown, -1 none
+    const int dev = current_device();
+    if (dev < 0) return 0;
+    if (n[dev] == 0) {
+        pair_func_attr<false>();
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)(sm_count() / 2 * 2)); cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = (size_t)smem_bytes_pair();
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int c = 0;
+        if (cudaOccupancyMaxActiveClusters(&c, k_tc_pair<false>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); c = 0; }
+        n[dev] = c > 0 ? c : -1;
+    }
+    return n[dev] > 0 ? n[dev] : 0;
+}
+
+static bool g_wide_cta_pairs = true;   // wide passes on CTA pairs (k_tc_pair) instead of single CTAs (k_tc<., ., 16>)
+void tc_set_wide_cta_pairs(bool on) { g_wide_cta_pairs = on; }
 
 bool tc_set_split_penalty(int per_mille) {
     if (per_mille < 0 || per_mille > 1000) return false;
@@ -648,10 +1044,20 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsig
     if (pair && (a.n_mats != 2 || a.n_end[1] != 2 * a.n_end[0])) return -1;
     const int nb = a.nb > 1 ? kWideBlocks : 1;
     if (a.nb > 1 && a.nb != kWideBlocks) return -1;
-    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false, pair, nb);
+    const bool cta_pair = nb > 1 && g_wide_cta_pairs && max_pair_clusters() > 0;
+    TcPlan* pl = get_plan(cache, a.W, a.n_end, a.n_mats, a.K, a.act, false, pair, nb, cta_pair);
     if (!pl) return -1;
     TcParams p = pl->p;
     p.out = a.out; p.n_total = a.n_total; p.r0 = a.r0; p.m = a.m; p.status = status;
+    if (cta_pair) {
+        if (pair) {
+            p.swiglu_out = reinterpret_cast<__nv_bfloat16*>(a.swiglu_out);
+            if (!launch_pair<true>(st, pl, p)) return -1;
+        } else {
+            if (!launch_pair<false>(st, pl, p)) return -1;
+        }
+        return p.S;
+    }
     if (a.next_W[0] && g_l2_next_every > 0 && nb == 1) {   // announce a later pair-mode GEMM: same plan that GEMM will use
         const void* nW[2] = {a.next_W[0], a.next_W[1]};
         int n_end[2] = {a.next_rows, 2 * a.next_rows};

@@ -28,6 +28,9 @@ bool tc_set_tuning(int stages, int ctas_per_sm);
 bool tc_set_l2_prefetch(int every);
 // cost the host's work decomposition charges for each additional k split, per mille of the streaming time
 bool tc_set_split_penalty(int per_mille);
+// wide passes (GemmArgs::nb > 1): true (default) = clusters of two CTAs sharing one activation tile (cta_group::2),
+// false = one CTA per work item
+void tc_set_wide_cta_pairs(bool on);
 // returns the number of split-K partials written to a.out, or -1 if no TMA descriptor could be made
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status);
 bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status);

@@ -151,7 +151,60 @@ __global__ void k_rope_append(RopeArgs a) {
         dst[i + half] = from_f32<T>(x1);
     }
 }
+// The same for the many rows of a wide prefill pass: four rotation pairs per thread (128-bit loads and stores), eight
+// heads per block.  grid = (ceil((H + 2 Hkv) / 8), m), block = 8 * hd / 8 threads.  Same arithmetic, same results.
+template <typename T>
+__global__ void k_rope_append_wide(RopeArgs a) {
+    pdl_trigger();
+    pdl_wait();
+    const int half = a.hd >> 1, per_head = half >> 2;            // threads per head
+    const int head = blockIdx.x * 8 + threadIdx.x / per_head;
+    if (head >= a.H + 2 * a.Hkv) return;
+    const int i = (threadIdx.x % per_head) * 4;                  // first of this thread's four rotation pairs
+    const int row = a.r0 + blockIdx.y;
+    const int pos = a.pos0 + row;
+    const int qd = a.H * a.hd, kvd = a.Hkv * a.hd, ntot = qd + 2 * kvd;
+    const int col = head * a.hd;
+    const int blk = row / kMaxW;
+    const float* p0 = a.qkv + ((size_t)blk * a.n_split * kMaxW + (row - blk * kMaxW)) * ntot + col + i;
+    const size_t stride4 = (size_t)kMaxW * ntot / 4;
+    float4 x0 = sum_splits4(reinterpret_cast<const float4*>(p0), stride4, a.n_split);
+    float4 x1 = sum_splits4(reinterpret_cast<const float4*>(p0 + half), stride4, a.n_split);
+    const bool is_v = head >= a.H + a.Hkv;
+    if (!is_v) {
+        rope_apply(rope_fetch(a.inv_freq, a.rope_tab, half, pos, i), x0.x, x1.x);
+        rope_apply(rope_fetch(a.inv_freq, a.rope_tab, half, pos, i + 1), x0.y, x1.y);
+        rope_apply(rope_fetch(a.inv_freq, a.rope_tab, half, pos, i + 2), x0.z, x1.z);
+        rope_apply(rope_fetch(a.inv_freq, a.rope_tab, half, pos, i + 3), x0.w, x1.w);
+    }
+    if (head < a.H) {
+        float* q = a.q + (size_t)row * qd + col;
+        *reinterpret_cast<float4*>(q + i) = x0;
+        *reinterpret_cast<float4*>(q + i + half) = x1;
+    } else {
+        const int kvh = is_v ? head - a.H - a.Hkv : head - a.H;
+        T* cache = reinterpret_cast<T*>(is_v ? a.v_cache : a.k_cache);
+        const int page = a.page_table[pos >> a.page_shift];
+        T* dst = cache + ((size_t)page * a.page + (pos & (a.page - 1))) * kvd + kvh * a.hd;
+        if constexpr (sizeof(T) == 2) {   // four rounded values per 8-byte store
+            auto pack4 = [](float4 x) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+                return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+            };
+            *reinterpret_cast<uint2*>(dst + i) = pack4(x0);
+            *reinterpret_cast<uint2*>(dst + i + half) = pack4(x1);
+        } else {
+            *reinterpret_cast<float4*>(dst + i) = x0;
+            *reinterpret_cast<float4*>(dst + i + half) = x1;
+        }
+    }
+}
 template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a) {
+    if (a.m > kMaxW && a.hd % 8 == 0 && a.hd <= 128) {   // wide prefill pass
+        dim3 grid((a.H + 2 * a.Hkv + 7) / 8, a.m);
+        launch_k(k_rope_append_wide<T>, grid, dim3(a.hd), 0, st, a);
+        return;
+    }
     dim3 grid(a.H + 2 * a.Hkv, a.m);
     launch_k(k_rope_append<T>, grid, dim3(a.hd / 2), 0, st, a);
 }

@@ -1,5 +1,7 @@
 // Internal declarations shared by the translation units of the SpecBound sm_100a library.
 #pragma once
+#include <cstdio>
+#include <cstdlib>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -108,6 +110,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 extern bool g_use_pdl;
+// With SB_DEBUG set in the environment, CUDA errors are also written to stderr where they are first seen.
+inline cudaError_t report_cuda(const char* where, cudaError_t err) {
+    if (err != cudaSuccess) {
+        static const bool on = getenv("SB_DEBUG") != nullptr;
+        if (on) fprintf(stderr, "[specbound] %s: %s (%s)\n", where, cudaGetErrorName(err), cudaGetErrorString(err));
+    }
+    return err;
+}
 // Index of the current device for the per-device host-side caches (function attributes, SM count, ...); -1 on error.
 constexpr int kMaxDevices = 64;
 inline int current_device() {
@@ -122,10 +132,10 @@ inline int device_sm_count() {   // SMs of the current device (148 if the query 
     if (!n[dev] && (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0)) n[dev] = 148;
     return n[dev];
 }
-// cluster.y > 1 launches thread-block clusters of that many CTAs along y (grid.y must be a multiple of it);
+// cluster with more than one CTA: launches thread-block clusters of that shape (the grid must be a multiple of it);
 // pdl: launch with programmatic stream serialisation (the kernel may start while its predecessor drains)
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kcp(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,
+inline cudaError_t launch_kcp(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, dim3 cluster,
                               bool pdl, Args&&... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
@@ -136,11 +146,11 @@ inline cudaError_t launch_kcp(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
         attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
         ++n_attr;
     }
-    if (cluster_y > 1) {
+    if (cluster.x * cluster.y * cluster.z > 1) {
         attr[n_attr].id = cudaLaunchAttributeClusterDimension;
-        attr[n_attr].val.clusterDim.x = 1;
-        attr[n_attr].val.clusterDim.y = (unsigned)cluster_y;
-        attr[n_attr].val.clusterDim.z = 1;
+        attr[n_attr].val.clusterDim.x = cluster.x;
+        attr[n_attr].val.clusterDim.y = cluster.y;
+        attr[n_attr].val.clusterDim.z = cluster.z;
         ++n_attr;
     }
     cfg.attrs = attr;
@@ -158,7 +168,13 @@ inline cudaError_t launch_kcp(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
             if (n_seen[dev] < 32) seen[dev][n_seen[dev]++] = (void*)kernel;
         }
     }
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    return report_cuda("kernel launch", cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+}
+// clusters of cluster_y CTAs along y
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kcp(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,
+                              bool pdl, Args&&... args) {
+    return launch_kcp(kernel, grid, block, smem, st, dim3(1, cluster_y > 1 ? (unsigned)cluster_y : 1u, 1), pdl, static_cast<Args&&>(args)...);
 }
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kc(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_y,

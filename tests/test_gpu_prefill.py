@@ -29,8 +29,9 @@ def _hidden_after_prefill(ctx, prompt, n_layers):
 
 # 16: the smallest wide pass; 64, 70, 100: one ragged wide pass (70 and 100 end in a partial block of 8 rows); 128: a
 # whole pass; 130: a whole pass + 2 rows through an 8-row pass; 300: two whole passes and a ragged one.  Page size 16
-# wide_mode 1: the tiled tensor-core attention kernel of the wide passes (the default); 2: the decode attention kernels
-@pytest.mark.parametrize("wide_mode", [1, 2])
+# wide_mode 1: wide GEMMs on CTA pairs + the tiled tensor-core attention kernel (the default); 2: the decode attention
+# kernels; 3: as 1 with the wide GEMMs on single CTAs
+@pytest.mark.parametrize("wide_mode", [1, 2, 3])
 @pytest.mark.parametrize("n_prompt", [16, 64, 70, 100, 128, 130, 300])
 def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt, wide_mode):
     shape = SMALL_BF16
