@@ -73,22 +73,27 @@ __global__ void __launch_bounds__(kPfWarps * 32) k_attn_prefill(PrefillAttnArgs 
     const int n_blocks = last_pos / kPfBlock + 1;
     pdl_wait();
 
-    auto stage = [&](int blk, int buf) {                 // cached rows blk * 64 .. + 63 of K and V into buffer buf
+    // cached rows blk * 64 .. + 63 of K and V into buffer buf: a thread owns one 16-byte column of pieces and walks the
+    // rows; the row's page and offset are computed once and serve both the K and the V copy
+    auto stage = [&](int blk, int buf) {
         unsigned char* base = smem + (size_t)buf * 2 * kTile;
-        constexpr int kPieces = HD * 2 / 16;
-        for (int idx = threadIdx.x; idx < 2 * kPfBlock * kPieces; idx += blockDim.x) {
-            const int which = idx / (kPfBlock * kPieces);
-            const int rem = idx - which * (kPfBlock * kPieces);
-            const int r = rem / kPieces, piece = rem - r * kPieces;
+        constexpr int kPieces = HD * 2 / 16;                         // 16-byte pieces per row (8 or 16)
+        constexpr int kRowsPerSweep = kPfWarps * 32 / kPieces;       // rows the CTA covers per sweep
+        const int piece = threadIdx.x % kPieces;
+        const unsigned char* kc = reinterpret_cast<const unsigned char*>(a.k_cache) + (size_t)kvh * HD * 2 + piece * 16;
+        const unsigned char* vc = reinterpret_cast<const unsigned char*>(a.v_cache) + (size_t)kvh * HD * 2 + piece * 16;
+#pragma unroll 4
+        for (int r = threadIdx.x / kPieces; r < kPfBlock; r += kRowsPerSweep) {
             const int t = blk * kPfBlock + r;
-            unsigned char* dst = base + (size_t)which * kTile + (size_t)r * ROWB + piece * 16;
+            unsigned char* dst = base + (size_t)r * ROWB + piece * 16;
             if (t <= last_pos) {
                 const int page = a.page_table[t >> a.page_shift];
-                const unsigned char* src = reinterpret_cast<const unsigned char*>(which ? a.v_cache : a.k_cache) +
-                                           (((size_t)page * a.page + (t & (a.page - 1))) * kvd + (size_t)kvh * HD) * 2 + piece * 16;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+                const size_t off = ((size_t)page * a.page + (t & (a.page - 1))) * kvd * 2;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(kc + off) : "memory");
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst + kTile)), "l"(vc + off) : "memory");
             } else {   // beyond the tile's last position: the probabilities are 0 there, and 0 * garbage must stay 0
                 *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(dst + kTile) = make_uint4(0u, 0u, 0u, 0u);
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -138,7 +143,9 @@ __global__ void __launch_bounds__(kPfWarps * 32) k_attn_prefill(PrefillAttnArgs 
         const int p0 = blk * kPfBlock + warp * 16;        // this warp's 16 positions of the block
         if (p0 <= last_pos) {
             // ---- scores: two n tiles (positions p0 .. p0+7, p0+8 .. p0+15) ----
+            // (the high and the low halves of q accumulate separately: four independent chains of MMAs instead of two)
             float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            float sl[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 // matrices: (positions 0-7, channels lo), (0-7, hi), (8-15, lo), (8-15, hi)
@@ -146,10 +153,14 @@ __global__ void __launch_bounds__(kPfWarps * 32) k_attn_prefill(PrefillAttnArgs 
                 const int r = warp * 16 + (lane & 7) + ((lane >> 4) << 3), cbyte = (16 * ks + ((lane >> 3) & 1) * 8) * 2;
                 ldmatrix_x4(kb, k_s + (uint32_t)(r * ROWB + cbyte));
                 mma_bf16(s[0], qh[ks], kb[0], kb[1]);
-                mma_bf16(s[0], ql[ks], kb[0], kb[1]);
+                mma_bf16(sl[0], ql[ks], kb[0], kb[1]);
                 mma_bf16(s[1], qh[ks], kb[2], kb[3]);
-                mma_bf16(s[1], ql[ks], kb[2], kb[3]);
+                mma_bf16(sl[1], ql[ks], kb[2], kb[3]);
             }
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s[nt][j] += sl[nt][j];
             // ---- online softmax of rows g (values [.][0], [.][1]) and g + 8 ([.][2], [.][3]) ----
             float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
