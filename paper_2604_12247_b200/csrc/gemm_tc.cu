@@ -479,27 +479,34 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
 }
 
 // ---------------------------------------------------------------------------------------------
-// Wide passes (prefill, 128 activation rows) on CTA PAIRS: tcgen05.mma.cta_group::2, M = 256, N = 256.
+// Wide passes (prefill, 128 activation rows) on CTA PAIRS: tcgen05.mma.cta_group::2, M = 256, N = 16 .. 256.
 //
-// In the one-CTA wide form every CTA re-reads the whole [256][K] activation operand from L2 for its 128 weight rows:
-// 3 bytes reach the SMs per weight byte, and that L2 -> SM traffic, not HBM, bounds the pass.  Here two CTAs of a
-// cluster (one per SM) share one activation tile: each stages ITS 128 weight rows (the M half it accumulates in its
-// own tensor memory) and ITS HALF of the activation operand (operand rows 128 r .. 128 r + 127 of the [256][64]
-// tile = blocks 8 r .. 8 r + 7); the MMA, issued by one thread of the first CTA, reads both halves out of both CTAs'
-// shared memory.  2 bytes per weight byte, stages of 32 KB, six of them, both accumulators double-buffered.
+// At 128 rows the pass is bound by the tensor pipe, so the operands swap roles against the 8-row kernel: the
+// ACTIVATIONS are the MMA's M operand (256 operand rows = 128 rows x high/low halves; each CTA of the pair holds 128 of
+// them = 64 rows, and accumulates them in its own tensor memory), the WEIGHT rows of a work item are the N operand
+// (2 R rows, R of them staged by each CTA), and N can be any multiple of 16: the host picks the tile width that
+// spreads a matrix evenly over the clusters (gate/up of the 7B shape: 22016 rows are 1.16 rounds of 128-row tiles,
+// i.e. 2 rounds at 62 % fill with weights as M; as N they are two rounds of 160 columns).  An MMA's time is
+// proportional to N.  Both CTAs stage their operand halves with plain TMA copies (no cluster multicast anywhere); the
+// MMA, issued by one thread of the first CTA, reads both halves out of both CTAs' shared memory.
+//
+// Accumulator of a CTA: lane = operand row (block b = lanes 16 b .. 16 b + 15: high halves of rows 8 b .. 8 b + 7, then
+// their low halves), column = weight row of the item.  The epilogue adds the low half's lane to the high half's with
+// a shuffle and writes 16-byte pieces.  Gate/up: the first CTA stages the item's gate rows, the second its up rows,
+// so a lane holds gate (columns 0 .. h-1) and up (columns h .. 2 h - 1) of the same output and applies SwiGLU itself.
 //
 // Barriers: "full" lives in the first CTA (the leader) and counts the bytes of BOTH CTAs' copies (each CTA issues its
-// own TMA copies with the pair form of the instruction, which may complete on the peer's barrier -- no cluster
-// multicast anywhere); "stage empty" and "accumulator full" exist in both CTAs and are signalled together by the
-// leader's tcgen05.commit; "accumulator empty" lives in the leader and takes the arrivals of both CTAs' epilogue
-// warps.  Every wait is bounded as in k_tc.
+// own copies with the pair form of the instruction, which may complete on the peer's barrier); "stage empty" and
+// "accumulator full" exist in both CTAs and are signalled together by the leader's tcgen05.commit; "accumulator
+// empty" lives in the leader and takes the arrivals of both CTAs' epilogue warps.  Every wait is bounded as in k_tc.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPairStages = 6;
 constexpr int kStageB2 = 128 * kBK * 2;       // this CTA's half of the activation tile: 16 KB
 constexpr uint32_t kPairCols = 256;           // TMEM columns of one accumulator (16 per block of 8 rows)
 static int smem_bytes_pair() { return kPairStages * (kStageA + kStageB2) + 1024 + 256; }
 static_assert(kPairStages * (kStageA + kStageB2) + 1280 + 16384 + 512 <= 227 * 1024, "pair stages exceed shared memory");
-__host__ __device__ constexpr uint32_t idesc_pair() { return (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24); }
+// D = f32, A = B = bf16, both K-major, M = 256 (the pair), N columns
+__host__ __device__ constexpr uint32_t idesc_pair(uint32_t n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24); }
 
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
@@ -554,25 +561,35 @@ __device__ __forceinline__ void tc_ld64_nowait(uint32_t taddr, uint32_t (&v)[64]
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Work items of the pair kernel: (slab of 2 R weight rows, k split); CTA r of the pair takes rows row0 + r R ..
-// (gate/up: columns row0 + r h .. of both matrices).  Clusters stride over the items.
-__device__ __forceinline__ ItemInfo decode_item_pair(const TcParams& p, int item, int rank) {
+// Work items of the pair kernel: (slab of 2 R weight rows, k split); CTA r of the pair stages rows row0 + r R ..
+// (gate/up: the h columns row0 .. of the gate matrix for r = 0, of the up matrix for r = 1).  Clusters stride over
+// the items.  first_row: the first weight row (output column) of the item.
+__device__ __forceinline__ ItemInfo decode_item_pair(const TcParams& p, int item, int rank, int* first_row) {
     ItemInfo it = decode_item(p, item);
-    if (p.pair_half) it.row0 = (item % p.n_chunks) * 2 * p.pair_half + rank * p.pair_half;
-    else it.row0 = 2 * it.row0 + rank * p.R;       // decode_item counted slabs of R rows; a pair slab is 2 R
+    if (p.pair_half) {
+        it.row0 = (item % p.n_chunks) * p.pair_half;
+        *first_row = it.row0;
+    } else {
+        *first_row = 2 * it.row0;                  // decode_item counted slabs of R rows; a pair slab is 2 R
+        it.row0 = 2 * it.row0 + rank * p.R;
+    }
     return it;
 }
 
 template <bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant__ TcParams p) {
-    constexpr int NB = kWideBlocks;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_s;
-    __shared__ float xch_s[kPair ? 2 : 1][kPair ? 4 : 1][kMaxW][kPair ? 64 : 1];   // gate/up: exchange area of the epilogue warps
-    __shared__ volatile int ok_s[8];
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -609,8 +626,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
     cluster_sync_pair();        // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
-    const uint32_t a_bytes = kPair ? 2u * (uint32_t)p.pair_half * (kBK * 2) : (uint32_t)p.R * (kBK * 2);
-    const uint32_t stage_bytes = 2u * (a_bytes + (uint32_t)kStageB2);   // what both CTAs bring per fill
+    const int R = kPair ? p.pair_half : p.R;                             // weight rows this CTA stages per fill
+    const uint32_t stage_bytes = 2u * ((uint32_t)R * (kBK * 2) + (uint32_t)kStageB2);   // what both CTAs bring per fill
 
     if (warp < kProducers) {
         // ------------------------------ TMA producers (both CTAs) ------------------------------
@@ -623,7 +640,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
             // position in this cluster's sequence of (item, k block) fills
             int item = cluster_id, kb = 0;
             ItemInfo it{};
-            auto start_item = [&]() { if (item < p.n_items) { it = decode_item_pair(p, item, (int)rank); kb = it.kb0; } };
+            int first_row_unused = 0;
+            auto start_item = [&]() { if (item < p.n_items) { it = decode_item_pair(p, item, (int)rank, &first_row_unused); kb = it.kb0; } };
             auto advance = [&]() {
                 if (item >= p.n_items) return;
                 if (++kb < it.kb1) return;
@@ -632,13 +650,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
             };
             start_item();
             for (int j = 0; j < warp; ++j) advance();
-            auto load_a = [&](int st, uint32_t bar) {
-                if (kPair) {
-                    tma_load_2d_pair(smA + st * kStageA, &p.tmA[0], kb * kBK, it.row0, bar, pol_w);
-                    tma_load_2d_pair(smA + st * kStageA + 64 * kBK * 2, &p.tmA[1], kb * kBK, it.row0, bar, pol_w);
-                } else {
-                    tma_load_2d_pair(smA + st * kStageA, &p.tmA[it.mat], kb * kBK, it.row0, bar, pol_w);
-                }
+            auto load_a = [&](int st, uint32_t bar) {   // this CTA's weight rows (gate/up: the first CTA's are gate rows, the second's up rows)
+                tma_load_2d_pair(smA + st * kStageA, &p.tmA[kPair ? (int)rank : it.mat], kb * kBK, it.row0, bar, pol_w);
             };
             // The weight tiles of the first pipeline fill do not depend on the preceding kernel: requested before the
             // grid-dependency wait; the activation tiles follow after it.
@@ -673,6 +686,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
         // ------------------------------ MMA issuer (one thread of the leader) ------------------------------
         pdl_wait();
         if (rank == 0 && lane == 0) {
+            const uint32_t idesc = idesc_pair(2u * (uint32_t)R);
             int stage = 0, phase = 0, n_local = 0;
             bool ok = true;
             for (int item = cluster_id; item < p.n_items && ok; item += n_clusters, ++n_local) {
@@ -685,10 +699,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
                 for (int kb = it.kb0; kb < it.kb1; ++kb) {
                     if (!(ok = mbar_wait(full_bar(stage), phase, &abort_s, p.status, 3u))) break;
                     tc_fence_after();
-                    const uint64_t da = smem_desc(smA + stage * kStageA), db = smem_desc(smB + stage * kStageB2);
+                    // A = the activation halves (M), B = the weight rows (N)
+                    const uint64_t da = smem_desc(smB + stage * kStageB2), db = smem_desc(smA + stage * kStageA);
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k)
-                        tc_mma_pair(d_tmem, da + 2u * k, db + 2u * k, idesc_pair(), (kb > it.kb0 || k > 0) ? 1u : 0u);
+                        tc_mma_pair(d_tmem, da + 2u * k, db + 2u * k, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
                     tc_commit_pair(empty_bar(stage));     // frees the stage in both CTAs once these MMAs have read it
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
@@ -697,119 +712,107 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
         }
     } else {
         // ------------------------------ epilogue (128 threads of each CTA) ------------------------------
-        // An item's mainloop is short at 128 rows (a few microseconds), so the epilogue must not be a chain of small
-        // tensor-memory loads: four loads of 64 columns (4 blocks of 8 rows) per item, the next one in flight while
-        // the current one is stored.
+        // An item's main loop is short at 128 rows (a few microseconds), so the epilogue must be short too: tensor-memory
+        // loads of 32-64 columns, the next one in flight while the current one is stored, and compact code (a loop,
+        // not thousands of straight-line instructions that would all be instruction-cache misses).
         pdl_wait();
         const int q = warp & 3;
-        const int row_in_tile = q * 32 + lane;
-        const int n_groups = (p.r0 + p.m + 4 * kMaxW - 1) / (4 * kMaxW);   // groups of 4 blocks that hold rows of this pass (<= 4)
+        const int o = 128 * (int)rank + 32 * q + lane;      // operand row of this lane
+        const int blk = o >> 4, i_row = o & 7;              // block of 8 rows, row in the block
+        const int row = blk * kMaxW + i_row;
+        const bool row_ok = (o & 8) == 0 && row >= p.r0 && row < p.r0 + p.m;   // high-half lanes store; lane + 8 holds the low half
+        const int N = 2 * R;
         int n_local = 0;
         bool ok = true;
         for (int item = cluster_id; item < p.n_items && ok; item += n_clusters, ++n_local) {
-            const ItemInfo it = decode_item_pair(p, item, (int)rank);
+            int first_row = 0;
+            const ItemInfo it = decode_item_pair(p, item, (int)rank, &first_row);
             const int buf = n_local & 1;
             const uint32_t use = (uint32_t)(n_local >> 1);
             if (lane == 0) ok = mbar_wait_relaxed(tfull_bar(buf), use & 1u, &abort_s, p.status, 4u);
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            if (kPair) ok = epi_vote(ok, ok_s, n_local, q, lane);
             if (!ok) break;
             tc_fence_after();
             const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * kPairCols;
-            // One group of 4 blocks: finish what sits in v.  The code of a group is kept small and the loop over the
-            // groups is NOT unrolled beyond the two register buffers: an item's epilogue runs once, straight-line code
-            // of thousands of instructions would all be cold instruction-cache misses (measured: 7 us per item).
-            auto finish_group = [&](int g, const uint32_t (&v)[64]) {
-                if constexpr (kPair) {
-                    // tile rows 0-63 (warps 0-1) hold gate projections, rows 64-127 (warps 2-3) the up projections of the
-                    // same columns.  Of the group's four blocks the gate warps finish blocks 0-1 and the up warps blocks
-                    // 2-3: each side hands the other its values for the blocks it does not finish, through a
-                    // double-buffered exchange area (one barrier per group).
-                    float (*xb)[kMaxW][64] = xch_s[g & 1];
-                    const int c = row_in_tile & 63;
-                    const bool up_side = q >= 2;
-                    // (register indices stay compile-time: both candidates are formed, one is selected)
-                    float mine[2][kMaxW];
-#pragma unroll
-                    for (int b = 0; b < 2; ++b) {
-#pragma unroll
-                        for (int i = 0; i < kMaxW; ++i) {
-                            const float lo2 = __uint_as_float(v[b * 16 + i]) + __uint_as_float(v[b * 16 + 8 + i]);
-                            const float hi2 = __uint_as_float(v[(b + 2) * 16 + i]) + __uint_as_float(v[(b + 2) * 16 + 8 + i]);
-                            xb[up_side ? b : b + 2][i][c] = up_side ? lo2 : hi2;    // the block the other side finishes
-                            mine[b][i] = up_side ? hi2 : lo2;
-                        }
-                    }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    const int col = it.row0 + c;
-                    if (c < p.pair_half && col < p.n_rows[0]) {
-                        const size_t F = (size_t)p.n_rows[0];
-#pragma unroll
-                        for (int b = 0; b < 2; ++b) {
-                            const int bk = up_side ? b + 2 : b;    // block (within the group) finished here
-                            const int blk = g * 4 + bk;
-                            __nv_bfloat16* dst = p.swiglu_out + (size_t)blk * 16 * F + col;
-#pragma unroll
-                            for (int i = 0; i < kMaxW; ++i) {
-                                const int row = blk * kMaxW + i;
-                                if (row >= p.r0 && row < p.r0 + p.m) {
-                                    const float other = xb[bk][i][c];
-                                    const float gt = up_side ? other : mine[b][i], u = up_side ? mine[b][i] : other;
-                                    const float val = gt / (1.f + expf(-gt)) * u;
-                                    const __nv_bfloat16 hi = __float2bfloat16_rn(val);
-                                    dst[(size_t)i * F] = hi;
-                                    dst[(size_t)(i + 8) * F] = __float2bfloat16_rn(val - __bfloat162float(hi));
-                                }
-                            }
-                        }
-                    }
-                } else {
-                    const int n = it.row0 + row_in_tile;
-                    if (row_in_tile < p.R && n < p.n_rows[it.mat]) {
-                        const int s = item / p.n_chunks;
-                        // partials [block][split][8][n_total]
-                        float* o = p.out + (((size_t)(g * 4) * p.S + s) * kMaxW) * p.n_total + p.n_off[it.mat] + n;
-                        const size_t blk_stride = (size_t)p.S * kMaxW * p.n_total;
-#pragma unroll
-                        for (int b = 0; b < 4; ++b) {
-#pragma unroll
-                            for (int i = 0; i < kMaxW; ++i) {
-                                const int row = (g * 4 + b) * kMaxW + i;
-                                if (row >= p.r0 && row < p.r0 + p.m)
-                                    o[b * blk_stride + (size_t)i * p.n_total] = __uint_as_float(v[b * 16 + i]) + __uint_as_float(v[b * 16 + 8 + i]);
-                            }
-                        }
-                    }
-                }
-            };
-            if constexpr (kPair) {     // one register buffer: the exchange needs the registers
-                uint32_t va[64];
+            if constexpr (kPair) {
+                // columns 0 .. h-1: gate projections, h .. 2 h - 1: up projections of FFN columns first_row ..
+                const int h = R, F = p.n_rows[0];
+                __nv_bfloat16* dst = p.swiglu_out + ((size_t)blk * 16 + i_row) * F + first_row;   // high halves; low halves 8 rows on
+                uint32_t g[32], u[32];
 #pragma unroll 1
-                for (int g = 0; g < n_groups; ++g) {
-                    tc_ld64_nowait(t0 + (uint32_t)g * 64u, va);
+                for (int c0 = 0; c0 < h; c0 += 32) {
+                    tc_ld32_nowait(t0 + (uint32_t)c0, g);
+                    tc_ld32_nowait(t0 + (uint32_t)(h + c0), u);
                     tc_wait_ld();
-                    finish_group(g, va);
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t hi[4], lo[4];
+#pragma unroll
+                        for (int c2 = 0; c2 < 4; ++c2) {
+                            float val[2];
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                const int c = c8 * 8 + c2 * 2 + e;
+                                const float gh = __uint_as_float(g[c]), uh = __uint_as_float(u[c]);
+                                const float gt = gh + __shfl_down_sync(0xffffffffu, gh, 8), up = uh + __shfl_down_sync(0xffffffffu, uh, 8);
+                                val[e] = gt / (1.f + expf(-gt)) * up;
+                            }
+                            const __nv_bfloat162 vh = __floats2bfloat162_rn(val[0], val[1]);
+                            const __nv_bfloat162 vl = __floats2bfloat162_rn(val[0] - __bfloat162float(vh.x), val[1] - __bfloat162float(vh.y));
+                            hi[c2] = *reinterpret_cast<const uint32_t*>(&vh);
+                            lo[c2] = *reinterpret_cast<const uint32_t*>(&vl);
+                        }
+                        const int c = c0 + c8 * 8;
+                        if (row_ok && c < h && first_row + c < F) {     // h and F are multiples of 8: a piece is all in or all out
+                            *reinterpret_cast<uint4*>(dst + c) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                            *reinterpret_cast<uint4*>(dst + (size_t)8 * F + c) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                        }
+                    }
                 }
             } else {
+                // partials [block][split][8][n_total]; columns first_row .. first_row + N - 1 of matrix it.mat
+                const int s = item / p.n_chunks;
+                float* orow = p.out + (((size_t)blk * p.S + s) * kMaxW + i_row) * p.n_total + p.n_off[it.mat] + first_row;
+                const int n_lim = min(N, p.n_rows[it.mat] - first_row);
+                auto finish_group = [&](int c0, const uint32_t (&v)[64]) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 16; ++c4) {
+                        float x[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float hi = __uint_as_float(v[c4 * 4 + e]);
+                            x[e] = hi + __shfl_down_sync(0xffffffffu, hi, 8);
+                        }
+                        const int c = c0 + c4 * 4;
+                        if (row_ok && c < n_lim) {
+                            if (c + 3 < n_lim) {
+                                *reinterpret_cast<float4*>(orow + c) = make_float4(x[0], x[1], x[2], x[3]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    if (c + e < n_lim) orow[c + e] = x[e];
+                            }
+                        }
+                    }
+                };
                 uint32_t va[64], vb[64];
                 tc_ld64_nowait(t0, va);
 #pragma unroll 1
-                for (int g = 0; g < n_groups; g += 2) {     // two groups per trip: one register buffer each, the next load in flight
+                for (int c0 = 0; c0 < N; c0 += 128) {     // two groups of 64 columns per trip: one register buffer each
                     tc_wait_ld();
-                    if (g + 1 < n_groups) tc_ld64_nowait(t0 + (uint32_t)(g + 1) * 64u, vb);
-                    finish_group(g, va);
-                    if (g + 1 < n_groups) {
+                    if (c0 + 64 < N) tc_ld64_nowait(t0 + (uint32_t)(c0 + 64), vb);
+                    finish_group(c0, va);
+                    if (c0 + 64 < N) {
                         tc_wait_ld();
-                        if (g + 2 < n_groups) tc_ld64_nowait(t0 + (uint32_t)(g + 2) * 64u, va);
-                        finish_group(g + 1, vb);
+                        if (c0 + 128 < N) tc_ld64_nowait(t0 + (uint32_t)(c0 + 128), va);
+                        finish_group(c0 + 64, vb);
                     }
                 }
             }
-            // every load of this accumulator has completed (the last group's wait): it may be overwritten
+            // every load of this accumulator has completed: it may be overwritten
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0));
-            if (kPair) asm volatile("bar.sync 1, 128;" ::: "memory");   // the exchange buffers are free for the next item
         }
     }
 
@@ -867,22 +870,16 @@ static int sm_count() { return device_sm_count(); }
 
 // Slab height R (multiple of 8 in [64,128]) and split count S that minimise what the busiest
 // CTA streams.  Depends on the shape only, never on the number of rows.
-// per_item: CTAs that share a work item (a slab is then per_item * R rows); penalty_pm: cost of one more split.
-static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out, int per_item = 1,
-                         int penalty_pm = -1) {
-    if (penalty_pm < 0) penalty_pm = g_split_penalty_pm;
+static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out) {
     double best = 1e300;
     int bR = 128, bS = 1;
     for (int S = 1; S <= max_split && S <= KB; ++S)
         for (int R = 128; R >= 64; R -= 8) {
             long long chunks = 0;
-            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + per_item * R - 1) / (per_item * R);
+            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + R - 1) / R;
             long long items = chunks * S;
             long long per = (items + G - 1) / G;
-            // what a CTA moves into its shared memory per k block: its R weight rows and, for CTA pairs in a wide pass
-            // (bound by the L2 -> SM traffic), its 128-row half of the activation tile as well
-            const int rows_moved = per_item == 2 ? R + 128 : R;
-            double cost = (double)per * rows_moved * ((KB + S - 1) / S) * (1.0 + 0.001 * penalty_pm * S);   // each split adds partial traffic and consumer loads
+            double cost = (double)per * R * ((KB + S - 1) / S) * (1.0 + 0.001 * g_split_penalty_pm * S);   // each split adds partial traffic and consumer loads
             if (cost < best - 1e-9) { best = cost; bR = R; bS = S; }
         }
     *R_out = bR;
@@ -890,12 +887,45 @@ static void choose_split(const int* n_rows, int n_mats, int KB, int max_split, i
 }
 
 // Pair mode: rows of each kind per item (multiple of 8 in [32,64]) that minimise what the busiest CTA streams.
-static int choose_pair_half(int n_rows, int G, int per_item = 1) {
+static int choose_pair_half(int n_rows, int G) {
     double best = 1e300;
     int bh = 64;
     for (int h = 64; h >= 32; h -= 8) {
-        long long items = (n_rows + per_item * h - 1) / (per_item * h);
-        double cost = (double)((items + G - 1) / G) * (per_item == 2 ? 2 * h + 128 : h);   // rows moved per k block, as in choose_split
+        long long items = (n_rows + h - 1) / h;
+        double cost = (double)((items + G - 1) / G) * h;
+        if (cost < best - 1e-9) { best = cost; bh = h; }
+    }
+    return bh;
+}
+
+// Work decomposition of the CTA-pair kernel: R (multiple of 8, <= 128) and the split count that minimise what the
+// busiest cluster spends.  G = clusters.  Measured: a k block costs a cluster 0.34-0.38 us whatever the tile width
+// (N = 112, 160, 176 or 256 columns: the six-stage pipeline is bound by the round trip of a stage, not by the MMA's
+// width), so narrow tiles buy nothing below ~96 rows per CTA: the cost of an item is charged as if it had at least
+// that many (floor 32 / 64 / 96 / 128: 512-token prefill 22.4 / 20.2 / 20.0 / 20.4 ms).
+static int g_pair_floor_rows = 96, g_pair_split_pm = 30;
+static void choose_split_cta_pair(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out) {
+    double best = 1e300;
+    int bR = 128, bS = 1;
+    for (int S = 1; S <= max_split && S <= KB; ++S)
+        for (int R = 128; R >= 8; R -= 8) {
+            long long chunks = 0;
+            for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + 2 * R - 1) / (2 * R);
+            const long long per = (chunks * S + G - 1) / G;
+            const double cost = (double)per * (R > g_pair_floor_rows ? R : g_pair_floor_rows) * ((KB + S - 1) / S) *
+                                (1.0 + 0.001 * g_pair_split_pm * (S - 1));
+            if (cost < best - 1e-9) { best = cost; bR = R; bS = S; }
+        }
+    *R_out = bR;
+    *S_out = bS;
+}
+// gate/up: FFN columns per item (the first CTA stages that many gate rows, the second as many up rows; never split along k)
+static int choose_cols_cta_pair(int n_rows, int G) {
+    double best = 1e300;
+    int bh = 128;
+    for (int h = 128; h >= 8; h -= 8) {
+        const long long items = (n_rows + h - 1) / h;
+        const double cost = (double)((items + G - 1) / G) * (h > g_pair_floor_rows ? h : g_pair_floor_rows);
         if (cost < best - 1e-9) { best = cost; bh = h; }
     }
     return bh;
@@ -925,14 +955,21 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     for (int j = 0; j < n_mats; ++j) { p.n_rows[j] = n_end[j] - prev; p.n_off[j] = prev; prev = n_end[j]; }
     int chunks = 0;
     const int per_item = cta_pair ? 2 : 1;   // CTAs that share a work item
-    if (pair) {
-        p.pair_half = choose_pair_half(p.n_rows[0], G, per_item);
+    if (pair && cta_pair) {
+        p.pair_half = choose_cols_cta_pair(p.n_rows[0], G);
+        p.R = p.pair_half;
+        p.S = 1;
+        chunks = (p.n_rows[0] + p.pair_half - 1) / p.pair_half;
+        for (int j = 0; j < 3; ++j) p.chunk_end[j] = chunks;
+    } else if (pair) {
+        p.pair_half = choose_pair_half(p.n_rows[0], G);
         p.R = 2 * p.pair_half;
         p.S = 1;
-        chunks = (p.n_rows[0] + per_item * p.pair_half - 1) / (per_item * p.pair_half);
+        chunks = (p.n_rows[0] + p.pair_half - 1) / p.pair_half;
         for (int j = 0; j < 3; ++j) p.chunk_end[j] = chunks;
     } else {
-        choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S, per_item, cta_pair ? 30 : g_split_penalty_pm);
+        if (cta_pair) choose_split_cta_pair(p.n_rows, n_mats, p.KB, kMaxSplit, G, &p.R, &p.S);
+        else choose_split(p.n_rows, n_mats, p.KB, head ? 1 : kMaxSplit, G, &p.R, &p.S);
         for (int j = 0; j < 3; ++j) {
             if (j < n_mats) chunks += (p.n_rows[j] + per_item * p.R - 1) / (per_item * p.R);
             p.chunk_end[j] = chunks;
