@@ -487,7 +487,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_tc(const __grid_constant__ Tc
 // (2 R rows, R of them staged by each CTA), and N can be any multiple of 16: the host picks the tile width that
 // spreads a matrix evenly over the clusters (gate/up of the 7B shape: 22016 rows are 1.16 rounds of 128-row tiles,
 // i.e. 2 rounds at 62 % fill with weights as M; as N they are two rounds of 160 columns).  Measured, a k block costs a
-// cluster the same 0.34-0.38 us at every width (the pipeline is bound by a stage's round trip), so the decomposition
+// cluster the same 0.34-0.38 us at every width tried (at N = 256 that is the measured tensor peak), so the decomposition
 // prefers wide tiles and few k blocks per cluster.  Both CTAs stage their operand halves with plain TMA copies, each into its own shared memory; the
 // MMA, issued by one thread of the first CTA, reads both halves out of both CTAs' shared memory.
 //
@@ -901,8 +901,8 @@ static int choose_pair_half(int n_rows, int G) {
 
 // Work decomposition of the CTA-pair kernel: R (multiple of 8, <= 128) and the split count that minimise what the
 // busiest cluster spends.  G = clusters.  Measured: a k block costs a cluster 0.34-0.38 us whatever the tile width
-// (N = 112, 160, 176 or 256 columns: the six-stage pipeline is bound by the round trip of a stage, not by the MMA's
-// width), so narrow tiles buy nothing below ~96 rows per CTA: the cost of an item is charged as if it had at least
+// (N = 112, 160, 176 or 256 columns; at 256 that is the measured tensor peak, and 4 stages instead of 6 cost 5 % only),
+// so narrow tiles buy nothing below ~96 rows per CTA: the cost of an item is charged as if it had at least
 // that many (floor 32 / 64 / 96 / 128: 512-token prefill 22.4 / 20.2 / 20.0 / 20.4 ms).
 static int g_pair_floor_rows = 96, g_pair_split_pm = 30;
 static void choose_split_cta_pair(const int* n_rows, int n_mats, int KB, int max_split, int G, int* R_out, int* S_out) {
