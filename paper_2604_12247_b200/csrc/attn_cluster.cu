@@ -22,7 +22,10 @@ constexpr int kMaxPairGroup = 8;
 
 // PG = (row, query head) pairs handled per sweep over the staged tile: the largest of 8, 4, 2, 1 that
 // divides what each warp gets, so that the inner loops carry no run-time predicates.
-template <typename T, int HD, int PG>
+// kBig: clusters of 9 .. 16 chunk CTAs (contexts of up to 2048 positions; a non-portable cluster size, used for models
+// with so few KV heads that all clusters are resident at once): the chunk partials are folded in two groups of eight
+// and the groups in order -- the two-level fold of the chunk merge kernel, which for a single group is the plain one.
+template <typename T, int HD, int PG, bool kBig>
 __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     constexpr int kPairGroup = PG;
     constexpr int E = HD / 32;                       // channels per lane in P.V
@@ -270,26 +273,37 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
             int row = a.r0 + i;
             int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own (<= cluster size)
             float M = -INFINITY, L = 0.f, O = 0.f;
-            float mc[kBatch], lc[kBatch], oc[kBatch];
+            float Mf = -INFINITY, Lf = 0.f, Of = 0.f;   // kBig: the fold over the groups
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                mc[u] = -INFINITY; lc[u] = 0.f; oc[u] = 0.f;
-                if (u < n_chunks) {
-                    uint32_t base;
-                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(base) : "r"(out_local + (uint32_t)(p * (HD + 2)) * 4u), "r"(u));
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mc[u]) : "r"(base + (uint32_t)HD * 4u) : "memory");
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(lc[u]) : "r"(base + (uint32_t)(HD + 1) * 4u) : "memory");
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(oc[u]) : "r"(base + (uint32_t)e * 4u) : "memory");
+            for (int g0 = 0; g0 < (kBig ? 2 : 1); ++g0) {
+                float mc[kBatch], lc[kBatch], oc[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    mc[u] = -INFINITY; lc[u] = 0.f; oc[u] = 0.f;
+                    if (g0 * kBatch + u < n_chunks) {
+                        uint32_t base;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(base) : "r"(out_local + (uint32_t)(p * (HD + 2)) * 4u), "r"(g0 * kBatch + u));
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mc[u]) : "r"(base + (uint32_t)HD * 4u) : "memory");
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(lc[u]) : "r"(base + (uint32_t)(HD + 1) * 4u) : "memory");
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(oc[u]) : "r"(base + (uint32_t)e * 4u) : "memory");
+                    }
                 }
-            }
+                if (kBig) { M = -INFINITY; L = 0.f; O = 0.f; }
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                if (mc[u] > -INFINITY) {
+                for (int u = 0; u < kBatch; ++u) {
+                    if (mc[u] > -INFINITY) {
+                        float f0, f1;
+                        attn_fold(M, L, mc[u], lc[u], f0, f1);
+                        O = attn_fold_out(O, oc[u], f0, f1);
+                    }
+                }
+                if (kBig && M > -INFINITY) {
                     float f0, f1;
-                    attn_fold(M, L, mc[u], lc[u], f0, f1);
-                    O = attn_fold_out(O, oc[u], f0, f1);
+                    attn_fold(Mf, Lf, M, L, f0, f1);
+                    Of = attn_fold_out(Of, O, f0, f1);
                 }
             }
+            if (kBig) { L = Lf; O = Of; }
             using A = Act<T>;
             A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (kvh * G + g) * HD + e, a.H * HD, attn_finish(O, L));
         }
@@ -304,18 +318,19 @@ static size_t cluster_attn_smem(int P, int HD, size_t elt) {
            (size_t)kPosWarps * P * (HD + 2) * 4 + (size_t)P * (HD + 2) * 4;
 }
 // Returns false if the device cannot co-schedule such a cluster or the pairs do not fit (nothing is launched then).
-template <typename T, int HD, int PG>
+template <typename T, int HD, int PG, bool kBig>
 static bool launch_cluster_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem, int cluster_y) {
-    auto kernel = k_attn_cluster<T, HD, PG>;
+    auto kernel = k_attn_cluster<T, HD, PG, kBig>;
     static bool configured[kMaxDevices];             // function attributes are per device
     const int dev = current_device();
     if (dev < 0 || smem > 200 * 1024) return false;
     if (!configured[dev]) {
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
+        if (kBig && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) (void)cudaGetLastError();
         configured[dev] = true;
     }
     if (cluster_y > 1) {
-        static int fits_dev[kMaxDevices][9];             // per device and cluster size: 0 unknown, 1 yes, -1 no
+        static int fits_dev[kMaxDevices][17];            // per device and cluster size: 0 unknown, 1 yes, -1 no
         int* fits = fits_dev[dev];
         if (fits[cluster_y] == 0) {
             cudaLaunchConfig_t cfg{};
@@ -326,7 +341,9 @@ static bool launch_cluster_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, siz
             cfg.attrs = at; cfg.numAttrs = 1;
             int n = 0;
             if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-            fits[cluster_y] = n > 0 ? 1 : -1;
+            // big clusters only where every cluster of the grid is resident at once (one per KV head)
+            fits[cluster_y] = (kBig ? n >= (int)grid.x : n > 0) ? 1 : -1;
+            if (getenv("SB_DEBUG")) fprintf(stderr, "[specbound] attention clusters of %d CTAs: %d resident at once, %u wanted\n", cluster_y, n, grid.x);
         }
         if (fits[cluster_y] < 0) return false;
     }
@@ -339,15 +356,23 @@ static bool launch_cluster_hd(cudaStream_t st, const AttnArgs& a, dim3 grid, int
     // pairs per sweep: the largest of 8, 4, 2, 1 that divides what each of a block's two warps gets
     const int P0 = (P + 1) / 2, P1 = P - P0;
     auto divides = [&](int g) { return P0 % g == 0 && P1 % g == 0; };
-    if (divides(8)) return launch_cluster_pg<T, HD, 8>(st, a, grid, smem, cluster_y);
-    if (divides(4)) return launch_cluster_pg<T, HD, 4>(st, a, grid, smem, cluster_y);
-    if (divides(2)) return launch_cluster_pg<T, HD, 2>(st, a, grid, smem, cluster_y);
-    return launch_cluster_pg<T, HD, 1>(st, a, grid, smem, cluster_y);
+    if (cluster_y > 8) {
+        if (divides(8)) return launch_cluster_pg<T, HD, 8, true>(st, a, grid, smem, cluster_y);
+        if (divides(4)) return launch_cluster_pg<T, HD, 4, true>(st, a, grid, smem, cluster_y);
+        if (divides(2)) return launch_cluster_pg<T, HD, 2, true>(st, a, grid, smem, cluster_y);
+        return launch_cluster_pg<T, HD, 1, true>(st, a, grid, smem, cluster_y);
+    }
+    if (divides(8)) return launch_cluster_pg<T, HD, 8, false>(st, a, grid, smem, cluster_y);
+    if (divides(4)) return launch_cluster_pg<T, HD, 4, false>(st, a, grid, smem, cluster_y);
+    if (divides(2)) return launch_cluster_pg<T, HD, 2, false>(st, a, grid, smem, cluster_y);
+    return launch_cluster_pg<T, HD, 1, false>(st, a, grid, smem, cluster_y);
 }
 
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a) {
     int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
-    if (n_chunks > 8) return false;   // portable cluster size
+    // up to 8 chunks: the portable cluster size.  9 .. 16: only where all clusters fit on the device at once, one CTA
+    // per SM (models with few KV heads); elsewhere the chunk kernel with its three CTAs per SM does better
+    if (n_chunks > 16 || (n_chunks > 8 && a.Hkv * n_chunks > device_sm_count())) return false;
     dim3 grid(a.Hkv, n_chunks);
     switch (a.hd) {
         case 32: return launch_cluster_hd<T, 32>(st, a, grid, n_chunks);
