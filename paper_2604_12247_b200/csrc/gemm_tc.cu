@@ -756,7 +756,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_pair(const __grid_constant
                                 const int c = c8 * 8 + c2 * 2 + e;
                                 const float gh = __uint_as_float(g[c]), uh = __uint_as_float(u[c]);
                                 const float gt = gh + __shfl_down_sync(0xffffffffu, gh, 8), up = uh + __shfl_down_sync(0xffffffffu, uh, 8);
-                                val[e] = gt / (1.f + expf(-gt)) * up;
+                                val[e] = __fdividef(gt, 1.f + __expf(-gt)) * up;   // fast exponential and division: this epilogue is a chain of dependent instructions on one warp per scheduler
                             }
                             const __nv_bfloat162 vh = __floats2bfloat162_rn(val[0], val[1]);
                             const __nv_bfloat162 vl = __floats2bfloat162_rn(val[0] - __bfloat162float(vh.x), val[1] - __bfloat162float(vh.y));
