@@ -11,8 +11,8 @@
 // out of one another's shared memory.  The arithmetic is that of attn_common.cuh: bit-identical to the chunk kernel +
 // chunk merge that longer contexts use (kernels_small.cu).  This is the latency-critical variant: at these lengths a
 // CTA per SM is all there is, and every microsecond between the QKV GEMM and the output projection is on the layer's
-// critical path; the chunk kernel of the long contexts (3 CTAs per SM, asynchronous 16-byte staging, block partials
-// over the K tile) measured 1.3 us per layer slower here.
+// critical path; the layout of the long contexts' chunk kernel (3 CTAs per SM, block partials over the K tile) measured
+// about 1 us per layer slower here.
 #include "attn_common.cuh"
 
 namespace sb {

@@ -246,6 +246,19 @@ struct AttnLayout {
     }
 };
 
+// mbarrier wait that lets the hardware park the thread for up to `ns` nanoseconds instead of spinning
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
 // PG = (row, query head) pairs handled per sweep over a staged block: 1, 2, 4 or 8; the pair count is padded to a
 // multiple of it (padding pairs compute on zero queries and are never written), so the inner loops carry no
 // run-time predicates and each K element is unpacked once for up to 8 pairs.
@@ -277,8 +290,6 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
-    const int g_shift = (G & (G - 1)) == 0 ? __ffs(G) - 1 : -1;   // G is 1, 2 or 4 in practice: a shift instead of a division
-    auto row_of = [&](int p) { return g_shift >= 0 ? p >> g_shift : p / G; };
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const int Ppad = lay.Ppad;
@@ -294,44 +305,67 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         return lay.alias ? reinterpret_cast<float*>(k_tiles + (size_t)w * 32 * ROWB_K)
                          : reinterpret_cast<float*>(smem + lay.off_mrg) + (size_t)w * Ppad * (HD + 2);
     };
+    __shared__ __align__(8) unsigned long long stage_bar[kPosWarps];
+    if (threadIdx.x < kPosWarps) mbar_init(smem_u32(&stage_bar[threadIdx.x]), WPB);   // one arrival per warp of the block
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+
     const int pos_last = a.pos0 + a.r0 + a.m - 1;
     const int pos_new0 = kFront ? a.pos0 + a.r0 : pos_last + 1;   // first position whose K,V this launch creates
     const int tbase = c * kAttnChunk + v * 32;
     const int my_t = tbase + lane;
+    // The page table is set up when the context is created (or, for the stateless call, before the call)
+    // and no kernel of a launch sequence writes it: like the weights it may be read before the wait.
+    int my_page = 0;
+    if (my_t < pos_new0) my_page = a.page_table[my_t >> a.page_shift];
     // Rows of EARLIER steps of this layer (positions below pos_done) are complete when this kernel starts: between such
     // steps the stream holds a launch without programmatic overlap (the embedding kernel that starts every step, or
     // the clear of a stateless call).  Their copies -- the long, cold loads of this kernel -- start before the
     // grid-dependency wait.  Separate form: the RoPE/append kernel right before this one wrote the rows from
-    // pos_done on; they are staged after the wait.  (The page table is set up when the context is created -- or, for
-    // the stateless call, before the call -- and no kernel of a launch sequence writes it: like the weights it may be
-    // read before the wait.)
+    // pos_done on; they are staged after the wait, on the same barrier (the warp arrives with the second batch).
     const int pos_done = kFront ? pos_new0 : pos_pred0;
-    // 1. stage the chunk's K and V rows with 16-byte asynchronous copies (each thread a column of pieces: the copies of
-    //    a warp cover two whole rows); rows beyond the last position are zeroed (their probabilities are 0, but
+    __syncthreads();   // barriers initialised
+    // 1. stage the block's K and V rows: one TMA copy per row of an earlier launch (two warps per block: the first
+    //    takes K, the second V); rows beyond the last position are zeroed (their probabilities are 0, but
     //    0 * garbage must stay 0); rows this launch creates are written in step 2
     constexpr uint32_t kRowBytes = HD * (uint32_t)sizeof(T);
-    constexpr int kPieces = (int)kRowBytes / 16;                 // 16-byte pieces per row
-    auto stage_rows = [&](int lo, int hi, bool zero_tail) {      // rows of this chunk at positions [lo, hi)
-        for (int idx = threadIdx.x; idx < 2 * kAttnChunk * kPieces; idx += blockDim.x) {
-            const int which = idx / (kAttnChunk * kPieces);      // 0 = K, 1 = V
-            const int rem = idx - which * (kAttnChunk * kPieces);
-            const int r = rem / kPieces, piece = rem - r * kPieces;
-            const int t = c * kAttnChunk + r;
-            unsigned char* dst = (which ? v_tiles + (size_t)r * ROWB_V : k_tiles + (size_t)r * ROWB_K) + piece * 16;
-            if (t >= lo && t < hi) {
-                const int page = a.page_table[t >> a.page_shift];
-                const unsigned char* src = reinterpret_cast<const unsigned char*>(which ? a.v_cache : a.k_cache) +
-                                           (((size_t)page * a.page + (t & (a.page - 1))) * kvd + (size_t)kvh * HD) * sizeof(T) + piece * 16;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-            } else if (zero_tail && t > pos_last) {
-                *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+    const int which0 = WPB == 2 ? hsel : 0, which1 = WPB == 2 ? hsel + 1 : 2;   // 0 = K, 1 = V
+    {
+        const bool early = my_t < pos_done;
+        const uint32_t bar = smem_u32(&stage_bar[v]);
+        const unsigned n_early = __popc(__ballot_sync(0xffffffffu, early));
+        if (lane == 0) {
+            if (kFront) mbar_expect_tx(bar, (uint32_t)(which1 - which0) * n_early * kRowBytes);
+            else mbar_expect_tx_only(bar, (uint32_t)(which1 - which0) * n_early * kRowBytes);
+        }
+        __syncwarp();
+        for (int which = which0; which < which1; ++which) {
+            unsigned char* row = which ? V_w + lane * ROWB_V : K_w + lane * ROWB_K;
+            if (early) {
+                const T* src = reinterpret_cast<const T*>(which ? a.v_cache : a.k_cache) +
+                               ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                bulk_load(smem_u32(row), src, kRowBytes, bar);
+            } else if (my_t > pos_last) {
+#pragma unroll
+                for (int j = 0; j < (int)kRowBytes / 16; ++j) reinterpret_cast<uint4*>(row)[j] = make_uint4(0u, 0u, 0u, 0u);
             }
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-    stage_rows(0, pos_done, true);
+    }
     pdl_wait();
-    if (!kFront) stage_rows(pos_done, pos_new0, false);   // the rows the RoPE/append kernel just wrote
+    if (!kFront) {   // the rows the RoPE/append kernel just wrote
+        const bool late = my_t >= pos_done && my_t < pos_new0;
+        const uint32_t bar = smem_u32(&stage_bar[v]);
+        const unsigned n_late = __popc(__ballot_sync(0xffffffffu, late));
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(which1 - which0) * n_late * kRowBytes);
+        __syncwarp();
+        if (late) {
+            for (int which = which0; which < which1; ++which) {
+                unsigned char* row = which ? V_w + lane * ROWB_V : K_w + lane * ROWB_K;
+                const T* src = reinterpret_cast<const T*>(which ? a.v_cache : a.k_cache) +
+                               ((size_t)my_page * a.page + (my_t & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                bulk_load(smem_u32(row), src, kRowBytes, bar);
+            }
+        }
+    }
     // 2. while those copies fly: q, and (front end) the new positions' K and V
     for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[idx] = 0.f;   // padding pairs
     if (kFront) {
@@ -348,7 +382,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         auto item_of = [&](int idx) -> Item {
             if (idx < n_q) {
                 int p = idx / half;
-                return Item{0, a.pos0 + a.r0 + row_of(p), idx - p * half, p};
+                return Item{0, a.pos0 + a.r0 + p / G, idx - p * half, p};
             }
             int j = idx - n_q, it = j % HD;
             return Item{it >= half ? 2 : 1, lo + j / HD, it >= half ? it - half : it, 0};
@@ -367,7 +401,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 if (idx < n_items) {
                     const Item it = item_of(idx);
                     const float* p0 = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
-                                      (it.kind == 0 ? (kvh * G + (it.p - row_of(it.p) * G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+                                      (it.kind == 0 ? (kvh * G + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
                     x0[u] = sum_splits(p0, sstride, a.n_split);
                     x1[u] = sum_splits(p0 + half, sstride, a.n_split);
                     if (it.kind != 2) cs[u] = rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2);
@@ -400,11 +434,22 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     } else {
         for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
             int p = idx / HD, e = idx - p * HD;
-            int i = row_of(p), g = p - i * G;
+            int i = p / G, g = p - i * G;
             q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
         }
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");   // this thread's copies have landed
+    {   // bounded wait for this block's copies
+        const uint32_t bar = smem_u32(&stage_bar[v]);
+        if (!mbar_try_wait(bar, 0)) {
+            const unsigned long long t0 = clock64();
+            while (!mbar_try_wait_parked(bar, 0, 2000u)) {
+                if (clock64() - t0 > kStageWaitCycles) {
+                    if (a.status) atomicExch(a.status, 5u);
+                    break;
+                }
+            }
+        }
+    }
     __syncthreads();   // q_s, the rows of step 2 and every block's tiles are complete
 
     const float scale = attn_score_scale(HD);
@@ -446,7 +491,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         float mx[kPairGroup], ls[kPairGroup];
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
-            int i = row_of(pg + pp);
+            int i = (pg + pp) / G;
             bool on = my_t <= a.pos0 + a.r0 + i;         // causal: a row sees positions <= its own
             P_w[pp * 32 + lane] = attn_block_softmax(sc[pp], scale, on, mx[pp], ls[pp]);
         }
@@ -504,7 +549,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     // merge the four blocks in block order; thread -> (pair, two channels)
     for (int idx = threadIdx.x; idx < P * (HD / 2); idx += blockDim.x) {
         const int p = idx / (HD / 2), e = (idx - p * (HD / 2)) * 2;
-        const int i = row_of(p), g = p - i * G;
+        const int i = p / G, g = p - i * G;
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kPosWarps; ++w) M = fmaxf(M, mrg_blk(w)[(size_t)p * (HD + 2) + HD]);
