@@ -34,9 +34,11 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     constexpr int ROWB = HD * (int)sizeof(T) + 16;   // padded row pitch: lane-per-row 16-byte reads are conflict-free
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
-    const int kvh = blockIdx.x, c = blockIdx.y;
+    const int gs = a.gsplit > 1 ? a.gsplit : 1;      // CTAs that share a KV head's query heads
+    const int kvh = (int)blockIdx.x / gs, gsub = (int)blockIdx.x - kvh * gs, c = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
+    const int G = a.H / a.Hkv / gs, P = a.m * G;     // this CTA's query heads of the group; pair p = i * G + g: row r0 + i, query head head0 + g
+    const int head0 = kvh * (a.H / a.Hkv) + gsub * G;
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD]
     unsigned char* kv_s = smem + (size_t)P * HD * 4;                                // per warp: K[32], V[32]
@@ -118,7 +120,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
                 if (idx < n_items) {
                     const Item it = item_of(idx);
                     const float* p0 = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
-                                      (it.kind == 0 ? (kvh * G + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+                                      (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
                     x0[u] = sum_splits(p0, sstride, a.n_split);
                     x1[u] = sum_splits(p0 + half, sstride, a.n_split);
                     if (it.kind != 2) cs[u] = rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2);
@@ -139,8 +141,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
                     const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
                     T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
                     T* dst = cache + ((size_t)page[u] * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
-                    dst[it.e2] = y0;
-                    dst[it.e2 + half] = y1;
+                    if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
+                        dst[it.e2] = y0;
+                        dst[it.e2 + half] = y1;
+                    }
                     int tl = it.pos - c * kAttnChunk;
                     T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
                     srow[it.e2] = y0;
@@ -305,7 +309,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
             }
             if (kBig) { L = Lf; O = Of; }
             using A = Act<T>;
-            A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (kvh * G + g) * HD + e, a.H * HD, attn_finish(O, L));
+            A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (head0 + g) * HD + e, a.H * HD, attn_finish(O, L));
         }
     }
     __syncthreads();
@@ -330,9 +334,9 @@ static bool launch_cluster_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, siz
         configured[dev] = true;
     }
     if (cluster_y > 1) {
-        static int fits_dev[kMaxDevices][17];            // per device and cluster size: 0 unknown, 1 yes, -1 no
-        int* fits = fits_dev[dev];
-        if (fits[cluster_y] == 0) {
+        static int resident_dev[kMaxDevices][17];        // per device and cluster size: clusters resident at once + 1 (0 = not asked yet)
+        int* resident = resident_dev[dev];
+        if (resident[cluster_y] == 0) {
             cudaLaunchConfig_t cfg{};
             cfg.gridDim = grid; cfg.blockDim = dim3(kAttnWarps * 32); cfg.dynamicSmemBytes = 200 * 1024;
             cudaLaunchAttribute at[1];
@@ -341,17 +345,17 @@ static bool launch_cluster_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, siz
             cfg.attrs = at; cfg.numAttrs = 1;
             int n = 0;
             if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-            // big clusters only where every cluster of the grid is resident at once (one per KV head)
-            fits[cluster_y] = (kBig ? n >= (int)grid.x : n > 0) ? 1 : -1;
-            if (getenv("SB_DEBUG")) fprintf(stderr, "[specbound] attention clusters of %d CTAs: %d resident at once, %u wanted\n", cluster_y, n, grid.x);
+            resident[cluster_y] = n + 1;
+            if (getenv("SB_DEBUG")) fprintf(stderr, "[specbound] attention clusters of %d CTAs: %d resident at once\n", cluster_y, n);
         }
-        if (fits[cluster_y] < 0) return false;
+        // big clusters only where every cluster of the grid is resident at once
+        if (resident[cluster_y] - 1 < (kBig ? (int)grid.x : 1)) return false;
     }
     return launch_kc(kernel, grid, dim3(kAttnWarps * 32), smem, st, cluster_y, a) == cudaSuccess;
 }
 template <typename T, int HD>
 static bool launch_cluster_hd(cudaStream_t st, const AttnArgs& a, dim3 grid, int cluster_y) {
-    const int P = a.m * (a.H / a.Hkv);
+    const int P = a.m * (a.H / a.Hkv) / (a.gsplit > 1 ? a.gsplit : 1);
     size_t smem = cluster_attn_smem(P, HD, sizeof(T));
     // pairs per sweep: the largest of 8, 4, 2, 1 that divides what each of a block's two warps gets
     const int P0 = (P + 1) / 2, P1 = P - P0;
@@ -372,13 +376,27 @@ template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArg
     int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
     // up to 8 chunks: the portable cluster size.  9 .. 16: only where all clusters fit on the device at once, one CTA
     // per SM (models with few KV heads); elsewhere the chunk kernel with its three CTAs per SM does better
-    if (n_chunks > 16 || (n_chunks > 8 && a.Hkv * n_chunks > device_sm_count())) return false;
-    dim3 grid(a.Hkv, n_chunks);
-    switch (a.hd) {
-        case 32: return launch_cluster_hd<T, 32>(st, a, grid, n_chunks);
-        case 64: return launch_cluster_hd<T, 64>(st, a, grid, n_chunks);
-        default: return launch_cluster_hd<T, 128>(st, a, grid, n_chunks);
+    if (n_chunks > 16) return false;
+    // Grouped-query models: with few KV heads there are fewer CTAs than SMs, each doing the CUDA-core work of all its
+    // group's (row, head) pairs; spread a group's query heads over 2 or 4 CTAs while all CTAs still fit the device at once
+    // (every one of them stages the KV head's rows: a few MB more out of L2).  A split that cannot be launched (big
+    // clusters that are not all resident) falls back to the next smaller one.
+    const int Gfull = a.H / a.Hkv, sms = device_sm_count();
+    for (int gs = 4; gs >= 1; gs >>= 1) {
+        if (Gfull % gs || (gs > 1 && a.Hkv * gs * n_chunks > sms)) continue;
+        if (n_chunks > 8 && a.Hkv * gs * n_chunks > sms) continue;      // big clusters: one wave only
+        AttnArgs b = a;
+        b.gsplit = gs;
+        dim3 grid(a.Hkv * gs, n_chunks);
+        bool ok;
+        switch (a.hd) {
+            case 32: ok = launch_cluster_hd<T, 32>(st, b, grid, n_chunks); break;
+            case 64: ok = launch_cluster_hd<T, 64>(st, b, grid, n_chunks); break;
+            default: ok = launch_cluster_hd<T, 128>(st, b, grid, n_chunks); break;
+        }
+        if (ok) return true;
     }
+    return false;
 }
 
 template bool launch_attention_fused<float>(cudaStream_t, const AttnArgs&);

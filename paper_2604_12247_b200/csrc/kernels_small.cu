@@ -279,7 +279,8 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     constexpr int ROWB_K = HD * (int)sizeof(T) + 16, ROWB_V = HD * (int)sizeof(T);
     extern __shared__ __align__(16) unsigned char smem[];
     pdl_trigger();
-    const int kvh = blockIdx.x, c = blockIdx.y;
+    const int gs = a.gsplit > 1 ? a.gsplit : 1;      // CTAs that share a KV head's query heads
+    const int kvh = (int)blockIdx.x / gs, gsub = (int)blockIdx.x - kvh * gs, c = blockIdx.y;
     const int pos_pred0 = a.pos_pred0 >= 0 ? a.pos_pred0 : a.pos0 + a.r0;   // separate form: first position the preceding RoPE/append launch wrote
     if (!kFront && a.n_blocks > 1) {                 // several blocks of 8 rows in one launch: this CTA's block
         const int blk = blockIdx.z;
@@ -289,7 +290,8 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         if (c * kAttnChunk > a.pos0 + a.r0 + a.m - 1) return;   // a chunk beyond this block's last position
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = a.H / a.Hkv, P = a.m * G;          // pair p = i * G + g: row r0 + i, query head kvh * G + g
+    const int G = a.H / a.Hkv / gs, P = a.m * G;     // this CTA's query heads of the group; pair p = i * G + g: row r0 + i, query head head0 + g
+    const int head0 = kvh * (a.H / a.Hkv) + gsub * G;
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const int Ppad = lay.Ppad;
@@ -401,7 +403,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 if (idx < n_items) {
                     const Item it = item_of(idx);
                     const float* p0 = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
-                                      (it.kind == 0 ? (kvh * G + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+                                      (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
                     x0[u] = sum_splits(p0, sstride, a.n_split);
                     x1[u] = sum_splits(p0 + half, sstride, a.n_split);
                     if (it.kind != 2) cs[u] = rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2);
@@ -422,8 +424,10 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                     const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
                     T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
                     T* dst = cache + ((size_t)page[u] * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
-                    dst[it.e2] = y0;
-                    dst[it.e2 + half] = y1;
+                    if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
+                        dst[it.e2] = y0;
+                        dst[it.e2 + half] = y1;
+                    }
                     int tl = it.pos - c * kAttnChunk;
                     T* srow = reinterpret_cast<T*>(is_v ? v_tiles + (size_t)tl * ROWB_V : k_tiles + (size_t)tl * ROWB_K);
                     srow[it.e2] = y0;
@@ -435,7 +439,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
             int p = idx / HD, e = idx - p * HD;
             int i = p / G, g = p - i * G;
-            q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (kvh * G + g) * HD + e];
+            q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (head0 + g) * HD + e];
         }
     }
     {   // bounded wait for this block's copies
@@ -568,7 +572,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 }
             }
         }
-        float* dst = a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + kvh * G + g) * (HD + 2);
+        float* dst = a.part + (((size_t)c * kMaxW + (a.r0 + i)) * a.H + head0 + g) * (HD + 2);
         *reinterpret_cast<float2*>(dst + e) = make_float2(O0, O1);
         if (e == 0) {
             dst[HD] = M;
@@ -658,7 +662,7 @@ __global__ void __launch_bounds__(kChunkGroup * 32) k_attn_combine(AttnArgs a) {
 template <typename T, int HD, int PG, bool kFront, int WPB>
 static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid) {
     auto kernel = k_attn_partial<T, HD, PG, kFront, WPB>;
-    const int P = a.m * (a.H / a.Hkv);
+    const int P = a.m * (a.H / a.Hkv) / (a.gsplit > 1 ? a.gsplit : 1);
     const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const dim3 block(kPosWarps * WPB * 32);
     static bool configured[kMaxDevices];             // function attributes are per device
@@ -673,7 +677,7 @@ static bool launch_attn_pg(cudaStream_t st, const AttnArgs& a, dim3 grid) {
 }
 template <typename T, int HD, bool kFront>
 static bool launch_attn_partial(cudaStream_t st, const AttnArgs& a, dim3 grid) {
-    const int P = a.m * (a.H / a.Hkv);
+    const int P = a.m * (a.H / a.Hkv) / (a.gsplit > 1 ? a.gsplit : 1);
     // Two warps per 32-position block share the pairs (latency hides behind warps, not behind instruction-level
     // parallelism: one warp per block with twice the pairs measured slower at every context length); pairs per sweep =
     // what one of the two warps gets, padded to 1, 2, 4 or 8.
@@ -704,10 +708,18 @@ template <typename T> void launch_attention_combine(cudaStream_t st, const AttnA
 }
 
 // Contexts of any length in two launches: the chunk kernel with its front end (RoPE, cache append) and the chunk merge.
-template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a) {
-    if (a.n_blocks > 1) return false;
-    int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
-    dim3 grid(a.Hkv, n_chunks);
+template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a0) {
+    if (a0.n_blocks > 1) return false;
+    int n_chunks = (a0.pos0 + a0.r0 + a0.m - 1) / kAttnChunk + 1;
+    // grouped-query models: a KV head's query heads over 2 or 4 CTAs (see launch_attention_fused) while the grid stays
+    // within two CTAs per SM: beyond that the copies of the KV rows that every CTA of a group stages cost more than
+    // the shorter sweeps save (Llama-3 geometry, one row, 3000 positions: 97.4 us per layer split, 95.9 unsplit)
+    AttnArgs a = a0;
+    const int Gfull = a.H / a.Hkv, slots = 2 * device_sm_count();
+    a.gsplit = 1;
+    for (int gs = 4; gs > 1; gs >>= 1)
+        if (Gfull % gs == 0 && a.Hkv * gs * n_chunks <= slots) { a.gsplit = gs; break; }
+    dim3 grid(a.Hkv * a.gsplit, n_chunks);
     bool ok;
     switch (a.hd) {
         case 32: ok = launch_attn_partial<T, 32, true>(st, a, grid); break;

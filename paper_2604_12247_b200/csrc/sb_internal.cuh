@@ -396,6 +396,9 @@ struct AttnArgs {
     // separate kernels only: first position that the RoPE/append launch preceding this one wrote (-1: pos0 + r0).
     // K/V rows below it belong to earlier steps and may be fetched before the grid-dependency wait.
     int pos_pred0 = -1;
+    // grouped-query models: the query heads of a KV head spread over gsplit CTAs (1, 2 or 4, a divisor of H / Hkv;
+    // grid.x = Hkv * gsplit), each staging the KV head's rows for itself.  Set by the launchers.
+    int gsplit = 1;
 };
 
 struct RopeArgs {
