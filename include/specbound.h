@@ -298,9 +298,10 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                       SwiGLU as the down projection's operand (otherwise SwiGLU is a kernel of its own).
  *                       The fused GEMM is never split along k, so its sums may round differently from the
  *                       separate kernels' (fp32 rounding level).
- *                    2: RoPE, KV-cache append, attention and the merge of its 128-position chunks run as one
- *                       launch (chunk CTAs of a KV head form a thread-block cluster; up to 8 chunks, longer
- *                       contexts use the separate kernels).  Bit-identical to the separate kernels.
+ *                    2: RoPE, KV-cache append and attention run inside the attention kernel: up to 8 chunks of 128
+ *                       positions (11 for models with few KV heads) in one launch whose chunk CTAs form a
+ *                       thread-block cluster and merge the chunks; longer contexts in two (chunk kernel, chunk merge).
+ *                       Off: three launches (RoPE/append, chunk kernel, chunk merge).  Bit-identical either way.
  *                    Each setting by itself is deterministic and row-invariant.
  *   SB_OPT_QKV_AHEAD (default option only) 1 (default) = while sb_generate waits for an exit decision it already
  *                    issues the RMSNorm and QKV GEMM of the layer step that follows if the row does not exit
