@@ -240,16 +240,40 @@ def oracle_check(ctx, run: inputs.Run, weights_cpu: dict, n_prompt: int, n_gen: 
     t0 = time.perf_counter()
     o = oracle.Oracle(run.shape, weights_cpu, len(toks) + 1)
     top1, _, margin, deficit = o.teacher_forced(toks, n_prompt)
+    off = top1 != sp["tokens"]
+    # How far the free-running GPU state has drifted from the oracle's at the position with the smallest margin (or the
+    # first one that is not the oracle's top-1): the row that decides that token is run again on both sides layer by
+    # layer (the oracle's cache holds the earlier positions from the pass above), and the ORACLE's head is applied to
+    # both final hidden states.  The drift comes from K/V cache entries that land on a neighbouring bf16 value on one
+    # side; it grows with depth and says how large a margin a legitimate difference can flip.
+    j = int(np.nonzero(off)[0][0]) if off.any() else int(np.argmin(margin))
+    drift = None
+    if j >= 1:
+        pos = n_prompt + j - 1
+        ctx.reset()
+        ctx.prefill(toks[:pos])
+        ctx.draft_push(int(toks[pos]))
+        ctx.draft_advance(run.shape.n_layers)
+        h_gpu = ctx.read_hidden(0).astype(np.float64)
+        ctx.reset()
+        h_orc = o.embed(int(toks[pos]))[None, :]
+        for l in range(1, run.shape.n_layers + 1):
+            h_orc = o.layer_forward(l, h_orc, pos)
+        z_o, z_g = o.final_logits(h_orc[0]), o.final_logits(h_gpu)
+        drift = {"generated_index": j, "margin_there": float(margin[j]),
+                 "hidden_rel_err_last_layer": float(np.abs(h_gpu - h_orc[0]).max() / np.abs(h_orc[0]).max()),
+                 "logit_diff_rms": float(np.sqrt(np.mean((z_g - z_o) ** 2))), "logit_diff_max": float(np.abs(z_g - z_o).max())}
     o.close()
     dt = time.perf_counter() - t0
-    off = top1 != sp["tokens"]
     return {"prompt_tokens": n_prompt, "positions": int(n_gen), "not_top1": int(off.sum()),
             "near_ties": int((margin < 2 * tol).sum()), "wrong": int((off & (margin >= 2 * tol)).sum()),
             "worst_deficit": float(deficit.min()), "logit_tolerance": tol, "smallest_margin": float(margin.min()),
             "tokens_equal_ar": bool(np.array_equal(sp["tokens"], ar["tokens"])), "oracle_seconds": dt,
+            "free_running_drift": drift,
             "what": "teacher-forced oracle pass over a short-prompt generation of this workload (same weights, d_max, w_max, "
                     "tau, threshold); wrong = GPU token differs from the oracle's top-1 at a position whose top-2 margin is "
-                    "not below twice the tolerance"}
+                    "not below twice the tolerance; free_running_drift = the oracle's head applied to the GPU's and to the "
+                    "oracle's final hidden state of the row that decides the token with the smallest margin"}
 
 
 def side_arm(args, workload: str, peak: float, masked: bool = False, steps: int = 3) -> dict:
