@@ -13,6 +13,9 @@ pytestmark = pytest.mark.gpu
 
 SMALL_BF16 = inputs.scaled(inputs.LLAMA3_8B, name="small-bf16", n_layers=4, d_model=512, n_heads=8, n_kv_heads=2,
                            head_dim=64, d_ffn=1408, vocab=2048, head_scale=16.0)
+# the same with an FFN width that is not a multiple of the GEMMs' 64-wide k block (the down projection's last k block
+# is filled up with zeros by the tensor-map's out-of-range rule) nor of the widest tile
+ODD_FFN_BF16 = inputs.scaled(SMALL_BF16, name="small-bf16-odd-ffn", d_ffn=1416)
 OPT_WIDE_PREFILL = 9
 
 
@@ -34,7 +37,15 @@ def _hidden_after_prefill(ctx, prompt, n_layers):
 @pytest.mark.parametrize("wide_mode", [1, 2, 3])
 @pytest.mark.parametrize("n_prompt", [16, 64, 70, 100, 128, 130, 300])
 def test_wide_prefill_matches_narrow_passes_and_oracle(n_prompt, wide_mode):
-    shape = SMALL_BF16
+    _wide_against_narrow_and_oracle(SMALL_BF16, n_prompt, wide_mode)
+
+
+@pytest.mark.parametrize("n_prompt", [70, 130])
+def test_wide_prefill_with_a_ragged_last_k_block(n_prompt):
+    _wide_against_narrow_and_oracle(ODD_FFN_BF16, n_prompt, 1)
+
+
+def _wide_against_narrow_and_oracle(shape, n_prompt, wide_mode):
     w = inputs.make_weights(shape, 5, damp_rho=0.3)
     pr = inputs.make_prompt(shape, n_prompt, 17).numpy()
     max_seq = n_prompt + 24
