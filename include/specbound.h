@@ -316,8 +316,20 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
 enum { SB_OPT_GEMM = 1, SB_OPT_TRACE = 2, SB_OPT_TC_TUNING = 3, SB_OPT_PDL = 4, SB_OPT_L2_PREFETCH = 5,
        SB_OPT_SPLIT_PENALTY = 6, SB_OPT_FUSE = 7, SB_OPT_QKV_AHEAD = 8, SB_OPT_WIDE_PREFILL = 9 };
 int sb_set_option(sb_ctx* ctx, int32_t key, int32_t value);
+
 /* Process-wide default for contexts and stateless calls created afterwards. */
 int sb_set_default_option(int32_t key, int32_t value);
+
+/* The work decomposition the weight-streaming GEMMs of a layer pass use (Section 3.3: the skinny-M GEMMs of the draft
+ * steps and of the unified pass; Section 4.3: prefill).  Host arithmetic only: no device is touched, nothing is launched;
+ * meant for tests and for sizing studies.
+ *   mode 0: the 8-row kernel on `units` CTAs; 1: its gate/up form (n_rows[0] = FFN width, n_mats = 1);
+ *   mode 2: the 128-row kernel on `units` clusters of two CTAs; 3: its gate/up form.
+ *   n_rows[n_mats] (1..3 matrices that share k and the activation operand, HOST array), k = inner dimension.
+ * Out (HOST): rows_per_cta = weight rows a CTA stages per work item (gate/up: FFN columns per item), k_splits, n_items =
+ * slabs x splits.  Returns SB_ERR_ARG for null pointers, mode outside 0..3, n_mats outside 1..3 or non-positive sizes. */
+int sb_plan_gemm(int32_t mode, const int32_t* n_rows, int32_t n_mats, int32_t k, int32_t units, int32_t* rows_per_cta,
+                 int32_t* k_splits, int32_t* n_items);
 
 const char* sb_strerror(int status);
 

@@ -68,7 +68,7 @@ EXPORTS = ("sb_workspace_bytes", "sb_create", "sb_destroy", "sb_load_weights", "
            "sb_read_hidden", "sb_prefill", "sb_draft_push", "sb_draft_advance", "sb_exit_confidence", "sb_verify",
            "sb_generate", "sb_generate_ar", "sb_set_sampling", "sb_sample_uniform", "sb_k_sample", "sb_k_sample_scratch_bytes", "sb_k_scratch_bytes", "sb_k_exit_confidence", "sb_k_exit_confidence_static",
            "sb_k_layer", "sb_k_layer_chain", "sb_k_rope_table", "sb_k_rope_table_bytes",
-           "sb_tau_schedule", "sb_model_speedup", "sb_set_option", "sb_set_default_option", "sb_strerror")
+           "sb_tau_schedule", "sb_model_speedup", "sb_plan_gemm", "sb_set_option", "sb_set_default_option", "sb_strerror")
 
 _lib = None
 
@@ -118,6 +118,7 @@ def lib():
         L.sb_tau_schedule.argtypes = [f32, i32, vp]
         L.sb_model_speedup.restype = C.c_double
         L.sb_model_speedup.argtypes = [i32, C.c_double, i32, i32]
+        L.sb_plan_gemm.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp]
         L.sb_set_option.argtypes = [vp, i32, i32]
         L.sb_set_default_option.argtypes = [i32, i32]
         L.sb_strerror.restype = C.c_char_p
@@ -156,6 +157,14 @@ def tau_schedule(alpha: float, L: int) -> np.ndarray:
 
 def model_speedup(L: int, a: float, w: int, d_max: int) -> float:
     return lib().sb_model_speedup(L, a, w, d_max)
+
+
+def plan_gemm(mode: int, n_rows: Sequence[int], k: int, units: int):
+    """sb_plan_gemm: (rows per CTA, k splits, work items) of a weight-streaming GEMM on `units` CTAs or clusters."""
+    nr = np.ascontiguousarray(n_rows, dtype=np.int32)
+    r, s_, n = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib().sb_plan_gemm(mode, _np_ptr(nr), len(nr), k, units, C.byref(r), C.byref(s_), C.byref(n)), "sb_plan_gemm")
+    return r.value, s_.value, n.value
 
 
 def sample_uniform(seed: int, pos: int) -> float:

@@ -1236,6 +1236,15 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max) {
     return num / ((1.0 - a) * ((double)w * d_max + L - d_max));
 }
 
+int sb_plan_gemm(int32_t mode, const int32_t* n_rows, int32_t n_mats, int32_t k, int32_t units, int32_t* rows_per_cta,
+                 int32_t* k_splits, int32_t* n_items) {
+    if (!rows_per_cta || !k_splits || !n_items) return SB_ERR_ARG;
+    int R = 0, S = 0, items = 0;
+    if (!tc_plan_query(mode, n_rows, n_mats, k, units, &R, &S, &items)) return SB_ERR_ARG;
+    *rows_per_cta = R; *k_splits = S; *n_items = items;
+    return SB_OK;
+}
+
 const char* sb_strerror(int s) {
     switch (s) {
         case SB_OK: return "ok";

@@ -986,6 +986,27 @@ static TcPlan* get_plan(TcPlanCache* cache, const void* const* W, const int* n_e
     return pl;
 }
 
+// The decomposition the launches use, for a given number of CTAs (8-row kernel) or clusters (CTA-pair kernel): host
+// arithmetic only.  mode 0: 8-row kernel, 1: its gate/up form, 2: 128-row CTA-pair kernel, 3: its gate/up form.
+bool tc_plan_query(int mode, const int* n_rows, int n_mats, int K, int units, int* R, int* S, int* n_items) {
+    if (mode < 0 || mode > 3 || !n_rows || n_mats < 1 || n_mats > 3 || K < 1 || units < 1) return false;
+    for (int j = 0; j < n_mats; ++j)
+        if (n_rows[j] < 1) return false;
+    const int KB = (K + kBK - 1) / kBK;
+    if (mode == 1 || mode == 3) {
+        const int h = mode == 3 ? choose_cols_cta_pair(n_rows[0], units) : choose_pair_half(n_rows[0], units);
+        *R = h; *S = 1; *n_items = (n_rows[0] + h - 1) / h;
+        return true;
+    }
+    if (mode == 2) choose_split_cta_pair(n_rows, n_mats, KB, kMaxSplit, units, R, S);
+    else choose_split(n_rows, n_mats, KB, kMaxSplit, units, R, S);
+    const int per = mode == 2 ? 2 : 1;
+    int chunks = 0;
+    for (int j = 0; j < n_mats; ++j) chunks += (n_rows[j] + per * *R - 1) / (per * *R);
+    *n_items = chunks * *S;
+    return true;
+}
+
 template <bool kHead, bool kPair, int NB = 1> static void launch(cudaStream_t st, const TcPlan* pl, const TcParams& p) {
     static bool attr_set[kMaxDevices];   // function attributes are per device
     const int dev = current_device();

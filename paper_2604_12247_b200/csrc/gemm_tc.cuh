@@ -31,6 +31,9 @@ bool tc_set_split_penalty(int per_mille);
 // wide passes (GemmArgs::nb > 1): true (default) = clusters of two CTAs sharing one activation tile (cta_group::2),
 // false = one CTA per work item
 void tc_set_wide_cta_pairs(bool on);
+// the work decomposition for `units` CTAs (modes 0, 1: 8-row kernel, its gate/up form) or clusters (modes 2, 3: CTA-pair
+// kernel, its gate/up form): rows per CTA (gate/up: columns per item), k splits, work items.  Host arithmetic only.
+bool tc_plan_query(int mode, const int* n_rows, int n_mats, int K, int units, int* R, int* S, int* n_items);
 // returns the number of split-K partials written to a.out, or -1 if no TMA descriptor could be made
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& a, TcPlanCache* cache, unsigned int* status);
 bool launch_head_tc(cudaStream_t st, const HeadArgs& a, TcPlanCache* cache, unsigned int* status);
