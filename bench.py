@@ -580,8 +580,11 @@ def micro_arm(args):
     build.build()
     torch.cuda.set_device(0)
     peak, peak_src = measured_peak()
-    s = inputs.scaled(inputs.LLAMA2_7B, n_layers=1)
-    out = {"mode": "micro", "peak_gbs": peak, "peak_source": peak_src, "iters": args.iters, "layer": [], "exit": []}
+    base = inputs.RUNS[args.workload].shape            # --workload picks the layer's geometry (default: the 7B shape)
+    if base.dtype != "bf16":
+        raise SystemExit("--micro needs a bf16 workload")
+    s = inputs.scaled(base, n_layers=1)
+    out = {"mode": "micro", "shape": base.name, "peak_gbs": peak, "peak_source": peak_src, "iters": args.iters, "layer": [], "exit": []}
     ev = lambda: torch.cuda.Event(enable_timing=True)
     cases = [c for c in args.micro_case.split(",") if c] if args.micro_case else None
 

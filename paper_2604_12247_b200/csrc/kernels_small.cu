@@ -711,14 +711,31 @@ template <typename T> void launch_attention_combine(cudaStream_t st, const AttnA
 template <typename T> bool launch_attention_front(cudaStream_t st, const AttnArgs& a0) {
     if (a0.n_blocks > 1) return false;
     int n_chunks = (a0.pos0 + a0.r0 + a0.m - 1) / kAttnChunk + 1;
-    // grouped-query models: a KV head's query heads over 2 or 4 CTAs (see launch_attention_fused) while the grid stays
-    // within two CTAs per SM: beyond that the copies of the KV rows that every CTA of a group stages cost more than
-    // the shorter sweeps save (Llama-3 geometry, one row, 3000 positions: 97.4 us per layer split, 95.9 unsplit)
+    // Grouped-query models: a KV head's query heads over 2 or 4 CTAs (see launch_attention_fused), for two reasons.
+    // (1) Many pairs: beyond 16 (row, head) pairs a CTA needs a second sweep per warp, loses the overlay of its block
+    //     partials on the K tile and with it all but one of its places on an SM (Llama-3 geometry, 6 rows: 131 us per
+    //     layer against 108 at 4 rows): split until a CTA has at most 16, and on to at most 8 (three CTAs per SM instead
+    //     of two) where that does not add a wave of CTAs.
+    // (2) Few CTAs: split further while the grid stays within two CTAs per SM; beyond that the copies of the KV rows that
+    //     every CTA of a group stages cost more than the shorter sweeps save (one row, 3000 positions: 97.4 vs 95.9 us).
+    // Measured on the Llama-3 geometry, us per layer unsplit / chosen: 2500 positions 8 rows 140 / 114, 4 rows 108 / 104;
+    // 8192 positions 8 rows 193 / 164, 6 rows 176 / 162.  The choice depends on the number of rows, the result does not.
     AttnArgs a = a0;
-    const int Gfull = a.H / a.Hkv, slots = 2 * device_sm_count();
-    a.gsplit = 1;
-    for (int gs = 4; gs > 1; gs >>= 1)
-        if (Gfull % gs == 0 && a.Hkv * gs * n_chunks <= slots) { a.gsplit = gs; break; }
+    const int Gfull = a.H / a.Hkv, sms = device_sm_count(), pairs = a.m * Gfull;
+    auto waves = [&](int gs) {   // rounds of resident CTAs the grid needs with that split
+        const int pc = pairs / gs, pg = pc > 8 ? 8 : pc > 4 ? 4 : pc > 2 ? 2 : 1;
+        const AttnLayout lay(pc, a.hd, (int)sizeof(T), pg, 2);
+        int per_sm = (int)((228 * 1024) / (lay.total + 1024));
+        const int by_regs = pc > 8 ? 2 : 3;          // the 8-pair sweep needs twice the registers
+        per_sm = per_sm < 1 ? 1 : per_sm > by_regs ? by_regs : per_sm;
+        return (a.Hkv * gs * n_chunks + per_sm * sms - 1) / (per_sm * sms);
+    };
+    int gs = 1;
+    while (gs < 4 && Gfull % (2 * gs) == 0 && pairs / gs > 16) gs *= 2;
+    if (gs < 4 && Gfull % (2 * gs) == 0 && pairs / gs > 8 && waves(2 * gs) <= waves(gs)) gs *= 2;
+    for (int g = 4; g > gs; g >>= 1)
+        if (Gfull % g == 0 && a.Hkv * g * n_chunks <= 2 * sms) { gs = g; break; }
+    a.gsplit = gs;
     dim3 grid(a.Hkv * a.gsplit, n_chunks);
     bool ok;
     switch (a.hd) {
