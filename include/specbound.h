@@ -299,7 +299,7 @@ double sb_model_speedup(int32_t L, double a, int32_t w, int32_t d_max);
  *                       The fused GEMM is never split along k, so its sums may round differently from the
  *                       separate kernels' (fp32 rounding level).
  *                    2: RoPE, KV-cache append and attention run inside the attention kernel: up to 8 chunks of 128
- *                       positions (11 for models with few KV heads) in one launch whose chunk CTAs form a
+ *                       positions in one launch whose chunk CTAs form a
  *                       thread-block cluster and merge the chunks; longer contexts in two (chunk kernel, chunk merge).
  *                       Off: three launches (RoPE/append, chunk kernel, chunk merge).  Bit-identical either way.
  *                    Each setting by itself is deterministic and row-invariant.

@@ -22,10 +22,7 @@ constexpr int kMaxPairGroup = 8;
 
 // PG = (row, query head) pairs handled per sweep over the staged tile: the largest of 8, 4, 2, 1 that
 // divides what each warp gets, so that the inner loops carry no run-time predicates.
-// kBig: clusters of 9 .. 16 chunk CTAs (contexts of up to 2048 positions; a non-portable cluster size, used for models
-// with so few KV heads that all clusters are resident at once): the chunk partials are folded in two groups of eight
-// and the groups in order -- the two-level fold of the chunk merge kernel, which for a single group is the plain one.
-template <typename T, int HD, int PG, bool kBig>
+template <typename T, int HD, int PG>
 __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     constexpr int kPairGroup = PG;
     constexpr int E = HD / 32;                       // channels per lane in P.V
@@ -277,37 +274,26 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
             int row = a.r0 + i;
             int n_chunks = (a.pos0 + row) / kAttnChunk + 1;   // chunks that hold positions <= this row's own (<= cluster size)
             float M = -INFINITY, L = 0.f, O = 0.f;
-            float Mf = -INFINITY, Lf = 0.f, Of = 0.f;   // kBig: the fold over the groups
+            float mc[kBatch], lc[kBatch], oc[kBatch];
 #pragma unroll
-            for (int g0 = 0; g0 < (kBig ? 2 : 1); ++g0) {
-                float mc[kBatch], lc[kBatch], oc[kBatch];
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    mc[u] = -INFINITY; lc[u] = 0.f; oc[u] = 0.f;
-                    if (g0 * kBatch + u < n_chunks) {
-                        uint32_t base;
-                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(base) : "r"(out_local + (uint32_t)(p * (HD + 2)) * 4u), "r"(g0 * kBatch + u));
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mc[u]) : "r"(base + (uint32_t)HD * 4u) : "memory");
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(lc[u]) : "r"(base + (uint32_t)(HD + 1) * 4u) : "memory");
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(oc[u]) : "r"(base + (uint32_t)e * 4u) : "memory");
-                    }
-                }
-                if (kBig) { M = -INFINITY; L = 0.f; O = 0.f; }
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    if (mc[u] > -INFINITY) {
-                        float f0, f1;
-                        attn_fold(M, L, mc[u], lc[u], f0, f1);
-                        O = attn_fold_out(O, oc[u], f0, f1);
-                    }
-                }
-                if (kBig && M > -INFINITY) {
-                    float f0, f1;
-                    attn_fold(Mf, Lf, M, L, f0, f1);
-                    Of = attn_fold_out(Of, O, f0, f1);
+            for (int u = 0; u < kBatch; ++u) {
+                mc[u] = -INFINITY; lc[u] = 0.f; oc[u] = 0.f;
+                if (u < n_chunks) {
+                    uint32_t base;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(base) : "r"(out_local + (uint32_t)(p * (HD + 2)) * 4u), "r"(u));
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(mc[u]) : "r"(base + (uint32_t)HD * 4u) : "memory");
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(lc[u]) : "r"(base + (uint32_t)(HD + 1) * 4u) : "memory");
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(oc[u]) : "r"(base + (uint32_t)e * 4u) : "memory");
                 }
             }
-            if (kBig) { L = Lf; O = Of; }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                if (mc[u] > -INFINITY) {
+                    float f0, f1;
+                    attn_fold(M, L, mc[u], lc[u], f0, f1);
+                    O = attn_fold_out(O, oc[u], f0, f1);
+                }
+            }
             using A = Act<T>;
             A::store(reinterpret_cast<typename A::type*>(a.act_out), row, (head0 + g) * HD + e, a.H * HD, attn_finish(O, L));
         }
@@ -322,19 +308,18 @@ static size_t cluster_attn_smem(int P, int HD, size_t elt) {
            (size_t)kPosWarps * P * (HD + 2) * 4 + (size_t)P * (HD + 2) * 4;
 }
 // Returns false if the device cannot co-schedule such a cluster or the pairs do not fit (nothing is launched then).
-template <typename T, int HD, int PG, bool kBig>
+template <typename T, int HD, int PG>
 static bool launch_cluster_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, size_t smem, int cluster_y) {
-    auto kernel = k_attn_cluster<T, HD, PG, kBig>;
+    auto kernel = k_attn_cluster<T, HD, PG>;
     static bool configured[kMaxDevices];             // function attributes are per device
     const int dev = current_device();
     if (dev < 0 || smem > 200 * 1024) return false;
     if (!configured[dev]) {
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
-        if (kBig && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) (void)cudaGetLastError();
         configured[dev] = true;
     }
     if (cluster_y > 1) {
-        static int resident_dev[kMaxDevices][17];        // per device and cluster size: clusters resident at once + 1 (0 = not asked yet)
+        static int resident_dev[kMaxDevices][9];         // per device and cluster size: clusters resident at once + 1 (0 = not asked yet)
         int* resident = resident_dev[dev];
         if (resident[cluster_y] == 0) {
             cudaLaunchConfig_t cfg{};
@@ -348,8 +333,7 @@ static bool launch_cluster_pg(cudaStream_t st, const AttnArgs& a, dim3 grid, siz
             resident[cluster_y] = n + 1;
             if (getenv("SB_DEBUG")) fprintf(stderr, "[specbound] attention clusters of %d CTAs: %d resident at once\n", cluster_y, n);
         }
-        // big clusters only where every cluster of the grid is resident at once
-        if (resident[cluster_y] - 1 < (kBig ? (int)grid.x : 1)) return false;
+        if (resident[cluster_y] - 1 < 1) return false;
     }
     return launch_kc(kernel, grid, dim3(kAttnWarps * 32), smem, st, cluster_y, a) == cudaSuccess;
 }
@@ -360,31 +344,30 @@ static bool launch_cluster_hd(cudaStream_t st, const AttnArgs& a, dim3 grid, int
     // pairs per sweep: the largest of 8, 4, 2, 1 that divides what each of a block's two warps gets
     const int P0 = (P + 1) / 2, P1 = P - P0;
     auto divides = [&](int g) { return P0 % g == 0 && P1 % g == 0; };
-    if (cluster_y > 8) {
-        if (divides(8)) return launch_cluster_pg<T, HD, 8, true>(st, a, grid, smem, cluster_y);
-        if (divides(4)) return launch_cluster_pg<T, HD, 4, true>(st, a, grid, smem, cluster_y);
-        if (divides(2)) return launch_cluster_pg<T, HD, 2, true>(st, a, grid, smem, cluster_y);
-        return launch_cluster_pg<T, HD, 1, true>(st, a, grid, smem, cluster_y);
-    }
-    if (divides(8)) return launch_cluster_pg<T, HD, 8, false>(st, a, grid, smem, cluster_y);
-    if (divides(4)) return launch_cluster_pg<T, HD, 4, false>(st, a, grid, smem, cluster_y);
-    if (divides(2)) return launch_cluster_pg<T, HD, 2, false>(st, a, grid, smem, cluster_y);
-    return launch_cluster_pg<T, HD, 1, false>(st, a, grid, smem, cluster_y);
+    if (divides(8)) return launch_cluster_pg<T, HD, 8>(st, a, grid, smem, cluster_y);
+    if (divides(4)) return launch_cluster_pg<T, HD, 4>(st, a, grid, smem, cluster_y);
+    if (divides(2)) return launch_cluster_pg<T, HD, 2>(st, a, grid, smem, cluster_y);
+    return launch_cluster_pg<T, HD, 1>(st, a, grid, smem, cluster_y);
 }
 
 template <typename T> bool launch_attention_fused(cudaStream_t st, const AttnArgs& a) {
     int n_chunks = (a.pos0 + a.r0 + a.m - 1) / kAttnChunk + 1;
-    // up to 8 chunks: the portable cluster size.  9 .. 16: only where all clusters fit on the device at once, one CTA
-    // per SM (models with few KV heads); elsewhere the chunk kernel with its three CTAs per SM does better
-    if (n_chunks > 16) return false;
+    // up to 8 chunks: the portable cluster size.  (Clusters of 9-16 chunk CTAs, which fit the device at once only for
+    // models with few KV heads, were built and measured: slower than the chunk kernel with its query-head split, e.g.
+    // Llama-3 geometry at 1030 positions, 8 rows: 116.6 vs 104.8 us per layer.)
+    if (n_chunks > 8) return false;
     // Grouped-query models: with few KV heads there are fewer CTAs than SMs, each doing the CUDA-core work of all its
-    // group's (row, head) pairs; spread a group's query heads over 2 or 4 CTAs while all CTAs still fit the device at once
-    // (every one of them stages the KV head's rows: a few MB more out of L2).  A split that cannot be launched (big
-    // clusters that are not all resident) falls back to the next smaller one.
-    const int Gfull = a.H / a.Hkv, sms = device_sm_count();
+    // group's (row, head) pairs; spread a group's query heads over 2 or 4 CTAs (every one of them stages the KV head's rows:
+    // a few MB more out of L2) while the grid stays about within one CTA per SM, or within two where a CTA would
+    // otherwise sweep 16 pairs or more (two CTAs of up to 8 pairs fit an SM).  Llama-3 geometry, 512 positions, us per
+    // layer at 1 / 2 / 4 / 6 / 8 rows: unsplit 93.3 / 97.5 / 101.8 / 110.6 / 116.3, two CTAs per KV head 89.8 / 92.1 / 97.2 /
+    // 105.2 / 103.1, four 88.9 / 89.9 / 93.0 / 98.6 / 99.1; at 900 positions four CTAs lose to two at 1-2 rows (92.1 vs
+    // 89.6).  A split that cannot be launched falls back to the next smaller one.
+    const int Gfull = a.H / a.Hkv, sms = device_sm_count(), pairs = a.m * Gfull;
     for (int gs = 4; gs >= 1; gs >>= 1) {
-        if (Gfull % gs || (gs > 1 && a.Hkv * gs * n_chunks > sms)) continue;
-        if (n_chunks > 8 && a.Hkv * gs * n_chunks > sms) continue;      // big clusters: one wave only
+        const int ctas = a.Hkv * gs * n_chunks;
+        if (Gfull % gs) continue;
+        if (gs > 1 && !(ctas <= sms + sms / 8 || (pairs >= 16 && ctas <= 2 * sms))) continue;
         AttnArgs b = a;
         b.gsplit = gs;
         dim3 grid(a.Hkv * gs, n_chunks);

@@ -30,9 +30,9 @@ K_SCALE = 3.0
 
 # (rows, first position).  511/512: the round straddles / starts on the 4th -> 5th chunk boundary; 896: 8 chunks;
 # 1016: the last row sits at 1023, the last position the one-launch kernel takes; 1017 with 8 rows, 1023 with 4,
-# 1024, 1025: hand-over to the long-context kernels (9 chunks; with few KV heads clusters of 9-11 chunk CTAs take
-# these); 1150, 1279, 1404: 10 and 11 chunks and the last row the big clusters take (position 1407); 2048: 17
-# chunks; 8184: 64 chunks, the longest context of the micro-benchmarks
+# 1024, 1025: hand-over to the long-context kernels (9 chunks); 1150, 1279, 1404: 10 and 11 chunks, where the
+# grouped-query geometry changes how many CTAs share a KV head's query heads; 2048: 17 chunks; 8184: 64 chunks, the
+# longest context of the micro-benchmarks
 CASES = [(1, 511), (8, 511), (4, 512), (8, 896), (8, 1016), (1, 1023), (8, 1017), (4, 1023), (1, 1024), (8, 1024),
          (4, 1025), (6, 1150), (3, 1279), (5, 1404), (2, 1500), (3, 1790), (1, 2048), (8, 2048), (6, 2500), (5, 4000),
          (4, 8184), (8, 8184), (1, 8191)]
@@ -155,9 +155,9 @@ def test_dropping_one_chunk_would_be_seen(geometry):
 @pytest.mark.parametrize("first_pos", [1021, 1405, 2050])
 def test_long_context_rows_do_not_depend_on_companions(geometry, first_pos):
     """Row i of a 6-row pass is bit-identical to the same row run alone once the earlier rows' K,V are cached, also
-    where the pass straddles a hand-over between the attention kernels (1021: rows at 1021 .. 1023 alone go through
-    the 8-chunk clusters, in company through the 9-chunk path; 1405: the 11 -> 12 chunk boundary, where a model with
-    few KV heads leaves the big clusters for the two-launch kernels) and deep inside a long context: what
+    where the pass straddles the hand-over between the attention kernels (1021: rows at 1021 .. 1023 alone go through
+    the 8-chunk clusters, in company through the two-launch kernels), where the number of rows changes how a KV head's
+    query heads are spread over CTAs (a row alone and in a pass of six), and deep inside a long context: what
     makes speculative decoding return exactly the autoregressive tokens at any length."""
     g = geometry
     m = 6
