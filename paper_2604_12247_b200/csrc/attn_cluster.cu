@@ -86,7 +86,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     // 2. while those copies fly: q, and the new positions' K and V
     {
         constexpr int half = HD / 2;
-        constexpr int kBatch = 4;   // work items whose partial sums are requested together
+        // work items whose partial sums are requested together: one.  Batches of 4 (everything four items need requested
+        // before the first value is used) measured 0.5-1.2 us per layer SLOWER at every width, batches of 6 another 1 us at
+        // one row: the first loads leave later behind the longer address arithmetic, and that is on the critical path
+        constexpr int kBatch = 1;
         const int ntot = qd + 2 * kvd;
         const size_t sstride = (size_t)kMaxW * ntot;
         // work items: P * half rotation pairs of q, then, for each new position of this chunk, half rotation pairs

@@ -372,7 +372,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[idx] = 0.f;   // padding pairs
     if (kFront) {
         constexpr int half = HD / 2;
-        constexpr int kBatch = 4;   // work items whose partial sums are requested together
+        constexpr int kBatch = 1;   // work items whose partial sums are requested together: one (see k_attn_cluster; here 4 were 0.7-2.7 us per layer slower)
         const int ntot = qd + 2 * kvd;
         const size_t sstride = (size_t)kMaxW * ntot;
         // work items: P * half rotation pairs of q, then, for each new position of this chunk, half rotation pairs
