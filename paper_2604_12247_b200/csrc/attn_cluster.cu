@@ -82,75 +82,59 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
             for (int j = 0; j < (int)kRowBytes / 16; ++j) reinterpret_cast<uint4*>(row)[j] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
+    // 2. while those copies fly: q, and the new positions' K and V.
+    // Work items: P * half rotation pairs of q, then, for each new position of this chunk, half rotation pairs of K and
+    // half element pairs of V (rounded to the storage type, written to the cache and into the staged tile of the warp
+    // that owns the position).  One item's operands are requested at a time: batches of 4 (everything four items need
+    // requested before the first value is used) measured 0.5-1.2 us per layer SLOWER at every width, batches of 6
+    // another 1 us at one row -- the first loads leave later behind the longer address arithmetic, and that is on the
+    // critical path.  For the same reason what an item needs that does not depend on the preceding kernel (its
+    // addresses, its rotation angle, its page) is prepared for a thread's first item BEFORE the grid-dependency wait.
+    constexpr int half = HD / 2;
+    const int ntot = qd + 2 * kvd;
+    const size_t sstride = (size_t)kMaxW * ntot;
+    const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
+    const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
+    struct Item { int kind, pos, e2, p; const float* src; float2 cs; int page; };   // kind 0: q pair of (row, head) pair p; 1: K pair; 2: V pair of position pos
+    auto item_of = [&](int idx) -> Item {
+        Item it;
+        if (idx < n_q) {
+            const int p = idx / half;
+            it.kind = 0; it.pos = a.pos0 + a.r0 + p / G; it.e2 = idx - p * half; it.p = p;
+        } else {
+            const int j = idx - n_q, e = j % HD;
+            it.kind = e >= half ? 2 : 1; it.pos = lo + j / HD; it.e2 = e >= half ? e - half : e; it.p = 0;
+        }
+        it.src = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
+                 (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+        it.cs = it.kind != 2 ? rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2) : make_float2(1.f, 0.f);
+        it.page = it.kind != 0 ? a.page_table[it.pos >> a.page_shift] : 0;   // (the page table is constant: see above)
+        return it;
+    };
+    Item first{};
+    if ((int)threadIdx.x < n_items) first = item_of(threadIdx.x);
     pdl_wait();
-    // 2. while those copies fly: q, and the new positions' K and V
-    {
-        constexpr int half = HD / 2;
-        // work items whose partial sums are requested together: one.  Batches of 4 (everything four items need requested
-        // before the first value is used) measured 0.5-1.2 us per layer SLOWER at every width, batches of 6 another 1 us at
-        // one row: the first loads leave later behind the longer address arithmetic, and that is on the critical path
-        constexpr int kBatch = 1;
-        const int ntot = qd + 2 * kvd;
-        const size_t sstride = (size_t)kMaxW * ntot;
-        // work items: P * half rotation pairs of q, then, for each new position of this chunk, half rotation pairs
-        // of K and half element pairs of V (rounded to the storage type, written to the cache and into the staged
-        // tile of the warp that owns the position)
-        const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
-        const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
-        struct Item { int kind, pos, e2, p; };   // kind 0: q pair of (row, head) pair p; 1: K pair; 2: V pair of position pos
-        auto item_of = [&](int idx) -> Item {
-            if (idx < n_q) {
-                int p = idx / half;
-                return Item{0, a.pos0 + a.r0 + p / G, idx - p * half, p};
+    for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
+        const Item it = idx == (int)threadIdx.x ? first : item_of(idx);
+        float x0 = sum_splits(it.src, sstride, a.n_split);
+        float x1 = sum_splits(it.src + half, sstride, a.n_split);
+        if (it.kind != 2) rope_apply(it.cs, x0, x1);
+        if (it.kind == 0) {
+            q_s[it.p * HD + it.e2] = x0;
+            q_s[it.p * HD + it.e2 + half] = x1;
+        } else {
+            const bool is_v = it.kind == 2;
+            const T y0 = from_f32<T>(x0), y1 = from_f32<T>(x1);
+            T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
+            T* dst = cache + ((size_t)it.page * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
+            if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
+                dst[it.e2] = y0;
+                dst[it.e2 + half] = y1;
             }
-            int j = idx - n_q, it = j % HD;
-            return Item{it >= half ? 2 : 1, lo + j / HD, it >= half ? it - half : it, 0};
-        };
-        for (int base = threadIdx.x; base < n_items; base += kBatch * blockDim.x) {
-            // everything a thread's items need from memory is requested before the first value is used
-            float x0[kBatch], x1[kBatch];
-            float2 cs[kBatch];
-            int page[kBatch];
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                int idx = base + u * blockDim.x;
-                x0[u] = x1[u] = 0.f;
-                cs[u] = make_float2(1.f, 0.f);
-                page[u] = 0;
-                if (idx < n_items) {
-                    const Item it = item_of(idx);
-                    const float* p0 = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
-                                      (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
-                    x0[u] = sum_splits(p0, sstride, a.n_split);
-                    x1[u] = sum_splits(p0 + half, sstride, a.n_split);
-                    if (it.kind != 2) cs[u] = rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2);
-                    if (it.kind != 0) page[u] = a.page_table[it.pos >> a.page_shift];
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                int idx = base + u * blockDim.x;
-                if (idx >= n_items) continue;
-                const Item it = item_of(idx);
-                if (it.kind != 2) rope_apply(cs[u], x0[u], x1[u]);
-                if (it.kind == 0) {
-                    q_s[it.p * HD + it.e2] = x0[u];
-                    q_s[it.p * HD + it.e2 + half] = x1[u];
-                } else {
-                    const bool is_v = it.kind == 2;
-                    const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
-                    T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
-                    T* dst = cache + ((size_t)page[u] * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
-                    if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
-                        dst[it.e2] = y0;
-                        dst[it.e2 + half] = y1;
-                    }
-                    int tl = it.pos - c * kAttnChunk;
-                    T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
-                    srow[it.e2] = y0;
-                    srow[it.e2 + half] = y1;
-                }
-            }
+            const int tl = it.pos - c * kAttnChunk;
+            T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
+            srow[it.e2] = y0;
+            srow[it.e2 + half] = y1;
         }
     }
     {   // bounded wait for this block's copies
