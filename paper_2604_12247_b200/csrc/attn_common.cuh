@@ -82,6 +82,30 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// acc[e] = fma(p, v[e], acc[e]) for a lane's E channels: one rounding per channel, two channels per instruction
+// (fma.rn.f32x2 is two independent IEEE fused multiply-adds) where E is even
+template <int E> __device__ __forceinline__ void fma_channels(float p, const float (&v)[E], float (&acc)[E]) {
+    if constexpr (E % 2 == 0) {
+        const float2 pp = make_float2(p, p);
+#pragma unroll
+        for (int e = 0; e < E; e += 2) {
+            const float2 r = __ffma2_rn(pp, make_float2(v[e], v[e + 1]), make_float2(acc[e], acc[e + 1]));
+            acc[e] = r.x;
+            acc[e + 1] = r.y;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = fmaf(p, v[e], acc[e]);
+    }
+}
+
+// (s0, s1) = (fma(q0, k, s0), fma(q1, k, s1)): the score chains of two pairs advanced by one packed instruction
+__device__ __forceinline__ void fma_pairs(float q0, float q1, float k, float& s0, float& s1) {
+    const float2 r = __ffma2_rn(make_float2(q0, q1), make_float2(k, k), make_float2(s0, s1));
+    s0 = r.x;
+    s1 = r.y;
+}
+
 // 1 / sqrt(head_dim) as every kernel forms it
 __device__ __forceinline__ float attn_score_scale(int hd) { return rsqrtf((float)hd); }
 

@@ -295,7 +295,10 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const int Ppad = lay.Ppad;
-    float* q_s = reinterpret_cast<float*>(smem);                                   // [Ppad][HD]
+    float* q_s = reinterpret_cast<float*>(smem);                                   // [Ppad][HD], see q_at
+    // Where a sweep takes two or more pairs, the queries of pairs 2j and 2j+1 are interleaved channel by channel, so that
+    // one packed fused multiply-add advances both pairs' score chains (attn_common.cuh: fma_pairs)
+    auto q_at = [](int p, int ch) -> int { return PG >= 2 ? ((p >> 1) * HD + ch) * 2 + (p & 1) : p * HD + ch; };
     unsigned char* k_tiles = smem + lay.off_k;
     unsigned char* v_tiles = smem + lay.off_v;
     const int v = warp & (kPosWarps - 1), hsel = warp / kPosWarps;   // position block; which share of the pair groups
@@ -369,7 +372,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         }
     }
     // 2. while those copies fly: q, and (front end) the new positions' K and V
-    for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[idx] = 0.f;   // padding pairs
+    for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[q_at(idx / HD, idx % HD)] = 0.f;   // padding pairs
     if (kFront) {
         constexpr int half = HD / 2;
         constexpr int kBatch = 1;   // work items whose partial sums are requested together: one (see k_attn_cluster; here 4 were 0.7-2.7 us per layer slower)
@@ -417,8 +420,8 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 const Item it = item_of(idx);
                 if (it.kind != 2) rope_apply(cs[u], x0[u], x1[u]);
                 if (it.kind == 0) {
-                    q_s[it.p * HD + it.e2] = x0[u];
-                    q_s[it.p * HD + it.e2 + half] = x1[u];
+                    q_s[q_at(it.p, it.e2)] = x0[u];
+                    q_s[q_at(it.p, it.e2 + half)] = x1[u];
                 } else {
                     const bool is_v = it.kind == 2;
                     const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
@@ -439,7 +442,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
             int p = idx / HD, e = idx - p * HD;
             int i = p / G, g = p - i * G;
-            q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (head0 + g) * HD + e];
+            q_s[q_at(p, e)] = a.q[(size_t)(a.r0 + i) * qd + (head0 + g) * HD + e];
         }
     }
     {   // bounded wait for this block's copies
@@ -475,20 +478,27 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
             float kf[EPP];
             unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB_K + piece * 16), kf);
             // per pair one fmaf chain over the channels in order; the pairs' chains are independent and interleaved
+            if constexpr (kPairGroup >= 2) {
 #pragma unroll
-            for (int v4 = 0; v4 < EPP / 4; ++v4) {
-                float4 qq[kPairGroup];
+                for (int c2 = 0; c2 < EPP / 2; ++c2) {   // two channels of two pairs per 16-byte read
+                    float4 qq[kPairGroup / 2];
 #pragma unroll
-                for (int pp = 0; pp < kPairGroup; ++pp)
-                    qq[pp] = *reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP + 4 * v4);
+                    for (int j = 0; j < kPairGroup / 2; ++j)
+                        qq[j] = *reinterpret_cast<const float4*>(q_s + ((size_t)((pg >> 1) + j) * HD + piece * EPP + 2 * c2) * 2);
 #pragma unroll
-                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].x, kf[4 * v4], sc[pp]);
+                    for (int j = 0; j < kPairGroup / 2; ++j) fma_pairs(qq[j].x, qq[j].y, kf[2 * c2], sc[2 * j], sc[2 * j + 1]);
 #pragma unroll
-                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].y, kf[4 * v4 + 1], sc[pp]);
+                    for (int j = 0; j < kPairGroup / 2; ++j) fma_pairs(qq[j].z, qq[j].w, kf[2 * c2 + 1], sc[2 * j], sc[2 * j + 1]);
+                }
+            } else {
 #pragma unroll
-                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].z, kf[4 * v4 + 2], sc[pp]);
-#pragma unroll
-                for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = fmaf(qq[pp].w, kf[4 * v4 + 3], sc[pp]);
+                for (int v4 = 0; v4 < EPP / 4; ++v4) {
+                    const float4 qq = *reinterpret_cast<const float4*>(q_s + (size_t)pg * HD + piece * EPP + 4 * v4);
+                    sc[0] = fmaf(qq.x, kf[4 * v4], sc[0]);
+                    sc[0] = fmaf(qq.y, kf[4 * v4 + 1], sc[0]);
+                    sc[0] = fmaf(qq.z, kf[4 * v4 + 2], sc[0]);
+                    sc[0] = fmaf(qq.w, kf[4 * v4 + 3], sc[0]);
+                }
             }
         }
         // ---- softmax pieces of this warp's 32 positions (warp-shuffle max and sum) ----
@@ -511,26 +521,19 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
             float vf[4][E];
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) load_channels<T, E>(V_w + (t4 * 4 + tt) * ROWB_V + lane * E * (int)sizeof(T), vf[tt]);
-            // per (pair, channel) one fmaf chain over the positions in order; the chains are independent and interleaved
+            // per (pair, channel) one fmaf chain over the positions in order; the chains are independent and interleaved.
+            // Two neighbouring channels' chains share one packed instruction (fma.rn.f32x2: two IEEE fused
+            // multiply-adds, the same roundings as two scalar ones) where a lane has an even number of channels.
             float4 p4[kPairGroup];
 #pragma unroll
             for (int pp = 0; pp < kPairGroup; ++pp) p4[pp] = *reinterpret_cast<const float4*>(P_w + pp * 32 + t4 * 4);
 #pragma unroll
-            for (int pp = 0; pp < kPairGroup; ++pp)
+            for (int tt = 0; tt < 4; ++tt)
 #pragma unroll
-                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].x, vf[0][e], o[pp][e]);
-#pragma unroll
-            for (int pp = 0; pp < kPairGroup; ++pp)
-#pragma unroll
-                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].y, vf[1][e], o[pp][e]);
-#pragma unroll
-            for (int pp = 0; pp < kPairGroup; ++pp)
-#pragma unroll
-                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].z, vf[2][e], o[pp][e]);
-#pragma unroll
-            for (int pp = 0; pp < kPairGroup; ++pp)
-#pragma unroll
-                for (int e = 0; e < E; ++e) o[pp][e] = fmaf(p4[pp].w, vf[3][e], o[pp][e]);
+                for (int pp = 0; pp < kPairGroup; ++pp) {
+                    const float pt = tt == 0 ? p4[pp].x : tt == 1 ? p4[pp].y : tt == 2 ? p4[pp].z : p4[pp].w;
+                    fma_channels<E>(pt, vf[tt], o[pp]);
+                }
         }
         __syncwarp();   // every lane is done with its K row and with P_w
         if (pair_barrier && !arrived) {   // ... and so is the block's other warp, before the block partial goes over the K tile
