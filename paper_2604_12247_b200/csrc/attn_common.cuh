@@ -106,6 +106,17 @@ __device__ __forceinline__ void fma_pairs(float q0, float q1, float k, float& s0
     s1 = r.y;
 }
 
+// x / d for a small non-negative x and the query-head group size d: a shift where d is a power of two (the usual
+// group sizes; a run-time integer division costs about twenty instructions, and the kernels divide once per work item)
+struct GroupDiv {
+    int d, sh;
+    __device__ explicit GroupDiv(int d_) : d(d_), sh(-1) {
+        if ((d_ & (d_ - 1)) == 0)
+            for (sh = 0; (1 << sh) < d_; ++sh) {}
+    }
+    __device__ __forceinline__ int operator()(int x) const { return sh >= 0 ? x >> sh : (int)((unsigned)x / (unsigned)d); }
+};
+
 // 1 / sqrt(head_dim) as every kernel forms it
 __device__ __forceinline__ float attn_score_scale(int hd) { return rsqrtf((float)hd); }
 

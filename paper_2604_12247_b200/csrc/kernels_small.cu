@@ -292,6 +292,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.H / a.Hkv / gs, P = a.m * G;     // this CTA's query heads of the group; pair p = i * G + g: row r0 + i, query head head0 + g
     const int head0 = kvh * (a.H / a.Hkv) + gsub * G;
+    const GroupDiv divG(G);
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const int Ppad = lay.Ppad;
@@ -387,7 +388,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         auto item_of = [&](int idx) -> Item {
             if (idx < n_q) {
                 int p = idx / half;
-                return Item{0, a.pos0 + a.r0 + p / G, idx - p * half, p};
+                return Item{0, a.pos0 + a.r0 + divG(p), idx - p * half, p};
             }
             int j = idx - n_q, it = j % HD;
             return Item{it >= half ? 2 : 1, lo + j / HD, it >= half ? it - half : it, 0};
@@ -406,7 +407,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 if (idx < n_items) {
                     const Item it = item_of(idx);
                     const float* p0 = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
-                                      (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+                                      (it.kind == 0 ? (head0 + (it.p - divG(it.p) * G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
                     x0[u] = sum_splits(p0, sstride, a.n_split);
                     x1[u] = sum_splits(p0 + half, sstride, a.n_split);
                     if (it.kind != 2) cs[u] = rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2);
@@ -441,7 +442,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     } else {
         for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
             int p = idx / HD, e = idx - p * HD;
-            int i = p / G, g = p - i * G;
+            int i = divG(p), g = p - i * G;
             q_s[q_at(p, e)] = a.q[(size_t)(a.r0 + i) * qd + (head0 + g) * HD + e];
         }
     }
@@ -505,7 +506,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         float mx[kPairGroup], ls[kPairGroup];
 #pragma unroll
         for (int pp = 0; pp < kPairGroup; ++pp) {
-            int i = (pg + pp) / G;
+            int i = divG(pg + pp);
             bool on = my_t <= a.pos0 + a.r0 + i;         // causal: a row sees positions <= its own
             P_w[pp * 32 + lane] = attn_block_softmax(sc[pp], scale, on, mx[pp], ls[pp]);
         }
@@ -556,7 +557,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     // merge the four blocks in block order; thread -> (pair, two channels)
     for (int idx = threadIdx.x; idx < P * (HD / 2); idx += blockDim.x) {
         const int p = idx / (HD / 2), e = (idx - p * (HD / 2)) * 2;
-        const int i = p / G, g = p - i * G;
+        const int i = divG(p), g = p - i * G;
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kPosWarps; ++w) M = fmaxf(M, mrg_blk(w)[(size_t)p * (HD + 2) + HD]);
