@@ -37,10 +37,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     const int G = a.H / a.Hkv / gs, P = a.m * G;     // this CTA's query heads of the group; pair p = i * G + g: row r0 + i, query head head0 + g
     const int head0 = kvh * (a.H / a.Hkv) + gsub * G;
     const int kvd = a.Hkv * HD, qd = a.H * HD;
-    float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD], see q_at
-    // Where a sweep takes two or more pairs, the queries of pairs 2j and 2j+1 are interleaved channel by channel, so that
-    // one packed fused multiply-add advances both pairs' score chains (attn_common.cuh: fma_pairs)
-    auto q_at = [](int p, int ch) -> int { return PG >= 2 ? ((p >> 1) * HD + ch) * 2 + (p & 1) : p * HD + ch; };
+    float* q_s = reinterpret_cast<float*>(smem);                                   // [P][HD]
     unsigned char* kv_s = smem + (size_t)P * HD * 4;                                // per warp: K[32], V[32]
     const int v = warp & (kPosWarps - 1), hsel = warp / kPosWarps;   // position block; which half of the pairs
     unsigned char* K_w = kv_s + (size_t)v * 64 * ROWB;
@@ -123,8 +120,8 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
         float x1 = sum_splits(it.src + half, sstride, a.n_split);
         if (it.kind != 2) rope_apply(it.cs, x0, x1);
         if (it.kind == 0) {
-            q_s[q_at(it.p, it.e2)] = x0;
-            q_s[q_at(it.p, it.e2 + half)] = x1;
+            q_s[it.p * HD + it.e2] = x0;
+            q_s[it.p * HD + it.e2 + half] = x1;
         } else {
             const bool is_v = it.kind == 2;
             const T y0 = from_f32<T>(x0), y1 = from_f32<T>(x1);
@@ -158,37 +155,28 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     const int P0 = (P + 1) / 2;   // pairs [0, P0) go to the first warp of a block, [P0, P) to the second
     for (int pg = hsel ? P0 : 0; pg < (hsel ? P : P0); pg += kPairGroup) {
         // ---- scores: lane = position ----
-        float sc[kPairGroup];
+        float2 sc2[kPairGroup];   // per pair: the sums over the even and over the odd channels (attn_score_step)
 #pragma unroll
-        for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = 0.f;
+        for (int pp = 0; pp < kPairGroup; ++pp) sc2[pp] = make_float2(0.f, 0.f);
 #pragma unroll 2
         for (int piece = 0; piece < PPR; ++piece) {
             float kf[EPP];
             unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB + piece * 16), kf);
-            // per pair one fmaf chain over the channels in order; the pairs' chains are independent and interleaved
-            if constexpr (kPairGroup >= 2) {
+            // the pairs' chains are independent and interleaved
 #pragma unroll
-                for (int c2 = 0; c2 < EPP / 2; ++c2) {   // two channels of two pairs per 16-byte read
-                    float4 qq[kPairGroup / 2];
+            for (int v4 = 0; v4 < EPP / 4; ++v4) {
+                float4 qq[kPairGroup];
 #pragma unroll
-                    for (int j = 0; j < kPairGroup / 2; ++j)
-                        qq[j] = *reinterpret_cast<const float4*>(q_s + ((size_t)((pg >> 1) + j) * HD + piece * EPP + 2 * c2) * 2);
+                for (int pp = 0; pp < kPairGroup; ++pp)
+                    qq[pp] = *reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP + 4 * v4);
 #pragma unroll
-                    for (int j = 0; j < kPairGroup / 2; ++j) fma_pairs(qq[j].x, qq[j].y, kf[2 * c2], sc[2 * j], sc[2 * j + 1]);
-#pragma unroll
-                    for (int j = 0; j < kPairGroup / 2; ++j) fma_pairs(qq[j].z, qq[j].w, kf[2 * c2 + 1], sc[2 * j], sc[2 * j + 1]);
-                }
-            } else {
-#pragma unroll
-                for (int v4 = 0; v4 < EPP / 4; ++v4) {
-                    const float4 qq = *reinterpret_cast<const float4*>(q_s + (size_t)pg * HD + piece * EPP + 4 * v4);
-                    sc[0] = fmaf(qq.x, kf[4 * v4], sc[0]);
-                    sc[0] = fmaf(qq.y, kf[4 * v4 + 1], sc[0]);
-                    sc[0] = fmaf(qq.z, kf[4 * v4 + 2], sc[0]);
-                    sc[0] = fmaf(qq.w, kf[4 * v4 + 3], sc[0]);
-                }
+                for (int pp = 0; pp < kPairGroup; ++pp)
+                    attn_score_step(qq[pp], kf[4 * v4], kf[4 * v4 + 1], kf[4 * v4 + 2], kf[4 * v4 + 3], sc2[pp]);
             }
         }
+        float sc[kPairGroup];
+#pragma unroll
+        for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = attn_score_finish(sc2[pp]);
         // ---- softmax pieces of this warp's 32 positions (warp-shuffle max and sum) ----
         float mx[kPairGroup], ls[kPairGroup];
 #pragma unroll

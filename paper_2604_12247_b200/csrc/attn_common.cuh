@@ -1,8 +1,9 @@
 // Arithmetic shared by the attention kernels (one-launch cluster kernel, separate chunk kernel, streaming kernel
 // for long contexts, chunk merge).  Every kernel computes a (row, query head) pair's attention the same way:
 //
-//   32-position block : scores by one fmaf chain per position over the channels in order; block maximum and sum of
-//                       exp(score - maximum) by warp butterflies; out = sum_t p_t V_t by one fmaf chain per channel
+//   32-position block : a position's score = (fmaf chain over the even channels, in order) + (fmaf chain over the odd
+//                       channels, in order); block maximum and sum of exp(score - maximum) by warp butterflies;
+//                       out = sum_t p_t V_t by one fmaf chain per channel over the positions in order
 //   128-position chunk: its four blocks merged at once: M = max m_j, L = sum_j l_j f_j, O = sum_j o_j f_j with
 //                       f_j = exp(m_j - M), in block order
 //   8-chunk group     : the chunks folded one after the other, in chunk order
@@ -99,12 +100,15 @@ template <int E> __device__ __forceinline__ void fma_channels(float p, const flo
     }
 }
 
-// (s0, s1) = (fma(q0, k, s0), fma(q1, k, s1)): the score chains of two pairs advanced by one packed instruction
-__device__ __forceinline__ void fma_pairs(float q0, float q1, float k, float& s0, float& s1) {
-    const float2 r = __ffma2_rn(make_float2(q0, q1), make_float2(k, k), make_float2(s0, s1));
-    s0 = r.x;
-    s1 = r.y;
+// One step of a position's score: channels c .. c+3 of q and K enter the accumulator, whose halves are the running sums
+// over the even and over the odd channels (each a fused-multiply-add chain in channel order, advanced together by packed
+// instructions: neither operand has to be duplicated, and the dependent chain is half as long as one sum over all
+// channels would be).  attn_score_finish adds the two halves.
+__device__ __forceinline__ void attn_score_step(const float4& q, float k0, float k1, float k2, float k3, float2& acc) {
+    acc = __ffma2_rn(make_float2(q.x, q.y), make_float2(k0, k1), acc);
+    acc = __ffma2_rn(make_float2(q.z, q.w), make_float2(k2, k3), acc);
 }
+__device__ __forceinline__ float attn_score_finish(const float2& acc) { return __fadd_rn(acc.x, acc.y); }
 
 // x / d for a small non-negative x and the query-head group size d: a shift where d is a power of two (the usual
 // group sizes; a run-time integer division costs about twenty instructions, and the kernels divide once per work item)

@@ -296,10 +296,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     const int kvd = a.Hkv * HD, qd = a.H * HD;
     const AttnLayout lay(P, HD, (int)sizeof(T), PG, WPB);
     const int Ppad = lay.Ppad;
-    float* q_s = reinterpret_cast<float*>(smem);                                   // [Ppad][HD], see q_at
-    // Where a sweep takes two or more pairs, the queries of pairs 2j and 2j+1 are interleaved channel by channel, so that
-    // one packed fused multiply-add advances both pairs' score chains (attn_common.cuh: fma_pairs)
-    auto q_at = [](int p, int ch) -> int { return PG >= 2 ? ((p >> 1) * HD + ch) * 2 + (p & 1) : p * HD + ch; };
+    float* q_s = reinterpret_cast<float*>(smem);                                   // [Ppad][HD]
     unsigned char* k_tiles = smem + lay.off_k;
     unsigned char* v_tiles = smem + lay.off_v;
     const int v = warp & (kPosWarps - 1), hsel = warp / kPosWarps;   // position block; which share of the pair groups
@@ -373,7 +370,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         }
     }
     // 2. while those copies fly: q, and (front end) the new positions' K and V
-    for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[q_at(idx / HD, idx % HD)] = 0.f;   // padding pairs
+    for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[idx] = 0.f;   // padding pairs
     if (kFront) {
         constexpr int half = HD / 2;
         constexpr int kBatch = 1;   // work items whose partial sums are requested together: one (see k_attn_cluster; here 4 were 0.7-2.7 us per layer slower)
@@ -421,8 +418,8 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
                 const Item it = item_of(idx);
                 if (it.kind != 2) rope_apply(cs[u], x0[u], x1[u]);
                 if (it.kind == 0) {
-                    q_s[q_at(it.p, it.e2)] = x0[u];
-                    q_s[q_at(it.p, it.e2 + half)] = x1[u];
+                    q_s[it.p * HD + it.e2] = x0[u];
+                    q_s[it.p * HD + it.e2 + half] = x1[u];
                 } else {
                     const bool is_v = it.kind == 2;
                     const T y0 = from_f32<T>(x0[u]), y1 = from_f32<T>(x1[u]);
@@ -443,7 +440,7 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
         for (int idx = threadIdx.x; idx < P * HD; idx += blockDim.x) {
             int p = idx / HD, e = idx - p * HD;
             int i = divG(p), g = p - i * G;
-            q_s[q_at(p, e)] = a.q[(size_t)(a.r0 + i) * qd + (head0 + g) * HD + e];
+            q_s[idx] = a.q[(size_t)(a.r0 + i) * qd + (head0 + g) * HD + e];
         }
     }
     {   // bounded wait for this block's copies
@@ -471,37 +468,28 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     bool arrived = false;
     for (int pg = pg_begin; pg < pg_end; pg += kPairGroup) {
         // ---- scores: lane = position ----
-        float sc[kPairGroup];
+        float2 sc2[kPairGroup];   // per pair: the sums over the even and over the odd channels (attn_score_step)
 #pragma unroll
-        for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = 0.f;
+        for (int pp = 0; pp < kPairGroup; ++pp) sc2[pp] = make_float2(0.f, 0.f);
 #pragma unroll 2
         for (int piece = 0; piece < PPR; ++piece) {
             float kf[EPP];
             unpack16<T>(*reinterpret_cast<const uint4*>(K_w + lane * ROWB_K + piece * 16), kf);
-            // per pair one fmaf chain over the channels in order; the pairs' chains are independent and interleaved
-            if constexpr (kPairGroup >= 2) {
+            // the pairs' chains are independent and interleaved
 #pragma unroll
-                for (int c2 = 0; c2 < EPP / 2; ++c2) {   // two channels of two pairs per 16-byte read
-                    float4 qq[kPairGroup / 2];
+            for (int v4 = 0; v4 < EPP / 4; ++v4) {
+                float4 qq[kPairGroup];
 #pragma unroll
-                    for (int j = 0; j < kPairGroup / 2; ++j)
-                        qq[j] = *reinterpret_cast<const float4*>(q_s + ((size_t)((pg >> 1) + j) * HD + piece * EPP + 2 * c2) * 2);
+                for (int pp = 0; pp < kPairGroup; ++pp)
+                    qq[pp] = *reinterpret_cast<const float4*>(q_s + (size_t)(pg + pp) * HD + piece * EPP + 4 * v4);
 #pragma unroll
-                    for (int j = 0; j < kPairGroup / 2; ++j) fma_pairs(qq[j].x, qq[j].y, kf[2 * c2], sc[2 * j], sc[2 * j + 1]);
-#pragma unroll
-                    for (int j = 0; j < kPairGroup / 2; ++j) fma_pairs(qq[j].z, qq[j].w, kf[2 * c2 + 1], sc[2 * j], sc[2 * j + 1]);
-                }
-            } else {
-#pragma unroll
-                for (int v4 = 0; v4 < EPP / 4; ++v4) {
-                    const float4 qq = *reinterpret_cast<const float4*>(q_s + (size_t)pg * HD + piece * EPP + 4 * v4);
-                    sc[0] = fmaf(qq.x, kf[4 * v4], sc[0]);
-                    sc[0] = fmaf(qq.y, kf[4 * v4 + 1], sc[0]);
-                    sc[0] = fmaf(qq.z, kf[4 * v4 + 2], sc[0]);
-                    sc[0] = fmaf(qq.w, kf[4 * v4 + 3], sc[0]);
-                }
+                for (int pp = 0; pp < kPairGroup; ++pp)
+                    attn_score_step(qq[pp], kf[4 * v4], kf[4 * v4 + 1], kf[4 * v4 + 2], kf[4 * v4 + 3], sc2[pp]);
             }
         }
+        float sc[kPairGroup];
+#pragma unroll
+        for (int pp = 0; pp < kPairGroup; ++pp) sc[pp] = attn_score_finish(sc2[pp]);
         // ---- softmax pieces of this warp's 32 positions (warp-shuffle max and sum) ----
         float mx[kPairGroup], ls[kPairGroup];
 #pragma unroll
