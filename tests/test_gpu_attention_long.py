@@ -24,6 +24,10 @@ pytestmark = pytest.mark.gpu
 
 GEOM_7B = inputs.scaled(inputs.LLAMA2_7B, name="attn-7b-geometry", n_layers=1, d_model=512, d_ffn=512, vocab=64)
 GEOM_L3 = inputs.scaled(inputs.LLAMA3_8B, name="attn-l3-geometry", n_layers=1, d_model=512, d_ffn=512, vocab=64)
+# three query heads per KV head: a group size that is not a power of two (the kernels' index arithmetic has a fast path
+# for powers of two), that no split over several CTAs divides, and that gives a warp more than one sweep at 6-8 rows
+GEOM_G3 = inputs.scaled(inputs.LLAMA3_8B, name="attn-3-per-kv-geometry", n_layers=1, d_model=512, d_ffn=512, vocab=64,
+                        n_heads=24, n_kv_heads=8)
 MAX_SEQ = 8200
 PAGE = 64
 K_SCALE = 3.0
@@ -101,7 +105,7 @@ class Geometry:
         return out, np.stack([k for k, _ in kv]), np.stack([v for _, v in kv])
 
 
-@pytest.fixture(scope="module", params=[GEOM_7B, GEOM_L3], ids=lambda s: s.name)
+@pytest.fixture(scope="module", params=[GEOM_7B, GEOM_L3, GEOM_G3], ids=lambda s: s.name)
 def geometry(request):
     g = Geometry(request.param)
     yield g
