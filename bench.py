@@ -394,7 +394,7 @@ def product_arm(args, run: inputs.Run):
                 "peak_source": peak_src, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
                 "bytes_per_launch": uni_bytes / max(uni_steps, 1), "us_per_launch": uni_us / max(uni_steps, 1),
                 "launches": uni_steps, "traffic": captured_traffic(f"layer_pass:{s.name}")}
-    probes, probe_us = S("probes_timed"), S("us_probe_kernels")   # one probe in eight is bracketed by events
+    probes, probe_us = S("probes_timed"), S("us_probe_kernels")   # one probe in 32 is bracketed by events
     ach_p = probes * wb["head"] / (probe_us * 1e-6) / 1e9 if probe_us > 0 else 0.0
     roofline_exit = {"kernel": "exit-confidence kernel (final RMSNorm'd row x LM head, fused temperature softmax max/argmax)",
                      "bound": "hbm", "achieved": ach_p, "peak": peak, "unit": "GB/s", "frac": ach_p / peak,

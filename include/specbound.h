@@ -87,7 +87,7 @@ typedef struct {
     int64_t unified_layer_steps;          /* layer passes inside us_unified                          */
     int64_t unified_kv_positions;         /* sum over those passes of the KV length they attended over */
     double us_probe_kernels;              /* device time of the exit-confidence kernels of the draft phase that were
-                                             timed: one probe in eight is bracketed by CUDA events     */
+                                             timed: one probe in 32 is bracketed by CUDA events        */
     int64_t kernel_launches;              /* kernels launched by the call                            */
     int64_t h2d_bytes, d2h_bytes;         /* bytes copied host->device / device->host by the call    */
     int64_t probes_timed;                 /* probes behind us_probe_kernels                          */

@@ -851,9 +851,9 @@ static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf
                  sb_stats* st = nullptr, bool more_layers = false) {
     int r = c->rows - 1;
     ensure_act(c->e, c->norm_of(layer), r, 1);
-    // One probe in eight is bracketed by events (which needs the copy + synchronise path and keeps the kernel from
+    // One probe in 32 is bracketed by events (which needs the copy + synchronise path and keeps the kernel from
     // overlapping its predecessor); the others report through the mirror.
-    const bool timed = st && (c->probes_issued++ & 7) == 0;
+    const bool timed = st && (c->probes_issued++ & 31) == 0;
     if (timed) {
         cudaEventRecord(c->ev[5], c->e.st);
         head(c->e, c->head_of(layer), r, 1, tau_l, threshold, c->conf_d(), c->token_d(), c->flag_d(), nullptr);
