@@ -81,6 +81,9 @@ typedef struct {
     int64_t width_hist[SB_MAX_W + 1];     /* [w] = rounds verified with w rows                       */
     double us_prefill, us_decode;         /* host wall time around the two phases                    */
     double us_decode_dev;                 /* device time of the decode phase (CUDA events on the stream) */
+    /* The next five cover the TIMED rounds only (rounds_timed of them: the first round and every fourth after it).
+     * A CUDA event between two kernels keeps the later one from overlapping the earlier one's tail, so bracketing
+     * every round would slow down what it measures. */
     double us_draft, us_verify;           /* device time of draft phases / of verification (alignment,
                                              unified pass, final head, acceptance)                    */
     double us_unified;                    /* device time of the unified passes alone (layers D+1..L) */
@@ -91,6 +94,7 @@ typedef struct {
     int64_t kernel_launches;              /* kernels launched by the call                            */
     int64_t h2d_bytes, d2h_bytes;         /* bytes copied host->device / device->host by the call    */
     int64_t probes_timed;                 /* probes behind us_probe_kernels                          */
+    int64_t rounds_timed;                 /* rounds behind us_draft, us_verify, us_unified           */
 } sb_stats;
 
 typedef struct { /* trace of one speculation round, filled by sb_generate when asked to */

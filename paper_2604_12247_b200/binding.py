@@ -44,7 +44,7 @@ class Stats(C.Structure):
         ("us_prefill", C.c_double), ("us_decode", C.c_double), ("us_decode_dev", C.c_double), ("us_draft", C.c_double),
         ("us_verify", C.c_double), ("us_unified", C.c_double), ("unified_layer_steps", C.c_int64),
         ("unified_kv_positions", C.c_int64), ("us_probe_kernels", C.c_double), ("kernel_launches", C.c_int64),
-        ("h2d_bytes", C.c_int64), ("d2h_bytes", C.c_int64), ("probes_timed", C.c_int64)]
+        ("h2d_bytes", C.c_int64), ("d2h_bytes", C.c_int64), ("probes_timed", C.c_int64), ("rounds_timed", C.c_int64)]
 
 
 class Round(C.Structure):

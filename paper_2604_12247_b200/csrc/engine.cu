@@ -439,6 +439,7 @@ struct sb_ctx {
     struct { int layer = 0, r0 = 0, m = 0, s_qkv = 0; } ahead;   // QKV issued ahead for the next layer step (layer 0: none)
     int64_t probes_at[SB_MAX_LAYERS + 1] = {}, exits_at[SB_MAX_LAYERS + 1] = {};   // per layer, of the current sb_generate call
     int64_t probes_issued = 0;
+    bool time_round = true;      // the current round of sb_generate is bracketed by events (one round in kTimedRoundEvery)
     int n = 0, pending = -1, rows = 0;
     int depth[SB_MAX_W];
     float sample_temperature = 0.f;      // sampling decoding (Section 4.3): 0 = greedy
@@ -847,6 +848,9 @@ static void qkv_ahead(sb_ctx* c, int layer) {
     c->ahead.layer = layer + 1; c->ahead.r0 = r0; c->ahead.m = m;
 }
 
+// sb_generate brackets one round in this many with CUDA events (phase times, the unified pass's time and counters)
+constexpr int kTimedRoundEvery = 4;
+
 static int probe(sb_ctx* c, int layer, float tau_l, float threshold, float* conf, int32_t* token, int32_t* flag,
                  sb_stats* st = nullptr, bool more_layers = false) {
     int r = c->rows - 1;
@@ -894,12 +898,16 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     for (int i = 0; i < w; ++i) D = c->depth[i] > D ? c->depth[i] : D;
     for (int l = 1; l <= D; ++l) advance_suffix(c, l, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm, st);
     c->ahead.layer = 0;   // the unified pass is timed as a whole: it never starts from work issued ahead of its window
-    cudaEventRecord(c->ev[3], e.st);
+    // An event between two kernels keeps the second from overlapping the first (its weight tiles are requested only
+    // after the event): the rounds that are timed pay a few microseconds per event, so only some are (sb_generate).
+    const bool timed = st && c->time_round;
+    if (timed) cudaEventRecord(c->ev[3], e.st);
     for (int l = D + 1; l <= e.D.L; ++l) {
         run_layer(c, l, 0, w, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
-        if (st) { st->layer_steps++; st->layer_row_steps += w; st->unified_layer_steps++; st->unified_kv_positions += c->n + w; }
+        if (st) { st->layer_steps++; st->layer_row_steps += w; }
+        if (timed) { st->unified_layer_steps++; st->unified_kv_positions += c->n + w; }
     }
-    cudaEventRecord(c->ev[4], e.st);
+    if (timed) cudaEventRecord(c->ev[4], e.st);
     ensure_act(e, c->w.final_norm, 0, w);
     final_tokens(c, 0, w, (long long)c->n + 1, c->token_d(), Mirror{nullptr, nullptr, 0u});   // row i holds position n + i
     int d8[kMaxW];
@@ -907,11 +915,11 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     const Mirror mir = next_mirror(c);
     launch_accept(e.st, c->token_d(), d8, w, max_emit, c->accept_d(), mir);
     e.launches++;
-    cudaEventRecord(c->ev[2], e.st);
+    if (timed) cudaEventRecord(c->ev[2], e.st);
     int rc = wait_results(c, mir);
     if (rc) return rc;
-    if (st) cudaEventSynchronize(c->ev[2]);   // the round's events are read below and by the caller
-    if (st) {
+    if (timed) cudaEventSynchronize(c->ev[2]);   // the round's events are read below and by the caller
+    if (timed) {
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]) == cudaSuccess) st->us_unified += 1e3 * ms;
     }
@@ -975,7 +983,8 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
         int drafts[kMaxW];
         for (int i = 0; i < kMaxW; ++i) { drafts[i] = -1; R.draft[i] = -1; }
         int cur = c->pending;
-        cudaEventRecord(c->ev[0], e.st);
+        c->time_round = (nr % kTimedRoundEvery) == 0;
+        if (c->time_round) cudaEventRecord(c->ev[0], e.st);
         for (;;) {                              // draft phase (Section 3.3)
             if ((rc = sb_draft_push(c, cur))) return rc;
             int r = c->rows - 1;
@@ -999,13 +1008,16 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
             if (c->rows == w_max) break;        // long shallow chain: the width bound ends the round
             cur = drafts[r];
         }
-        cudaEventRecord(c->ev[1], e.st);
+        if (c->time_round) cudaEventRecord(c->ev[1], e.st);
         int w = c->rows, emit = 0;
         if ((rc = verify_rows(c, drafts, w, n_gen - produced, out_tokens + produced, &emit, st, &R))) return rc;
         produced += emit;
-        float ms = 0.f;
-        if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]) == cudaSuccess) st->us_draft += 1e3 * ms;
-        if (cudaEventElapsedTime(&ms, c->ev[1], c->ev[2]) == cudaSuccess) st->us_verify += 1e3 * ms;
+        if (c->time_round) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]) == cudaSuccess) st->us_draft += 1e3 * ms;
+            if (cudaEventElapsedTime(&ms, c->ev[1], c->ev[2]) == cudaSuccess) st->us_verify += 1e3 * ms;
+            st->rounds_timed++;
+        }
         if (rounds && nr < max_rounds) rounds[nr] = R;
         ++nr;
     }
