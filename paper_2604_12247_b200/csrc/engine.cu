@@ -116,7 +116,7 @@ constexpr int kWideRows = kWideBlocks * kMaxW;   // rows of one wide prefill pas
 struct Work {
     int* page_table;
     float* h;              // [8][d] hidden-state cache: one vector per in-flight row
-    void *act_a, *act_o, *act_f;
+    void *act_a, *act_b, *act_o, *act_f;   // act_b: the hidden rows under a second norm (layer_step's next_gain2)
     float *p_qkv, *p_o, *p_gu, *p_down;   // split-K partials [kMaxSplit][8][N]
     float* q;              // [8][qd]
     float* attn_part;
@@ -157,6 +157,7 @@ static size_t carve(const Dims& D, char* base, bool with_state, Work* w) {
     c.take(W.page_table, sizeof(int) * D.n_pages);
     c.take(W.h, sizeof(float) * kMaxW * D.d);
     c.take(W.act_a, es * act_rows * D.d);
+    c.take(W.act_b, es * act_rows * D.d);
     c.take(W.act_o, es * act_rows * D.qd);
     c.take(W.act_f, es * act_rows * D.F);
     size_t ps = sizeof(float) * kMaxSplit * kMaxW;
@@ -213,6 +214,7 @@ struct Exec {   // everything a launch sequence needs
     // which normalised activation act_a currently holds
     const void* act_gain = nullptr;
     int act_r0 = 0, act_m = 0;
+    const void* act2_gain = nullptr;      // ... and act_b (same rows), null = nothing valid
     TcPlanCache* plans = nullptr;
     unsigned int* clear_next = nullptr;   // 16 words that the next RMSNorm launch of ensure_act zeroes (stateless calls)
     int err = 0;   // sticky host-side error of a launch sequence (a TMA descriptor could not be built)
@@ -229,6 +231,7 @@ static void ensure_act(Exec& e, const void* gain, int r0, int m) {
     SB_T(e, launch_resid_norm<T>(e.st, e.W.h, nullptr, 0, e.D.d, (const T*)gain, e.D.eps, e.W.act_a, r0, m, e.clear_next));
     e.clear_next = nullptr;
     e.launches++;
+    if (r0 != e.act_r0 || m != e.act_m) e.act2_gain = nullptr;   // the row range describes both buffers
     e.act_gain = gain; e.act_r0 = r0; e.act_m = m;
 }
 
@@ -262,18 +265,22 @@ static int gemm(Exec& e, const void* const* W, const int* N, int n_mats, int K, 
 // issue them ahead of time (qkv_ahead) while the host still waits for an exit decision.  Returns the split count.
 static int layer_qkv(Exec& e, const sb_layer_weights& lw, int r0, int m) {
     const Dims& D = e.D;
-    ensure_act(e, lw.attn_norm, r0, m);
+    // the step that produced these rows may have left them under this layer's norm in the second operand buffer (it
+    // knew that an exit test would take the first): no RMSNorm launch then
+    const bool second = e.act2_gain == lw.attn_norm && e.act_gain != lw.attn_norm && r0 >= e.act_r0 && r0 + m <= e.act_r0 + e.act_m;
+    if (!second) ensure_act(e, lw.attn_norm, r0, m);
     const void* wqkv[3] = {lw.wq, lw.wk, lw.wv};
     int nqkv[3] = {D.qd, D.kvd, D.kvd};
     SB_MARK("norm");
-    int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, e.W.act_a, e.W.p_qkv, r0, m);
+    int s_qkv = gemm(e, wqkv, nqkv, 3, D.d, second ? e.W.act_b : e.W.act_a, e.W.p_qkv, r0, m);
     SB_MARK("qkv");
     return s_qkv;
 }
 
 // s_qkv_ahead > 0: layer_qkv was already issued for exactly these rows of this layer, with that split count
+// next_gain2 (nullable): a second gain under which the rows' RMSNorm is left as well (in act_b)
 static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, void* v_cache_l, int r0, int m, int pos0,
-                       const void* next_gain, int s_qkv_ahead = 0) {
+                       const void* next_gain, int s_qkv_ahead = 0, const void* next_gain2 = nullptr) {
     const Dims& D = e.D;
     Work& W = e.W;
     const int s_qkv = s_qkv_ahead > 0 ? s_qkv_ahead : layer_qkv(e, lw, r0, m);
@@ -331,10 +338,13 @@ static void layer_step(Exec& e, const sb_layer_weights& lw, void* k_cache_l, voi
     int nd[1] = {D.d};
     int s_d = gemm(e, wd, nd, 1, D.F, W.act_f, W.p_down, r0, m);
     SB_MARK("down");
-    SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_down, s_d, D.d, (const T*)next_gain, D.eps, W.act_a, r0, m));
+    if (!next_gain) next_gain2 = nullptr;
+    SB_T(e, launch_resid_norm<T>(e.st, W.h, W.p_down, s_d, D.d, (const T*)next_gain, D.eps, W.act_a, r0, m, nullptr,
+                                 (const T*)next_gain2, W.act_b));
     SB_MARK("resid");
     e.launches += 2;
     e.act_gain = next_gain; e.act_r0 = r0; e.act_m = m;
+    e.act2_gain = next_gain2;
 }
 
 // Wide prefill pass: one decoder layer for M <= 8 * kWideBlocks prompt rows at positions pos0 .. pos0+M-1 (bf16
@@ -502,11 +512,11 @@ static int wait_results(sb_ctx* c, const Mirror& m) {
     return SB_OK;
 }
 
-static void run_layer(sb_ctx* c, int layer, int r0, int m, const void* next_gain) {
+static void run_layer(sb_ctx* c, int layer, int r0, int m, const void* next_gain, const void* next_gain2 = nullptr) {
     // a QKV issued ahead is good for the very next layer step only (the scratch it wrote is reused by every step)
     const int s_ahead = (c->ahead.layer == layer && c->ahead.r0 == r0 && c->ahead.m == m) ? c->ahead.s_qkv : 0;
     c->ahead.layer = 0;
-    layer_step(c->e, c->layers[layer - 1], c->kc(layer), c->vc(layer), r0, m, c->n, next_gain, s_ahead);
+    layer_step(c->e, c->layers[layer - 1], c->kc(layer), c->vc(layer), r0, m, c->n, next_gain, s_ahead, next_gain2);
     for (int i = r0; i < r0 + m; ++i) c->depth[i] = layer;
 }
 
@@ -528,12 +538,12 @@ static void final_tokens(sb_ctx* c, int r0, int m, long long pos0, int* token, c
     e.launches++;
 }
 
-static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats* st) {
+static int advance_suffix(sb_ctx* c, int layer, const void* next_gain, sb_stats* st, const void* next_gain2 = nullptr) {
     int r0 = c->rows;
     while (r0 > 0 && c->depth[r0 - 1] == layer - 1) --r0;
     int m = c->rows - r0;
     if (m == 0) return 0;
-    run_layer(c, layer, r0, m, next_gain);
+    run_layer(c, layer, r0, m, next_gain, next_gain2);
     if (st) { st->layer_steps++; st->layer_row_steps += m; }
     return m;
 }
@@ -670,7 +680,7 @@ int sb_load_weights(sb_ctx* c, const sb_weights* w) {
 int sb_reset(sb_ctx* c) {
     if (!c) return SB_ERR_ARG;
     c->n = 0; c->pending = -1; c->rows = 0;
-    c->e.act_gain = nullptr;
+    c->e.act_gain = nullptr; c->e.act2_gain = nullptr;
     // a sticky host error or an expired device wait of an earlier call is forgotten with the sequence
     c->e.err = 0;
     if (cudaMemsetAsync(c->e.W.status, 0, 64, c->e.st) != cudaSuccess) return SB_ERR_CUDA;
@@ -784,7 +794,7 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
                 if (cudaMemcpyAsync(e.W.h, e.W.pf_h + (size_t)(nblk - 1) * kMaxW * e.D.d, sizeof(float) * m * e.D.d,
                                     cudaMemcpyDeviceToDevice, e.st) != cudaSuccess)
                     return SB_ERR_CUDA;
-                e.act_gain = nullptr;
+                e.act_gain = nullptr; e.act2_gain = nullptr;
             }
         }
     }
@@ -793,7 +803,7 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
         bool last = p0 + m == n_prompt;
         SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, e.W.toks + p0, 0, 0, m, e.W.h));
         e.launches++;
-        e.act_gain = nullptr;
+        e.act_gain = nullptr; e.act2_gain = nullptr;
         c->n = p0;
         for (int l = 1; l <= e.D.L; ++l) {
             const void* next = l < e.D.L ? c->layers[l].attn_norm : (last ? c->w.final_norm : nullptr);
@@ -934,7 +944,7 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     c->n += emit;                       // rollback: KV at positions >= n is dead and will be overwritten
     c->pending = c->mailbox[26 + emit - 1];
     c->rows = 0;
-    e.act_gain = nullptr;
+    e.act_gain = nullptr; e.act2_gain = nullptr;
     return SB_OK;
 }
 
@@ -993,7 +1003,10 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
                 // a layer whose temperature is <= 0 is walked but not probed: its step hands the rows straight to the
                 // next layer's attention norm
                 const bool probed = tau[l - 1] > 0.f;
-                advance_suffix(c, l, probed ? c->norm_of(l) : c->layers[l].attn_norm, st);
+                // a probed layer leaves its rows under the exit test's norm and, for the step that follows if the row
+                // stays, under the next layer's attention norm as well (one RMSNorm launch less per exit test)
+                advance_suffix(c, l, probed ? c->norm_of(l) : c->layers[l].attn_norm, st,
+                               probed && l < e.D.L ? c->layers[l].attn_norm : nullptr);
                 if (!probed) continue;
                 float conf; int tok, flag;
                 if ((rc = probe(c, l, tau[l - 1], threshold, &conf, &tok, &flag, st, l < d_max))) return rc;
@@ -1063,7 +1076,7 @@ int sb_generate_ar(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n
     for (int i = 1; i < n_gen; ++i) {
         SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, log + i - 1, 0, 0, 1, e.W.h));
         e.launches++;
-        e.act_gain = nullptr;
+        e.act_gain = nullptr; e.act2_gain = nullptr;
         for (int l = 1; l <= e.D.L; ++l)
             layer_step(e, c->layers[l - 1], c->kc(l), c->vc(l), 0, 1, c->n, l < e.D.L ? c->layers[l].attn_norm : c->w.final_norm);
         final_tokens(c, 0, 1, (long long)c->n + 1, log + i, Mirror{nullptr, nullptr, 0u});

@@ -35,14 +35,18 @@ void launch_embed(cudaStream_t st, const T* embed, int d, const int* toks_dev, i
 // ------------------------------------------------------------------------------------------------
 // h[row] += sum_s part[s][row][:]   (if part != null; split-K partials are summed in split order)
 // act[row] = h[row] / sqrt(mean(h[row]^2) + eps) * gain      (if gain != null)
+// act2[row] = the same with gain2                             (if gain2 != null: the rows are about to be read under two
+//                                                              norms, the exit test's and the next layer's)
 // One CTA per row; the reduction order is fixed by the thread layout only.
 // ------------------------------------------------------------------------------------------------
 constexpr int kNormThreads = 1024;
 constexpr int kNormVec = 2;   // float4 per thread: rows up to 1024 * 2 * 4 = 8192 wide
-template <typename T, bool kWide>
+// kDual: a second gain and output (an instantiation of its own: the common form stays as small as it was)
+template <typename T, bool kWide, bool kDual>
 __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__ h, const float* __restrict__ part,
                                                             int n_split, int d, const T* __restrict__ gain, float eps,
-                                                            void* __restrict__ act, int r0, unsigned int* __restrict__ clear16) {
+                                                            void* __restrict__ act, int r0, unsigned int* __restrict__ clear16,
+                                                            const T* __restrict__ gain2, void* __restrict__ act2) {
     __shared__ float red[kNormThreads / 32];
     pdl_trigger();
     // the gains are weights: no kernel writes them, so they are requested before the grid-dependency wait (a layer's
@@ -54,6 +58,14 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
         for (int j = 0; j < kNormVec; ++j) {
             int k4 = threadIdx.x + j * kNormThreads;
             if (k4 < nv) g4[j] = load_gain4(gain, k4 << 2);
+        }
+    }
+    float4 g4b[kNormVec];
+    if (kDual) {
+#pragma unroll
+        for (int j = 0; j < kNormVec; ++j) {
+            int k4 = threadIdx.x + j * kNormThreads;
+            if (k4 < nv) g4b[j] = load_gain4(gain2, k4 << 2);
         }
     }
     pdl_wait();
@@ -97,12 +109,27 @@ __global__ void __launch_bounds__(kNormThreads) k_resid_norm(float* __restrict__
             A::store4(a, row, k4 << 2, d, make_float4(v[j].x * inv * g4[j].x, v[j].y * inv * g4[j].y, v[j].z * inv * g4[j].z,
                                                      v[j].w * inv * g4[j].w));
     }
+    if (kDual) {
+        typename A::type* a2 = reinterpret_cast<typename A::type*>(act2) + (size_t)blk * A::rows * d;
+#pragma unroll
+        for (int j = 0; j < kNormVec; ++j) {
+            int k4 = threadIdx.x + j * kNormThreads;
+            if (k4 < nv)
+                A::store4(a2, row, k4 << 2, d, make_float4(v[j].x * inv * g4b[j].x, v[j].y * inv * g4b[j].y,
+                                                          v[j].z * inv * g4b[j].z, v[j].w * inv * g4b[j].w));
+        }
+    }
 }
 template <typename T>
 void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d, const T* gain, float eps,
-                       void* act, int r0, int m, unsigned int* clear16) {
-    if (r0 + m > kMaxW) launch_k(k_resid_norm<T, true>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16);
-    else launch_k(k_resid_norm<T, false>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16);
+                       void* act, int r0, int m, unsigned int* clear16, const T* gain2, void* act2) {
+    if (!gain || !act2) gain2 = nullptr;
+    if (gain2) {   // draft steps only: at most 8 rows
+        launch_k(k_resid_norm<T, false, true>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16, gain2, act2);
+        return;
+    }
+    if (r0 + m > kMaxW) launch_k(k_resid_norm<T, true, false>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16, gain2, act2);
+    else launch_k(k_resid_norm<T, false, false>, dim3(m), dim3(kNormThreads), 0, st, h, part, n_split, d, gain, eps, act, r0, clear16, gain2, act2);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1125,7 +1152,7 @@ void launch_init_pages(cudaStream_t st, int* page_table, int n_pages) {
 // explicit instantiations
 #define SB_INST(T)                                                                                                  \
     template void launch_embed<T>(cudaStream_t, const T*, int, const int*, int, int, int, float*);                  \
-    template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int, unsigned int*); \
+    template void launch_resid_norm<T>(cudaStream_t, float*, const float*, int, int, const T*, float, void*, int, int, unsigned int*, const T*, void*); \
     template void launch_rope_append<T>(cudaStream_t, const RopeArgs&);                                             \
     template bool launch_attention<T>(cudaStream_t, const AttnArgs&);                                               \
     template void launch_attention_combine<T>(cudaStream_t, const AttnArgs&);                                       \

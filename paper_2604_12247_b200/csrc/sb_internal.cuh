@@ -420,7 +420,7 @@ template <typename T> void launch_embed(cudaStream_t st, const T* embed, int d, 
                                         int row0, int m, float* h);
 template <typename T> void launch_resid_norm(cudaStream_t st, float* h, const float* part, int n_split, int d,
                                              const T* gain, float eps, void* act, int r0, int m,
-                                             unsigned int* clear16 = nullptr);
+                                             unsigned int* clear16 = nullptr, const T* gain2 = nullptr, void* act2 = nullptr);
 template <typename T> void launch_rope_append(cudaStream_t st, const RopeArgs& a);
 // cos/sin of pos * inv_freq[i] for pos < n_pos, i < half, as [pos][half]
 void launch_rope_table(cudaStream_t st, float2* tab, int n_pos, int half, const double* inv_freq);
