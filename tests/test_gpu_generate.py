@@ -48,6 +48,12 @@ def test_tiny_run_matches_oracle_tokens_and_trace(which, tiny_weights, tiny_damp
     assert st.probes == sum(r.probes for r in orc_rounds)
     assert st.layer_steps == sum(r.layer_steps for r in orc_rounds)
     assert st.kernel_launches > 0
+    # the phase timings and the unified-pass counters cover the event-bracketed rounds: the first and every fourth after it
+    timed = [r for i, r in enumerate(orc_rounds) if i % 4 == 0]
+    assert st.rounds_timed == len(timed)
+    assert st.unified_layer_steps == sum(run.shape.n_layers - r.D for r in timed)   # layers D+1 .. L of each
+    assert st.us_unified > 0 and st.us_draft > 0 and st.us_verify >= st.us_unified
+    assert 1 <= st.probes_timed <= st.probes
     # determinism: a second run is identical down to the confidence bits
     sp2 = ctx.generate(pr, run.n_gen, run.d_max, run.w_max, run.tau, run.threshold, trace=True)
     assert np.array_equal(sp2["tokens"], sp["tokens"])
