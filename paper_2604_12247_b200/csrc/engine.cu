@@ -450,6 +450,8 @@ struct sb_ctx {
     int64_t probes_at[SB_MAX_LAYERS + 1] = {}, exits_at[SB_MAX_LAYERS + 1] = {};   // per layer, of the current sb_generate call
     int64_t probes_issued = 0;
     bool time_round = true;      // the current round of sb_generate is bracketed by events (one round in kTimedRoundEvery)
+    bool round_ahead = false;    // sb_generate: verify_rows may issue the start of the next round behind the acceptance kernel
+    bool embed_ahead = false;    // ... and did: row 0 already holds the embedding of the last emitted token
     int n = 0, pending = -1, rows = 0;
     int depth[SB_MAX_W];
     float sample_temperature = 0.f;      // sampling decoding (Section 4.3): 0 = greedy
@@ -680,6 +682,7 @@ int sb_load_weights(sb_ctx* c, const sb_weights* w) {
 int sb_reset(sb_ctx* c) {
     if (!c) return SB_ERR_ARG;
     c->n = 0; c->pending = -1; c->rows = 0;
+    c->ahead.layer = 0; c->embed_ahead = false; c->round_ahead = false;
     c->e.act_gain = nullptr; c->e.act2_gain = nullptr;
     // a sticky host error or an expired device wait of an earlier call is forgotten with the sequence
     c->e.err = 0;
@@ -829,8 +832,12 @@ int sb_draft_push(sb_ctx* c, int32_t token) {
     if (c->rows >= SB_MAX_W) return SB_ERR_CAPACITY;
     if (c->n + c->rows + 1 > c->e.D.max_seq) return SB_ERR_CAPACITY;
     Exec& e = c->e;
-    SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, nullptr, token, c->rows, 1, e.W.h));
-    e.launches++;
+    if (c->embed_ahead && c->rows == 0) {
+        c->embed_ahead = false;   // issued behind the last round's acceptance kernel, from the same token on the device
+    } else {
+        SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, nullptr, token, c->rows, 1, e.W.h));
+        e.launches++;
+    }
     c->depth[c->rows++] = 0;
     return SB_OK;
 }
@@ -926,6 +933,17 @@ static int verify_rows(sb_ctx* c, const int32_t* drafts, int w, int max_emit, in
     launch_accept(e.st, c->token_d(), d8, w, max_emit, c->accept_d(), mir);
     e.launches++;
     if (timed) cudaEventRecord(c->ev[2], e.st);
+    // While the host waits for the outcome, the GPU would idle: the next round always starts by embedding the last
+    // emitted token, which the acceptance kernel has left on the device, and by the RMSNorm + QKV GEMM of layer 1 on
+    // row 0.  They touch the hidden row, the operand buffer and scratch only (the rows of this round are done with).
+    if (c->round_ahead && e.D.L > 1) {
+        SB_T(e, launch_embed<T>(e.st, (const T*)c->w.embed, e.D.d, c->accept_d() + 10, 0, 0, 1, e.W.h));
+        e.launches++;
+        e.act_gain = nullptr; e.act2_gain = nullptr;
+        c->ahead.s_qkv = layer_qkv(e, c->layers[0], 0, 1);
+        c->ahead.layer = 1; c->ahead.r0 = 0; c->ahead.m = 1;
+        c->embed_ahead = true;
+    }
     int rc = wait_results(c, mir);
     if (rc) return rc;
     if (timed) cudaEventSynchronize(c->ev[2]);   // the round's events are read below and by the caller
@@ -1023,6 +1041,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
         }
         if (c->time_round) cudaEventRecord(c->ev[1], e.st);
         int w = c->rows, emit = 0;
+        c->round_ahead = g_qkv_ahead && produced + w < n_gen;   // this round cannot be the last one
         if ((rc = verify_rows(c, drafts, w, n_gen - produced, out_tokens + produced, &emit, st, &R))) return rc;
         produced += emit;
         if (c->time_round) {
@@ -1034,6 +1053,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
         if (rounds && nr < max_rounds) rounds[nr] = R;
         ++nr;
     }
+    c->round_ahead = false; c->embed_ahead = false; c->ahead.layer = 0;
     cudaEventRecord(c->ev[8], e.st);
     cudaEventSynchronize(c->ev[8]);
     st->us_decode = now_us() - t1;

@@ -790,7 +790,7 @@ template <typename T> void launch_swiglu(cudaStream_t st, const float* part, int
 
 // ------------------------------------------------------------------------------------------------
 // Greedy acceptance: the longest prefix of drafts equal to the full model's tokens, then the
-// model's own token.  result = {n_emit, n_accepted_drafts, g[0..7]}
+// model's own token.  result = {n_emit, n_accepted_drafts, g[0..7], last emitted token}
 // ------------------------------------------------------------------------------------------------
 struct Drafts8 { int v[kMaxW]; };
 __global__ void k_accept(const int* __restrict__ g, Drafts8 drafts, int w, int max_emit, int* __restrict__ result, Mirror mirror) {
@@ -804,6 +804,7 @@ __global__ void k_accept(const int* __restrict__ g, Drafts8 drafts, int w, int m
         result[0] = emit;
         result[1] = acc;
         for (int i = 0; i < kMaxW; ++i) result[2 + i] = i < w ? g[i] : -1;
+        result[10] = g[emit - 1];   // the token the next round starts from: the embedding kernel issued ahead reads it here
     }
     publish_results(mirror);
 }
