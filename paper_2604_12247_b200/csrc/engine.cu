@@ -825,8 +825,10 @@ int sb_prefill(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t* firs
     return SB_OK;
 }
 
-int sb_draft_push(sb_ctx* c, int32_t token) {
+// from_generate: the call comes from sb_generate's round loop, which alone may have issued the embedding ahead
+static int draft_push(sb_ctx* c, int32_t token, bool from_generate) {
     if (!c) return SB_ERR_ARG;
+    if (!from_generate) c->embed_ahead = false;
     if (!c->loaded || c->pending < 0) return SB_ERR_STATE;
     if (token < 0 || token >= c->e.D.V) return SB_ERR_ARG;
     if (c->rows >= SB_MAX_W) return SB_ERR_CAPACITY;
@@ -841,6 +843,7 @@ int sb_draft_push(sb_ctx* c, int32_t token) {
     c->depth[c->rows++] = 0;
     return SB_OK;
 }
+int sb_draft_push(sb_ctx* c, int32_t token) { return draft_push(c, token, false); }
 
 int sb_draft_advance(sb_ctx* c, int32_t to_layer) {
     if (!c) return SB_ERR_ARG;
@@ -1014,7 +1017,7 @@ int sb_generate(sb_ctx* c, const int32_t* prompt, int32_t n_prompt, int32_t n_ge
         c->time_round = (nr % kTimedRoundEvery) == 0;
         if (c->time_round) cudaEventRecord(c->ev[0], e.st);
         for (;;) {                              // draft phase (Section 3.3)
-            if ((rc = sb_draft_push(c, cur))) return rc;
+            if ((rc = draft_push(c, cur, true))) return rc;
             int r = c->rows - 1;
             bool exited = false;
             for (int l = 1; l <= d_max; ++l) {
