@@ -94,47 +94,111 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
     const int ntot = qd + 2 * kvd;
     const size_t sstride = (size_t)kMaxW * ntot;
     const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
-    const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
-    struct Item { int kind, pos, e2, p; const float* src; float2 cs; int page; };   // kind 0: q pair of (row, head) pair p; 1: K pair; 2: V pair of position pos
-    auto item_of = [&](int idx) -> Item {
-        Item it;
-        if (idx < n_q) {
-            const int p = idx / half;
-            it.kind = 0; it.pos = a.pos0 + a.r0 + p / G; it.e2 = idx - p * half; it.p = p;
-        } else {
-            const int j = idx - n_q, e = j % HD;
-            it.kind = e >= half ? 2 : 1; it.pos = lo + j / HD; it.e2 = e >= half ? e - half : e; it.p = 0;
-        }
-        it.src = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
-                 (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
-        it.cs = it.kind != 2 ? rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2) : make_float2(1.f, 0.f);
-        it.page = it.kind != 0 ? a.page_table[it.pos >> a.page_shift] : 0;   // (the page table is constant: see above)
-        return it;
-    };
-    Item first{};
-    if ((int)threadIdx.x < n_items) first = item_of(threadIdx.x);
-    pdl_wait();
-    for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
-        const Item it = idx == (int)threadIdx.x ? first : item_of(idx);
-        float x0 = sum_splits(it.src, sstride, a.n_split);
-        float x1 = sum_splits(it.src + half, sstride, a.n_split);
-        if (it.kind != 2) rope_apply(it.cs, x0, x1);
-        if (it.kind == 0) {
-            q_s[it.p * HD + it.e2] = x0;
-            q_s[it.p * HD + it.e2 + half] = x1;
-        } else {
-            const bool is_v = it.kind == 2;
-            const T y0 = from_f32<T>(x0), y1 = from_f32<T>(x1);
-            T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
-            T* dst = cache + ((size_t)it.page * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
-            if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
-                dst[it.e2] = y0;
-                dst[it.e2 + half] = y1;
+    // Two forms of the same loop.  The narrow one (PG = 1: rounds of one to three rows, the latency-critical ones) is kept
+    // exactly as it was measured: written as the VEC = 1 case of the wide form it compiled to code that ran 1-1.5 us per
+    // layer slower, for no visible reason but its shape.
+    if constexpr (PG < 2) {   // one rotation pair per work item
+        const int n_q = P * half, n_items = n_q + max(hi - lo + 1, 0) * HD;
+        struct Item { int kind, pos, e2, p; const float* src; float2 cs; int page; };   // kind 0: q pair of (row, head) pair p; 1: K pair; 2: V pair of position pos
+        auto item_of = [&](int idx) -> Item {
+            Item it;
+            if (idx < n_q) {
+                const int p = idx / half;
+                it.kind = 0; it.pos = a.pos0 + a.r0 + p / G; it.e2 = idx - p * half; it.p = p;
+            } else {
+                const int j = idx - n_q, e = j % HD;
+                it.kind = e >= half ? 2 : 1; it.pos = lo + j / HD; it.e2 = e >= half ? e - half : e; it.p = 0;
             }
-            const int tl = it.pos - c * kAttnChunk;
-            T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
-            srow[it.e2] = y0;
-            srow[it.e2 + half] = y1;
+            it.src = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
+                     (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+            it.cs = it.kind != 2 ? rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2) : make_float2(1.f, 0.f);
+            it.page = it.kind != 0 ? a.page_table[it.pos >> a.page_shift] : 0;   // (the page table is constant: see above)
+            return it;
+        };
+        Item first{};
+        if ((int)threadIdx.x < n_items) first = item_of(threadIdx.x);
+        pdl_wait();
+        for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
+            const Item it = idx == (int)threadIdx.x ? first : item_of(idx);
+            float x0 = sum_splits(it.src, sstride, a.n_split);
+            float x1 = sum_splits(it.src + half, sstride, a.n_split);
+            if (it.kind != 2) rope_apply(it.cs, x0, x1);
+            if (it.kind == 0) {
+                q_s[it.p * HD + it.e2] = x0;
+                q_s[it.p * HD + it.e2 + half] = x1;
+            } else {
+                const bool is_v = it.kind == 2;
+                const T y0 = from_f32<T>(x0), y1 = from_f32<T>(x1);
+                T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
+                T* dst = cache + ((size_t)it.page * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
+                    dst[it.e2] = y0;
+                    dst[it.e2 + half] = y1;
+                }
+                const int tl = it.pos - c * kAttnChunk;
+                T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
+                srow[it.e2] = y0;
+                srow[it.e2 + half] = y1;
+            }
+        }
+    } else {
+        // Wide rounds (PG >= 2) take two neighbouring rotation pairs per item (8-byte loads of the partial sums, packed
+        // stores): half as many passes over the items, and the CTA that also appends the new rows -- eight rows are 1024
+        // single-pair items on 256 threads -- is what the cluster's other CTAs wait for at the merge.
+        constexpr int VEC = PG >= 2 ? 2 : 1;
+        constexpr int hv = half / VEC, per_pos = HD / VEC;
+        const int n_q = P * hv, n_items = n_q + max(hi - lo + 1, 0) * per_pos;
+        struct Item { int kind, pos, e2, p; const float* src; float2 cs[VEC]; int page; };   // kind 0: q pairs of (row, head) pair p; 1: K pairs; 2: V pairs of position pos
+        auto item_of = [&](int idx) -> Item {
+            Item it;
+            if (idx < n_q) {
+                const int p = idx / hv;
+                it.kind = 0; it.pos = a.pos0 + a.r0 + p / G; it.e2 = (idx - p * hv) * VEC; it.p = p;
+            } else {
+                const int j = idx - n_q, e = (j % per_pos) * VEC;
+                it.kind = e >= half ? 2 : 1; it.pos = lo + j / per_pos; it.e2 = e >= half ? e - half : e; it.p = 0;
+            }
+            it.src = a.qkv + (size_t)(it.pos - a.pos0) * ntot +
+                     (it.kind == 0 ? (head0 + (it.p % G)) * HD : qd + (it.kind == 2 ? kvd : 0) + kvh * HD) + it.e2;
+    #pragma unroll
+            for (int v2 = 0; v2 < VEC; ++v2)
+                it.cs[v2] = it.kind != 2 ? rope_fetch(a.inv_freq, a.rope_tab, half, it.pos, it.e2 + v2) : make_float2(1.f, 0.f);
+            it.page = it.kind != 0 ? a.page_table[it.pos >> a.page_shift] : 0;   // (the page table is constant: see above)
+            return it;
+        };
+        Item first{};
+        if ((int)threadIdx.x < n_items) first = item_of(threadIdx.x);
+        pdl_wait();
+        for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
+            const Item it = idx == (int)threadIdx.x ? first : item_of(idx);
+            float x0[VEC], x1[VEC];
+            if constexpr (VEC == 2) {
+                const float2 lo2 = sum_splits2(it.src, sstride, a.n_split), hi2 = sum_splits2(it.src + half, sstride, a.n_split);
+                x0[0] = lo2.x; x0[1] = lo2.y; x1[0] = hi2.x; x1[1] = hi2.y;
+            } else {
+                x0[0] = sum_splits(it.src, sstride, a.n_split);
+                x1[0] = sum_splits(it.src + half, sstride, a.n_split);
+            }
+            if (it.kind != 2) {
+    #pragma unroll
+                for (int v2 = 0; v2 < VEC; ++v2) rope_apply(it.cs[v2], x0[v2], x1[v2]);
+            }
+            if (it.kind == 0) {
+                store_run<float, VEC>(q_s + it.p * HD + it.e2, x0);
+                store_run<float, VEC>(q_s + it.p * HD + it.e2 + half, x1);
+            } else {
+                const bool is_v = it.kind == 2;
+                T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
+                T* dst = cache + ((size_t)it.page * a.page + (it.pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
+                    store_run<T, VEC>(dst + it.e2, x0);
+                    store_run<T, VEC>(dst + it.e2 + half, x1);
+                }
+                const int tl = it.pos - c * kAttnChunk;
+                T* srow = reinterpret_cast<T*>(kv_s + (size_t)(tl >> 5) * 64 * ROWB + (is_v ? 32 * ROWB : 0) + (tl & 31) * ROWB);
+                store_run<T, VEC>(srow + it.e2, x0);
+                store_run<T, VEC>(srow + it.e2 + half, x1);
+            }
         }
     }
     {   // bounded wait for this block's copies

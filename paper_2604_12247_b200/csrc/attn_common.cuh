@@ -121,6 +121,20 @@ struct GroupDiv {
     __device__ __forceinline__ int operator()(int x) const { return sh >= 0 ? x >> sh : (int)((unsigned)x / (unsigned)d); }
 };
 
+// N (1 or 2) consecutive values rounded to the storage type and stored at p (N * sizeof(T)-byte aligned), as one store
+template <typename T, int N> __device__ __forceinline__ void store_run(T* p, const float (&v)[N]);
+template <> __device__ __forceinline__ void store_run<float, 1>(float* p, const float (&v)[1]) { p[0] = v[0]; }
+template <> __device__ __forceinline__ void store_run<float, 2>(float* p, const float (&v)[2]) {
+    *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]);
+}
+template <> __device__ __forceinline__ void store_run<__nv_bfloat16, 1>(__nv_bfloat16* p, const float (&v)[1]) { p[0] = from_f32<__nv_bfloat16>(v[0]); }
+template <> __device__ __forceinline__ void store_run<__nv_bfloat16, 2>(__nv_bfloat16* p, const float (&v)[2]) {
+    __nv_bfloat162 r;
+    r.x = from_f32<__nv_bfloat16>(v[0]);
+    r.y = from_f32<__nv_bfloat16>(v[1]);
+    *reinterpret_cast<__nv_bfloat162*>(p) = r;
+}
+
 // 1 / sqrt(head_dim) as every kernel forms it
 __device__ __forceinline__ float attn_score_scale(int hd) { return rsqrtf((float)hd); }
 

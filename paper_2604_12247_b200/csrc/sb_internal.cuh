@@ -206,6 +206,16 @@ __device__ __forceinline__ float sum_splits(const float* __restrict__ first, siz
     for (int s = 1; s < kMaxSplitK; ++s) acc += v[s];
     return acc;
 }
+__device__ __forceinline__ float2 sum_splits2(const float* __restrict__ first, size_t split_stride, int n_split) {   // two neighbouring elements
+    float2 v[kMaxSplitK];
+#pragma unroll
+    for (int s = 0; s < kMaxSplitK; ++s)
+        v[s] = s < n_split ? __ldcg(reinterpret_cast<const float2*>(first + (size_t)s * split_stride)) : make_float2(0.f, 0.f);
+    float2 acc = v[0];
+#pragma unroll
+    for (int s = 1; s < kMaxSplitK; ++s) { acc.x += v[s].x; acc.y += v[s].y; }
+    return acc;
+}
 __device__ __forceinline__ float4 sum_splits4(const float4* __restrict__ first, size_t split_stride4, int n_split) {
     float4 v[kMaxSplitK];
 #pragma unroll
