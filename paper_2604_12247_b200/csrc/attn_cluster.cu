@@ -118,8 +118,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
         Item first{};
         if ((int)threadIdx.x < n_items) first = item_of(threadIdx.x);
         pdl_wait();
-        for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
-            const Item it = idx == (int)threadIdx.x ? first : item_of(idx);
+        auto process = [&](const Item& it) {
             float x0 = sum_splits(it.src, sstride, a.n_split);
             float x1 = sum_splits(it.src + half, sstride, a.n_split);
             if (it.kind != 2) rope_apply(it.cs, x0, x1);
@@ -140,7 +139,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) k_attn_cluster(AttnArgs a) {
                 srow[it.e2] = y0;
                 srow[it.e2 + half] = y1;
             }
-        }
+        };
+        // the item prepared above goes first, with its loads right behind the wait; the others, if any, through the loop
+        if ((int)threadIdx.x < n_items) process(first);
+        for (int idx = threadIdx.x + blockDim.x; idx < n_items; idx += blockDim.x) process(item_of(idx));
     } else {
         // Wide rounds (PG >= 2) take two neighbouring rotation pairs per item (8-byte loads of the partial sums, packed
         // stores): half as many passes over the items, and the CTA that also appends the new rows -- eight rows are 1024
