@@ -398,7 +398,50 @@ __global__ void __launch_bounds__(kPosWarps * WPB * 32) k_attn_partial(AttnArgs 
     }
     // 2. while those copies fly: q, and (front end) the new positions' K and V
     for (int idx = P * HD + threadIdx.x; idx < Ppad * HD; idx += blockDim.x) q_s[idx] = 0.f;   // padding pairs
-    if (kFront) {
+    if (kFront && PG >= 4) {
+        // Wide rounds: two neighbouring rotation pairs per work item (8-byte loads of the partial sums, packed stores), as in
+        // the cluster kernel: every chunk CTA redoes the q rotation, and this halves its passes over the items.
+        constexpr int half = HD / 2, VEC = 2, hv = half / VEC, per_pos = HD / VEC;
+        const int ntot = qd + 2 * kvd;
+        const size_t sstride = (size_t)kMaxW * ntot;
+        const int lo = max(pos_new0, c * kAttnChunk), hi = min(pos_last, c * kAttnChunk + kAttnChunk - 1);
+        const int n_q = P * hv, n_items = n_q + max(hi - lo + 1, 0) * per_pos;
+        for (int idx = threadIdx.x; idx < n_items; idx += blockDim.x) {
+            int kind, pos, e2, p = 0;   // kind 0: q pairs of (row, head) pair p; 1: K pairs; 2: V pairs of position pos
+            if (idx < n_q) {
+                p = idx / hv;
+                kind = 0; pos = a.pos0 + a.r0 + divG(p); e2 = (idx - p * hv) * VEC;
+            } else {
+                const int j = idx - n_q, e = (j % per_pos) * VEC;
+                kind = e >= half ? 2 : 1; pos = lo + j / per_pos; e2 = e >= half ? e - half : e;
+            }
+            const float* src = a.qkv + (size_t)(pos - a.pos0) * ntot +
+                               (kind == 0 ? (head0 + (p - divG(p) * G)) * HD : qd + (kind == 2 ? kvd : 0) + kvh * HD) + e2;
+            const float2 lo2 = sum_splits2(src, sstride, a.n_split), hi2 = sum_splits2(src + half, sstride, a.n_split);
+            float x0[VEC] = {lo2.x, lo2.y}, x1[VEC] = {hi2.x, hi2.y};
+            if (kind != 2) {
+#pragma unroll
+                for (int v2 = 0; v2 < VEC; ++v2) rope_apply(rope_fetch(a.inv_freq, a.rope_tab, half, pos, e2 + v2), x0[v2], x1[v2]);
+            }
+            if (kind == 0) {
+                store_run<float, VEC>(q_s + p * HD + e2, x0);
+                store_run<float, VEC>(q_s + p * HD + e2 + half, x1);
+            } else {
+                const bool is_v = kind == 2;
+                const int page = a.page_table[pos >> a.page_shift];
+                T* cache = reinterpret_cast<T*>(const_cast<void*>(is_v ? a.v_cache : a.k_cache));
+                T* dst = cache + ((size_t)page * a.page + (pos & (a.page - 1))) * kvd + (size_t)kvh * HD;
+                if (gsub == 0) {   // one of the CTAs that share the KV head appends; all of them put the rows in their tile
+                    store_run<T, VEC>(dst + e2, x0);
+                    store_run<T, VEC>(dst + e2 + half, x1);
+                }
+                const int tl = pos - c * kAttnChunk;
+                T* srow = reinterpret_cast<T*>(is_v ? v_tiles + (size_t)tl * ROWB_V : k_tiles + (size_t)tl * ROWB_K);
+                store_run<T, VEC>(srow + e2, x0);
+                store_run<T, VEC>(srow + e2 + half, x1);
+            }
+        }
+    } else if (kFront) {
         constexpr int half = HD / 2;
         constexpr int kBatch = 1;   // work items whose partial sums are requested together: one (see k_attn_cluster; here 4 were 0.7-2.7 us per layer slower)
         const int ntot = qd + 2 * kvd;
